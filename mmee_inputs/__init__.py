@@ -1,0 +1,142 @@
+"""Synthetic, deterministic inputs for the MMEE search path.
+
+Only shapes and accelerator constants live here: attention workload tuples, accelerator
+parameter sets and search options, as plain dicts whose keys are the field names of the
+three input structs (workload, arch, objective).  No part of the cost model is computed in
+this module; both the CUDA library's binding and the CPU oracle receive these dicts and do
+their own set-up.
+"""
+from __future__ import annotations
+
+import random
+
+OBJ_ENERGY, OBJ_LATENCY, OBJ_EDP = 0, 1, 2
+TILE_POW2, TILE_ALL_DIVISORS = 0, 1
+ORD_NORECOMP2, ORD_ALL6 = 0, 1
+FUSE_FUSED, FUSE_SOFTMAX_IN_OP1, FUSE_SEPARATE = 1, 2, 4
+FUSE_ALL = 7
+
+KiB = 1024
+MiB = 1024 * 1024
+
+
+def workload(batch, q_heads, kv_heads, seq_q, seq_kv, d_qk, d_v, word_bytes=2):
+    return dict(batch=batch, q_heads=q_heads, kv_heads=kv_heads, seq_q=seq_q, seq_kv=seq_kv,
+                d_qk=d_qk, d_v=d_v, word_bytes=word_bytes)
+
+
+def arch(pe_rows, pe_cols, n_arrays, gb_bytes, rf_bytes, dram_words_per_cycle,
+         e_dram_pj, e_gb_pj, e_rf_pj, e_mac_pj, c_softmax=10.0, energy_quantum_pj=1.0):
+    return dict(pe_rows=pe_rows, pe_cols=pe_cols, n_arrays=n_arrays, gb_bytes=gb_bytes,
+                rf_bytes=rf_bytes, dram_words_per_cycle=dram_words_per_cycle,
+                e_dram_pj=e_dram_pj, e_gb_pj=e_gb_pj, e_rf_pj=e_rf_pj, e_mac_pj=e_mac_pj,
+                c_softmax=c_softmax, energy_quantum_pj=energy_quantum_pj)
+
+
+def objective(objective=OBJ_ENERGY, topk=1, tiling_set=TILE_ALL_DIVISORS, order_set=ORD_ALL6,
+              fuse_mask=FUSE_ALL, t_begin=0, t_end=0):
+    return dict(objective=objective, topk=topk, tiling_set=tiling_set, order_set=order_set,
+                fuse_mask=fuse_mask, t_begin=t_begin, t_end=t_end)
+
+
+# --- accelerators -----------------------------------------------------------------------------
+
+def arch_tiny():
+    """8x8 PE array, DRAM + 32 KB global buffer, no register-file level."""
+    return arch(8, 8, 1, 32 * KiB, 0, 64, 200.0, 6.0, 0.0, 1.0)
+
+
+def arch_edge():
+    """16x16 PE array, DRAM / 256 KB global buffer / 1 KB register file per PE."""
+    return arch(16, 16, 1, 256 * KiB, 1 * KiB, 32, 200.0, 6.0, 1.0, 1.0)
+
+
+def arch_cloud():
+    """128x128 PE array, HBM / 8 MB global buffer / 2 KB register file per PE."""
+    return arch(128, 128, 1, 8 * MiB, 2 * KiB, 512, 120.0, 4.0, 0.8, 0.5, energy_quantum_pj=0.1)
+
+
+def arch_accel1():
+    """The paper's first evaluation accelerator (Section VII-A): 4 arrays of 32x32 PEs, 1 MB buffer,
+    60 GB/s DRAM at 1 GHz with 2-byte words = 30 words/cycle.  Energy constants are stand-ins."""
+    return arch(32, 32, 4, 1 * MiB, 1 * KiB, 30, 200.0, 6.0, 1.0, 1.0)
+
+
+# --- the five benchmark configurations --------------------------------------------------------
+
+def config1():
+    """Tiny single-head attention, power-of-two tilings, two loop orders, fuse / no-fuse."""
+    return dict(name="tiny_s64_d64", workload=workload(1, 1, 1, 64, 64, 64, 64),
+                arch=arch_tiny(),
+                searches=[objective(OBJ_ENERGY, 1, TILE_POW2, ORD_NORECOMP2,
+                                    FUSE_FUSED | FUSE_SEPARATE)])
+
+
+def config2():
+    """BERT-base-shaped attention on the edge accelerator; energy, then latency."""
+    return dict(name="bert_base_s512", workload=workload(1, 12, 12, 512, 512, 64, 64),
+                arch=arch_edge(),
+                searches=[objective(OBJ_ENERGY, 1), objective(OBJ_LATENCY, 1)])
+
+
+def config3():
+    """Llama-style prefill attention on the cloud accelerator; energy and latency, top-16."""
+    return dict(name="llama_prefill_s4096", workload=workload(1, 32, 32, 4096, 4096, 128, 128),
+                arch=arch_cloud(),
+                searches=[objective(OBJ_ENERGY, 16), objective(OBJ_LATENCY, 16)])
+
+
+def config4():
+    """Grouped-query attention (32 query heads on 8 KV heads), latency and energy-delay product."""
+    return dict(name="gqa_b4_s8192", workload=workload(4, 32, 8, 8192, 8192, 128, 128),
+                arch=arch_cloud(),
+                searches=[objective(OBJ_LATENCY, 1), objective(OBJ_EDP, 1)])
+
+
+SWEEP_SEQS = (1024, 2048, 4096, 8192, 16384, 32768, 65536)
+SWEEP_HEAD_DIMS = (64, 128)
+
+
+def config5():
+    """Sweep: single-head attention at seq 1K..64K, d in {64,128}, edge and cloud, energy."""
+    points = []
+    for arch_name, mk in (("edge", arch_edge), ("cloud", arch_cloud)):
+        for d in SWEEP_HEAD_DIMS:
+            for s in SWEEP_SEQS:
+                points.append(dict(name="sweep_%s_d%d_s%d" % (arch_name, d, s),
+                                   workload=workload(1, 1, 1, s, s, d, d), arch=mk(),
+                                   searches=[objective(OBJ_ENERGY, 1)]))
+    return points
+
+
+def all_configs():
+    return [config1(), config2(), config3(), config4()] + config5()
+
+
+# --- seeded tiny problems for exhaustive parity ----------------------------------------------
+
+def random_tiny_problem(seed: int):
+    """A small random attention shape with a random accelerator, fully determined by `seed`.
+    Dimensions are products of small primes so that divisor lists are ragged; capacities are
+    chosen so that some, but not all, candidates fit."""
+    rng = random.Random(seed)
+    pick = lambda xs: xs[rng.randrange(len(xs))]
+    seq_q = pick([4, 6, 8, 9, 12, 16, 18, 24])
+    seq_kv = pick([4, 6, 8, 10, 12, 16, 20])
+    d_qk = pick([2, 3, 4, 6, 8])
+    d_v = pick([2, 4, 5, 6, 8])
+    g = pick([1, 1, 2])
+    kv = pick([1, 2])
+    w = workload(pick([1, 2]), g * kv, kv, seq_q, seq_kv, d_qk, d_v, pick([1, 2, 4]))
+    pe = pick([2, 4, 8])
+    gb_words = pick([24, 48, 96, 200, 400, 1000])
+    quantum = pick([1.0, 0.5, 0.25])
+    a = arch(pe, pick([2, 4, 8]), pick([1, 2, 4]), gb_words * w["word_bytes"],
+             pick([0, 64]), pick([1, 2, 3, 8]),
+             quantum * rng.randrange(50, 400), quantum * rng.randrange(2, 20),
+             quantum * rng.randrange(1, 4), quantum * rng.randrange(1, 4),
+             c_softmax=float(rng.randrange(1, 12)), energy_quantum_pj=quantum)
+    o = objective(pick([OBJ_ENERGY, OBJ_LATENCY, OBJ_EDP]), pick([1, 3, 16]),
+                  pick([TILE_POW2, TILE_ALL_DIVISORS]), pick([ORD_NORECOMP2, ORD_ALL6]),
+                  pick([1, 5, 7, 7, 3, 6]))
+    return dict(name="tiny_seed%d" % seed, workload=w, arch=a, searches=[o])

@@ -1,0 +1,284 @@
+"""Pins of the CPU oracle to the paper and to mathematics (no GPU needed).
+
+Each test fixes the oracle to something that is not the oracle itself: values the paper prints for
+its worked example, an independent tile-by-tile execution of the loop nest, closed forms, counting
+arguments and brute force.
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+import mmee_inputs as mi
+import oracle
+from helpers import candidate_index, divisor_lists, exponent_vector, row_index, tiling_index
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _read_golden(name):
+    rows = []
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                rows.append(line.split())
+    return rows
+
+
+# Eight distinct primes as loop bounds: a monomial in the bounds is then identified uniquely by
+# the prime factorisation of its value.      i_D k_D l_D j_D i_G k_G l_G j_G
+PRIME_BOUNDS = (2, 3, 5, 7, 11, 13, 17, 19)
+
+
+def _prime_problem(**obj):
+    iD, kD, lD, jD, iG, kG, lG, jG = PRIME_BOUNDS
+    w = mi.workload(1, 1, 1, iD * iG, lD * lG, kD * kG, jD * jG, 1)
+    a = mi.arch(4, 4, 1, 10 ** 9, 64, 2, 200.0, 6.0, 1.0, 1.0)
+    o = mi.objective(**obj)
+    return oracle.make_problem(w, a, o)
+
+
+EXAMPLE_PI = 0                      # i2 > l2 > j2, k2 innermost
+EXAMPLE_BETA = (4, 3, 3, 3, 5)      # A at L4, E at L5, B/C/D at L3
+
+
+def test_worked_example_monomials_match_the_paper():
+    p = _prime_problem(fuse_mask=mi.FUSE_FUSED)
+    idx = candidate_index(p, PRIME_BOUNDS[4:], 0, EXAMPLE_PI, EXAMPLE_BETA)
+    r = oracle.evaluate(p, idx)
+    assert tuple(r.bound) == PRIME_BOUNDS
+    got = {"BS_A": r.bs_x[0], "DA_A": r.da_x[0], "DA_D": r.da_x[3]}
+    tau = None
+    for row in _read_golden("worked_example.txt"):
+        if row[0] == "TAU":
+            tau = [int(v) for v in row[1:]]
+        else:
+            assert exponent_vector(got[row[0]], PRIME_BOUNDS) == [int(v) for v in row[1:]], row[0]
+    # Eq. (3) with the example's tau: BS^Op1 = BS_A + BS_B + BS_C + BS_E
+    assert tau == [1, 0, 0, 0, 1]
+    assert r.bs_op1 == r.bs_x[0] + r.bs_x[1] + r.bs_x[2] + tau[3] * r.bs_x[3] + tau[4] * r.bs_x[4]
+    assert r.bs_op1 == r.bs_x[0] + r.bs_x[1] + r.bs_x[2] + r.bs_x[4]
+    # Eq. (2) second line and Eq. (5)
+    assert r.bs_op2 == r.bs_x[2] + r.bs_x[3] + r.bs_x[4] + r.bs_x[0]
+    assert r.bs == max(r.bs_op1, r.bs_op2)
+    # DA_C = 0 and DA = DA_A + DA_B + DA_D + DA_E (Section V-C)
+    assert r.da_x[2] == 0
+    assert r.n[0] == r.da_x[0] + r.da_x[1] + r.da_x[3] + r.da_x[4]
+    # "each element is fetched from DRAM exactly once" / "i_D copies of matrix D"
+    iD, kD, lD, jD, iG, kG, lG, jG = PRIME_BOUNDS
+    assert r.da_x[0] == (iD * iG) * (kD * kG)
+    assert r.da_x[3] == iD * (lD * lG) * (jD * jG)
+
+
+def test_buffer_chart_of_section_iv():
+    """Unit tiles, k_D = j_D = 2: usage goes 3 -> 4 (a1 a2 b3 c1) -> 3 over the first three stages,
+    and the peak over all stages is the buffer requirement of Eq. (2)-(5)."""
+    want = [int(v) for row in _read_golden("paper_numbers.txt") if row[0] == "buffer_chart_first_stages"
+            for v in row[1:]]
+    bound = (2, 2, 2, 2, 1, 1, 1, 1)
+    sim = oracle.simulate(bound, EXAMPLE_PI, EXAMPLE_BETA)
+    assert list(sim.trace[:3]) == want
+    assert list(sim.trace_kind[:5]) == [1, 1, 2, 3, 3]      # two producer stages, softmax, two consumer stages
+    w = mi.workload(1, 1, 1, 2, 2, 2, 2, 1)
+    p = oracle.make_problem(w, mi.arch(2, 2, 1, 10 ** 6, 0, 1, 1, 1, 0, 1), mi.objective(fuse_mask=1))
+    r = oracle.evaluate(p, candidate_index(p, (1, 1, 1, 1), 0, EXAMPLE_PI, EXAMPLE_BETA))
+    assert sim.peak == r.bs == 6
+
+
+@pytest.mark.parametrize("dims,tile", [((4, 6, 6, 4), (2, 3, 2, 2)), ((6, 4, 9, 6), (2, 2, 3, 2)),
+                                       ((8, 2, 4, 6), (2, 1, 2, 3))])
+def test_closed_forms_against_tile_level_simulation(dims, tile):
+    """Every fused row (6 orders x 5^5 levels) of one tiling whose inter-tile bounds are all >= 2 is
+    executed tile by tile.  Where consecutive stages cannot share a tile that the closed form
+    assumes refetched, both agree exactly; elsewhere the closed form is an upper bound."""
+    I, K, L, J = dims
+    p = oracle.make_problem(mi.workload(1, 1, 1, I, L, K, J, 1),
+                            mi.arch(2, 2, 1, 10 ** 9, 0, 1, 1, 1, 0, 1),
+                            mi.objective(fuse_mask=mi.FUSE_FUSED))
+    assert p.R == 18750
+    t = tiling_index(p, tile)
+    exact_rows = 0
+    for r in range(18750):
+        rec = oracle.evaluate(p, (t * p.R + r) * 9)
+        assert min(rec.bound[:4]) >= 2
+        sim = oracle.simulate(list(rec.bound), rec.pi, list(rec.beta))
+        rho = rec.bound[3] if rec.recompute else 1
+        # producer invocations: recomputation regenerates each C tile j_D times (Section III-C)
+        assert sim.c_productions == rho * rec.bound[0] * rec.bound[2]
+        assert sim.op1_stages == rho * rec.bound[0] * rec.bound[1] * rec.bound[2]
+        assert sim.op2_stages == rec.bound[0] * rec.bound[2] * rec.bound[3]
+        assert rec.n[3] == sim.op1_stages * rec.bound[4] * rec.bound[5] * rec.bound[6] \
+            + sim.op2_stages * rec.bound[4] * rec.bound[6] * rec.bound[7]
+        # producer operands and the consumer-side buffer: always exact
+        assert rec.da_x[0] == sim.loads[0] and rec.da_x[1] == sim.loads[1]
+        assert rec.bs_op2 == sim.peak_op2
+        for x in (3, 4):
+            if rec.pi in (0, 1) or rec.beta[x] >= 4:
+                assert rec.da_x[x] == sim.loads[x]
+            else:
+                assert rec.da_x[x] >= sim.loads[x]
+        if rec.pi in (0, 1):
+            assert rec.bs_op1 == sim.peak_op1
+            exact_rows += 1
+        else:
+            assert rec.bs_op1 >= sim.peak_op1
+    assert exact_rows == 6250
+
+
+def test_mac_and_softmax_counts():
+    """Section V-D: MACs = N_op1 + N_op2, or j_D N_op1 + N_op2 under recomputation; softmax work
+    c_softmax * i * l (times j_D under recomputation).  MACs do not depend on tiling, levels or
+    stationary mode inside a recomputation group."""
+    p = _prime_problem()
+    I, K, L, J = [int(v) for v in p.dim]
+    rng = np.random.default_rng(7)
+    seen = {0: 0, 1: 0}
+    for idx in rng.integers(0, p.N, size=4000):
+        r = oracle.evaluate(p, int(idx))
+        rho = r.bound[3] if r.recompute else 1
+        assert r.n[3] == rho * I * K * L + I * L * J
+        assert r.n[4] == rho * I * L
+        seen[r.recompute] += 1
+        if r.phi != 0:
+            assert r.recompute == 0
+    assert seen[0] and seen[1]
+    # energy of the softmax term: c_softmax MAC-energies per element
+    assert p.cq_sfu == 10 * p.cq_mac
+
+
+def test_dram_traffic_not_below_compulsory_and_buffer_not_below_tiles():
+    for seed in range(6):
+        cfg = mi.random_tiny_problem(seed)
+        p = oracle.make_problem(cfg["workload"], cfg["arch"], cfg["searches"][0])
+        I, K, L, J = [int(v) for v in p.dim]
+        recs = oracle.evaluate_range(p, 0, min(p.N, 60000))
+        for r in recs:
+            iG, kG, lG, jG = r.bound[4:]
+            assert r.n[0] >= I * K + K * L + L * J + I * J
+            assert r.bs_op1 >= iG * kG + kG * lG + iG * lG
+            assert r.bs_op2 >= iG * lG + lG * jG + iG * jG
+            assert r.n[1] == r.n[0] + r.br
+            assert r.feasible == (r.bs <= p.cap_words)
+
+
+def test_row_space_counts():
+    """6 orders x 5 levels for each of 5 operands = 18 750 fused rows; with the 16*13*15*13
+    factorisations of the FFN dims this is the paper's 7.6e8 mappings; recompute x stationary
+    pairs partition the rows into 18 groups."""
+    nums = {row[0]: row[1:] for row in _read_golden("paper_numbers.txt") if not row[0].startswith("table1")}
+    dims = [int(v) for v in nums["ffn_dims"]]
+    p = oracle.make_problem(mi.workload(1, 1, 1, dims[0], dims[2], dims[1], dims[3], 2),
+                            mi.arch(32, 32, 1, 2 ** 20, 0, 1, 1.0, 1.0, 0.0, 1.0),
+                            mi.objective(fuse_mask=mi.FUSE_FUSED))
+    assert p.R == 6 * 5 ** 5 == 18750
+    assert abs(p.R - float(nums["rows_per_group_unpruned_approx"][0])) / 20000 < 0.1
+    assert list(p.ndiv) == [16, 13, 15, 13]
+    mappings = p.T * p.R
+    assert mappings == 760500000
+    assert round(mappings / 1e8, 1) == float(nums["mappings_ffn_task"][0]) / 1e8
+    assert p.N == mappings * 9
+
+    q = _prime_problem(fuse_mask=mi.FUSE_FUSED)
+    groups = set()
+    for r in range(q.R):
+        for s in range(9):
+            rec = oracle.evaluate(q, r * 9 + s)
+            groups.add((rec.recompute, rec.sm[0], rec.sm[1]))
+    assert len(groups) == int(nums["groups"][0])
+
+
+def test_table1_accel1_latency_closed_form():
+    """Table I, Accel. 1, BERT-Base: 0.10 / 6.29 / 100.66 ms = 3 heads per array x 2 S^2 64 MACs on
+    1024 PEs at 1 GHz.  The oracle's latency for a mapping whose tiles fill the array is that
+    number, and no mapping is faster."""
+    for row in _read_golden("paper_numbers.txt"):
+        if row[0] != "table1_accel1_bert_latency_ms":
+            continue
+        S, ms = int(row[1]), float(row[2])
+        cycles = 3 * 2 * S * S * 64 // 1024
+        assert round(cycles / 1e6, 2) == ms
+        w = mi.workload(1, 12, 12, S, S, 64, 64, 2)
+        o = mi.objective(mi.OBJ_LATENCY, 1, mi.TILE_ALL_DIVISORS, mi.ORD_NORECOMP2, mi.FUSE_FUSED)
+        p = oracle.make_problem(w, mi.arch_accel1(), o)
+        t = tiling_index(p, (256, 64, 32, 64))
+        o.update(t_begin=max(0, t - 3), t_end=t + 3)
+        p = oracle.make_problem(w, mi.arch_accel1(), o)
+        res = oracle.search(p)
+        assert res.topk[0].latency_cycles == float(cycles)
+        keys, feas = oracle.keys_range(p, p.t_begin * p.R * 9, (p.t_end - p.t_begin) * p.R * 9)
+        assert keys.min() == cycles // 3 * 30
+
+
+def test_search_is_the_sorted_prefix_of_all_keys():
+    """argmin / top-k against a full sort of (key, idx) over every candidate of tiny problems."""
+    for seed in (1, 2, 3, 4, 5, 8):
+        cfg = mi.random_tiny_problem(seed)
+        o = dict(cfg["searches"][0], topk=16)
+        p = oracle.make_problem(cfg["workload"], cfg["arch"], o)
+        if p.N > 3_000_000:
+            o.update(t_begin=0, t_end=max(1, 3_000_000 // (p.R * 9)))
+            p = oracle.make_problem(cfg["workload"], cfg["arch"], o)
+        begin, count = p.t_begin * p.R * 9, (p.t_end - p.t_begin) * p.R * 9
+        keys, feas = oracle.keys_range(p, begin, count)
+        idx = np.arange(begin, begin + count, dtype=np.uint64)
+        keep = feas.astype(bool)
+        order = np.lexsort((idx[keep], keys[keep]))[:16]
+        want = [(int(keys[keep][i]), int(idx[keep][i])) for i in order]
+        res = oracle.search(p, threads=3)
+        key_of = {mi.OBJ_ENERGY: lambda r: r.e_key, mi.OBJ_LATENCY: lambda r: r.l_key,
+                  mi.OBJ_EDP: lambda r: int(np.float64(r.edp_key).view(np.int64))}[o["objective"]]
+        got = [(key_of(r), r.idx) for r in res.topk]
+        assert got == want
+        assert res.n_feasible == int(keep.sum()) and res.n_total == count
+        # thread count must not change the answer
+        assert [(r.idx) for r in oracle.search(p, threads=1).topk] == [g[1] for g in got]
+
+
+def test_edp_key_is_one_ieee_product():
+    p = _prime_problem(objective=mi.OBJ_EDP)
+    for idx in (0, 12345, p.N - 1):
+        r = oracle.evaluate(p, idx)
+        assert r.edp_key == float(r.e_key) * float(r.l_key)
+
+
+def test_index_layout_round_trip():
+    """idx = (t*R + r)*9 + s with t mixed-radix over ascending divisor lists (j fastest) and rows
+    ordered order-major, then levels of A, B, C, D, E."""
+    cfg = mi.config1()
+    p = oracle.make_problem(cfg["workload"], cfg["arch"], cfg["searches"][0])
+    assert (p.T, p.R, p.N) == (2401, 7500, 162067500)
+    divs = divisor_lists(p)
+    assert divs[0] == [1, 2, 4, 8, 16, 32, 64]
+    rng = np.random.default_rng(3)
+    for idx in rng.integers(0, p.N, size=300):
+        r = oracle.evaluate(p, int(idx))
+        assert candidate_index(p, tuple(r.bound[4:]), r.phi, r.pi, tuple(r.beta), tuple(r.sm)) == idx
+        assert all(r.bound[d] * r.bound[4 + d] == p.dim[d] for d in range(4))
+        assert r.phi in (0, 2) and r.pi in (0, 1)
+
+
+def test_benchmark_candidate_counts():
+    want = {"tiny_s64_d64": 162067500, "bert_base_s512": 1157625000,
+            "llama_prefill_s4096": 2555280000, "gqa_b4_s8192": 3386880000}
+    for cfg in (mi.config1(), mi.config2(), mi.config3(), mi.config4()):
+        p = oracle.make_problem(cfg["workload"], cfg["arch"], cfg["searches"][0])
+        assert p.N == want[cfg["name"]]
+    total = 0
+    for cfg in mi.config5():
+        total += oracle.make_problem(cfg["workload"], cfg["arch"], cfg["searches"][0]).N
+    assert total == 2 * 158200 * 26250 * 9
+
+
+def test_bad_inputs_are_rejected():
+    w, a = mi.workload(1, 1, 1, 8, 8, 4, 4), mi.arch_tiny()
+    with pytest.raises(oracle.OracleError):
+        oracle.make_problem(dict(w, seq_q=0), a, mi.objective())
+    with pytest.raises(oracle.OracleError):
+        oracle.make_problem(dict(w, q_heads=3, kv_heads=2), a, mi.objective())
+    with pytest.raises(oracle.OracleError):
+        oracle.make_problem(w, a, mi.objective(fuse_mask=0))
+    with pytest.raises(oracle.OracleError) as e:
+        oracle.make_problem(w, dict(a, e_gb_pj=6.3), mi.objective())
+    assert e.value.code == oracle.ERR_QUANTUM
