@@ -300,7 +300,7 @@ int mo_eval(const mo_problem* p, uint64_t idx, mo_record* o)
         }
         int tau[5];
         for (int x = 0; x < 5; ++x) tau[x] = o->beta[x] >= 4;
-        /* Eq. (2), (3), (5) */
+        /* Eq. (1), (2), (4) */
         bs1 = bs[OPD_A] + bs[OPD_B] + bs[OPD_C] + tau[OPD_D] * bs[OPD_D] + tau[OPD_E] * bs[OPD_E];
         bs2 = bs[OPD_C] + bs[OPD_D] + bs[OPD_E] + tau[OPD_A] * bs[OPD_A] + tau[OPD_B] * bs[OPD_B];
     } else {

@@ -60,7 +60,7 @@ def test_worked_example_monomials_match_the_paper():
     assert tau == [1, 0, 0, 0, 1]
     assert r.bs_op1 == r.bs_x[0] + r.bs_x[1] + r.bs_x[2] + tau[3] * r.bs_x[3] + tau[4] * r.bs_x[4]
     assert r.bs_op1 == r.bs_x[0] + r.bs_x[1] + r.bs_x[2] + r.bs_x[4]
-    # Eq. (2) second line and Eq. (5)
+    # Eq. (2) and Eq. (4)
     assert r.bs_op2 == r.bs_x[2] + r.bs_x[3] + r.bs_x[4] + r.bs_x[0]
     assert r.bs == max(r.bs_op1, r.bs_op2)
     # DA_C = 0 and DA = DA_A + DA_B + DA_D + DA_E (Section V-C)
@@ -74,7 +74,7 @@ def test_worked_example_monomials_match_the_paper():
 
 def test_buffer_chart_of_section_iv():
     """Unit tiles, k_D = j_D = 2: usage goes 3 -> 4 (a1 a2 b3 c1) -> 3 over the first three stages,
-    and the peak over all stages is the buffer requirement of Eq. (2)-(5)."""
+    and the peak over all stages is the buffer requirement of Eq. (1)-(4)."""
     want = [int(v) for row in _read_golden("paper_numbers.txt") if row[0] == "buffer_chart_first_stages"
             for v in row[1:]]
     bound = (2, 2, 2, 2, 1, 1, 1, 1)
