@@ -1,0 +1,231 @@
+/*
+ * libmmee -- exhaustive search over fused-attention dataflow mappings on one NVIDIA B200.
+ *
+ * The library evaluates the analytical buffer-size / DRAM-access / energy / latency model of
+ * "Fast Cross-Operator Optimization of Attention Dataflow" (MMEE) for EVERY mapping of a fused
+ * two-GEMM chain  C = A*B (Q*K^T), softmax, E = C*D (P*V)  onto a spatial accelerator, discards
+ * the mappings that do not fit the on-chip buffer and returns the k best under one objective.
+ * All model arithmetic runs in CUDA kernels (sm_100a); there is no CPU fallback.
+ *
+ * Plain C ABI: structs of fixed-width integers and doubles, raw pointers.  Every pointer
+ * argument says below whether it is HOST or DEVICE memory.  All functions return an int status
+ * (MMEE_OK = 0); nothing throws, aborts or traps.
+ *
+ * Candidate space (Sections III, IV, VI-A of the paper; dims I,K,L,J with I = query rows,
+ * L = key/value rows, K = J = head dims):
+ *   tiling t   : (i_G,k_G,l_G,j_G), each a divisor of its dim; x_D = X / x_G.  t is the mixed-radix
+ *                number over the ascending divisor lists, j fastest.
+ *   order pi   : order of the inter-tile loops (i2,l2,j2), outer->inner; k2 is always innermost
+ *                (constraint "No Psum Propagation", Section III-C):
+ *                0 (i,l,j) 1 (l,i,j) 2 (i,j,l) 3 (l,j,i) 4 (j,i,l) 5 (j,l,i)
+ *   levels     : beta_X in 3..7 for X in A,B,C,D,E (Section IV-A "Buffering Level");
+ *                L3 = one tile, L4 = k2, L5/L6/L7 = inner/middle/outer loop of the order
+ *   stationary : sm1, sm2 in {0 weight, 1 input, 2 output} for the two operators (Section V-D)
+ *   fusion phi : 0 fused (the paper's space), 1 unfused GEMMs with softmax in the first one's
+ *                epilogue, 2 fully unfused (separate softmax pass)
+ *   row r      : fused rows first, r = o*3125 + (bA-3)*625 + (bB-3)*125 + (bC-3)*25 + (bD-3)*5 + (bE-3)
+ *                with o the position of pi in the order set; then one block of 625 rows per order for
+ *                each unfused mode (bC = 3): o*625 + (bA-3)*125 + (bB-3)*25 + (bD-3)*5 + (bE-3)
+ *   index      : idx = (t*R + r)*9 + 3*sm1 + sm2,  R rows per tiling,  N = T*R*9 candidates
+ */
+#ifndef MMEE_H
+#define MMEE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* objective */
+#define MMEE_OBJ_ENERGY   0u   /* energy-driven search (Section VII-D)                         */
+#define MMEE_OBJ_LATENCY  1u   /* latency-driven search                                         */
+#define MMEE_OBJ_EDP      2u   /* energy-delay product (Section VII-K)                          */
+/* tiling_set */
+#define MMEE_TILE_POW2          0u   /* only power-of-two tile extents                          */
+#define MMEE_TILE_ALL_DIVISORS  1u   /* every integer factorisation (Section VI-A)              */
+/* order_set */
+#define MMEE_ORD_NORECOMP2  0u   /* orders 0 and 1 (j2 innermost: no recomputation)             */
+#define MMEE_ORD_ALL6       1u   /* all six orders (recomputation included, Section III-C)      */
+/* fuse_mask bits */
+#define MMEE_FUSE_FUSED            1u
+#define MMEE_FUSE_SOFTMAX_IN_OP1   2u
+#define MMEE_FUSE_SEPARATE         4u
+
+#define MMEE_MAX_TOPK      16u
+#define MMEE_MAX_DIVISORS  64u    /* per dimension */
+#define MMEE_NO_INDEX      UINT64_MAX
+
+/* status codes */
+#define MMEE_OK               0
+#define MMEE_ERR_ARG          1   /* NULL pointer, zero dimension, value out of range              */
+#define MMEE_ERR_OVERFLOW     2   /* a worst-case key of this problem does not fit 62 bits         */
+#define MMEE_ERR_QUANTUM      3   /* an energy is not an integer multiple of energy_quantum_pj     */
+#define MMEE_ERR_NO_FEASIBLE  4   /* no mapping fits the buffer (reported in mmee_result_t.status) */
+#define MMEE_ERR_CUDA         5   /* a CUDA runtime call failed (no device, launch error, ...)     */
+#define MMEE_ERR_TIMEOUT      6   /* reserved: the kernels contain no device-side wait             */
+#define MMEE_ERR_RANGE        7   /* request exceeds a documented maximum                          */
+
+/* Attention workload.  Heads are independent instances of one search (Section V, first
+ * paragraph); the q_heads/kv_heads query heads that share a K/V head are stacked along I. */
+typedef struct {
+    uint32_t batch, q_heads, kv_heads;       /* instances = batch*kv_heads                       */
+    uint32_t seq_q, seq_kv, d_qk, d_v;       /* I = (q_heads/kv_heads)*seq_q, L = seq_kv, K, J   */
+    uint32_t word_bytes;                     /* operand word size                                 */
+} mmee_workload_t;
+
+/* Spatial accelerator template (Section II-B): PE arrays with register files, one global
+ * buffer, DRAM.  Energies are per word moved / per MAC, in pJ. */
+typedef struct {
+    uint32_t pe_rows, pe_cols, n_arrays;
+    uint64_t gb_bytes;                       /* global buffer capacity                            */
+    uint64_t rf_bytes;                       /* per-PE register file; 0 = no register-file level  */
+    uint32_t dram_words_per_cycle;
+    double   e_dram_pj, e_gb_pj, e_rf_pj, e_mac_pj;
+    double   c_softmax;                      /* softmax cost per score element, in MAC energies   */
+    double   energy_quantum_pj;              /* every energy must be an integer multiple of this  */
+} mmee_arch_t;
+
+typedef struct {
+    uint32_t objective;                      /* MMEE_OBJ_*                                        */
+    uint32_t topk;                           /* 1..MMEE_MAX_TOPK                                  */
+    uint32_t tiling_set;                     /* MMEE_TILE_*                                       */
+    uint32_t order_set;                      /* MMEE_ORD_*                                        */
+    uint32_t fuse_mask;                      /* OR of MMEE_FUSE_*, at least one bit               */
+    uint64_t t_begin, t_end;                 /* tiling sub-range [t_begin,t_end); 0,0 = all       */
+} mmee_objective_t;
+
+/* One fully evaluated mapping.  Counts are per instance. */
+typedef struct {
+    uint64_t idx;                            /* MMEE_NO_INDEX when the slot is empty              */
+    uint64_t t;
+    uint32_t row;
+    uint32_t bound[8];                       /* i_D,k_D,l_D,j_D,i_G,k_G,l_G,j_G (Section V-E)     */
+    uint8_t  phi, pi, beta[5], sm[2], recompute, feasible, reserved[5];
+    int32_t  status;                         /* MMEE_OK or MMEE_ERR_NO_FEASIBLE                   */
+    int64_t  bs_x[5];                        /* buffer words of A,B,C,D,E (Section V-B)           */
+    int64_t  bs_op1, bs_op2, bs;             /* Eq. (1), (2), (4)                                 */
+    int64_t  da_x[5];                        /* DRAM words of A,B,C,D,E (Section V-C); C only unfused */
+    int64_t  da_sm;                          /* separate softmax pass, phi = 2                    */
+    int64_t  br, cyc1, cyc2;                 /* buffer<->PE words; compute cycles per operator    */
+    int64_t  n[5];                           /* N_DRAM, N_GB, N_RF, N_MAC, N_SFU                  */
+    int64_t  e_key;                          /* energy in quanta                                  */
+    int64_t  l_key;                          /* latency in words = cycles * dram_words_per_cycle  */
+    double   edp_key;                        /* (double)e_key * (double)l_key                     */
+    double   energy_pj;                      /* e_key * quantum * instances                       */
+    double   latency_cycles;                 /* l_key / words_per_cycle * ceil(instances/n_arrays) */
+    uint64_t n_total;                        /* candidates of the searched range (in out_best)    */
+    uint64_t n_feasible;                     /* of which fit the buffer (in out_best)             */
+} mmee_result_t;
+
+typedef struct mmee_handle mmee_handle_t;
+
+/*
+ * mmee_create -- plan one search (problem statement of Section VI-A: workload dims, accelerator,
+ * objective in; optimal mapping out).  Enumerates the tilings by integer factorisation, derives
+ * the query vectors of every (order, operand, level) (Section V-E, Section VI-A "offline"
+ * enumeration), quantises the energies and bounds the largest possible key.
+ *   workload, arch, objective : HOST, read only during the call.
+ *   out                       : HOST, receives the handle.  The handle owns a few KB of DEVICE
+ *                               scratch on the device that is current at the call.
+ * Errors: MMEE_ERR_ARG, _OVERFLOW, _QUANTUM, _RANGE (more than MMEE_MAX_DIVISORS divisors), _CUDA.
+ */
+int mmee_create(const mmee_workload_t* workload, const mmee_arch_t* arch,
+                const mmee_objective_t* objective, mmee_handle_t** out);
+
+/*
+ * mmee_search -- evaluate every mapping of the handle's range, drop those whose buffer need
+ * (Eq. 4) exceeds the global buffer, and select the k smallest (key, idx) (Section VI-A; ties
+ * broken by the lower index).  Asynchronous on `cuda_stream` (a cudaStream_t, may be 0).
+ *   out_best : DEVICE, one mmee_result_t; also carries n_total / n_feasible and, when nothing
+ *              fits, status = MMEE_ERR_NO_FEASIBLE with idx = MMEE_NO_INDEX.
+ *   out_topk : DEVICE, objective.topk entries, best first, unused slots idx = MMEE_NO_INDEX;
+ *              may be NULL.
+ * Caller owns both buffers.  Calls on one handle must not overlap on the GPU.
+ */
+int mmee_search(mmee_handle_t* handle, void* cuda_stream, mmee_result_t* out_best,
+                mmee_result_t* out_topk);
+
+int mmee_destroy(mmee_handle_t* handle);
+
+/* Number of candidates / tilings / rows of the full space of the handle (HOST values). */
+uint64_t mmee_num_candidates(const mmee_handle_t* handle);
+uint64_t mmee_num_tilings(const mmee_handle_t* handle);
+uint64_t mmee_num_rows(const mmee_handle_t* handle);
+
+const char* mmee_strerror(int status);
+
+/*
+ * mmee_eval -- evaluate `count` consecutive candidates from `idx_begin` on the device with the
+ * query-vector form of the model, exp(q . ln b) taken exactly as an integer product
+ * (Section V-E, Eq. 8), and write one full record each.
+ *   out : DEVICE, count records.  Asynchronous on the stream.
+ */
+int mmee_eval(mmee_handle_t* handle, void* cuda_stream, uint64_t idx_begin, uint64_t count,
+              mmee_result_t* out);
+
+/*
+ * mmee_dump_keys -- run the search kernel's own evaluation path over the handle's tiling range
+ * and store every candidate's objective key instead of reducing (Eq. 11: the full result matrix).
+ *   out_keys : DEVICE, (t_end - t_begin) * R * 9 int64; entry idx - t_begin*R*9.  Energy and
+ *              latency keys as integers, EDP keys as the bit pattern of the double; INT64_MAX
+ *              for a mapping that does not fit the buffer.
+ * Meant for small ranges (parity checks).  MMEE_ERR_RANGE above 2^31 candidates.
+ */
+int mmee_dump_keys(mmee_handle_t* handle, void* cuda_stream, int64_t* out_keys);
+
+/*
+ * mmee_solve_host -- whole path with HOST buffers: plan, upload, search, copy the results back,
+ * release.  Synchronous.  out_best: HOST, one record; out_topk: HOST, objective.topk records or
+ * NULL.  h2d_bytes / d2h_bytes (HOST, may be NULL) receive the bytes copied in each direction.
+ */
+int mmee_solve_host(const mmee_workload_t* workload, const mmee_arch_t* arch,
+                    const mmee_objective_t* objective, mmee_result_t* out_best,
+                    mmee_result_t* out_topk, uint64_t* h2d_bytes, uint64_t* d2h_bytes);
+
+/*
+ * mmee_query_vector -- HOST only, no device needed.  The query vector q in {0,1}^8 over
+ * b = [i_D,k_D,l_D,j_D,i_G,k_G,l_G,j_G] (Section V-E) of one metric of one operand:
+ *   metric 0 = operand buffer size BS_X (Section V-B), 1 = operand DRAM access DA_X (Section V-C).
+ *   phi, pi, operand (0..4 = A..E), beta (3..7), recompute (0/1; only read for DA of A and B).
+ * Returns MMEE_ERR_ARG for values out of range or for DA of the fused intermediate C (which is 0).
+ */
+int mmee_query_vector(uint32_t metric, uint32_t phi, uint32_t pi, uint32_t operand, uint32_t beta,
+                      uint32_t recompute, uint8_t out_q[8]);
+
+/* HOST only: whether order `pi` with C buffered at level `beta_c` regenerates C (Section III-C). */
+int mmee_recompute_flag(uint32_t pi, uint32_t beta_c, uint32_t* out_flag);
+
+/*
+ * mmee_last_search_stats -- HOST counters of the most recent mmee_search on the handle, valid
+ * after the stream has been synchronised: kernels launched by that call, persistent CTAs,
+ * threads per CTA, dynamic shared memory per CTA, tasks (groups of 225 consecutive mappings) and,
+ * when mmee_kernel_timing is on, the device time of the search kernel and of the finalize kernel
+ * in milliseconds (CUDA events recorded on the search's stream; -1 when timing is off).
+ */
+typedef struct {
+    uint32_t kernels_launched, grid, block, smem_bytes;
+    uint64_t tasks;
+    float    search_ms, finalize_ms;
+} mmee_launch_stats_t;
+int mmee_last_search_stats(const mmee_handle_t* handle, mmee_launch_stats_t* out);
+
+/* mmee_kernel_timing -- switch per-kernel CUDA-event timing of mmee_search on (1) or off (0). */
+int mmee_kernel_timing(mmee_handle_t* handle, int enable);
+
+/*
+ * mmee_alu_peak -- measure the integer instruction rates of the current device with register-only
+ * kernels (the denominators of the search kernel's roofline).  out: HOST, four doubles:
+ *   [0] 32-bit logic instructions, 10^9 per second (integer ALU pipe alone)
+ *   [1] 32-bit add + logic pairs, 10^9 instructions per second
+ *   [2] the search kernel's candidate mix -- a 64-bit add and a 64-bit signed compare, counted as
+ *       four 32-bit instructions -- 10^9 instructions per second
+ *   [3] SM clock in MHz during the measurement
+ * Synchronous; a few milliseconds; allocates and frees 4 KB of device memory.
+ */
+int mmee_alu_peak(double out[4]);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MMEE_H */

@@ -1,0 +1,49 @@
+// Internal: device scratch layout and kernel launchers (mmee_search.cu), used by the C ABI.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+
+#include "mmee_plan.h"
+
+namespace mmee {
+
+constexpr int kSearchThreads = 256;
+
+// One CTA's k best (key, idx) pairs, best first.
+struct Partial {
+    int64_t key[MMEE_MAX_TOPK];
+    uint64_t idx[MMEE_MAX_TOPK];
+    int32_t count;
+    int32_t pad;
+};
+
+// Global scratch of one handle: a work counter, the feasible-row count, the shared pruning bound
+// and one partial list per CTA.  The header is reset by the finalize kernel.
+struct Scratch {
+    unsigned long long next_task;
+    unsigned long long feasible_rows;
+    long long G;
+    long long pad;
+    Partial partial[1];     // grid entries follow
+};
+
+struct LaunchShape {
+    uint32_t grid;          // persistent CTAs
+    uint32_t range_tasks;   // tasks a CTA takes per pull (multiple of kSearchThreads)
+    uint32_t slots;         // tilings one range can touch
+    uint32_t smem_bytes;
+};
+
+inline size_t scratch_bytes(uint32_t grid) { return sizeof(Scratch) + (size_t)(grid ? grid - 1 : 0) * sizeof(Partial); }
+
+size_t search_smem_bytes(const Plan& p, uint32_t slots);
+cudaError_t search_occupancy(const Plan& p, size_t smem, int* blocks_per_sm);
+cudaError_t launch_search(const Plan& p, const LaunchShape& shape, Scratch* scratch, int64_t* dump, cudaStream_t st);
+cudaError_t launch_finalize(const Plan& p, Scratch* scratch, int n_partials, mmee_result_t* out_best,
+                            mmee_result_t* out_topk, cudaStream_t st);
+cudaError_t launch_reset(Scratch* scratch, cudaStream_t st);
+cudaError_t launch_eval(const Plan& p, uint64_t idx_begin, uint64_t count, mmee_result_t* out, cudaStream_t st);
+cudaError_t measure_alu_peak(double* giops);
+
+}  // namespace mmee
