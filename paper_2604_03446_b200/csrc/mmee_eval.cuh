@@ -1,0 +1,191 @@
+// Device-side model arithmetic shared by the kernels: exact monomials from query vectors
+// (Section V-E), array-level terms per stationary mode, and the full evaluation of one mapping.
+#pragma once
+
+#include "mmee_plan.h"
+
+namespace mmee {
+
+// exp(q . ln b) taken exactly: the product of the bounds the query vector selects (Eq. 8).
+__device__ __forceinline__ int64_t monomial(uint32_t q, const uint32_t b[8]) {
+    int64_t v = 1;
+#pragma unroll
+    for (int d = 0; d < 8; ++d)
+        if (q & (1u << d)) v *= (int64_t)b[d];
+    return v;
+}
+
+__device__ __forceinline__ int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// Compute cycles of one (m x r) * (r x n) tile on a rows x cols array.
+// 0 weight stationary: r x n weights folded onto the array, m inputs streamed per fold;
+// 1 input stationary:  m x r inputs folded, n weight columns streamed;
+// 2 output stationary: m x n outputs folded, r reduction steps streamed.
+__device__ __forceinline__ int64_t tile_cycles(int sm, int64_t m, int64_t r, int64_t n, int64_t rows, int64_t cols) {
+    if (sm == 0) return ceil_div64(r, rows) * ceil_div64(n, cols) * m;
+    if (sm == 1) return ceil_div64(m, rows) * ceil_div64(r, cols) * n;
+    return ceil_div64(m, rows) * ceil_div64(n, cols) * r;
+}
+
+// Words moved between the global buffer and the array for one tile: the stationary operand
+// once, the streamed operand once per fold of the other dimension, partial sums read and
+// written between reduction folds (2*folds - 1 transfers per output element).
+__device__ __forceinline__ int64_t tile_traffic(int sm, int64_t m, int64_t r, int64_t n, int64_t rows, int64_t cols) {
+    if (sm == 0) return r * n + m * r * ceil_div64(n, cols) + m * n * (2 * ceil_div64(r, rows) - 1);
+    if (sm == 1) return m * r + r * n * ceil_div64(m, rows) + m * n * (2 * ceil_div64(r, cols) - 1);
+    return m * r * ceil_div64(n, cols) + r * n * ceil_div64(m, rows) + m * n;
+}
+
+// Everything about one tiling that does not depend on order or levels.
+struct TilingTerms {
+    int64_t br1[3], br2[3];     // per-tile buffer<->PE words by stationary mode
+    int64_t cy1[3], cy2[3];     // per-tile cycles by stationary mode
+    int64_t t1, t2;             // tile invocations of Op1 (without recomputation) and Op2
+    int64_t carry1, carry2;     // partial sums carried between reduction steps (rho = 1)
+    int64_t ikl, ilj, il;       // I*K*L, I*L*J, I*L
+};
+
+__device__ __forceinline__ void tiling_terms(const Plan& p, const uint32_t b[8], TilingTerms& tt) {
+    const int64_t iD = b[0], kD = b[1], lD = b[2], jD = b[3], iG = b[4], kG = b[5], lG = b[6], jG = b[7];
+#pragma unroll
+    for (int sm = 0; sm < 3; ++sm) {
+        tt.br1[sm] = tile_traffic(sm, iG, kG, lG, p.pe_rows, p.pe_cols);
+        tt.br2[sm] = tile_traffic(sm, iG, lG, jG, p.pe_rows, p.pe_cols);
+        tt.cy1[sm] = tile_cycles(sm, iG, kG, lG, p.pe_rows, p.pe_cols);
+        tt.cy2[sm] = tile_cycles(sm, iG, lG, jG, p.pe_rows, p.pe_cols);
+    }
+    tt.t1 = iD * kD * lD;
+    tt.t2 = iD * lD * jD;
+    tt.carry1 = (tt.t1 - tt.t1 / kD) * iG * lG;
+    tt.carry2 = (tt.t2 - tt.t2 / lD) * iG * jG;
+    tt.ikl = (int64_t)p.dim[0] * p.dim[1] * p.dim[2];
+    tt.ilj = (int64_t)p.dim[0] * p.dim[2] * p.dim[3];
+    tt.il = (int64_t)p.dim[0] * p.dim[2];
+}
+
+// Tiling index -> boundary vector b (one column of the boundary matrix, Section VI-A).
+__device__ __forceinline__ void tiling_bounds(const Plan& p, uint64_t t, uint32_t b[8]) {
+#pragma unroll
+    for (int d = 3; d >= 0; --d) {
+        const uint32_t a = (uint32_t)(t % p.ndiv[d]);
+        t /= p.ndiv[d];
+        const uint32_t g = p.divs[d][a];
+        b[4 + d] = g;
+        b[d] = p.dim[d] / g;
+    }
+}
+
+// Task index inside a tiling -> (block, levels of A, B, C).  Rows of a task: levels of D, E.
+struct TaskChoice {
+    uint32_t block, phi, order_slot, order;
+    uint32_t la, lb, lc;        // beta - 3
+};
+
+__device__ __forceinline__ TaskChoice decode_task(const Plan& p, uint32_t w) {
+    TaskChoice c;
+    if (w < p.fused_tasks) {
+        c.block = w / 125u;
+        const uint32_t rem = w - c.block * 125u;
+        c.la = rem / 25u;
+        c.lb = (rem / 5u) % 5u;
+        c.lc = rem % 5u;
+    } else {
+        const uint32_t u = w - p.fused_tasks;
+        c.block = p.n_fused_blocks + u / 25u;
+        const uint32_t rem = u % 25u;
+        c.la = rem / 5u;
+        c.lb = rem % 5u;
+        c.lc = 0;
+    }
+    c.phi = p.block_phi[c.block];
+    c.order_slot = p.block_order_slot[c.block];
+    c.order = p.order_id[c.order_slot];
+    return c;
+}
+
+// Full evaluation of one mapping: all five metric groups of Section VI-A (buffer sizes of
+// producer and consumer, DRAM access, compute latency of both operators, buffer<->register
+// traffic), then energy and latency (Section V-D).
+__device__ inline void evaluate_candidate(const Plan& p, uint64_t idx, mmee_result_t& o) {
+    const uint64_t per_t = (uint64_t)p.rows_per_tiling * 9u;
+    const uint64_t t = idx / per_t;
+    const uint32_t rem = (uint32_t)(idx - t * per_t);
+    const uint32_t row = rem / 9u, s = rem % 9u;
+    const uint32_t w = row / 25u, de = row % 25u;
+    const TaskChoice c = decode_task(p, w);
+    const uint32_t lv[5] = {c.la, c.lb, c.lc, de / 5u, de % 5u};
+    const int sm1 = (int)(s / 3u), sm2 = (int)(s % 3u);
+
+    uint32_t b[8];
+    tiling_bounds(p, t, b);
+    TilingTerms tt;
+    tiling_terms(p, b, tt);
+
+    o.idx = idx; o.t = t; o.row = row;
+    for (int d = 0; d < 8; ++d) o.bound[d] = b[d];
+    o.phi = (uint8_t)c.phi; o.pi = (uint8_t)c.order;
+    for (int x = 0; x < 5; ++x) o.beta[x] = (uint8_t)(lv[x] + 3);
+    o.sm[0] = (uint8_t)sm1; o.sm[1] = (uint8_t)sm2;
+    for (int i = 0; i < 5; ++i) o.reserved[i] = 0;
+    o.status = MMEE_OK;
+
+    const QueryTables& q = p.q;
+    const bool fused = c.phi == 0;
+    const uint32_t rc = fused ? q.recompute[c.order][c.lc] : 0u;
+    const int64_t rho = rc ? (int64_t)b[3] : 1;
+
+    int64_t bs[5], da[5];
+    for (int x = 0; x < 5; ++x) {
+        bs[x] = monomial(q.bs[c.order][x][lv[x]], b);
+        if (fused) da[x] = (x == OP_C) ? 0 : monomial(q.da[c.order][x][lv[x]][rc], b);
+        else da[x] = monomial(q.da_unfused[c.order][x][lv[x]], b);
+    }
+    int64_t bs1, bs2, da_sm = 0, da1 = 0, da2 = 0;
+    if (fused) {
+        // Eq. (1)/(2): operands of the other operator count only when retained (tau = 1).
+        bs1 = bs[OP_A] + bs[OP_B] + bs[OP_C] + (lv[OP_D] ? bs[OP_D] : 0) + (lv[OP_E] ? bs[OP_E] : 0);
+        bs2 = bs[OP_C] + bs[OP_D] + bs[OP_E] + (lv[OP_A] ? bs[OP_A] : 0) + (lv[OP_B] ? bs[OP_B] : 0);
+    } else {
+        bs1 = bs[OP_A] + bs[OP_B] + bs[OP_C];
+        bs2 = bs[OP_C] + bs[OP_D] + bs[OP_E];
+        const int64_t c_write = tt.il;                 // Op1 stores C, Op2 reads it back
+        da1 = da[OP_A] + da[OP_B] + c_write;
+        da2 = da[OP_C] + da[OP_D] + da[OP_E];
+        da[OP_C] += c_write;
+        if (c.phi == 2) da_sm = 2 * tt.il;             // separate softmax pass: read S, write P
+    }
+    const int64_t n_dram = da[0] + da[1] + da[2] + da[3] + da[4] + da_sm;
+    const int64_t n_mac = rho * tt.ikl + tt.ilj;
+    const int64_t n_sfu = rho * tt.il;
+    const int64_t t1 = rho * tt.t1;
+    const int64_t br = t1 * tt.br1[sm1] + rho * tt.carry1 + tt.t2 * tt.br2[sm2] + tt.carry2;
+    const int64_t cyc1 = t1 * tt.cy1[sm1], cyc2 = tt.t2 * tt.cy2[sm2];
+    const int64_t n_gb = n_dram + br;
+    const int64_t n_rf = p.has_rf ? br + 3 * n_mac : 0;
+
+    const int64_t e_key = p.cq[0] * n_dram + p.cq[1] * n_gb + p.cq[2] * n_rf + p.cq[3] * n_mac + p.cq[4] * n_sfu;
+    int64_t l_key;
+    if (fused) {
+        const int64_t comp = (cyc1 + cyc2) * (int64_t)p.bw;
+        l_key = n_dram > comp ? n_dram : comp;
+    } else {
+        const int64_t c1 = cyc1 * (int64_t)p.bw, c2 = cyc2 * (int64_t)p.bw;
+        l_key = (da1 > c1 ? da1 : c1) + da_sm + (da2 > c2 ? da2 : c2);
+    }
+
+    for (int x = 0; x < 5; ++x) { o.bs_x[x] = bs[x]; o.da_x[x] = da[x]; }
+    o.bs_op1 = bs1; o.bs_op2 = bs2; o.bs = bs1 > bs2 ? bs1 : bs2;
+    o.da_sm = da_sm;
+    o.br = br; o.cyc1 = cyc1; o.cyc2 = cyc2;
+    o.n[0] = n_dram; o.n[1] = n_gb; o.n[2] = n_rf; o.n[3] = n_mac; o.n[4] = n_sfu;
+    o.e_key = e_key; o.l_key = l_key;
+    o.recompute = (uint8_t)rc;
+    o.feasible = (uint8_t)(o.bs <= p.cap_words);
+    o.edp_key = __dmul_rn((double)e_key, (double)l_key);
+    o.energy_pj = __dmul_rn(__dmul_rn((double)e_key, p.quantum_pj), (double)p.instances);
+    const uint32_t waves = (p.instances + p.n_arrays - 1) / p.n_arrays;
+    o.latency_cycles = __dmul_rn(__ddiv_rn((double)l_key, (double)p.bw), (double)waves);
+    o.n_total = 0; o.n_feasible = 0;
+}
+
+}  // namespace mmee

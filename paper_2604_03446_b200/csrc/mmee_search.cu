@@ -1,0 +1,562 @@
+// The search kernels: exhaustive evaluation of every mapping, capacity pruning, top-k.
+//
+// Work decomposition.  A "task" is one (tiling, fusion mode, order, levels of A, B, C) choice; its
+// 25 rows are the levels of D and E and each row has 9 stationary pairs, so a task is 225
+// consecutive candidate indices: idx = task*225 + row*9 + s.  One thread owns one task at a time
+// and walks it in ascending index order, entirely in registers.
+//
+// The cost of a mapping is separable over operands (Section V-B/V-C: BS and DA are sums of
+// per-operand monomials; Section V-D: energy is linear in the access counts), so the query-matrix
+// product exp(Q . ln B) (Eq. 11) is evaluated once per (tiling, order, operand, level) into small
+// shared-memory tables -- each entry an exact integer monomial already multiplied by its energy
+// coefficient -- and a candidate's key is a handful of adds of table entries.  Nothing per
+// candidate ever touches global memory.
+//
+// CTAs are persistent and pull ranges of tasks from a global counter; per range they rebuild the
+// tables of the (at most a few) tilings the range touches.
+#include <cuda_runtime.h>
+
+#include "mmee_eval.cuh"
+#include "mmee_search.h"
+
+namespace mmee {
+
+namespace {
+
+constexpr unsigned kFull = 0xffffffffu;
+
+// ------------------------------------------------------------------------------------------------
+// shared-memory tables
+// ------------------------------------------------------------------------------------------------
+
+// Per (tiling, order): operand terms by level.  "g" entries are DRAM words times the objective's
+// scale (energy: quanta per DRAM word; latency/EDP: 1); "e" entries (EDP only) are the
+// energy-scaled copies.
+struct OrderTab {
+    int64_t A1[5], gA[5][2], B1[5], gB[5][2], C1[5];
+    int64_t D2[5], gD[5], gDu[5], E2[5], gE[5], gEu[5];
+    int64_t gCr;
+    int64_t eA[5][2], eB[5][2], eD[5], eDu[5], eE[5], eEu[5], eCr;
+    uint32_t rc[5];
+    uint32_t pad;
+};
+constexpr int kOrderEntries = 66;
+
+// Per tiling: array-level terms by stationary pair and recompute flag.
+struct TilingTab {
+    uint32_t b[8];
+    int64_t W[9][2];        // energy of buffer<->PE traffic, MACs and softmax, in quanta
+    int64_t CB[9][2];       // fused compute time in words (cycles * words per cycle)
+    int64_t QU[9][2];       // unfused Op2 compute time in words, by s (sm2 = s % 3)
+    int64_t C1w[3];         // unfused Op1 compute time in words, by sm1
+    int64_t cw, smx;        // C write-back words (I*L); separate softmax pass words (2*I*L)
+    int32_t live;           // smallest possible buffer need of this tiling fits
+    int32_t pad;
+};
+
+struct WarpTop {
+    int64_t key[MMEE_MAX_TOPK];
+    uint64_t idx[MMEE_MAX_TOPK];
+    int32_t count;
+    int32_t pad;
+};
+
+struct CtaShared {
+    long long G;             // upper bound on the final k-th smallest key (any full list's last key)
+    unsigned long long feasible_rows;
+    unsigned long long range_begin;
+};
+
+__device__ __forceinline__ bool pair_less(int64_t ka, uint64_t ia, int64_t kb, uint64_t ib) {
+    return ka < kb || (ka == kb && ia < ib);
+}
+
+// All 32 lanes call this converged.  Lane j holds list entry j.
+__device__ __forceinline__ bool warp_insert(WarpTop* wt, int k, int64_t nk, uint64_t ni, int lane) {
+    const int count = wt->count;
+    const bool have = lane < count;
+    const int64_t ek = have ? wt->key[lane] : kInfKey;
+    const uint64_t ei = have ? wt->idx[lane] : UINT64_MAX;
+    const unsigned smaller = __ballot_sync(kFull, have && pair_less(ek, ei, nk, ni));
+    const int pos = __popc(smaller);
+    if (pos >= k) return false;
+    __syncwarp();
+    if (have && lane >= pos && lane + 1 < k) { wt->key[lane + 1] = ek; wt->idx[lane + 1] = ei; }
+    if (lane == pos) { wt->key[pos] = nk; wt->idx[pos] = ni; }
+    if (lane == 0 && count < k) wt->count = count + 1;
+    __syncwarp();
+    return true;
+}
+
+// Threshold a lane compares keys against while it walks one task in ascending index order:
+// a key passes iff it can still enter the warp's list and is not above the CTA-wide bound G.
+// Strict against the list's last key when every index of the task lies above that entry's index.
+__device__ __forceinline__ int64_t lane_threshold(const WarpTop* wt, const CtaShared* cs, int k, uint64_t task_first_idx) {
+    int64_t thr = cs->G + 1;                       // G <= INT64_MAX - 1 always
+    if (wt->count == k) {
+        const int64_t tk = wt->key[k - 1];
+        const int64_t loc = (task_first_idx > wt->idx[k - 1]) ? tk : tk + 1;
+        thr = loc < thr ? loc : thr;
+    }
+    return thr;
+}
+
+__device__ __forceinline__ int64_t dbits(double v) { return __double_as_longlong(v); }
+
+template <int OBJ>
+__device__ __forceinline__ int64_t candidate_key(int64_t x, int64_t xe, int64_t w, int64_t p, int64_t q) {
+    if constexpr (OBJ == MMEE_OBJ_ENERGY) {
+        return x + w;
+    } else if constexpr (OBJ == MMEE_OBJ_LATENCY) {
+        return p + (x > q ? x : q);
+    } else {
+        const int64_t e = xe + w;
+        const int64_t l = p + (x > q ? x : q);
+        return dbits(__dmul_rn((double)e, (double)l));
+    }
+}
+
+// Rare path: some lane of the warp has a key below its threshold in this row.  Every lane
+// re-evaluates its nine candidates of the row from the shared tables and the warp inserts the
+// passing ones, one at a time, into its sorted list.
+template <int OBJ>
+__device__ __noinline__ int64_t slow_row(WarpTop* wt, CtaShared* cs, int k, int lane, bool f,
+                                         int64_t x, int64_t xe, const int64_t* wptr, const int64_t* qptr,
+                                         int64_t p0, int64_t p1, int64_t p2,
+                                         uint64_t row_first_idx, uint64_t task_first_idx) {
+    int64_t thr = lane_threshold(wt, cs, k, task_first_idx);
+    for (int s = 0; s < 9; ++s) {
+        const int64_t pp = s < 3 ? p0 : (s < 6 ? p1 : p2);
+        const int64_t key = candidate_key<OBJ>(x, xe, wptr[2 * s], pp, qptr[2 * s]);
+        bool pend = f && key < thr;
+        while (true) {
+            const unsigned m = __ballot_sync(kFull, pend);
+            if (!m) break;
+            const int leader = __ffs(m) - 1;
+            const int64_t lk = __shfl_sync(kFull, key, leader);
+            const uint64_t li = __shfl_sync(kFull, row_first_idx + (uint64_t)s, leader);
+            warp_insert(wt, k, lk, li, lane);
+            thr = lane_threshold(wt, cs, k, task_first_idx);
+            pend = (lane == leader) ? false : (pend && key < thr);
+        }
+    }
+    if (lane == 0 && wt->count == k) {
+        const long long last = wt->key[k - 1];
+        if (last < cs->G) atomicMin(&cs->G, last);
+    }
+    __syncwarp();
+    return lane_threshold(wt, cs, k, task_first_idx);
+}
+
+// ------------------------------------------------------------------------------------------------
+// table construction
+// ------------------------------------------------------------------------------------------------
+
+template <int OBJ>
+__device__ __forceinline__ void build_order_entry(const Plan& p, const uint32_t* b, uint32_t order, OrderTab* ot, int e) {
+    const QueryTables& q = p.q;
+    const int64_t scale = (OBJ == MMEE_OBJ_ENERGY) ? p.c_dram_gb : 1;
+    const int64_t escale = p.c_dram_gb;
+    if (e < 5) {
+        ot->A1[e] = monomial(q.bs[order][OP_A][e], b);
+    } else if (e < 15) {
+        const int l = (e - 5) >> 1, rc = (e - 5) & 1;
+        const int64_t v = monomial(q.da[order][OP_A][l][rc], b);
+        ot->gA[l][rc] = scale * v;
+        if (OBJ == MMEE_OBJ_EDP) ot->eA[l][rc] = escale * v;
+    } else if (e < 20) {
+        ot->B1[e - 15] = monomial(q.bs[order][OP_B][e - 15], b);
+    } else if (e < 30) {
+        const int l = (e - 20) >> 1, rc = (e - 20) & 1;
+        const int64_t v = monomial(q.da[order][OP_B][l][rc], b);
+        ot->gB[l][rc] = scale * v;
+        if (OBJ == MMEE_OBJ_EDP) ot->eB[l][rc] = escale * v;
+    } else if (e < 35) {
+        ot->C1[e - 30] = monomial(q.bs[order][OP_C][e - 30], b);
+        ot->rc[e - 30] = q.recompute[order][e - 30];
+    } else if (e < 40) {
+        ot->D2[e - 35] = monomial(q.bs[order][OP_D][e - 35], b);
+    } else if (e < 45) {
+        const int64_t v = monomial(q.da[order][OP_D][e - 40][0], b);
+        ot->gD[e - 40] = scale * v;
+        if (OBJ == MMEE_OBJ_EDP) ot->eD[e - 40] = escale * v;
+    } else if (e < 50) {
+        const int64_t v = monomial(q.da_unfused[order][OP_D][e - 45], b);
+        ot->gDu[e - 45] = scale * v;
+        if (OBJ == MMEE_OBJ_EDP) ot->eDu[e - 45] = escale * v;
+    } else if (e < 55) {
+        ot->E2[e - 50] = monomial(q.bs[order][OP_E][e - 50], b);
+    } else if (e < 60) {
+        const int64_t v = monomial(q.da[order][OP_E][e - 55][0], b);
+        ot->gE[e - 55] = scale * v;
+        if (OBJ == MMEE_OBJ_EDP) ot->eE[e - 55] = escale * v;
+    } else if (e < 65) {
+        const int64_t v = monomial(q.da_unfused[order][OP_E][e - 60], b);
+        ot->gEu[e - 60] = scale * v;
+        if (OBJ == MMEE_OBJ_EDP) ot->eEu[e - 60] = escale * v;
+    } else {
+        const int64_t v = monomial(q.da_unfused[order][OP_C][0], b);
+        ot->gCr = scale * v;
+        if (OBJ == MMEE_OBJ_EDP) ot->eCr = escale * v;
+    }
+}
+
+// One thread per tiling slot: bounds, array-level terms, liveness.
+__device__ __forceinline__ void build_tiling_tab(const Plan& p, uint64_t t, TilingTab* tb) {
+    uint32_t b[8];
+    tiling_bounds(p, t, b);
+    TilingTerms tt;
+    tiling_terms(p, b, tt);
+#pragma unroll
+    for (int d = 0; d < 8; ++d) tb->b[d] = b[d];
+    const int64_t bw = p.bw;
+    for (int s = 0; s < 9; ++s) {
+        const int sm1 = s / 3, sm2 = s % 3;
+        for (int rc = 0; rc < 2; ++rc) {
+            const int64_t rho = rc ? (int64_t)b[3] : 1;
+            const int64_t t1 = rho * tt.t1;
+            const int64_t br = t1 * tt.br1[sm1] + rho * tt.carry1 + tt.t2 * tt.br2[sm2] + tt.carry2;
+            const int64_t n_mac = rho * tt.ikl + tt.ilj;
+            const int64_t n_sfu = rho * tt.il;
+            tb->W[s][rc] = p.c_br * br + p.c_mac * n_mac + p.c_sfu * n_sfu;
+            tb->CB[s][rc] = (t1 * tt.cy1[sm1] + tt.t2 * tt.cy2[sm2]) * bw;
+            tb->QU[s][rc] = tt.t2 * tt.cy2[sm2] * bw;
+        }
+    }
+    for (int sm1 = 0; sm1 < 3; ++sm1) tb->C1w[sm1] = tt.t1 * tt.cy1[sm1] * bw;
+    tb->cw = tt.il;
+    tb->smx = 2 * tt.il;
+    // With every operand at L3 the buffer need is smallest: max(A+B+C, C+D+E) tiles (Eq. 1-4).
+    const int64_t ta = (int64_t)b[4] * b[5], tbb = (int64_t)b[5] * b[6], tc = (int64_t)b[4] * b[6];
+    const int64_t td = (int64_t)b[6] * b[7], te = (int64_t)b[4] * b[7];
+    const int64_t need1 = ta + tbb + tc, need2 = tc + td + te;
+    tb->live = ((need1 > need2 ? need1 : need2) <= p.cap_words) ? 1 : 0;
+    tb->pad = 0;
+}
+
+// ------------------------------------------------------------------------------------------------
+// the search kernel
+// ------------------------------------------------------------------------------------------------
+
+template <int OBJ, bool DUMP>
+__global__ void __launch_bounds__(kSearchThreads, 2)
+search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* __restrict__ scratch,
+              int64_t* __restrict__ dump) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    CtaShared* cs = reinterpret_cast<CtaShared*>(smem_raw);
+    WarpTop* wtops = reinterpret_cast<WarpTop*>(smem_raw + sizeof(CtaShared));
+    TilingTab* ttabs = reinterpret_cast<TilingTab*>(wtops + kSearchThreads / 32);
+    OrderTab* otabs = reinterpret_cast<OrderTab*>(ttabs + shape.slots);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int k = (int)p.topk;
+    WarpTop* wt = &wtops[warp];
+
+    if (tid == 0) {
+        cs->G = scratch->G;
+        cs->feasible_rows = 0;
+    }
+    if (lane == 0) wt->count = 0;
+    __syncthreads();
+
+    const uint32_t tpt = p.tasks_per_tiling;
+    const uint64_t task_begin = p.t_begin * tpt, task_end = p.t_end * tpt;
+    const uint64_t dump_origin = task_begin * kCandPerTask;
+    const int64_t cap = p.cap_words;
+    const uint32_t n_orders = p.n_orders;
+    unsigned long long my_rows = 0;
+
+    while (true) {
+        if (tid == 0) {
+            const unsigned long long got = atomicAdd(&scratch->next_task, (unsigned long long)shape.range_tasks);
+            cs->range_begin = task_begin + got;
+            // exchange the pruning bound with the other CTAs
+            const long long mine = cs->G;
+            const long long theirs = atomicMin(&scratch->G, mine);
+            if (theirs < mine) atomicMin(&cs->G, theirs);
+        }
+        __syncthreads();
+        const uint64_t r0 = cs->range_begin;
+        if (r0 >= task_end) break;
+        const uint64_t r1 = (r0 + shape.range_tasks < task_end) ? r0 + shape.range_tasks : task_end;
+        const uint64_t t_first = r0 / tpt, t_last = (r1 - 1) / tpt;
+        const uint32_t n_slots = (uint32_t)(t_last - t_first + 1);
+
+        // ---- tables of the tilings this range touches
+        if (tid < (int)n_slots) build_tiling_tab(p, t_first + tid, &ttabs[tid]);
+        __syncthreads();
+        const uint32_t items = n_slots * n_orders * kOrderEntries;
+        for (uint32_t it = tid; it < items; it += kSearchThreads) {
+            const uint32_t e = it % kOrderEntries;
+            const uint32_t so = it / kOrderEntries;
+            const uint32_t slot = so / n_orders, os = so % n_orders;
+            if (!ttabs[slot].live) continue;
+            build_order_entry<OBJ>(p, ttabs[slot].b, p.order_id[os], &otabs[slot * n_orders + os], (int)e);
+        }
+        __syncthreads();
+
+        // ---- tasks
+        for (uint64_t base = r0; base < r1; base += kSearchThreads) {
+            const uint64_t task = base + tid;
+            const bool valid = task < r1;
+            const uint64_t tq = valid ? task : r1 - 1;
+            const uint64_t t = tq / tpt;
+            const uint32_t w = (uint32_t)(tq - t * tpt);
+            const uint32_t slot = (uint32_t)(t - t_first);
+            const TilingTab* tb = &ttabs[slot];
+            const bool live = valid && tb->live;
+            if (DUMP && valid && !tb->live) {
+                for (int c = 0; c < kCandPerTask; ++c) dump[task * kCandPerTask - dump_origin + c] = kInfKey;
+            }
+            if (!__any_sync(kFull, live)) continue;
+
+            const TaskChoice c = decode_task(p, w);
+            const OrderTab* ot = &otabs[slot * n_orders + c.order_slot];
+            const bool fused = c.phi == 0;
+            const uint32_t rc = fused ? ot->rc[c.lc] : 0u;
+            const int64_t a1 = ot->A1[c.la], b1 = ot->B1[c.lb], c1 = ot->C1[c.lc];
+            // Eq. (1)/(2): a retained operand (level >= L4) of the other operator keeps its space.
+            const int64_t slack1 = cap - (a1 + b1 + c1);
+            const int64_t slack2 = cap - (c1 + ((fused && c.la) ? a1 : 0) + ((fused && c.lb) ? b1 : 0));
+            const int64_t gab = ot->gA[c.la][rc] + ot->gB[c.lb][rc];
+
+            int64_t x0, xe0 = 0, P[3], Q[9], W[9];
+            const int64_t* wptr = &tb->W[0][rc];
+            const int64_t* qptr;
+            if constexpr (OBJ == MMEE_OBJ_ENERGY) {
+                const int64_t extra = p.c_dram_gb * (tb->cw + (c.phi == 2 ? tb->smx : 0));
+                x0 = fused ? gab : gab + ot->gCr + extra;
+                P[0] = P[1] = P[2] = 0;
+                qptr = wptr;
+            } else {
+                const int64_t pass = (c.phi == 2) ? tb->smx : 0;
+                if (fused) {
+                    x0 = gab;
+                    P[0] = P[1] = P[2] = 0;
+                    qptr = &tb->CB[0][rc];
+                } else {
+                    // unfused latency: max(DA1, C1) + softmax pass + max(DA2, C2)
+                    x0 = ot->gCr;
+                    const int64_t da1 = gab + tb->cw;
+#pragma unroll
+                    for (int m = 0; m < 3; ++m) P[m] = (da1 > tb->C1w[m] ? da1 : tb->C1w[m]) + pass;
+                    qptr = &tb->QU[0][0];
+                }
+                if constexpr (OBJ == MMEE_OBJ_EDP) {
+                    const int64_t eab = ot->eA[c.la][rc] + ot->eB[c.lb][rc];
+                    xe0 = fused ? eab : eab + ot->eCr + p.c_dram_gb * (tb->cw + pass);
+                }
+            }
+#pragma unroll
+            for (int s = 0; s < 9; ++s) {
+                W[s] = wptr[2 * s];
+                Q[s] = qptr[2 * s];
+            }
+            int64_t E1[5], E2[5], gE[5], eE[5];
+#pragma unroll
+            for (int e = 0; e < 5; ++e) {
+                E2[e] = ot->E2[e];
+                E1[e] = (fused && e) ? E2[e] : 0;
+                gE[e] = fused ? ot->gE[e] : ot->gEu[e];
+                eE[e] = (OBJ == MMEE_OBJ_EDP) ? (fused ? ot->eE[e] : ot->eEu[e]) : 0;
+            }
+            const uint64_t task_first_idx = tq * kCandPerTask;
+            int64_t thr = lane_threshold(wt, cs, k, task_first_idx);
+            uint32_t rows = 0;
+
+#pragma unroll 1
+            for (int d = 0; d < 5; ++d) {
+                const int64_t d2 = ot->D2[d];
+                const int64_t s1 = slack1 - ((fused && d) ? d2 : 0);
+                const int64_t s2 = slack2 - d2;
+                const int64_t xd = x0 + (fused ? ot->gD[d] : ot->gDu[d]);
+                const int64_t xed = (OBJ == MMEE_OBJ_EDP) ? xe0 + (fused ? ot->eD[d] : ot->eDu[d]) : 0;
+#pragma unroll
+                for (int e = 0; e < 5; ++e) {
+                    const bool f = live && (E1[e] <= s1) && (E2[e] <= s2);     // Eq. (4) against the capacity
+                    rows += f ? 1u : 0u;
+                    const int64_t x = xd + gE[e];
+                    const int64_t xe = xed + eE[e];
+                    bool any = false;
+#pragma unroll
+                    for (int s = 0; s < 9; ++s) {
+                        const int64_t key = candidate_key<OBJ>(x, xe, W[s], P[s / 3], Q[s]);
+                        any |= key < thr;
+                        if (DUMP) {
+                            if (valid) dump[task_first_idx - dump_origin + (d * 5 + e) * 9 + s] = f ? key : kInfKey;
+                        }
+                    }
+                    any &= f;
+                    if (__any_sync(kFull, any)) {
+                        thr = slow_row<OBJ>(wt, cs, k, lane, f, x, xe, wptr, qptr, P[0], P[1], P[2],
+                                            task_first_idx + (uint64_t)((d * 5 + e) * 9), task_first_idx);
+                    }
+                }
+            }
+            my_rows += rows;
+        }
+        __syncthreads();      // tables are rebuilt at the top of the next range
+    }
+
+    // ---- feasible count
+    for (int off = 16; off; off >>= 1) my_rows += __shfl_down_sync(kFull, my_rows, off);
+    if (lane == 0 && my_rows) atomicAdd(&cs->feasible_rows, my_rows);
+    __syncthreads();
+
+    // ---- merge the warps' lists into warp 0's, then publish this CTA's partial list
+    if (warp == 0) {
+        for (int w2 = 1; w2 < kSearchThreads / 32; ++w2) {
+            const WarpTop* src = &wtops[w2];
+            const int n = src->count;
+            for (int j = 0; j < n; ++j)
+                if (!warp_insert(wt, k, src->key[j], src->idx[j], lane)) break;   // sorted: the rest is larger
+        }
+        Partial* out = &scratch->partial[blockIdx.x];
+        const int n = wt->count;
+        if (lane < n) { out->key[lane] = wt->key[lane]; out->idx[lane] = wt->idx[lane]; }
+        if (lane == 0) {
+            out->count = n;
+            if (cs->feasible_rows) atomicAdd(&scratch->feasible_rows, cs->feasible_rows);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// finalize: merge the CTAs' partial lists, evaluate the winners in full, reset the scratch header
+// ------------------------------------------------------------------------------------------------
+
+__global__ void __launch_bounds__(1024, 1)
+finalize_kernel(const __grid_constant__ Plan p, Scratch* __restrict__ scratch, int n_partials,
+                mmee_result_t* __restrict__ out_best, mmee_result_t* __restrict__ out_topk) {
+    __shared__ WarpTop tops[32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int k = (int)p.topk;
+    WarpTop* wt = &tops[warp];
+    if (lane == 0) wt->count = 0;
+    __syncwarp();
+    for (int c = warp; c < n_partials; c += 32) {
+        const Partial* src = &scratch->partial[c];
+        const int n = src->count;
+        for (int j = 0; j < n; ++j)
+            if (!warp_insert(wt, k, src->key[j], src->idx[j], lane)) break;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        for (int w2 = 1; w2 < 32; ++w2) {
+            const WarpTop* src = &tops[w2];
+            const int n = src->count;
+            for (int j = 0; j < n; ++j)
+                if (!warp_insert(wt, k, src->key[j], src->idx[j], lane)) break;
+        }
+        const int found = wt->count;
+        const uint64_t n_total = (p.t_end - p.t_begin) * (uint64_t)p.rows_per_tiling * 9u;
+        const uint64_t n_feasible = scratch->feasible_rows * 9ull;
+        if (lane < k) {
+            mmee_result_t r;
+            if (lane < found) {
+                evaluate_candidate(p, wt->idx[lane], r);
+            } else {
+                // empty slot
+                unsigned char* raw = reinterpret_cast<unsigned char*>(&r);
+                for (unsigned i = 0; i < sizeof(r); ++i) raw[i] = 0;
+                r.idx = MMEE_NO_INDEX;
+                r.status = found ? MMEE_OK : MMEE_ERR_NO_FEASIBLE;
+            }
+            if (out_topk) out_topk[lane] = r;
+            if (lane == 0) {
+                r.n_total = n_total;
+                r.n_feasible = n_feasible;
+                *out_best = r;
+            }
+        }
+        __syncwarp();
+        if (lane == 0) {         // ready for the next search on this handle
+            scratch->next_task = 0;
+            scratch->feasible_rows = 0;
+            scratch->G = kInfKey - 1;
+        }
+    }
+}
+
+__global__ void reset_kernel(Scratch* scratch) {
+    scratch->next_task = 0;
+    scratch->feasible_rows = 0;
+    scratch->G = kInfKey - 1;
+}
+
+__global__ void eval_kernel(const __grid_constant__ Plan p, uint64_t idx_begin, uint64_t count,
+                            mmee_result_t* __restrict__ out) {
+    for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < count;
+         i += (uint64_t)gridDim.x * blockDim.x) {
+        mmee_result_t r;
+        evaluate_candidate(p, idx_begin + i, r);
+        out[i] = r;
+    }
+}
+
+template <int OBJ, bool DUMP>
+cudaError_t launch_search_t(const Plan& p, const LaunchShape& shape, Scratch* scratch, int64_t* dump, cudaStream_t st) {
+    cudaError_t e = cudaFuncSetAttribute(search_kernel<OBJ, DUMP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)shape.smem_bytes);
+    if (e != cudaSuccess) return e;
+    search_kernel<OBJ, DUMP><<<shape.grid, kSearchThreads, shape.smem_bytes, st>>>(p, shape, scratch, dump);
+    return cudaGetLastError();
+}
+
+template <int OBJ, bool DUMP>
+cudaError_t occupancy_t(int* blocks_per_sm, size_t smem) {
+    cudaError_t e = cudaFuncSetAttribute(search_kernel<OBJ, DUMP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, search_kernel<OBJ, DUMP>, kSearchThreads, smem);
+}
+
+}  // namespace
+
+size_t search_smem_bytes(const Plan& p, uint32_t slots) {
+    return sizeof(CtaShared) + (kSearchThreads / 32) * sizeof(WarpTop) + slots * sizeof(TilingTab) +
+           (size_t)slots * p.n_orders * sizeof(OrderTab);
+}
+
+cudaError_t search_occupancy(const Plan& p, size_t smem, int* blocks_per_sm) {
+    switch (p.objective) {
+        case MMEE_OBJ_ENERGY: return occupancy_t<MMEE_OBJ_ENERGY, false>(blocks_per_sm, smem);
+        case MMEE_OBJ_LATENCY: return occupancy_t<MMEE_OBJ_LATENCY, false>(blocks_per_sm, smem);
+        default: return occupancy_t<MMEE_OBJ_EDP, false>(blocks_per_sm, smem);
+    }
+}
+
+cudaError_t launch_search(const Plan& p, const LaunchShape& shape, Scratch* scratch, int64_t* dump, cudaStream_t st) {
+    if (dump) {
+        switch (p.objective) {
+            case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, true>(p, shape, scratch, dump, st);
+            case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, true>(p, shape, scratch, dump, st);
+            default: return launch_search_t<MMEE_OBJ_EDP, true>(p, shape, scratch, dump, st);
+        }
+    }
+    switch (p.objective) {
+        case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, false>(p, shape, scratch, nullptr, st);
+        case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, false>(p, shape, scratch, nullptr, st);
+        default: return launch_search_t<MMEE_OBJ_EDP, false>(p, shape, scratch, nullptr, st);
+    }
+}
+
+cudaError_t launch_finalize(const Plan& p, Scratch* scratch, int n_partials, mmee_result_t* out_best,
+                            mmee_result_t* out_topk, cudaStream_t st) {
+    finalize_kernel<<<1, 1024, 0, st>>>(p, scratch, n_partials, out_best, out_topk);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_reset(Scratch* scratch, cudaStream_t st) {
+    reset_kernel<<<1, 1, 0, st>>>(scratch);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_eval(const Plan& p, uint64_t idx_begin, uint64_t count, mmee_result_t* out, cudaStream_t st) {
+    if (!count) return cudaSuccess;
+    const uint64_t want = (count + 127) / 128;
+    const int grid = (int)(want < 4096 ? want : 4096);
+    eval_kernel<<<grid, 128, 0, st>>>(p, idx_begin, count, out);
+    return cudaGetLastError();
+}
+
+}  // namespace mmee
