@@ -1,0 +1,230 @@
+// C ABI of libmmee (declared and documented in include/mmee.h).
+#include <cuda_runtime.h>
+
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "mmee_search.h"
+
+static_assert(sizeof(mmee_result_t) == 304, "mmee_result_t is part of the ABI");
+static_assert(sizeof(mmee::Plan) <= 4096, "the plan travels as a kernel parameter");
+
+struct mmee_handle {
+    mmee::Plan plan;
+    mmee::LaunchShape shape;
+    mmee::Scratch* scratch;      // device
+    int device;
+    mmee_launch_stats_t last;
+    bool timing;
+    cudaEvent_t ev[3];           // before search kernel, between, after finalize kernel
+};
+
+namespace {
+
+using namespace mmee;
+
+// Tasks a CTA pulls per visit of the global counter, and the tilings such a range can touch.
+int choose_shape(const Plan& p, int device, LaunchShape* shape) {
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return MMEE_ERR_CUDA;
+    const uint32_t rounds = 8;
+    shape->range_tasks = rounds * kSearchThreads;
+    shape->slots = (shape->range_tasks - 1) / p.tasks_per_tiling + 2;
+    size_t smem = search_smem_bytes(p, shape->slots);
+    // Many small tilings per range need many table slots: shrink the range until they fit.
+    while (smem > 96 * 1024 && shape->range_tasks > kSearchThreads) {
+        shape->range_tasks -= kSearchThreads;
+        shape->slots = (shape->range_tasks - 1) / p.tasks_per_tiling + 2;
+        smem = search_smem_bytes(p, shape->slots);
+    }
+    if (smem > (size_t)prop.sharedMemPerBlockOptin) return MMEE_ERR_RANGE;
+    shape->smem_bytes = (uint32_t)smem;
+    int per_sm = 0;
+    if (search_occupancy(p, smem, &per_sm) != cudaSuccess || per_sm < 1) return MMEE_ERR_CUDA;
+    if (per_sm > 2) per_sm = 2;
+    uint64_t grid = (uint64_t)prop.multiProcessorCount * (uint32_t)per_sm;
+    const uint64_t tasks = (p.t_end - p.t_begin) * p.tasks_per_tiling;
+    const uint64_t ranges = (tasks + shape->range_tasks - 1) / shape->range_tasks;
+    if (grid > ranges) grid = ranges ? ranges : 1;
+    shape->grid = (uint32_t)grid;
+    return MMEE_OK;
+}
+
+int cuda_status(cudaError_t e) { return e == cudaSuccess ? MMEE_OK : MMEE_ERR_CUDA; }
+
+}  // namespace
+
+extern "C" {
+
+int mmee_create(const mmee_workload_t* workload, const mmee_arch_t* arch, const mmee_objective_t* objective,
+                mmee_handle_t** out) {
+    if (!out) return MMEE_ERR_ARG;
+    *out = nullptr;
+    mmee_handle* h = new (std::nothrow) mmee_handle;
+    if (!h) return MMEE_ERR_ARG;
+    std::memset(h, 0, sizeof(*h));
+    int rc = build_plan(workload, arch, objective, &h->plan);
+    if (rc) { delete h; return rc; }
+    if (cudaGetDevice(&h->device) != cudaSuccess) { delete h; return MMEE_ERR_CUDA; }
+    rc = choose_shape(h->plan, h->device, &h->shape);
+    if (rc) { delete h; return rc; }
+    if (cudaMalloc(reinterpret_cast<void**>(&h->scratch), scratch_bytes(h->shape.grid)) != cudaSuccess) {
+        delete h;
+        return MMEE_ERR_CUDA;
+    }
+    if (launch_reset(h->scratch, 0) != cudaSuccess || cudaStreamSynchronize(0) != cudaSuccess) {
+        cudaFree(h->scratch);
+        delete h;
+        return MMEE_ERR_CUDA;
+    }
+    *out = h;
+    return MMEE_OK;
+}
+
+int mmee_search(mmee_handle_t* h, void* cuda_stream, mmee_result_t* out_best, mmee_result_t* out_topk) {
+    if (!h || !out_best) return MMEE_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (h->timing) cudaEventRecord(h->ev[0], st);
+    cudaError_t e = launch_search(h->plan, h->shape, h->scratch, nullptr, st);
+    if (e != cudaSuccess) return MMEE_ERR_CUDA;
+    if (h->timing) cudaEventRecord(h->ev[1], st);
+    e = launch_finalize(h->plan, h->scratch, (int)h->shape.grid, out_best, out_topk, st);
+    if (h->timing) cudaEventRecord(h->ev[2], st);
+    h->last.kernels_launched = 2;
+    h->last.grid = h->shape.grid;
+    h->last.block = kSearchThreads;
+    h->last.smem_bytes = h->shape.smem_bytes;
+    h->last.tasks = (h->plan.t_end - h->plan.t_begin) * h->plan.tasks_per_tiling;
+    return cuda_status(e);
+}
+
+int mmee_destroy(mmee_handle_t* h) {
+    if (!h) return MMEE_ERR_ARG;
+    cudaError_t e = cudaSuccess;
+    if (h->timing) for (int i = 0; i < 3; ++i) cudaEventDestroy(h->ev[i]);
+    if (h->scratch) e = cudaFree(h->scratch);
+    delete h;
+    return cuda_status(e);
+}
+
+uint64_t mmee_num_candidates(const mmee_handle_t* h) {
+    return h ? h->plan.n_tilings * (uint64_t)h->plan.rows_per_tiling * 9u : 0;
+}
+uint64_t mmee_num_tilings(const mmee_handle_t* h) { return h ? h->plan.n_tilings : 0; }
+uint64_t mmee_num_rows(const mmee_handle_t* h) { return h ? h->plan.rows_per_tiling : 0; }
+
+const char* mmee_strerror(int status) {
+    switch (status) {
+        case MMEE_OK: return "ok";
+        case MMEE_ERR_ARG: return "invalid argument";
+        case MMEE_ERR_OVERFLOW: return "a worst-case key of this problem does not fit 62 bits";
+        case MMEE_ERR_QUANTUM: return "an energy is not an integer multiple of the energy quantum";
+        case MMEE_ERR_NO_FEASIBLE: return "no mapping fits the global buffer";
+        case MMEE_ERR_CUDA: return "CUDA runtime error";
+        case MMEE_ERR_TIMEOUT: return "device-side wait timed out";
+        case MMEE_ERR_RANGE: return "request exceeds a documented maximum";
+        default: return "unknown status";
+    }
+}
+
+int mmee_eval(mmee_handle_t* h, void* cuda_stream, uint64_t idx_begin, uint64_t count, mmee_result_t* out) {
+    if (!h || (!out && count)) return MMEE_ERR_ARG;
+    const uint64_t n = mmee_num_candidates(h);
+    if (idx_begin > n || count > n - idx_begin) return MMEE_ERR_ARG;
+    return cuda_status(launch_eval(h->plan, idx_begin, count, out, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+int mmee_dump_keys(mmee_handle_t* h, void* cuda_stream, int64_t* out_keys) {
+    if (!h || !out_keys) return MMEE_ERR_ARG;
+    const uint64_t n = (h->plan.t_end - h->plan.t_begin) * (uint64_t)h->plan.rows_per_tiling * 9u;
+    if (n > (1ull << 31)) return MMEE_ERR_RANGE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = launch_search(h->plan, h->shape, h->scratch, out_keys, st);
+    if (e != cudaSuccess) return MMEE_ERR_CUDA;
+    return cuda_status(launch_reset(h->scratch, st));
+}
+
+int mmee_solve_host(const mmee_workload_t* workload, const mmee_arch_t* arch, const mmee_objective_t* objective,
+                    mmee_result_t* out_best, mmee_result_t* out_topk, uint64_t* h2d_bytes, uint64_t* d2h_bytes) {
+    if (!out_best || !objective) return MMEE_ERR_ARG;
+    mmee_handle_t* h = nullptr;
+    int rc = mmee_create(workload, arch, objective, &h);
+    if (rc) return rc;
+    const uint32_t k = h->plan.topk;
+    const size_t bytes = (size_t)(k + 1) * sizeof(mmee_result_t);
+    mmee_result_t* dev = nullptr;
+    if (cudaMalloc(reinterpret_cast<void**>(&dev), bytes) != cudaSuccess) { mmee_destroy(h); return MMEE_ERR_CUDA; }
+    rc = mmee_search(h, nullptr, dev, dev + 1);
+    if (rc == MMEE_OK) {
+        rc = cuda_status(cudaMemcpy(out_best, dev, sizeof(mmee_result_t), cudaMemcpyDeviceToHost));
+        if (rc == MMEE_OK && out_topk)
+            rc = cuda_status(cudaMemcpy(out_topk, dev + 1, (size_t)k * sizeof(mmee_result_t), cudaMemcpyDeviceToHost));
+    }
+    // The plan (divisor lists, query vectors, coefficients) travels to the device as the kernels'
+    // parameter block: once per launch.
+    if (h2d_bytes) *h2d_bytes = 2ull * sizeof(mmee::Plan);
+    if (d2h_bytes) *d2h_bytes = sizeof(mmee_result_t) * (uint64_t)(1 + (out_topk ? k : 0));
+    cudaFree(dev);
+    const int rc2 = mmee_destroy(h);
+    return rc ? rc : rc2;
+}
+
+int mmee_query_vector(uint32_t metric, uint32_t phi, uint32_t pi, uint32_t operand, uint32_t beta,
+                      uint32_t recompute, uint8_t out_q[8]) {
+    if (!out_q || metric > 1 || phi > 2 || pi > 5 || operand > 4 || beta < 3 || beta > 7 || recompute > 1)
+        return MMEE_ERR_ARG;
+    QueryTables tables;
+    build_query_tables(&tables);
+    uint8_t q;
+    if (metric == 0) {
+        q = tables.bs[pi][operand][beta - 3];
+    } else if (phi == 0) {
+        if (operand == OP_C) return MMEE_ERR_ARG;
+        q = tables.da[pi][operand][beta - 3][recompute];
+    } else {
+        q = tables.da_unfused[pi][operand][beta - 3];
+    }
+    for (int d = 0; d < 8; ++d) out_q[d] = (uint8_t)((q >> d) & 1u);
+    return MMEE_OK;
+}
+
+int mmee_recompute_flag(uint32_t pi, uint32_t beta_c, uint32_t* out_flag) {
+    if (!out_flag || pi > 5 || beta_c < 3 || beta_c > 7) return MMEE_ERR_ARG;
+    QueryTables tables;
+    build_query_tables(&tables);
+    *out_flag = tables.recompute[pi][beta_c - 3];
+    return MMEE_OK;
+}
+
+int mmee_last_search_stats(const mmee_handle_t* h, mmee_launch_stats_t* out) {
+    if (!h || !out) return MMEE_ERR_ARG;
+    *out = h->last;
+    out->search_ms = out->finalize_ms = -1.0f;
+    if (h->timing && h->last.kernels_launched) {
+        if (cudaEventElapsedTime(&out->search_ms, h->ev[0], h->ev[1]) != cudaSuccess ||
+            cudaEventElapsedTime(&out->finalize_ms, h->ev[1], h->ev[2]) != cudaSuccess)
+            return MMEE_ERR_CUDA;
+    }
+    return MMEE_OK;
+}
+
+int mmee_kernel_timing(mmee_handle_t* h, int enable) {
+    if (!h) return MMEE_ERR_ARG;
+    if (enable && !h->timing) {
+        for (int i = 0; i < 3; ++i)
+            if (cudaEventCreate(&h->ev[i]) != cudaSuccess) return MMEE_ERR_CUDA;
+        h->timing = true;
+    } else if (!enable && h->timing) {
+        for (int i = 0; i < 3; ++i) cudaEventDestroy(h->ev[i]);
+        h->timing = false;
+    }
+    return MMEE_OK;
+}
+
+int mmee_alu_peak(double out[4]) {
+    if (!out) return MMEE_ERR_ARG;
+    return cuda_status(measure_alu_peak(out));
+}
+
+}  // extern "C"
