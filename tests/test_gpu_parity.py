@@ -1,0 +1,269 @@
+"""GPU parity: the CUDA library against the CPU oracle, through the C ABI.
+
+Integer fields (access counts, buffer sizes, keys, indices, counters) must be bit-identical;
+floating-point outputs within 1e-12 relative.
+"""
+import glob
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import mmee_inputs as mi
+import oracle
+import paper_2604_03446_b200.binding as mm
+
+pytestmark = pytest.mark.gpu
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+REL_TOL = 1e-12
+INT_FIELDS = ("idx", "t", "row", "phi", "pi", "recompute", "feasible", "bs_op1", "bs_op2", "bs",
+              "da_sm", "br", "cyc1", "cyc2", "e_key", "l_key")
+ARRAY_FIELDS = ("bound", "beta", "sm", "bs_x", "da_x", "n")
+FLOAT_FIELDS = ("edp_key", "energy_pj", "latency_cycles")
+
+
+def assert_same_record(g, o, where=""):
+    for f in INT_FIELDS:
+        assert int(getattr(g, f)) == int(getattr(o, f)), "%s field %s" % (where, f)
+    for f in ARRAY_FIELDS:
+        assert list(getattr(g, f)) == list(getattr(o, f)), "%s field %s" % (where, f)
+    for f in FLOAT_FIELDS:
+        a, b = float(getattr(g, f)), float(getattr(o, f))
+        assert abs(a - b) <= REL_TOL * abs(b), "%s field %s: %r vs %r" % (where, f, a, b)
+
+
+class Handle:
+    def __init__(self, cfg, obj):
+        self.args = (cfg["workload"], cfg["arch"], obj)
+        self.h = None
+
+    def __enter__(self):
+        self.h = mm.mmee_create(*self.args)
+        return self.h
+
+    def __exit__(self, *exc):
+        mm.mmee_destroy(self.h)
+
+
+def gpu_search(cfg, obj):
+    k = obj["topk"]
+    best, topk = mm.result_buffer(1), mm.result_buffer(k)
+    with Handle(cfg, obj) as h:
+        mm.mmee_search(h, best, topk)
+        torch.cuda.synchronize()
+        stats = mm.mmee_last_search_stats(h)
+    return mm.read_results(best, 1)[0], mm.read_results(topk, k), stats
+
+
+def check_search(cfg, obj, threads=0):
+    p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
+    want = oracle.search(p, threads)
+    best, topk, _ = gpu_search(cfg, obj)
+    assert best.n_total == want.n_total
+    assert best.n_feasible == want.n_feasible
+    found = [r for r in topk if r.idx != mm.NO_INDEX]
+    assert [r.idx for r in found] == [r.idx for r in want.topk]
+    for g, o in zip(found, want.topk):
+        assert_same_record(g, o, cfg["name"])
+    if want.topk:
+        assert best.status == mm.OK and best.idx == want.topk[0].idx
+        assert_same_record(best, want.topk[0], cfg["name"])
+    else:
+        assert best.status == mm.ERR_NO_FEASIBLE and best.idx == mm.NO_INDEX
+    return best, found
+
+
+def shrink(cfg, obj, limit):
+    """Restrict the tiling range so that at most `limit` candidates are enumerated."""
+    p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
+    if p.N <= limit:
+        return dict(obj)
+    return dict(obj, t_begin=0, t_end=max(1, limit // (p.R * 9)))
+
+
+TINY_SEEDS = list(range(1, 13))
+
+
+@pytest.mark.parametrize("seed", TINY_SEEDS)
+def test_every_candidate_key_matches_the_oracle(seed):
+    """The search kernel's own evaluation path, element by element: one key per candidate,
+    INT64_MAX where the mapping does not fit the buffer."""
+    cfg = mi.random_tiny_problem(seed)
+    obj = shrink(cfg, cfg["searches"][0], 4_000_000)
+    p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
+    begin, count = p.t_begin * p.R * 9, (p.t_end - p.t_begin) * p.R * 9
+    keys, feas = oracle.keys_range(p, begin, count)
+    want = np.where(feas.astype(bool), keys, np.iinfo(np.int64).max)
+    out = torch.full((count,), -7, dtype=torch.int64, device="cuda")
+    with Handle(cfg, obj) as h:
+        assert mm.mmee_num_candidates(h) == p.N
+        mm.mmee_dump_keys(h, out)
+        torch.cuda.synchronize()
+    got = out.cpu().numpy()
+    bad = np.nonzero(got != want)[0]
+    assert bad.size == 0, "first mismatch at candidate %d: %d vs %d" % (begin + bad[0], got[bad[0]], want[bad[0]])
+
+
+@pytest.mark.parametrize("seed", TINY_SEEDS[:8])
+def test_every_candidate_record_matches_the_oracle(seed):
+    """The query-vector evaluation (mmee_eval): every field of every candidate."""
+    cfg = mi.random_tiny_problem(seed)
+    obj = cfg["searches"][0]
+    p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
+    count = min(p.N, 150_000)
+    begin = (p.N - count) // 2
+    want = oracle.evaluate_range(p, begin, count)
+    buf = mm.result_buffer(count)
+    with Handle(cfg, obj) as h:
+        mm.mmee_eval(h, begin, count, buf)
+        torch.cuda.synchronize()
+    got = mm.read_results(buf, count)
+    for g, o in zip(got, want):
+        assert_same_record(g, o, "seed %d idx %d" % (seed, o.idx))
+
+
+@pytest.mark.parametrize("seed", TINY_SEEDS)
+@pytest.mark.parametrize("k", [1, 16])
+def test_search_matches_the_oracle_on_tiny_problems(seed, k):
+    cfg = mi.random_tiny_problem(seed)
+    for objective in (mi.OBJ_ENERGY, mi.OBJ_LATENCY, mi.OBJ_EDP):
+        obj = shrink(cfg, dict(cfg["searches"][0], objective=objective, topk=k), 6_000_000)
+        check_search(cfg, obj)
+
+
+def test_config1_full_search():
+    cfg = mi.config1()
+    best, _ = check_search(cfg, cfg["searches"][0])
+    assert best.n_total == 162067500
+    check_search(cfg, dict(cfg["searches"][0], topk=16, objective=mi.OBJ_LATENCY))
+    check_search(cfg, dict(cfg["searches"][0], topk=16, objective=mi.OBJ_EDP))
+
+
+def _golden_files():
+    return sorted(glob.glob(os.path.join(GOLDEN, "search_*.json")))
+
+
+@pytest.mark.parametrize("path", _golden_files(), ids=lambda p: os.path.basename(p)[7:-5])
+def test_full_size_search_matches_stored_oracle_answers(path):
+    """Benchmark configurations at full size, in the launch configuration the benchmark times.
+    Expected values were written by tests/golden/make_search_goldens.py from the oracle alone."""
+    with open(path) as f:
+        gold = json.load(f)
+    cfg = dict(name=gold["name"], workload=gold["workload"], arch=gold["arch"])
+    for s in gold["searches"]:
+        best, topk, stats = gpu_search(cfg, s["objective"])
+        assert stats.kernels_launched == 2 and stats.grid >= 1
+        assert best.n_total == s["n_total"] and best.n_feasible == s["n_feasible"]
+        found = [r for r in topk if r.idx != mm.NO_INDEX]
+        assert [r.idx for r in found] == [r["idx"] for r in s["topk"]]
+        for g, o in zip(found, s["topk"]):
+            for f in ("t", "row", "phi", "pi", "recompute", "bs", "bs_op1", "bs_op2", "br", "cyc1", "cyc2",
+                      "e_key", "l_key"):
+                assert int(getattr(g, f)) == o[f], f
+            for f in ("bound", "beta", "sm", "n"):
+                assert list(getattr(g, f)) == o[f], f
+            for f in ("edp_key", "energy_pj", "latency_cycles"):
+                b = float.fromhex(o[f + "_hex"])
+                assert abs(float(getattr(g, f)) - b) <= REL_TOL * abs(b), f
+
+
+@pytest.mark.parametrize("maker", [mi.config2, mi.config3, mi.config4])
+def test_sampled_candidates_at_full_size(maker):
+    """Candidates drawn over the whole index space of the large configurations, each compared
+    field by field with the oracle's one-at-a-time evaluation."""
+    cfg = maker()
+    rng = np.random.default_rng(11)
+    for obj in cfg["searches"]:
+        p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
+        starts = [0, p.N - 64] + [int(v) for v in rng.integers(0, p.N - 64, size=30)]
+        with Handle(cfg, obj) as h:
+            for s in starts:
+                buf = mm.result_buffer(64)
+                mm.mmee_eval(h, s, 64, buf)
+                torch.cuda.synchronize()
+                for g, o in zip(mm.read_results(buf, 64), oracle.evaluate_range(p, s, 64)):
+                    assert_same_record(g, o, "%s idx %d" % (cfg["name"], o.idx))
+
+
+def test_sub_ranges_partition_the_search():
+    """Tiling sub-ranges: each range agrees with the oracle; the best over the ranges is the best
+    of the whole; feasible counts add up."""
+    cfg = mi.random_tiny_problem(5)
+    obj = dict(cfg["searches"][0], objective=mi.OBJ_ENERGY, topk=4)
+    p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
+    T = p.T
+    cuts = [0, T // 3, T // 3 + 1, T]
+    total_feasible, bests = 0, []
+    for lo, hi in zip(cuts[:-1], cuts[1:]):
+        best, found = check_search(cfg, dict(obj, t_begin=lo, t_end=hi))
+        total_feasible += best.n_feasible
+        bests += [(r.e_key, r.idx) for r in found]
+    whole, found = check_search(cfg, obj)
+    assert total_feasible == whole.n_feasible
+    assert sorted(bests)[:len(found)] == [(r.e_key, r.idx) for r in found]
+
+
+def test_nothing_fits():
+    cfg = mi.random_tiny_problem(3)
+    arch = dict(cfg["arch"], gb_bytes=cfg["workload"]["word_bytes"] * 2)
+    best, found = check_search(dict(cfg, arch=arch), dict(cfg["searches"][0], topk=3))
+    assert best.n_feasible == 0 and not found and best.status == mm.ERR_NO_FEASIBLE
+
+
+def test_fewer_feasible_mappings_than_k():
+    """A capacity that admits only a handful of mappings leaves the tail of the top-k empty."""
+    cfg = dict(name="scarce", workload=mi.workload(1, 1, 1, 4, 4, 2, 2, 1),
+               arch=mi.arch(2, 2, 1, 3, 0, 1, 10.0, 2.0, 0.0, 1.0))
+    obj = mi.objective(mi.OBJ_ENERGY, 16, mi.TILE_ALL_DIVISORS, mi.ORD_NORECOMP2, mi.FUSE_FUSED)
+    best, found = check_search(cfg, obj)
+    assert 0 < best.n_feasible // 9 and len(found) <= 16
+
+
+def test_massive_ties_keep_the_lowest_indices():
+    """Latency on a compute-bound problem: a large share of the mappings tie at the optimum and the
+    top-k must be exactly the k lowest indices among them."""
+    cfg = dict(name="ties", workload=mi.workload(1, 1, 1, 64, 64, 16, 16, 2),
+               arch=mi.arch(4, 4, 1, 64 * 1024, 64, 4096, 100.0, 5.0, 1.0, 1.0))
+    obj = mi.objective(mi.OBJ_LATENCY, 16, mi.TILE_POW2, mi.ORD_ALL6, mi.FUSE_ALL)
+    best, found = check_search(cfg, obj)
+    assert len({r.l_key for r in found}) == 1
+
+
+def test_repeated_searches_on_one_handle_are_identical():
+    cfg = mi.config1()
+    obj = dict(cfg["searches"][0], topk=16)
+    bufs = [(mm.result_buffer(1), mm.result_buffer(16)) for _ in range(3)]
+    with Handle(cfg, obj) as h:
+        for b, t in bufs:
+            mm.mmee_search(h, b, t)
+        torch.cuda.synchronize()
+    raws = [(bytes(b.cpu().numpy().tobytes()), bytes(t.cpu().numpy().tobytes())) for b, t in bufs]
+    assert raws[0] == raws[1] == raws[2]
+
+
+def test_host_buffer_entry_point_equals_device_path():
+    cfg = mi.config1()
+    obj = dict(cfg["searches"][0], topk=4)
+    best, topk, h2d, d2h = mm.mmee_solve_host(cfg["workload"], cfg["arch"], obj)
+    dbest, dtopk, _ = gpu_search(cfg, obj)
+    assert bytes(best) == bytes(dbest)
+    assert [bytes(r) for r in topk] == [bytes(r) for r in dtopk]
+    assert h2d > 0 and d2h == 5 * mm.RESULT_BYTES
+
+
+def test_search_on_a_side_stream():
+    cfg = mi.random_tiny_problem(2)
+    obj = shrink(cfg, dict(cfg["searches"][0], topk=2), 2_000_000)
+    p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
+    want = oracle.search(p)
+    st = torch.cuda.Stream()
+    best = mm.result_buffer(1)
+    with Handle(cfg, obj) as h:
+        with torch.cuda.stream(st):
+            mm.mmee_search(h, best, None, stream=st)
+        st.synchronize()
+    got = mm.read_results(best, 1)[0]
+    assert got.idx == (want.topk[0].idx if want.topk else mm.NO_INDEX)
