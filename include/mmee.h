@@ -155,6 +155,9 @@ uint64_t mmee_num_rows(const mmee_handle_t* handle);
 
 const char* mmee_strerror(int status);
 
+/* Text of the CUDA runtime error behind the calling thread's most recent MMEE_ERR_CUDA. */
+const char* mmee_last_cuda_error(void);
+
 /*
  * mmee_eval -- evaluate `count` consecutive candidates from `idx_begin` on the device with the
  * query-vector form of the model, exp(q . ln b) taken exactly as an integer product

@@ -20,7 +20,7 @@ NO_INDEX = 2 ** 64 - 1
 OK, ERR_ARG, ERR_OVERFLOW, ERR_QUANTUM, ERR_NO_FEASIBLE, ERR_CUDA, ERR_TIMEOUT, ERR_RANGE = range(8)
 
 EXPORTS = ("mmee_create", "mmee_search", "mmee_destroy", "mmee_num_candidates", "mmee_num_tilings",
-           "mmee_num_rows", "mmee_strerror", "mmee_eval", "mmee_dump_keys", "mmee_solve_host",
+           "mmee_num_rows", "mmee_strerror", "mmee_last_cuda_error", "mmee_eval", "mmee_dump_keys", "mmee_solve_host",
            "mmee_query_vector", "mmee_recompute_flag", "mmee_last_search_stats", "mmee_kernel_timing",
            "mmee_alu_peak")
 
@@ -71,6 +71,8 @@ RESULT_BYTES = C.sizeof(Result)
 class MmeeError(RuntimeError):
     def __init__(self, code: int, where: str):
         msg = library().mmee_strerror(code).decode() if _lib is not None else "status %d" % code
+        if code == ERR_CUDA and _lib is not None:
+            msg += ": " + library().mmee_last_cuda_error().decode()
         super().__init__("%s: %s (status %d)" % (where, msg, code))
         self.code = code
 
@@ -100,6 +102,8 @@ def library():
         getattr(L, name).restype = C.c_uint64
     L.mmee_strerror.argtypes = [C.c_int]
     L.mmee_strerror.restype = C.c_char_p
+    L.mmee_last_cuda_error.argtypes = []
+    L.mmee_last_cuda_error.restype = C.c_char_p
     L.mmee_eval.argtypes = [H, C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p]
     L.mmee_dump_keys.argtypes = [H, C.c_void_p, C.c_void_p]
     L.mmee_solve_host.argtypes = [C.POINTER(Workload), C.POINTER(Arch), C.POINTER(Objective),

@@ -51,7 +51,13 @@ int choose_shape(const Plan& p, int device, LaunchShape* shape) {
     return MMEE_OK;
 }
 
-int cuda_status(cudaError_t e) { return e == cudaSuccess ? MMEE_OK : MMEE_ERR_CUDA; }
+thread_local cudaError_t g_last_cuda_error = cudaSuccess;
+
+int cuda_status(cudaError_t e) {
+    if (e == cudaSuccess) return MMEE_OK;
+    g_last_cuda_error = e;
+    return MMEE_ERR_CUDA;
+}
 
 }  // namespace
 
@@ -221,6 +227,8 @@ int mmee_kernel_timing(mmee_handle_t* h, int enable) {
     }
     return MMEE_OK;
 }
+
+const char* mmee_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda_error); }
 
 int mmee_alu_peak(double out[4]) {
     if (!out) return MMEE_ERR_ARG;

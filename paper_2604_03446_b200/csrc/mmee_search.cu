@@ -313,7 +313,9 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
             const TaskChoice c = decode_task(p, w);
             const OrderTab* ot = &otabs[slot * n_orders + c.order_slot];
             const bool fused = c.phi == 0;
-            const uint32_t rc = fused ? ot->rc[c.lc] : 0u;
+            // Tables of a tiling that cannot fit are never built: a lane whose task lies in such a
+            // tiling must not index with what it reads from them.
+            const uint32_t rc = (fused && live) ? (ot->rc[c.lc] & 1u) : 0u;
             const int64_t a1 = ot->A1[c.la], b1 = ot->B1[c.lb], c1 = ot->C1[c.lc];
             // Eq. (1)/(2): a retained operand (level >= L4) of the other operator keeps its space.
             const int64_t slack1 = cap - (a1 + b1 + c1);
