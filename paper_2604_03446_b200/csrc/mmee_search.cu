@@ -116,6 +116,29 @@ __device__ __forceinline__ int64_t candidate_key(int64_t x, int64_t xe, int64_t 
     }
 }
 
+// One compare per candidate, OR-ed into one predicate.  Written as PTX so that the nine compares
+// against the common threshold stay nine compares: the compiler otherwise rewrites
+// (a < t) | (b < t) into min(a, b) < t, and a 64-bit min costs more than the compare it saves.
+__device__ __forceinline__ bool any_below(const int64_t (&k)[9], int64_t thr) {
+    unsigned r;
+    asm("{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.lt.s64 p, %1, %10;\n\t"
+        "setp.lt.or.s64 p, %2, %10, p;\n\t"
+        "setp.lt.or.s64 p, %3, %10, p;\n\t"
+        "setp.lt.or.s64 p, %4, %10, p;\n\t"
+        "setp.lt.or.s64 p, %5, %10, p;\n\t"
+        "setp.lt.or.s64 p, %6, %10, p;\n\t"
+        "setp.lt.or.s64 p, %7, %10, p;\n\t"
+        "setp.lt.or.s64 p, %8, %10, p;\n\t"
+        "setp.lt.or.s64 p, %9, %10, p;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}"
+        : "=r"(r)
+        : "l"(k[0]), "l"(k[1]), "l"(k[2]), "l"(k[3]), "l"(k[4]), "l"(k[5]), "l"(k[6]), "l"(k[7]), "l"(k[8]), "l"(thr));
+    return r != 0;
+}
+
 // Rare path: some lane of the warp has a key below its threshold in this row.  Every lane
 // re-evaluates its nine candidates of the row from the shared tables and the warp inserts the
 // passing ones, one at a time, into its sorted list.
@@ -379,16 +402,15 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                     rows += f ? 1u : 0u;
                     const int64_t x = xd + gE[e];
                     const int64_t xe = xed + eE[e];
-                    bool any = false;
+                    int64_t key[9];
 #pragma unroll
                     for (int s = 0; s < 9; ++s) {
-                        const int64_t key = candidate_key<OBJ>(x, xe, W[s], P[s / 3], Q[s]);
-                        any |= key < thr;
+                        key[s] = candidate_key<OBJ>(x, xe, W[s], P[s / 3], Q[s]);
                         if (DUMP) {
-                            if (valid) dump[task_first_idx - dump_origin + (d * 5 + e) * 9 + s] = f ? key : kInfKey;
+                            if (valid) dump[task_first_idx - dump_origin + (d * 5 + e) * 9 + s] = f ? key[s] : kInfKey;
                         }
                     }
-                    any &= f;
+                    const bool any = f && any_below(key, thr);
                     if (__any_sync(kFull, any)) {
                         thr = slow_row<OBJ>(wt, cs, k, lane, f, x, xe, wptr, qptr, P[0], P[1], P[2],
                                             task_first_idx + (uint64_t)((d * 5 + e) * 9), task_first_idx);
