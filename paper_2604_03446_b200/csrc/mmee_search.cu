@@ -119,7 +119,7 @@ __device__ __forceinline__ int64_t candidate_key(int64_t x, int64_t xe, int64_t 
 // One compare per candidate, OR-ed into one predicate.  Written as PTX so that the nine compares
 // against the common threshold stay nine compares: the compiler otherwise rewrites
 // (a < t) | (b < t) into min(a, b) < t, and a 64-bit min costs more than the compare it saves.
-__device__ __forceinline__ bool any_below(const int64_t (&k)[9], int64_t thr) {
+__device__ __forceinline__ unsigned any_below(const int64_t (&k)[9], int64_t thr) {
     unsigned r;
     asm("{\n\t"
         ".reg .pred p;\n\t"
@@ -136,7 +136,7 @@ __device__ __forceinline__ bool any_below(const int64_t (&k)[9], int64_t thr) {
         "}"
         : "=r"(r)
         : "l"(k[0]), "l"(k[1]), "l"(k[2]), "l"(k[3]), "l"(k[4]), "l"(k[5]), "l"(k[6]), "l"(k[7]), "l"(k[8]), "l"(thr));
-    return r != 0;
+    return r;
 }
 
 // Rare path: some lane of the warp has a key below its threshold in this row.  Every lane
@@ -341,8 +341,9 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
             const uint32_t rc = (fused && live) ? (ot->rc[c.lc] & 1u) : 0u;
             const int64_t a1 = ot->A1[c.la], b1 = ot->B1[c.lb], c1 = ot->C1[c.lc];
             // Eq. (1)/(2): a retained operand (level >= L4) of the other operator keeps its space.
-            const int64_t slack1 = cap - (a1 + b1 + c1);
-            const int64_t slack2 = cap - (c1 + ((fused && c.la) ? a1 : 0) + ((fused && c.lb) ? b1 : 0));
+            // A lane without a live task gets a negative slack, so that none of its rows fits.
+            const int64_t slack1 = live ? cap - (a1 + b1 + c1) : -1;
+            const int64_t slack2 = live ? cap - (c1 + ((fused && c.la) ? a1 : 0) + ((fused && c.lb) ? b1 : 0)) : -1;
             const int64_t gab = ot->gA[c.la][rc] + ot->gB[c.lb][rc];
 
             int64_t x0, xe0 = 0, P[3], Q[9], W[9];
@@ -396,10 +397,13 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                 const int64_t s2 = slack2 - d2;
                 const int64_t xd = x0 + (fused ? ot->gD[d] : ot->gDu[d]);
                 const int64_t xed = (OBJ == MMEE_OBJ_EDP) ? xe0 + (fused ? ot->eD[d] : ot->eDu[d]) : 0;
+                // Five rows (levels of E) are evaluated branch-free; one vote decides whether any
+                // lane of the warp has to enter the insertion path for this group.
+                unsigned fit[5], hit[5];
 #pragma unroll
                 for (int e = 0; e < 5; ++e) {
-                    const bool f = live && (E1[e] <= s1) && (E2[e] <= s2);     // Eq. (4) against the capacity
-                    rows += f ? 1u : 0u;
+                    fit[e] = (unsigned)(E1[e] <= s1) & (unsigned)(E2[e] <= s2);   // Eq. (4) against the capacity
+                    rows += fit[e];
                     const int64_t x = xd + gE[e];
                     const int64_t xe = xed + eE[e];
                     int64_t key[9];
@@ -407,13 +411,19 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                     for (int s = 0; s < 9; ++s) {
                         key[s] = candidate_key<OBJ>(x, xe, W[s], P[s / 3], Q[s]);
                         if (DUMP) {
-                            if (valid) dump[task_first_idx - dump_origin + (d * 5 + e) * 9 + s] = f ? key[s] : kInfKey;
+                            if (valid) dump[task_first_idx - dump_origin + (d * 5 + e) * 9 + s] = fit[e] ? key[s] : kInfKey;
                         }
                     }
-                    const bool any = f && any_below(key, thr);
-                    if (__any_sync(kFull, any)) {
-                        thr = slow_row<OBJ>(wt, cs, k, lane, f, x, xe, wptr, qptr, P[0], P[1], P[2],
-                                            task_first_idx + (uint64_t)((d * 5 + e) * 9), task_first_idx);
+                    hit[e] = any_below(key, thr) & fit[e];
+                }
+                if (__any_sync(kFull, (hit[0] | hit[1] | hit[2] | hit[3] | hit[4]) != 0u)) {
+#pragma unroll
+                    for (int e = 0; e < 5; ++e) {
+                        if (__any_sync(kFull, hit[e] != 0u)) {
+                            thr = slow_row<OBJ>(wt, cs, k, lane, fit[e] != 0u, xd + gE[e], xed + eE[e], wptr, qptr,
+                                                P[0], P[1], P[2],
+                                                task_first_idx + (uint64_t)((d * 5 + e) * 9), task_first_idx);
+                        }
                     }
                 }
             }
