@@ -15,60 +15,77 @@ __device__ __forceinline__ int64_t monomial(uint32_t q, const uint32_t b[8]) {
     return v;
 }
 
-__device__ __forceinline__ int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+// Ceiling of a / b for 32-bit operands (tile extents and array sizes), widened for the products.
+__device__ __forceinline__ int64_t ceil_div(uint32_t a, uint32_t b) { return (int64_t)((a + b - 1u) / b); }
 
 // Compute cycles of one (m x r) * (r x n) tile on a rows x cols array.
 // 0 weight stationary: r x n weights folded onto the array, m inputs streamed per fold;
 // 1 input stationary:  m x r inputs folded, n weight columns streamed;
 // 2 output stationary: m x n outputs folded, r reduction steps streamed.
-__device__ __forceinline__ int64_t tile_cycles(int sm, int64_t m, int64_t r, int64_t n, int64_t rows, int64_t cols) {
-    if (sm == 0) return ceil_div64(r, rows) * ceil_div64(n, cols) * m;
-    if (sm == 1) return ceil_div64(m, rows) * ceil_div64(r, cols) * n;
-    return ceil_div64(m, rows) * ceil_div64(n, cols) * r;
+__device__ __forceinline__ int64_t tile_cycles(int sm, uint32_t m, uint32_t r, uint32_t n, uint32_t rows, uint32_t cols) {
+    if (sm == 0) return ceil_div(r, rows) * ceil_div(n, cols) * (int64_t)m;
+    if (sm == 1) return ceil_div(m, rows) * ceil_div(r, cols) * (int64_t)n;
+    return ceil_div(m, rows) * ceil_div(n, cols) * (int64_t)r;
 }
 
 // Words moved between the global buffer and the array for one tile: the stationary operand
 // once, the streamed operand once per fold of the other dimension, partial sums read and
 // written between reduction folds (2*folds - 1 transfers per output element).
-__device__ __forceinline__ int64_t tile_traffic(int sm, int64_t m, int64_t r, int64_t n, int64_t rows, int64_t cols) {
-    if (sm == 0) return r * n + m * r * ceil_div64(n, cols) + m * n * (2 * ceil_div64(r, rows) - 1);
-    if (sm == 1) return m * r + r * n * ceil_div64(m, rows) + m * n * (2 * ceil_div64(r, cols) - 1);
-    return m * r * ceil_div64(n, cols) + r * n * ceil_div64(m, rows) + m * n;
+__device__ __forceinline__ int64_t tile_traffic(int sm, uint32_t m, uint32_t r, uint32_t n, uint32_t rows, uint32_t cols) {
+    const int64_t M = m, R = r, N = n;
+    if (sm == 0) return R * N + M * R * ceil_div(n, cols) + M * N * (2 * ceil_div(r, rows) - 1);
+    if (sm == 1) return M * R + R * N * ceil_div(m, rows) + M * N * (2 * ceil_div(r, cols) - 1);
+    return M * R * ceil_div(n, cols) + R * N * ceil_div(m, rows) + M * N;
 }
 
-// Everything about one tiling that does not depend on order or levels.
-struct TilingTerms {
-    int64_t br1[3], br2[3];     // per-tile buffer<->PE words by stationary mode
-    int64_t cy1[3], cy2[3];     // per-tile cycles by stationary mode
-    int64_t t1, t2;             // tile invocations of Op1 (without recomputation) and Op2
-    int64_t carry1, carry2;     // partial sums carried between reduction steps (rho = 1)
+// Tile invocations and carried partial sums of one tiling (no recomputation).
+struct TilingCounts {
+    int64_t t1, t2;             // tile invocations of Op1 and Op2
+    int64_t carry1, carry2;     // partial sums carried between consecutive reduction steps
     int64_t ikl, ilj, il;       // I*K*L, I*L*J, I*L
 };
 
-__device__ __forceinline__ void tiling_terms(const Plan& p, const uint32_t b[8], TilingTerms& tt) {
-    const int64_t iD = b[0], kD = b[1], lD = b[2], jD = b[3], iG = b[4], kG = b[5], lG = b[6], jG = b[7];
-#pragma unroll
-    for (int sm = 0; sm < 3; ++sm) {
-        tt.br1[sm] = tile_traffic(sm, iG, kG, lG, p.pe_rows, p.pe_cols);
-        tt.br2[sm] = tile_traffic(sm, iG, lG, jG, p.pe_rows, p.pe_cols);
-        tt.cy1[sm] = tile_cycles(sm, iG, kG, lG, p.pe_rows, p.pe_cols);
-        tt.cy2[sm] = tile_cycles(sm, iG, lG, jG, p.pe_rows, p.pe_cols);
-    }
-    tt.t1 = iD * kD * lD;
-    tt.t2 = iD * lD * jD;
-    tt.carry1 = (tt.t1 - tt.t1 / kD) * iG * lG;
-    tt.carry2 = (tt.t2 - tt.t2 / lD) * iG * jG;
-    tt.ikl = (int64_t)p.dim[0] * p.dim[1] * p.dim[2];
-    tt.ilj = (int64_t)p.dim[0] * p.dim[2] * p.dim[3];
-    tt.il = (int64_t)p.dim[0] * p.dim[2];
+__device__ __forceinline__ TilingCounts tiling_counts(const Plan& p, const uint32_t b[8]) {
+    const int64_t iD = b[0], kD = b[1], lD = b[2], jD = b[3], iG = b[4], lG = b[6], jG = b[7];
+    TilingCounts c;
+    c.t1 = iD * kD * lD;
+    c.t2 = iD * lD * jD;
+    c.carry1 = (c.t1 - iD * lD) * iG * lG;      // every reduction step but the first of each C tile
+    c.carry2 = (c.t2 - iD * jD) * iG * jG;
+    c.ikl = (int64_t)p.dim[0] * p.dim[1] * p.dim[2];
+    c.ilj = (int64_t)p.dim[0] * p.dim[2] * p.dim[3];
+    c.il = (int64_t)p.dim[0] * p.dim[2];
+    return c;
+}
+
+// Array-level terms of one (stationary pair, recompute flag) of one tiling: buffer<->PE words,
+// compute cycles of each operator, MAC and softmax counts.
+struct ArrayTerms {
+    int64_t br, cyc1, cyc2, n_mac, n_sfu;
+};
+
+__device__ __forceinline__ ArrayTerms array_terms(const Plan& p, const uint32_t b[8], const TilingCounts& c,
+                                                  int sm1, int sm2, bool recompute) {
+    const int64_t rho = recompute ? (int64_t)b[3] : 1;
+    const int64_t t1 = rho * c.t1;
+    ArrayTerms a;
+    a.br = t1 * tile_traffic(sm1, b[4], b[5], b[6], p.pe_rows, p.pe_cols) + rho * c.carry1 +
+           c.t2 * tile_traffic(sm2, b[4], b[6], b[7], p.pe_rows, p.pe_cols) + c.carry2;
+    a.cyc1 = t1 * tile_cycles(sm1, b[4], b[5], b[6], p.pe_rows, p.pe_cols);
+    a.cyc2 = c.t2 * tile_cycles(sm2, b[4], b[6], b[7], p.pe_rows, p.pe_cols);
+    a.n_mac = rho * c.ikl + c.ilj;
+    a.n_sfu = rho * c.il;
+    return a;
 }
 
 // Tiling index -> boundary vector b (one column of the boundary matrix, Section VI-A).
-__device__ __forceinline__ void tiling_bounds(const Plan& p, uint64_t t, uint32_t b[8]) {
+__device__ __forceinline__ void tiling_bounds(const Plan& p, uint64_t t64, uint32_t b[8]) {
+    uint32_t t = (uint32_t)t64;                 // at most MMEE_MAX_DIVISORS^4 = 2^24 tilings
 #pragma unroll
     for (int d = 3; d >= 0; --d) {
-        const uint32_t a = (uint32_t)(t % p.ndiv[d]);
-        t /= p.ndiv[d];
+        const uint32_t q = t / p.ndiv[d];
+        const uint32_t a = t - q * p.ndiv[d];
+        t = q;
         const uint32_t g = p.divs[d][a];
         b[4 + d] = g;
         b[d] = p.dim[d] / g;
@@ -118,8 +135,7 @@ __device__ inline void evaluate_candidate(const Plan& p, uint64_t idx, mmee_resu
 
     uint32_t b[8];
     tiling_bounds(p, t, b);
-    TilingTerms tt;
-    tiling_terms(p, b, tt);
+    const TilingCounts tt = tiling_counts(p, b);
 
     o.idx = idx; o.t = t; o.row = row;
     for (int d = 0; d < 8; ++d) o.bound[d] = b[d];
@@ -132,7 +148,6 @@ __device__ inline void evaluate_candidate(const Plan& p, uint64_t idx, mmee_resu
     const QueryTables& q = p.q;
     const bool fused = c.phi == 0;
     const uint32_t rc = fused ? q.recompute[c.order][c.lc] : 0u;
-    const int64_t rho = rc ? (int64_t)b[3] : 1;
 
     int64_t bs[5], da[5];
     for (int x = 0; x < 5; ++x) {
@@ -155,11 +170,8 @@ __device__ inline void evaluate_candidate(const Plan& p, uint64_t idx, mmee_resu
         if (c.phi == 2) da_sm = 2 * tt.il;             // separate softmax pass: read S, write P
     }
     const int64_t n_dram = da[0] + da[1] + da[2] + da[3] + da[4] + da_sm;
-    const int64_t n_mac = rho * tt.ikl + tt.ilj;
-    const int64_t n_sfu = rho * tt.il;
-    const int64_t t1 = rho * tt.t1;
-    const int64_t br = t1 * tt.br1[sm1] + rho * tt.carry1 + tt.t2 * tt.br2[sm2] + tt.carry2;
-    const int64_t cyc1 = t1 * tt.cy1[sm1], cyc2 = tt.t2 * tt.cy2[sm2];
+    const ArrayTerms at = array_terms(p, b, tt, sm1, sm2, rc != 0);
+    const int64_t n_mac = at.n_mac, n_sfu = at.n_sfu, br = at.br, cyc1 = at.cyc1, cyc2 = at.cyc2;
     const int64_t n_gb = n_dram + br;
     const int64_t n_rf = p.has_rf ? br + 3 * n_mac : 0;
 

@@ -3,7 +3,7 @@
 // Work decomposition.  A "task" is one (tiling, fusion mode, order, levels of A, B, C) choice; its
 // 25 rows are the levels of D and E and each row has 9 stationary pairs, so a task is 225
 // consecutive candidate indices: idx = task*225 + row*9 + s.  One thread owns one task at a time
-// and walks it in ascending index order, entirely in registers.
+// and walks it in ascending index order.
 //
 // The cost of a mapping is separable over operands (Section V-B/V-C: BS and DA are sums of
 // per-operand monomials; Section V-D: energy is linear in the access counts), so the query-matrix
@@ -29,18 +29,27 @@ constexpr unsigned kFull = 0xffffffffu;
 // shared-memory tables
 // ------------------------------------------------------------------------------------------------
 
-// Per (tiling, order): operand terms by level.  "g" entries are DRAM words times the objective's
-// scale (energy: quanta per DRAM word; latency/EDP: 1); "e" entries (EDP only) are the
-// energy-scaled copies.
+// Row-side terms (levels of D and E) of one (tiling, order), in the form the row loop consumes:
+// x1 = buffer words counted while Op1 runs (the operand's size if it is retained, else 0),
+// x2 = buffer words while Op2 runs, g = DRAM words times the objective's scale (energy: quanta
+// per DRAM word; latency / EDP: 1), e = energy-scaled copy (EDP only).  One instance for fused
+// rows, one for unfused rows, so that the loops need no selects.
+struct RowTab {
+    int64_t D1[5], D2[5], gD[5], eD[5];
+    int64_t E1[5], E2[5], gE[5], eE[5];
+};
+
+// Per (tiling, order): task-side terms (levels of A, B, C) and the two row tables.
 struct OrderTab {
-    int64_t A1[5], gA[5][2], B1[5], gB[5][2], C1[5];
-    int64_t D2[5], gD[5], gDu[5], E2[5], gE[5], gEu[5];
-    int64_t gCr;
-    int64_t eA[5][2], eB[5][2], eD[5], eDu[5], eE[5], eEu[5], eCr;
+    int64_t A1[5], A2[5], gA[5][2], eA[5][2];     // [level][recompute]; A2 = size if retained
+    int64_t B1[5], B2[5], gB[5][2], eB[5][2];
+    int64_t C1[5];
+    int64_t gCr, eCr;                             // unfused: C read back by Op2
     uint32_t rc[5];
     uint32_t pad;
+    RowTab rt[2];                                 // 0 fused, 1 unfused
 };
-constexpr int kOrderEntries = 66;
+constexpr int kOrderItems = 26;
 
 // Per tiling: array-level terms by stationary pair and recompute flag.
 struct TilingTab {
@@ -53,6 +62,7 @@ struct TilingTab {
     int32_t live;           // smallest possible buffer need of this tiling fits
     int32_t pad;
 };
+constexpr int kTilingItems = 21;    // 9 stationary pairs x 2 recompute flags, 3 unfused Op1 terms
 
 struct WarpTop {
     int64_t key[MMEE_MAX_TOPK];
@@ -116,27 +126,33 @@ __device__ __forceinline__ int64_t candidate_key(int64_t x, int64_t xe, int64_t 
     }
 }
 
-// One compare per candidate, OR-ed into one predicate.  Written as PTX so that the nine compares
-// against the common threshold stay nine compares: the compiler otherwise rewrites
-// (a < t) | (b < t) into min(a, b) < t, and a 64-bit min costs more than the compare it saves.
-__device__ __forceinline__ unsigned any_below(const int64_t (&k)[9], int64_t thr) {
-    unsigned r;
+// One row: the capacity test of Eq. (4) (e1 <= s1 and e2 <= s2: the two operator buffer sizes
+// against their slacks) and one compare per candidate key, OR-ed into one predicate.  Written as
+// PTX so that the nine compares against the common threshold stay nine compares: the compiler
+// otherwise rewrites (a < t) | (b < t) into min(a, b) < t, and a 64-bit min costs more than the
+// compare it saves.  Results as integers: fit = the row fits; hit = it fits and some key < thr.
+__device__ __forceinline__ void row_test(const int64_t (&k)[9], int64_t thr, int64_t e1, int64_t s1,
+                                         int64_t e2, int64_t s2, unsigned& fit, unsigned& hit) {
     asm("{\n\t"
-        ".reg .pred p;\n\t"
-        "setp.lt.s64 p, %1, %10;\n\t"
-        "setp.lt.or.s64 p, %2, %10, p;\n\t"
-        "setp.lt.or.s64 p, %3, %10, p;\n\t"
-        "setp.lt.or.s64 p, %4, %10, p;\n\t"
-        "setp.lt.or.s64 p, %5, %10, p;\n\t"
-        "setp.lt.or.s64 p, %6, %10, p;\n\t"
-        "setp.lt.or.s64 p, %7, %10, p;\n\t"
-        "setp.lt.or.s64 p, %8, %10, p;\n\t"
-        "setp.lt.or.s64 p, %9, %10, p;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t"
+        ".reg .pred p, q;\n\t"
+        "setp.le.s64 q, %12, %13;\n\t"
+        "setp.le.and.s64 q, %14, %15, q;\n\t"
+        "setp.lt.s64 p, %2, %11;\n\t"
+        "setp.lt.or.s64 p, %3, %11, p;\n\t"
+        "setp.lt.or.s64 p, %4, %11, p;\n\t"
+        "setp.lt.or.s64 p, %5, %11, p;\n\t"
+        "setp.lt.or.s64 p, %6, %11, p;\n\t"
+        "setp.lt.or.s64 p, %7, %11, p;\n\t"
+        "setp.lt.or.s64 p, %8, %11, p;\n\t"
+        "setp.lt.or.s64 p, %9, %11, p;\n\t"
+        "setp.lt.or.s64 p, %10, %11, p;\n\t"
+        "and.pred p, p, q;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t"
+        "selp.u32 %1, 1, 0, p;\n\t"
         "}"
-        : "=r"(r)
-        : "l"(k[0]), "l"(k[1]), "l"(k[2]), "l"(k[3]), "l"(k[4]), "l"(k[5]), "l"(k[6]), "l"(k[7]), "l"(k[8]), "l"(thr));
-    return r;
+        : "=r"(fit), "=r"(hit)
+        : "l"(k[0]), "l"(k[1]), "l"(k[2]), "l"(k[3]), "l"(k[4]), "l"(k[5]), "l"(k[6]), "l"(k[7]), "l"(k[8]), "l"(thr),
+          "l"(e1), "l"(s1), "l"(e2), "l"(s2));
 }
 
 // Rare path: some lane of the warp has a key below its threshold in this row.  Every lane
@@ -175,86 +191,83 @@ __device__ __noinline__ int64_t slow_row(WarpTop* wt, CtaShared* cs, int k, int 
 // table construction
 // ------------------------------------------------------------------------------------------------
 
+// One thread per (tiling slot, order, item): the monomials of one operand at one level.
 template <int OBJ>
-__device__ __forceinline__ void build_order_entry(const Plan& p, const uint32_t* b, uint32_t order, OrderTab* ot, int e) {
+__device__ __forceinline__ void build_order_item(const Plan& p, const uint32_t* b, uint32_t order, OrderTab* ot, int item) {
     const QueryTables& q = p.q;
     const int64_t scale = (OBJ == MMEE_OBJ_ENERGY) ? p.c_dram_gb : 1;
     const int64_t escale = p.c_dram_gb;
-    if (e < 5) {
-        ot->A1[e] = monomial(q.bs[order][OP_A][e], b);
-    } else if (e < 15) {
-        const int l = (e - 5) >> 1, rc = (e - 5) & 1;
-        const int64_t v = monomial(q.da[order][OP_A][l][rc], b);
-        ot->gA[l][rc] = scale * v;
-        if (OBJ == MMEE_OBJ_EDP) ot->eA[l][rc] = escale * v;
-    } else if (e < 20) {
-        ot->B1[e - 15] = monomial(q.bs[order][OP_B][e - 15], b);
-    } else if (e < 30) {
-        const int l = (e - 20) >> 1, rc = (e - 20) & 1;
-        const int64_t v = monomial(q.da[order][OP_B][l][rc], b);
-        ot->gB[l][rc] = scale * v;
-        if (OBJ == MMEE_OBJ_EDP) ot->eB[l][rc] = escale * v;
-    } else if (e < 35) {
-        ot->C1[e - 30] = monomial(q.bs[order][OP_C][e - 30], b);
-        ot->rc[e - 30] = q.recompute[order][e - 30];
-    } else if (e < 40) {
-        ot->D2[e - 35] = monomial(q.bs[order][OP_D][e - 35], b);
-    } else if (e < 45) {
-        const int64_t v = monomial(q.da[order][OP_D][e - 40][0], b);
-        ot->gD[e - 40] = scale * v;
-        if (OBJ == MMEE_OBJ_EDP) ot->eD[e - 40] = escale * v;
-    } else if (e < 50) {
-        const int64_t v = monomial(q.da_unfused[order][OP_D][e - 45], b);
-        ot->gDu[e - 45] = scale * v;
-        if (OBJ == MMEE_OBJ_EDP) ot->eDu[e - 45] = escale * v;
-    } else if (e < 55) {
-        ot->E2[e - 50] = monomial(q.bs[order][OP_E][e - 50], b);
-    } else if (e < 60) {
-        const int64_t v = monomial(q.da[order][OP_E][e - 55][0], b);
-        ot->gE[e - 55] = scale * v;
-        if (OBJ == MMEE_OBJ_EDP) ot->eE[e - 55] = escale * v;
-    } else if (e < 65) {
-        const int64_t v = monomial(q.da_unfused[order][OP_E][e - 60], b);
-        ot->gEu[e - 60] = scale * v;
-        if (OBJ == MMEE_OBJ_EDP) ot->eEu[e - 60] = escale * v;
+    const int l = item % 5;
+    if (item < 10) {                                   // A, B
+        const int x = item < 5 ? OP_A : OP_B;
+        const int64_t bs = monomial(q.bs[order][x][l], b);
+        const int64_t v0 = monomial(q.da[order][x][l][0], b), v1 = monomial(q.da[order][x][l][1], b);
+        int64_t* s1 = x == OP_A ? ot->A1 : ot->B1;
+        int64_t* s2 = x == OP_A ? ot->A2 : ot->B2;
+        int64_t (*g)[2] = x == OP_A ? ot->gA : ot->gB;
+        int64_t (*e)[2] = x == OP_A ? ot->eA : ot->eB;
+        s1[l] = bs;
+        s2[l] = l ? bs : 0;                            // retained (tau = 1) from L4 upwards
+        g[l][0] = scale * v0;
+        g[l][1] = scale * v1;
+        if (OBJ == MMEE_OBJ_EDP) { e[l][0] = escale * v0; e[l][1] = escale * v1; }
+    } else if (item < 15) {                            // C
+        ot->C1[l] = monomial(q.bs[order][OP_C][l], b);
+        ot->rc[l] = q.recompute[order][l];
+    } else if (item < 25) {                            // D, E
+        const int x = item < 20 ? OP_D : OP_E;
+        const int64_t bs = monomial(q.bs[order][x][l], b);
+        const int64_t vf = monomial(q.da[order][x][l][0], b);
+        const int64_t vu = monomial(q.da_unfused[order][x][l], b);
+        RowTab* f = &ot->rt[0];
+        RowTab* u = &ot->rt[1];
+        if (x == OP_D) {
+            f->D1[l] = l ? bs : 0; f->D2[l] = bs; f->gD[l] = scale * vf;
+            u->D1[l] = 0;          u->D2[l] = bs; u->gD[l] = scale * vu;
+            if (OBJ == MMEE_OBJ_EDP) { f->eD[l] = escale * vf; u->eD[l] = escale * vu; }
+        } else {
+            f->E1[l] = l ? bs : 0; f->E2[l] = bs; f->gE[l] = scale * vf;
+            u->E1[l] = 0;          u->E2[l] = bs; u->gE[l] = scale * vu;
+            if (OBJ == MMEE_OBJ_EDP) { f->eE[l] = escale * vf; u->eE[l] = escale * vu; }
+        }
     } else {
         const int64_t v = monomial(q.da_unfused[order][OP_C][0], b);
         ot->gCr = scale * v;
-        if (OBJ == MMEE_OBJ_EDP) ot->eCr = escale * v;
+        ot->eCr = escale * v;
     }
 }
 
-// One thread per tiling slot: bounds, array-level terms, liveness.
-__device__ __forceinline__ void build_tiling_tab(const Plan& p, uint64_t t, TilingTab* tb) {
+// One thread per tiling slot: bounds, liveness, the terms that need no division.
+__device__ __forceinline__ void build_tiling_head(const Plan& p, uint64_t t, TilingTab* tb) {
     uint32_t b[8];
     tiling_bounds(p, t, b);
-    TilingTerms tt;
-    tiling_terms(p, b, tt);
 #pragma unroll
     for (int d = 0; d < 8; ++d) tb->b[d] = b[d];
-    const int64_t bw = p.bw;
-    for (int s = 0; s < 9; ++s) {
-        const int sm1 = s / 3, sm2 = s % 3;
-        for (int rc = 0; rc < 2; ++rc) {
-            const int64_t rho = rc ? (int64_t)b[3] : 1;
-            const int64_t t1 = rho * tt.t1;
-            const int64_t br = t1 * tt.br1[sm1] + rho * tt.carry1 + tt.t2 * tt.br2[sm2] + tt.carry2;
-            const int64_t n_mac = rho * tt.ikl + tt.ilj;
-            const int64_t n_sfu = rho * tt.il;
-            tb->W[s][rc] = p.c_br * br + p.c_mac * n_mac + p.c_sfu * n_sfu;
-            tb->CB[s][rc] = (t1 * tt.cy1[sm1] + tt.t2 * tt.cy2[sm2]) * bw;
-            tb->QU[s][rc] = tt.t2 * tt.cy2[sm2] * bw;
-        }
-    }
-    for (int sm1 = 0; sm1 < 3; ++sm1) tb->C1w[sm1] = tt.t1 * tt.cy1[sm1] * bw;
-    tb->cw = tt.il;
-    tb->smx = 2 * tt.il;
+    const int64_t il = (int64_t)p.dim[0] * p.dim[2];
+    tb->cw = il;
+    tb->smx = 2 * il;
     // With every operand at L3 the buffer need is smallest: max(A+B+C, C+D+E) tiles (Eq. 1-4).
     const int64_t ta = (int64_t)b[4] * b[5], tbb = (int64_t)b[5] * b[6], tc = (int64_t)b[4] * b[6];
     const int64_t td = (int64_t)b[6] * b[7], te = (int64_t)b[4] * b[7];
     const int64_t need1 = ta + tbb + tc, need2 = tc + td + te;
     tb->live = ((need1 > need2 ? need1 : need2) <= p.cap_words) ? 1 : 0;
     tb->pad = 0;
+}
+
+// One thread per (tiling slot, item): stationary-pair terms with the cost coefficients applied.
+__device__ __forceinline__ void build_tiling_item(const Plan& p, TilingTab* tb, int item) {
+    const TilingCounts c = tiling_counts(p, tb->b);
+    const int64_t bw = p.bw;
+    if (item < 18) {
+        const int s = item >> 1, rc = item & 1;
+        const ArrayTerms a = array_terms(p, tb->b, c, s / 3, s % 3, rc != 0);
+        tb->W[s][rc] = p.c_br * a.br + p.c_mac * a.n_mac + p.c_sfu * a.n_sfu;
+        tb->CB[s][rc] = (a.cyc1 + a.cyc2) * bw;
+        tb->QU[s][rc] = a.cyc2 * bw;
+    } else {
+        const int sm1 = item - 18;
+        tb->C1w[sm1] = c.t1 * tile_cycles(sm1, tb->b[4], tb->b[5], tb->b[6], p.pe_rows, p.pe_cols) * bw;
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -306,44 +319,56 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
         const uint32_t n_slots = (uint32_t)(t_last - t_first + 1);
 
         // ---- tables of the tilings this range touches
-        if (tid < (int)n_slots) build_tiling_tab(p, t_first + tid, &ttabs[tid]);
+        if (tid < (int)n_slots) build_tiling_head(p, t_first + tid, &ttabs[tid]);
         __syncthreads();
-        const uint32_t items = n_slots * n_orders * kOrderEntries;
+        const uint32_t order_items = n_slots * n_orders * kOrderItems;
+        const uint32_t items = order_items + n_slots * kTilingItems;
         for (uint32_t it = tid; it < items; it += kSearchThreads) {
-            const uint32_t e = it % kOrderEntries;
-            const uint32_t so = it / kOrderEntries;
-            const uint32_t slot = so / n_orders, os = so % n_orders;
-            if (!ttabs[slot].live) continue;
-            build_order_entry<OBJ>(p, ttabs[slot].b, p.order_id[os], &otabs[slot * n_orders + os], (int)e);
+            if (it < order_items) {
+                const uint32_t e = it % kOrderItems;
+                const uint32_t so = it / kOrderItems;
+                const uint32_t slot = so / n_orders, os = so % n_orders;
+                if (!ttabs[slot].live) continue;
+                build_order_item<OBJ>(p, ttabs[slot].b, p.order_id[os], &otabs[slot * n_orders + os], (int)e);
+            } else {
+                const uint32_t j = it - order_items;
+                const uint32_t slot = j / kTilingItems;
+                if (!ttabs[slot].live) continue;
+                build_tiling_item(p, &ttabs[slot], (int)(j - slot * kTilingItems));
+            }
         }
         __syncthreads();
 
         // ---- tasks
-        for (uint64_t base = r0; base < r1; base += kSearchThreads) {
-            const uint64_t task = base + tid;
-            const bool valid = task < r1;
-            const uint64_t tq = valid ? task : r1 - 1;
-            const uint64_t t = tq / tpt;
-            const uint32_t w = (uint32_t)(tq - t * tpt);
-            const uint32_t slot = (uint32_t)(t - t_first);
+        const uint32_t w_first = (uint32_t)(r0 - t_first * tpt);      // task of r0 inside its tiling
+        const uint32_t n_range = (uint32_t)(r1 - r0);
+        for (uint32_t off = 0; off < n_range; off += kSearchThreads) {
+            const bool valid = off + tid < n_range;
+            const uint32_t o = valid ? off + tid : n_range - 1;
+            const uint32_t wa = w_first + o;
+            const uint32_t slot = wa / tpt;
+            const uint32_t w = wa - slot * tpt;
+            const uint64_t tq = r0 + o;
             const TilingTab* tb = &ttabs[slot];
             const bool live = valid && tb->live;
             if (DUMP && valid && !tb->live) {
-                for (int c = 0; c < kCandPerTask; ++c) dump[task * kCandPerTask - dump_origin + c] = kInfKey;
+                for (int c = 0; c < kCandPerTask; ++c) dump[tq * kCandPerTask - dump_origin + c] = kInfKey;
             }
             if (!__any_sync(kFull, live)) continue;
 
             const TaskChoice c = decode_task(p, w);
             const OrderTab* ot = &otabs[slot * n_orders + c.order_slot];
             const bool fused = c.phi == 0;
+            const RowTab* rt = &ot->rt[fused ? 0 : 1];
             // Tables of a tiling that cannot fit are never built: a lane whose task lies in such a
             // tiling must not index with what it reads from them.
             const uint32_t rc = (fused && live) ? (ot->rc[c.lc] & 1u) : 0u;
             const int64_t a1 = ot->A1[c.la], b1 = ot->B1[c.lb], c1 = ot->C1[c.lc];
+            const int64_t a2 = fused ? ot->A2[c.la] : 0, b2 = fused ? ot->B2[c.lb] : 0;
             // Eq. (1)/(2): a retained operand (level >= L4) of the other operator keeps its space.
             // A lane without a live task gets a negative slack, so that none of its rows fits.
             const int64_t slack1 = live ? cap - (a1 + b1 + c1) : -1;
-            const int64_t slack2 = live ? cap - (c1 + ((fused && c.la) ? a1 : 0) + ((fused && c.lb) ? b1 : 0)) : -1;
+            const int64_t slack2 = live ? cap - (c1 + a2 + b2) : -1;
             const int64_t gab = ot->gA[c.la][rc] + ot->gB[c.lb][rc];
 
             int64_t x0, xe0 = 0, P[3], Q[9], W[9];
@@ -378,49 +403,42 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                 W[s] = wptr[2 * s];
                 Q[s] = qptr[2 * s];
             }
-            int64_t E1[5], E2[5], gE[5], eE[5];
-#pragma unroll
-            for (int e = 0; e < 5; ++e) {
-                E2[e] = ot->E2[e];
-                E1[e] = (fused && e) ? E2[e] : 0;
-                gE[e] = fused ? ot->gE[e] : ot->gEu[e];
-                eE[e] = (OBJ == MMEE_OBJ_EDP) ? (fused ? ot->eE[e] : ot->eEu[e]) : 0;
-            }
             const uint64_t task_first_idx = tq * kCandPerTask;
             int64_t thr = lane_threshold(wt, cs, k, task_first_idx);
             uint32_t rows = 0;
 
 #pragma unroll 1
             for (int d = 0; d < 5; ++d) {
-                const int64_t d2 = ot->D2[d];
-                const int64_t s1 = slack1 - ((fused && d) ? d2 : 0);
-                const int64_t s2 = slack2 - d2;
-                const int64_t xd = x0 + (fused ? ot->gD[d] : ot->gDu[d]);
-                const int64_t xed = (OBJ == MMEE_OBJ_EDP) ? xe0 + (fused ? ot->eD[d] : ot->eDu[d]) : 0;
+                const int64_t s1 = slack1 - rt->D1[d];
+                const int64_t s2 = slack2 - rt->D2[d];
+                const int64_t xd = x0 + rt->gD[d];
+                const int64_t xed = (OBJ == MMEE_OBJ_EDP) ? xe0 + rt->eD[d] : 0;
                 // Five rows (levels of E) are evaluated branch-free; one vote decides whether any
                 // lane of the warp has to enter the insertion path for this group.
                 unsigned fit[5], hit[5];
 #pragma unroll
                 for (int e = 0; e < 5; ++e) {
-                    fit[e] = (unsigned)(E1[e] <= s1) & (unsigned)(E2[e] <= s2);   // Eq. (4) against the capacity
-                    rows += fit[e];
-                    const int64_t x = xd + gE[e];
-                    const int64_t xe = xed + eE[e];
+                    const int64_t x = xd + rt->gE[e];
+                    const int64_t xe = (OBJ == MMEE_OBJ_EDP) ? xed + rt->eE[e] : 0;
                     int64_t key[9];
 #pragma unroll
-                    for (int s = 0; s < 9; ++s) {
-                        key[s] = candidate_key<OBJ>(x, xe, W[s], P[s / 3], Q[s]);
-                        if (DUMP) {
-                            if (valid) dump[task_first_idx - dump_origin + (d * 5 + e) * 9 + s] = fit[e] ? key[s] : kInfKey;
+                    for (int s = 0; s < 9; ++s) key[s] = candidate_key<OBJ>(x, xe, W[s], P[s / 3], Q[s]);
+                    row_test(key, thr, rt->E1[e], s1, rt->E2[e], s2, fit[e], hit[e]);
+                    rows += fit[e];
+                    if (DUMP) {
+                        if (valid) {
+#pragma unroll
+                            for (int s = 0; s < 9; ++s)
+                                dump[task_first_idx - dump_origin + (d * 5 + e) * 9 + s] = fit[e] ? key[s] : kInfKey;
                         }
                     }
-                    hit[e] = any_below(key, thr) & fit[e];
                 }
                 if (__any_sync(kFull, (hit[0] | hit[1] | hit[2] | hit[3] | hit[4]) != 0u)) {
 #pragma unroll
                     for (int e = 0; e < 5; ++e) {
                         if (__any_sync(kFull, hit[e] != 0u)) {
-                            thr = slow_row<OBJ>(wt, cs, k, lane, fit[e] != 0u, xd + gE[e], xed + eE[e], wptr, qptr,
+                            thr = slow_row<OBJ>(wt, cs, k, lane, fit[e] != 0u, xd + rt->gE[e],
+                                                (OBJ == MMEE_OBJ_EDP) ? xed + rt->eE[e] : 0, wptr, qptr,
                                                 P[0], P[1], P[2],
                                                 task_first_idx + (uint64_t)((d * 5 + e) * 9), task_first_idx);
                         }
