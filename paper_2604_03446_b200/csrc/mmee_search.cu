@@ -16,6 +16,8 @@
 // tables of the (at most a few) tilings the range touches.
 #include <cuda_runtime.h>
 
+#include <cstddef>
+
 #include "mmee_eval.cuh"
 #include "mmee_search.h"
 
@@ -34,13 +36,14 @@ constexpr unsigned kFull = 0xffffffffu;
 // x2 = buffer words while Op2 runs, g = DRAM words times the objective's scale (energy: quanta
 // per DRAM word; latency / EDP: 1), e = energy-scaled copy (EDP only).  One instance for fused
 // rows, one for unfused rows, so that the loops need no selects.
-struct RowTab {
-    int64_t D1[5], D2[5], gD[5], eD[5];
-    int64_t E1[5], E2[5], gE[5], eE[5];
+struct alignas(16) RowTab {
+    int64_t D[5][4];        // per level of D: x1, x2, g, e
+    int64_t E[5][4];        // per level of E: x1, x2, g, e
 };
+static_assert(sizeof(RowTab) == 320 && offsetof(RowTab, E) == 160, "the row loop addresses RowTab by byte offset");
 
 // Per (tiling, order): task-side terms (levels of A, B, C) and the two row tables.
-struct OrderTab {
+struct alignas(16) OrderTab {
     int64_t A1[5], A2[5], gA[5][2], eA[5][2];     // [level][recompute]; A2 = size if retained
     int64_t B1[5], B2[5], gB[5][2], eB[5][2];
     int64_t C1[5];
@@ -52,7 +55,7 @@ struct OrderTab {
 constexpr int kOrderItems = 26;
 
 // Per tiling: array-level terms by stationary pair and recompute flag.
-struct TilingTab {
+struct alignas(16) TilingTab {
     uint32_t b[8];
     int64_t W[9][2];        // energy of buffer<->PE traffic, MACs and softmax, in quanta
     int64_t CB[9][2];       // fused compute time in words (cycles * words per cycle)
@@ -64,14 +67,14 @@ struct TilingTab {
 };
 constexpr int kTilingItems = 21;    // 9 stationary pairs x 2 recompute flags, 3 unfused Op1 terms
 
-struct WarpTop {
+struct alignas(16) WarpTop {
     int64_t key[MMEE_MAX_TOPK];
     uint64_t idx[MMEE_MAX_TOPK];
     int32_t count;
     int32_t pad;
 };
 
-struct CtaShared {
+struct alignas(16) CtaShared {
     long long G;             // upper bound on the final k-th smallest key (any full list's last key)
     unsigned long long feasible_rows;
     unsigned long long range_begin;
@@ -155,6 +158,101 @@ __device__ __forceinline__ void row_test(const int64_t (&k)[9], int64_t thr, int
           "l"(e1), "l"(s1), "l"(e2), "l"(s2));
 }
 
+// One group of five rows (levels of E at one level of D) in PTX: per row two 16-byte loads from the
+// row table, the row's base sum, the capacity test and nine add + compare pairs whose results
+// are OR-ed into one predicate for the group.  Outputs: hit = some fitting row has a key below
+// thr; fits = number of rows that fit.  rt_saddr is the shared-memory address of the RowTab.
+#define MMEE_ROW_HEAD(o1, o2)                                   \
+    "ld.shared.v2.s64 {e1, e2}, [%15+" o1 "];\n\t"              \
+    "ld.shared.v2.s64 {g, ge}, [%15+" o2 "];\n\t"               \
+    "add.s64 x, %2, g;\n\t"                                     \
+    "setp.le.s64 q, e1, %3;\n\t"                                \
+    "setp.le.and.s64 q, e2, %4, q;\n\t"
+#define MMEE_ROW_TAIL                                           \
+    "and.pred p, p, q;\n\t"                                     \
+    "or.pred h, h, p;\n\t"                                      \
+    "selp.u32 t, 1, 0, q;\n\t"                                  \
+    "add.u32 c, c, t;\n\t"
+#define MMEE_ENERGY_ROW(o1, o2)                                 \
+    MMEE_ROW_HEAD(o1, o2)                                       \
+    "add.s64 k, x, %6;\n\t"  "setp.lt.s64 p, k, %5;\n\t"        \
+    "add.s64 k, x, %7;\n\t"  "setp.lt.or.s64 p, k, %5, p;\n\t"  \
+    "add.s64 k, x, %8;\n\t"  "setp.lt.or.s64 p, k, %5, p;\n\t"  \
+    "add.s64 k, x, %9;\n\t"  "setp.lt.or.s64 p, k, %5, p;\n\t"  \
+    "add.s64 k, x, %10;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"  \
+    "add.s64 k, x, %11;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"  \
+    "add.s64 k, x, %12;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"  \
+    "add.s64 k, x, %13;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"  \
+    "add.s64 k, x, %14;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"  \
+    MMEE_ROW_TAIL
+
+__device__ __forceinline__ void group_test_energy(int64_t xd, int64_t s1, int64_t s2, int64_t thr,
+                                                  const int64_t (&W)[9], uint32_t rt_saddr,
+                                                  unsigned& hit, unsigned& fits) {
+    asm volatile("{\n\t"
+        ".reg .pred p, q, h;\n\t"
+        ".reg .s64 x, k, e1, e2, g, ge;\n\t"
+        ".reg .u32 c, t;\n\t"
+        "mov.u32 c, 0;\n\t"
+        "setp.ne.u32 h, 0, 0;\n\t"
+        MMEE_ENERGY_ROW("160", "176")
+        MMEE_ENERGY_ROW("192", "208")
+        MMEE_ENERGY_ROW("224", "240")
+        MMEE_ENERGY_ROW("256", "272")
+        MMEE_ENERGY_ROW("288", "304")
+        "selp.u32 %0, 1, 0, h;\n\t"
+        "mov.u32 %1, c;\n\t"
+        "}"
+        : "=r"(hit), "=r"(fits)
+        : "l"(xd), "l"(s1), "l"(s2), "l"(thr),
+          "l"(W[0]), "l"(W[1]), "l"(W[2]), "l"(W[3]), "l"(W[4]), "l"(W[5]), "l"(W[6]), "l"(W[7]), "l"(W[8]),
+          "r"(rt_saddr)
+        : "memory");
+}
+
+// Latency: key = max(x + P[s/3], Q[s] + P[s/3]) (= P + max(x, Q)); QP holds Q[s] + P[s/3].
+#define MMEE_LAT_ROW(o1, o2)                                                      \
+    "ld.shared.v2.s64 {e1, e2}, [%18+" o1 "];\n\t"                                \
+    "ld.shared.v2.s64 {g, ge}, [%18+" o2 "];\n\t"                                 \
+    "add.s64 x, %2, g;\n\t"                                                       \
+    "setp.le.s64 q, e1, %3;\n\t"                                                  \
+    "setp.le.and.s64 q, e2, %4, q;\n\t"                                           \
+    "add.s64 y0, x, %6;\n\t" "add.s64 y1, x, %7;\n\t" "add.s64 y2, x, %8;\n\t"    \
+    "max.s64 k, y0, %9;\n\t"  "setp.lt.s64 p, k, %5;\n\t"                         \
+    "max.s64 k, y0, %10;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"                   \
+    "max.s64 k, y0, %11;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"                   \
+    "max.s64 k, y1, %12;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"                   \
+    "max.s64 k, y1, %13;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"                   \
+    "max.s64 k, y1, %14;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"                   \
+    "max.s64 k, y2, %15;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"                   \
+    "max.s64 k, y2, %16;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"                   \
+    "max.s64 k, y2, %17;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"                   \
+    MMEE_ROW_TAIL
+
+__device__ __forceinline__ void group_test_latency(int64_t xd, int64_t s1, int64_t s2, int64_t thr,
+                                                   const int64_t (&P)[3], const int64_t (&QP)[9],
+                                                   uint32_t rt_saddr, unsigned& hit, unsigned& fits) {
+    asm volatile("{\n\t"
+        ".reg .pred p, q, h;\n\t"
+        ".reg .s64 x, k, e1, e2, g, ge, y0, y1, y2;\n\t"
+        ".reg .u32 c, t;\n\t"
+        "mov.u32 c, 0;\n\t"
+        "setp.ne.u32 h, 0, 0;\n\t"
+        MMEE_LAT_ROW("160", "176")
+        MMEE_LAT_ROW("192", "208")
+        MMEE_LAT_ROW("224", "240")
+        MMEE_LAT_ROW("256", "272")
+        MMEE_LAT_ROW("288", "304")
+        "selp.u32 %0, 1, 0, h;\n\t"
+        "mov.u32 %1, c;\n\t"
+        "}"
+        : "=r"(hit), "=r"(fits)
+        : "l"(xd), "l"(s1), "l"(s2), "l"(thr), "l"(P[0]), "l"(P[1]), "l"(P[2]),
+          "l"(QP[0]), "l"(QP[1]), "l"(QP[2]), "l"(QP[3]), "l"(QP[4]), "l"(QP[5]), "l"(QP[6]), "l"(QP[7]), "l"(QP[8]),
+          "r"(rt_saddr)
+        : "memory");
+}
+
 // Rare path: some lane of the warp has a key below its threshold in this row.  Every lane
 // re-evaluates its nine candidates of the row from the shared tables and the warp inserts the
 // passing ones, one at a time, into its sorted list.
@@ -221,15 +319,10 @@ __device__ __forceinline__ void build_order_item(const Plan& p, const uint32_t* 
         const int64_t vu = monomial(q.da_unfused[order][x][l], b);
         RowTab* f = &ot->rt[0];
         RowTab* u = &ot->rt[1];
-        if (x == OP_D) {
-            f->D1[l] = l ? bs : 0; f->D2[l] = bs; f->gD[l] = scale * vf;
-            u->D1[l] = 0;          u->D2[l] = bs; u->gD[l] = scale * vu;
-            if (OBJ == MMEE_OBJ_EDP) { f->eD[l] = escale * vf; u->eD[l] = escale * vu; }
-        } else {
-            f->E1[l] = l ? bs : 0; f->E2[l] = bs; f->gE[l] = scale * vf;
-            u->E1[l] = 0;          u->E2[l] = bs; u->gE[l] = scale * vu;
-            if (OBJ == MMEE_OBJ_EDP) { f->eE[l] = escale * vf; u->eE[l] = escale * vu; }
-        }
+        int64_t* fr = x == OP_D ? f->D[l] : f->E[l];
+        int64_t* ur = x == OP_D ? u->D[l] : u->E[l];
+        fr[0] = l ? bs : 0; fr[1] = bs; fr[2] = scale * vf; fr[3] = escale * vf;
+        ur[0] = 0;          ur[1] = bs; ur[2] = scale * vu; ur[3] = escale * vu;
     } else {
         const int64_t v = monomial(q.da_unfused[order][OP_C][0], b);
         ot->gCr = scale * v;
@@ -407,39 +500,59 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
             int64_t thr = lane_threshold(wt, cs, k, task_first_idx);
             uint32_t rows = 0;
 
+            const uint32_t rt_saddr = (uint32_t)__cvta_generic_to_shared(rt);
+            int64_t QP[9];
+#pragma unroll
+            for (int s = 0; s < 9; ++s) QP[s] = Q[s] + P[s / 3];
+
 #pragma unroll 1
             for (int d = 0; d < 5; ++d) {
-                const int64_t s1 = slack1 - rt->D1[d];
-                const int64_t s2 = slack2 - rt->D2[d];
-                const int64_t xd = x0 + rt->gD[d];
-                const int64_t xed = (OBJ == MMEE_OBJ_EDP) ? xe0 + rt->eD[d] : 0;
+                const int64_t s1 = slack1 - rt->D[d][0];
+                const int64_t s2 = slack2 - rt->D[d][1];
+                const int64_t xd = x0 + rt->D[d][2];
+                const int64_t xed = (OBJ == MMEE_OBJ_EDP) ? xe0 + rt->D[d][3] : 0;
                 // Five rows (levels of E) are evaluated branch-free; one vote decides whether any
                 // lane of the warp has to enter the insertion path for this group.
-                unsigned fit[5], hit[5];
+                unsigned hit_any, fits;
+                if constexpr (!DUMP && OBJ == MMEE_OBJ_ENERGY) {
+                    group_test_energy(xd, s1, s2, thr, W, rt_saddr, hit_any, fits);
+                } else if constexpr (!DUMP && OBJ == MMEE_OBJ_LATENCY) {
+                    group_test_latency(xd, s1, s2, thr, P, QP, rt_saddr, hit_any, fits);
+                } else {
+                    hit_any = 0; fits = 0;
 #pragma unroll
-                for (int e = 0; e < 5; ++e) {
-                    const int64_t x = xd + rt->gE[e];
-                    const int64_t xe = (OBJ == MMEE_OBJ_EDP) ? xed + rt->eE[e] : 0;
-                    int64_t key[9];
+                    for (int e = 0; e < 5; ++e) {
+                        const int64_t x = xd + rt->E[e][2];
+                        const int64_t xe = (OBJ == MMEE_OBJ_EDP) ? xed + rt->E[e][3] : 0;
+                        int64_t key[9];
 #pragma unroll
-                    for (int s = 0; s < 9; ++s) key[s] = candidate_key<OBJ>(x, xe, W[s], P[s / 3], Q[s]);
-                    row_test(key, thr, rt->E1[e], s1, rt->E2[e], s2, fit[e], hit[e]);
-                    rows += fit[e];
-                    if (DUMP) {
-                        if (valid) {
+                        for (int s = 0; s < 9; ++s) key[s] = candidate_key<OBJ>(x, xe, W[s], P[s / 3], Q[s]);
+                        unsigned fit, hit;
+                        row_test(key, thr, rt->E[e][0], s1, rt->E[e][1], s2, fit, hit);
+                        fits += fit;
+                        hit_any |= hit;
+                        if (DUMP) {
+                            if (valid) {
 #pragma unroll
-                            for (int s = 0; s < 9; ++s)
-                                dump[task_first_idx - dump_origin + (d * 5 + e) * 9 + s] = fit[e] ? key[s] : kInfKey;
+                                for (int s = 0; s < 9; ++s)
+                                    dump[task_first_idx - dump_origin + (d * 5 + e) * 9 + s] = fit ? key[s] : kInfKey;
+                            }
                         }
                     }
                 }
-                if (__any_sync(kFull, (hit[0] | hit[1] | hit[2] | hit[3] | hit[4]) != 0u)) {
-#pragma unroll
+                rows += fits;
+                if (__any_sync(kFull, hit_any != 0u)) {
+                    // rare: find the rows that passed and let the warp insert their candidates
+#pragma unroll 1
                     for (int e = 0; e < 5; ++e) {
-                        if (__any_sync(kFull, hit[e] != 0u)) {
-                            thr = slow_row<OBJ>(wt, cs, k, lane, fit[e] != 0u, xd + rt->gE[e],
-                                                (OBJ == MMEE_OBJ_EDP) ? xed + rt->eE[e] : 0, wptr, qptr,
-                                                P[0], P[1], P[2],
+                        const bool fit = (rt->E[e][0] <= s1) && (rt->E[e][1] <= s2);
+                        const int64_t x = xd + rt->E[e][2];
+                        const int64_t xe = (OBJ == MMEE_OBJ_EDP) ? xed + rt->E[e][3] : 0;
+                        bool below = false;
+                        for (int s = 0; s < 9; ++s)
+                            below |= candidate_key<OBJ>(x, xe, wptr[2 * s], P[s / 3], qptr[2 * s]) < thr;
+                        if (__any_sync(kFull, fit && below)) {
+                            thr = slow_row<OBJ>(wt, cs, k, lane, fit, x, xe, wptr, qptr, P[0], P[1], P[2],
                                                 task_first_idx + (uint64_t)((d * 5 + e) * 9), task_first_idx);
                         }
                     }
