@@ -16,6 +16,7 @@
 // tables of the (at most a few) tilings the range touches.
 #include <cuda_runtime.h>
 
+#include <climits>
 #include <cstddef>
 
 #include "mmee_eval.cuh"
@@ -158,99 +159,28 @@ __device__ __forceinline__ void row_test(const int64_t (&k)[9], int64_t thr, int
           "l"(e1), "l"(s1), "l"(e2), "l"(s2));
 }
 
-// One group of five rows (levels of E at one level of D) in PTX: per row two 16-byte loads from the
-// row table, the row's base sum, the capacity test and nine add + compare pairs whose results
-// are OR-ed into one predicate for the group.  Outputs: hit = some fitting row has a key below
-// thr; fits = number of rows that fit.  rt_saddr is the shared-memory address of the RowTab.
-#define MMEE_ROW_HEAD(o1, o2)                                   \
-    "ld.shared.v2.s64 {e1, e2}, [%15+" o1 "];\n\t"              \
-    "ld.shared.v2.s64 {g, ge}, [%15+" o2 "];\n\t"               \
-    "add.s64 x, %2, g;\n\t"                                     \
-    "setp.le.s64 q, e1, %3;\n\t"                                \
-    "setp.le.and.s64 q, e2, %4, q;\n\t"
-#define MMEE_ROW_TAIL                                           \
-    "and.pred p, p, q;\n\t"                                     \
-    "or.pred h, h, p;\n\t"                                      \
-    "selp.u32 t, 1, 0, q;\n\t"                                  \
-    "add.u32 c, c, t;\n\t"
-#define MMEE_ENERGY_ROW(o1, o2)                                 \
-    MMEE_ROW_HEAD(o1, o2)                                       \
-    "add.s64 k, x, %6;\n\t"  "setp.lt.s64 p, k, %5;\n\t"        \
-    "add.s64 k, x, %7;\n\t"  "setp.lt.or.s64 p, k, %5, p;\n\t"  \
-    "add.s64 k, x, %8;\n\t"  "setp.lt.or.s64 p, k, %5, p;\n\t"  \
-    "add.s64 k, x, %9;\n\t"  "setp.lt.or.s64 p, k, %5, p;\n\t"  \
-    "add.s64 k, x, %10;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"  \
-    "add.s64 k, x, %11;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"  \
-    "add.s64 k, x, %12;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"  \
-    "add.s64 k, x, %13;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"  \
-    "add.s64 k, x, %14;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"  \
-    MMEE_ROW_TAIL
+// ------------------------------------------------------------------------------------------------
+// 32-bit differential keys
+// ------------------------------------------------------------------------------------------------
+// Whether a candidate enters the top-k depends only on the sign of key - thr.  The row loop
+// therefore evaluates every candidate's key RELATIVE to the current threshold, saturated to 32
+// bits, and keeps the minimum over the group of five rows; a negative minimum sends the warp to
+// the exact 64-bit insertion path, which re-evaluates the rows in full.
+//
+// Energy: key = x + W[s].  With wmin = min_s W[s], B = thr - wmin, x' = x - B and W' = W - wmin >= 0:
+// key < thr  <=>  x' + W' < 0.  x' is saturated to [-2^31, 2^30 - 1] and W' to [0, 2^30].  If some
+// s of a row truly passes then either x' >= -2^31, where x' is exact and min(W', 2^30) <= W' keeps
+// the sum negative, or x' < -2^31, where s = argmin W (W' = 0) gives -2^31 < 0; conversely a
+// negative saturated sum implies x' < 0, i.e. the candidate with W' = 0 passes.  So a row is
+// flagged iff it holds a passing candidate, and no 32-bit sum can overflow.
+// Latency: key = max(x + P, Q + P); max(a, b) < thr <=> sat(a - thr) < 0 and sat(b - thr) < 0: exact
+// per candidate.
+constexpr int kRelCap = (1 << 30) - 1;
 
-__device__ __forceinline__ void group_test_energy(int64_t xd, int64_t s1, int64_t s2, int64_t thr,
-                                                  const int64_t (&W)[9], uint32_t rt_saddr,
-                                                  unsigned& hit, unsigned& fits) {
-    asm volatile("{\n\t"
-        ".reg .pred p, q, h;\n\t"
-        ".reg .s64 x, k, e1, e2, g, ge;\n\t"
-        ".reg .u32 c, t;\n\t"
-        "mov.u32 c, 0;\n\t"
-        "setp.ne.u32 h, 0, 0;\n\t"
-        MMEE_ENERGY_ROW("160", "176")
-        MMEE_ENERGY_ROW("192", "208")
-        MMEE_ENERGY_ROW("224", "240")
-        MMEE_ENERGY_ROW("256", "272")
-        MMEE_ENERGY_ROW("288", "304")
-        "selp.u32 %0, 1, 0, h;\n\t"
-        "mov.u32 %1, c;\n\t"
-        "}"
-        : "=r"(hit), "=r"(fits)
-        : "l"(xd), "l"(s1), "l"(s2), "l"(thr),
-          "l"(W[0]), "l"(W[1]), "l"(W[2]), "l"(W[3]), "l"(W[4]), "l"(W[5]), "l"(W[6]), "l"(W[7]), "l"(W[8]),
-          "r"(rt_saddr)
-        : "memory");
-}
-
-// Latency: key = max(x + P[s/3], Q[s] + P[s/3]) (= P + max(x, Q)); QP holds Q[s] + P[s/3].
-#define MMEE_LAT_ROW(o1, o2)                                                      \
-    "ld.shared.v2.s64 {e1, e2}, [%18+" o1 "];\n\t"                                \
-    "ld.shared.v2.s64 {g, ge}, [%18+" o2 "];\n\t"                                 \
-    "add.s64 x, %2, g;\n\t"                                                       \
-    "setp.le.s64 q, e1, %3;\n\t"                                                  \
-    "setp.le.and.s64 q, e2, %4, q;\n\t"                                           \
-    "add.s64 y0, x, %6;\n\t" "add.s64 y1, x, %7;\n\t" "add.s64 y2, x, %8;\n\t"    \
-    "max.s64 k, y0, %9;\n\t"  "setp.lt.s64 p, k, %5;\n\t"                         \
-    "max.s64 k, y0, %10;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"                   \
-    "max.s64 k, y0, %11;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"                   \
-    "max.s64 k, y1, %12;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"                   \
-    "max.s64 k, y1, %13;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"                   \
-    "max.s64 k, y1, %14;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"                   \
-    "max.s64 k, y2, %15;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"                   \
-    "max.s64 k, y2, %16;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"                   \
-    "max.s64 k, y2, %17;\n\t" "setp.lt.or.s64 p, k, %5, p;\n\t"                   \
-    MMEE_ROW_TAIL
-
-__device__ __forceinline__ void group_test_latency(int64_t xd, int64_t s1, int64_t s2, int64_t thr,
-                                                   const int64_t (&P)[3], const int64_t (&QP)[9],
-                                                   uint32_t rt_saddr, unsigned& hit, unsigned& fits) {
-    asm volatile("{\n\t"
-        ".reg .pred p, q, h;\n\t"
-        ".reg .s64 x, k, e1, e2, g, ge, y0, y1, y2;\n\t"
-        ".reg .u32 c, t;\n\t"
-        "mov.u32 c, 0;\n\t"
-        "setp.ne.u32 h, 0, 0;\n\t"
-        MMEE_LAT_ROW("160", "176")
-        MMEE_LAT_ROW("192", "208")
-        MMEE_LAT_ROW("224", "240")
-        MMEE_LAT_ROW("256", "272")
-        MMEE_LAT_ROW("288", "304")
-        "selp.u32 %0, 1, 0, h;\n\t"
-        "mov.u32 %1, c;\n\t"
-        "}"
-        : "=r"(hit), "=r"(fits)
-        : "l"(xd), "l"(s1), "l"(s2), "l"(thr), "l"(P[0]), "l"(P[1]), "l"(P[2]),
-          "l"(QP[0]), "l"(QP[1]), "l"(QP[2]), "l"(QP[3]), "l"(QP[4]), "l"(QP[5]), "l"(QP[6]), "l"(QP[7]), "l"(QP[8]),
-          "r"(rt_saddr)
-        : "memory");
+__device__ __forceinline__ int sat_s32(int64_t v) {
+    int r;
+    asm("cvt.sat.s32.s64 %0, %1;" : "=r"(r) : "l"(v));
+    return r;
 }
 
 // Rare path: some lane of the warp has a key below its threshold in this row.  Every lane
@@ -500,10 +430,30 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
             int64_t thr = lane_threshold(wt, cs, k, task_first_idx);
             uint32_t rows = 0;
 
-            const uint32_t rt_saddr = (uint32_t)__cvta_generic_to_shared(rt);
-            int64_t QP[9];
+            // threshold-relative forms (see "32-bit differential keys"); refreshed when thr moves
+            int64_t wmin = W[0];
+            int Wc[9], Qc[9];
+            int64_t B = 0, PmT[3];
+            if constexpr (OBJ == MMEE_OBJ_ENERGY) {
 #pragma unroll
-            for (int s = 0; s < 9; ++s) QP[s] = Q[s] + P[s / 3];
+                for (int s = 1; s < 9; ++s) wmin = W[s] < wmin ? W[s] : wmin;
+#pragma unroll
+                for (int s = 0; s < 9; ++s) {
+                    const int64_t wd = W[s] - wmin;
+                    Wc[s] = wd > (int64_t)(kRelCap + 1) ? (kRelCap + 1) : (int)wd;
+                }
+            }
+            auto refresh = [&](int64_t t) {
+                if constexpr (OBJ == MMEE_OBJ_ENERGY) {
+                    B = t - wmin;
+                } else if constexpr (OBJ == MMEE_OBJ_LATENCY) {
+#pragma unroll
+                    for (int j = 0; j < 3; ++j) PmT[j] = P[j] - t;
+#pragma unroll
+                    for (int s = 0; s < 9; ++s) Qc[s] = sat_s32(Q[s] + P[s / 3] - t);
+                }
+            };
+            refresh(thr);
 
 #pragma unroll 1
             for (int d = 0; d < 5; ++d) {
@@ -515,9 +465,37 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                 // lane of the warp has to enter the insertion path for this group.
                 unsigned hit_any, fits;
                 if constexpr (!DUMP && OBJ == MMEE_OBJ_ENERGY) {
-                    group_test_energy(xd, s1, s2, thr, W, rt_saddr, hit_any, fits);
+                    const int64_t xdb = xd - B;
+                    int acc = INT_MAX;
+                    fits = 0;
+#pragma unroll
+                    for (int e = 0; e < 5; ++e) {
+                        const unsigned fit = (unsigned)(rt->E[e][0] <= s1) & (unsigned)(rt->E[e][1] <= s2);   // Eq. (4)
+                        fits += fit;
+                        int xc = sat_s32(xdb + rt->E[e][2]);
+                        xc = xc < kRelCap ? xc : kRelCap;
+                        xc = fit ? xc : kRelCap;
+#pragma unroll
+                        for (int s = 0; s < 9; ++s) acc = __viaddmin_s32(xc, Wc[s], acc);     // min(key_s - thr)
+                    }
+                    hit_any = acc < 0;
                 } else if constexpr (!DUMP && OBJ == MMEE_OBJ_LATENCY) {
-                    group_test_latency(xd, s1, s2, thr, P, QP, rt_saddr, hit_any, fits);
+                    int acc = INT_MAX;
+                    fits = 0;
+#pragma unroll
+                    for (int e = 0; e < 5; ++e) {
+                        const unsigned fit = (unsigned)(rt->E[e][0] <= s1) & (unsigned)(rt->E[e][1] <= s2);   // Eq. (4)
+                        fits += fit;
+                        const int64_t x = xd + rt->E[e][2];
+                        int a[3];
+#pragma unroll
+                        for (int j = 0; j < 3; ++j) a[j] = sat_s32(x + PmT[j]);
+                        int racc = INT_MAX;
+#pragma unroll
+                        for (int s = 0; s < 9; ++s) racc = min(racc, max(a[s / 3], Qc[s]));       // min(key_s - thr)
+                        acc = min(acc, fit ? racc : INT_MAX);
+                    }
+                    hit_any = acc < 0;
                 } else {
                     hit_any = 0; fits = 0;
 #pragma unroll
@@ -556,6 +534,7 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                                                 task_first_idx + (uint64_t)((d * 5 + e) * 9), task_first_idx);
                         }
                     }
+                    refresh(thr);
                 }
             }
             my_rows += rows;
