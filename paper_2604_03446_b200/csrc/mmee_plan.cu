@@ -215,7 +215,8 @@ int build_plan(const mmee_workload_t* w, const mmee_arch_t* a, const mmee_object
     p->c_mac = p->cq[3] + (p->has_rf ? 3 * p->cq[2] : 0);
     p->c_sfu = p->cq[4];
 
-    if (a->gb_bytes / w->word_bytes > (uint64_t)INT64_MAX / 4) return MMEE_ERR_ARG;
+    // The row loop compares buffer sizes in 32 bits, saturated at 2^30 - 1 words.
+    if (a->gb_bytes / w->word_bytes >= (1ull << 30) - 1) return MMEE_ERR_RANGE;
     p->cap_words = (int64_t)(a->gb_bytes / w->word_bytes);
     p->bw = a->dram_words_per_cycle;
     p->pe_rows = a->pe_rows;

@@ -27,6 +27,8 @@ namespace mmee {
 namespace {
 
 constexpr unsigned kFull = 0xffffffffu;
+constexpr int kRelCap = (1 << 30) - 1;     // largest threshold-relative row term (see below)
+constexpr int kSizeCap = (1 << 30) - 1;    // buffer sizes saturate here; the capacity is smaller
 
 // ------------------------------------------------------------------------------------------------
 // shared-memory tables
@@ -40,8 +42,9 @@ constexpr unsigned kFull = 0xffffffffu;
 struct alignas(16) RowTab {
     int64_t D[5][4];        // per level of D: x1, x2, g, e
     int64_t E[5][4];        // per level of E: x1, x2, g, e
+    int32_t Dc[5][4];       // x1, x2 saturated to kSizeCap, g saturated to kRelCap + 1, unused
+    int32_t Ec[5][4];
 };
-static_assert(sizeof(RowTab) == 320 && offsetof(RowTab, E) == 160, "the row loop addresses RowTab by byte offset");
 
 // Per (tiling, order): task-side terms (levels of A, B, C) and the two row tables.
 struct alignas(16) OrderTab {
@@ -168,15 +171,16 @@ __device__ __forceinline__ void row_test(const int64_t (&k)[9], int64_t thr, int
 // the exact 64-bit insertion path, which re-evaluates the rows in full.
 //
 // Energy: key = x + W[s].  With wmin = min_s W[s], B = thr - wmin, x' = x - B and W' = W - wmin >= 0:
-// key < thr  <=>  x' + W' < 0.  x' is saturated to [-2^31, 2^30 - 1] and W' to [0, 2^30].  If some
-// s of a row truly passes then either x' >= -2^31, where x' is exact and min(W', 2^30) <= W' keeps
-// the sum negative, or x' < -2^31, where s = argmin W (W' = 0) gives -2^31 < 0; conversely a
-// negative saturated sum implies x' < 0, i.e. the candidate with W' = 0 passes.  So a row is
-// flagged iff it holds a passing candidate, and no 32-bit sum can overflow.
-// Latency: key = max(x + P, Q + P); max(a, b) < thr <=> sat(a - thr) < 0 and sat(b - thr) < 0: exact
-// per candidate.
-constexpr int kRelCap = (1 << 30) - 1;
-
+// key < thr  <=>  x' + W' < 0, and x' = u + v with u = (task and D-level terms) - B per group and
+// v = the E-level term >= 0.  u is saturated to [-2^31, 2^30 - 1], v and W' to [0, 2^30], u + v is
+// capped at 2^30 - 1 again: no 32-bit sum can overflow.  Saturation only ever lowers v and W' and
+// raises u only when u < -2^31, so: if a candidate of a row truly passes, the saturated sum of the
+// row's candidate with W' = 0 is negative (the row is flagged); a flagged row that holds no passing
+// candidate is possible only when u < -2^30 while v >= 2^30, and costs one visit of the exact path.
+// Latency: key = max(x + P, Q + P) and max(a, b) < thr <=> a - thr < 0 and b - thr < 0; the same
+// saturation is applied to x + P - thr = u + v.
+// Capacity (Eq. 4): sizes are saturated to kSizeCap, which is above every admissible capacity, so
+// "size <= slack" keeps its truth value in 32 bits.
 __device__ __forceinline__ int sat_s32(int64_t v) {
     int r;
     asm("cvt.sat.s32.s64 %0, %1;" : "=r"(r) : "l"(v));
@@ -253,6 +257,16 @@ __device__ __forceinline__ void build_order_item(const Plan& p, const uint32_t* 
         int64_t* ur = x == OP_D ? u->D[l] : u->E[l];
         fr[0] = l ? bs : 0; fr[1] = bs; fr[2] = scale * vf; fr[3] = escale * vf;
         ur[0] = 0;          ur[1] = bs; ur[2] = scale * vu; ur[3] = escale * vu;
+        int32_t* fc = x == OP_D ? f->Dc[l] : f->Ec[l];
+        int32_t* uc = x == OP_D ? u->Dc[l] : u->Ec[l];
+#pragma unroll
+        for (int i = 0; i < 3; ++i) {
+            const int64_t lim = i < 2 ? (int64_t)kSizeCap : (int64_t)kRelCap + 1;
+            fc[i] = (int32_t)(fr[i] < lim ? fr[i] : lim);
+            uc[i] = (int32_t)(ur[i] < lim ? ur[i] : lim);
+        }
+        fc[3] = 0;
+        uc[3] = 0;
     } else {
         const int64_t v = monomial(q.da_unfused[order][OP_C][0], b);
         ot->gCr = scale * v;
@@ -454,6 +468,14 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                 }
             };
             refresh(thr);
+            int E1c[5], E2c[5], Gc[5];
+#pragma unroll
+            for (int e = 0; e < 5; ++e) {
+                const int4 v = *reinterpret_cast<const int4*>(rt->Ec[e]);
+                E1c[e] = v.x; E2c[e] = v.y; Gc[e] = v.z;
+            }
+            const int slack1c = slack1 < 0 ? -1 : (int)slack1;      // slack <= capacity < 2^30
+            const int slack2c = slack2 < 0 ? -1 : (int)slack2;
 
 #pragma unroll 1
             for (int d = 0; d < 5; ++d) {
@@ -464,36 +486,42 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                 // Five rows (levels of E) are evaluated branch-free; one vote decides whether any
                 // lane of the warp has to enter the insertion path for this group.
                 unsigned hit_any, fits;
-                if constexpr (!DUMP && OBJ == MMEE_OBJ_ENERGY) {
-                    const int64_t xdb = xd - B;
+                if constexpr (!DUMP && OBJ != MMEE_OBJ_EDP) {
+                    const int s1c = slack1c - rt->Dc[d][0];
+                    const int s2c = slack2c - rt->Dc[d][1];
                     int acc = INT_MAX;
                     fits = 0;
+                    if constexpr (OBJ == MMEE_OBJ_ENERGY) {
+                        int uc = sat_s32(xd - B);
+                        uc = uc < kRelCap ? uc : kRelCap;
 #pragma unroll
-                    for (int e = 0; e < 5; ++e) {
-                        const unsigned fit = (unsigned)(rt->E[e][0] <= s1) & (unsigned)(rt->E[e][1] <= s2);   // Eq. (4)
-                        fits += fit;
-                        int xc = sat_s32(xdb + rt->E[e][2]);
-                        xc = xc < kRelCap ? xc : kRelCap;
-                        xc = fit ? xc : kRelCap;
+                        for (int e = 0; e < 5; ++e) {
+                            const unsigned fit = (unsigned)(E1c[e] <= s1c) & (unsigned)(E2c[e] <= s2c);   // Eq. (4)
+                            fits += fit;
+                            int xc = __viaddmin_s32(uc, Gc[e], kRelCap);
+                            xc = fit ? xc : kRelCap;
 #pragma unroll
-                        for (int s = 0; s < 9; ++s) acc = __viaddmin_s32(xc, Wc[s], acc);     // min(key_s - thr)
-                    }
-                    hit_any = acc < 0;
-                } else if constexpr (!DUMP && OBJ == MMEE_OBJ_LATENCY) {
-                    int acc = INT_MAX;
-                    fits = 0;
+                            for (int s = 0; s < 9; ++s) acc = __viaddmin_s32(xc, Wc[s], acc);     // min(key_s - thr)
+                        }
+                    } else {
+                        int uc[3];
 #pragma unroll
-                    for (int e = 0; e < 5; ++e) {
-                        const unsigned fit = (unsigned)(rt->E[e][0] <= s1) & (unsigned)(rt->E[e][1] <= s2);   // Eq. (4)
-                        fits += fit;
-                        const int64_t x = xd + rt->E[e][2];
-                        int a[3];
+                        for (int j = 0; j < 3; ++j) {
+                            uc[j] = sat_s32(xd + PmT[j]);
+                            uc[j] = uc[j] < kRelCap ? uc[j] : kRelCap;
+                        }
 #pragma unroll
-                        for (int j = 0; j < 3; ++j) a[j] = sat_s32(x + PmT[j]);
-                        int racc = INT_MAX;
+                        for (int e = 0; e < 5; ++e) {
+                            const unsigned fit = (unsigned)(E1c[e] <= s1c) & (unsigned)(E2c[e] <= s2c);   // Eq. (4)
+                            fits += fit;
+                            int a[3];
 #pragma unroll
-                        for (int s = 0; s < 9; ++s) racc = min(racc, max(a[s / 3], Qc[s]));       // min(key_s - thr)
-                        acc = min(acc, fit ? racc : INT_MAX);
+                            for (int j = 0; j < 3; ++j) a[j] = __viaddmin_s32(uc[j], Gc[e], kRelCap);
+                            int racc = INT_MAX;
+#pragma unroll
+                            for (int s = 0; s < 9; ++s) racc = min(racc, max(a[s / 3], Qc[s]));   // min(key_s - thr)
+                            acc = min(acc, fit ? racc : INT_MAX);
+                        }
                     }
                     hit_any = acc < 0;
                 } else {
