@@ -48,6 +48,14 @@ int choose_shape(const Plan& p, int device, LaunchShape* shape) {
     const uint64_t ranges = (tasks + shape->range_tasks - 1) / shape->range_tasks;
     if (grid > ranges) grid = ranges ? ranges : 1;
     shape->grid = (uint32_t)grid;
+    shape->n_ranges = ranges;
+    // golden-ratio stride, moved to the next value coprime to the number of ranges
+    uint64_t stride = ranges > 2 ? (uint64_t)((double)ranges * 0.6180339887498949) : 1;
+    if (stride < 1) stride = 1;
+    auto gcd = [](uint64_t a, uint64_t b) { while (b) { const uint64_t t = a % b; a = b; b = t; } return a; };
+    while (ranges > 1 && gcd(stride, ranges) != 1) ++stride;
+    shape->range_stride = ranges > 1 ? stride % ranges : 0;
+    if (ranges > 1 && shape->range_stride == 0) shape->range_stride = 1;
     return MMEE_OK;
 }
 

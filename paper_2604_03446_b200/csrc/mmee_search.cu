@@ -191,7 +191,7 @@ __device__ __forceinline__ int sat_s32(int64_t v) {
 // re-evaluates its nine candidates of the row from the shared tables and the warp inserts the
 // passing ones, one at a time, into its sorted list.
 template <int OBJ>
-__device__ __noinline__ int64_t slow_row(WarpTop* wt, CtaShared* cs, int k, int lane, bool f,
+__device__ __noinline__ int64_t slow_row(WarpTop* wt, CtaShared* cs, long long* global_g, int k, int lane, bool f,
                                          int64_t x, int64_t xe, const int64_t* wptr, const int64_t* qptr,
                                          int64_t p0, int64_t p1, int64_t p2,
                                          uint64_t row_first_idx, uint64_t task_first_idx) {
@@ -213,7 +213,10 @@ __device__ __noinline__ int64_t slow_row(WarpTop* wt, CtaShared* cs, int k, int 
     }
     if (lane == 0 && wt->count == k) {
         const long long last = wt->key[k - 1];
-        if (last < cs->G) atomicMin(&cs->G, last);
+        if (last < cs->G) {
+            atomicMin(&cs->G, last);
+            atomicMin(global_g, last);       // other CTAs pick it up at their next task
+        }
     }
     __syncwarp();
     return lane_threshold(wt, cs, k, task_first_idx);
@@ -341,8 +344,13 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
 
     while (true) {
         if (tid == 0) {
-            const unsigned long long got = atomicAdd(&scratch->next_task, (unsigned long long)shape.range_tasks);
-            cs->range_begin = task_begin + got;
+            // Ranges are visited in a stride-permuted order (stride coprime to their number), so that
+            // the first pull of every CTA samples the whole index space and the pruning bound G is
+            // near its final value from the start.
+            const unsigned long long got = atomicAdd(&scratch->next_task, 1ull);
+            cs->range_begin = got < shape.n_ranges
+                                  ? task_begin + ((got * shape.range_stride) % shape.n_ranges) * shape.range_tasks
+                                  : task_end;
             // exchange the pruning bound with the other CTAs
             const long long mine = cs->G;
             const long long theirs = atomicMin(&scratch->G, mine);
@@ -441,6 +449,11 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                 Q[s] = qptr[2 * s];
             }
             const uint64_t task_first_idx = tq * kCandPerTask;
+            if (lane == 0) {
+                const long long seen = *reinterpret_cast<volatile long long*>(&scratch->G);
+                if (seen < cs->G) atomicMin(&cs->G, seen);
+            }
+            __syncwarp();
             int64_t thr = lane_threshold(wt, cs, k, task_first_idx);
             uint32_t rows = 0;
 
@@ -558,7 +571,7 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                         for (int s = 0; s < 9; ++s)
                             below |= candidate_key<OBJ>(x, xe, wptr[2 * s], P[s / 3], qptr[2 * s]) < thr;
                         if (__any_sync(kFull, fit && below)) {
-                            thr = slow_row<OBJ>(wt, cs, k, lane, fit, x, xe, wptr, qptr, P[0], P[1], P[2],
+                            thr = slow_row<OBJ>(wt, cs, &scratch->G, k, lane, fit, x, xe, wptr, qptr, P[0], P[1], P[2],
                                                 task_first_idx + (uint64_t)((d * 5 + e) * 9), task_first_idx);
                         }
                     }

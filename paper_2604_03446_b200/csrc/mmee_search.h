@@ -33,6 +33,8 @@ struct LaunchShape {
     uint32_t range_tasks;   // tasks a CTA takes per pull (multiple of kSearchThreads)
     uint32_t slots;         // tilings one range can touch
     uint32_t smem_bytes;
+    uint64_t n_ranges;      // ranges of the searched task interval
+    uint64_t range_stride;  // ranges are visited as (i * range_stride) mod n_ranges; coprime to n_ranges
 };
 
 inline size_t scratch_bytes(uint32_t grid) { return sizeof(Scratch) + (size_t)(grid ? grid - 1 : 0) * sizeof(Partial); }
