@@ -61,14 +61,19 @@ constexpr int kOrderItems = 26;
 // Per tiling: array-level terms by stationary pair and recompute flag.
 struct alignas(16) TilingTab {
     uint32_t b[8];
+    int32_t Wc[2][12];      // W[s][rc] - wmin[rc], saturated to kRelCap + 1 (entries 9..11 unused)
     int64_t W[9][2];        // energy of buffer<->PE traffic, MACs and softmax, in quanta
     int64_t CB[9][2];       // fused compute time in words (cycles * words per cycle)
     int64_t QU[9][2];       // unfused Op2 compute time in words, by s (sm2 = s % 3)
     int64_t C1w[3];         // unfused Op1 compute time in words, by sm1
     int64_t cw, smx;        // C write-back words (I*L); separate softmax pass words (2*I*L)
+    int64_t wmin[2];        // min over the stationary pairs of W[.][rc]
     int32_t live;           // smallest possible buffer need of this tiling fits
-    int32_t pad;
+    int32_t pad[3];
 };
+static_assert(offsetof(TilingTab, Wc) % 16 == 0 && sizeof(int32_t[12]) % 16 == 0, "Wc rows are read as int4");
+static_assert(offsetof(RowTab, Ec) % 16 == 0 && offsetof(OrderTab, rt) % 16 == 0 && sizeof(RowTab) % 16 == 0,
+              "Ec rows are read as int4");
 constexpr int kTilingItems = 21;    // 9 stationary pairs x 2 recompute flags, 3 unfused Op1 terms
 
 struct alignas(16) WarpTop {
@@ -291,7 +296,7 @@ __device__ __forceinline__ void build_tiling_head(const Plan& p, uint64_t t, Til
     const int64_t td = (int64_t)b[6] * b[7], te = (int64_t)b[4] * b[7];
     const int64_t need1 = ta + tbb + tc, need2 = tc + td + te;
     tb->live = ((need1 > need2 ? need1 : need2) <= p.cap_words) ? 1 : 0;
-    tb->pad = 0;
+    tb->pad[0] = tb->pad[1] = tb->pad[2] = 0;
 }
 
 // One thread per (tiling slot, item): stationary-pair terms with the cost coefficients applied.
@@ -383,6 +388,21 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
             }
         }
         __syncthreads();
+        if (OBJ == MMEE_OBJ_ENERGY && tid < (int)(2 * n_slots)) {
+            // threshold-relative stationary-pair terms (see "32-bit differential keys")
+            TilingTab* tb = &ttabs[tid >> 1];
+            const int rc = tid & 1;
+            if (tb->live) {
+                int64_t m = tb->W[0][rc];
+                for (int s = 1; s < 9; ++s) m = tb->W[s][rc] < m ? tb->W[s][rc] : m;
+                tb->wmin[rc] = m;
+                for (int s = 0; s < 9; ++s) {
+                    const int64_t wd = tb->W[s][rc] - m;
+                    tb->Wc[rc][s] = wd > (int64_t)(kRelCap + 1) ? (kRelCap + 1) : (int32_t)wd;
+                }
+            }
+        }
+        __syncthreads();
 
         // ---- tasks
         const uint32_t w_first = (uint32_t)(r0 - t_first * tpt);      // task of r0 inside its tiling
@@ -458,17 +478,16 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
             uint32_t rows = 0;
 
             // threshold-relative forms (see "32-bit differential keys"); refreshed when thr moves
-            int64_t wmin = W[0];
+            int64_t wmin = 0;
             int Wc[9], Qc[9];
             int64_t B = 0, PmT[3];
             if constexpr (OBJ == MMEE_OBJ_ENERGY) {
-#pragma unroll
-                for (int s = 1; s < 9; ++s) wmin = W[s] < wmin ? W[s] : wmin;
-#pragma unroll
-                for (int s = 0; s < 9; ++s) {
-                    const int64_t wd = W[s] - wmin;
-                    Wc[s] = wd > (int64_t)(kRelCap + 1) ? (kRelCap + 1) : (int)wd;
-                }
+                wmin = tb->wmin[rc];
+                const int4* wc4 = reinterpret_cast<const int4*>(tb->Wc[rc]);
+                const int4 w0 = wc4[0], w1 = wc4[1], w2 = wc4[2];
+                Wc[0] = w0.x; Wc[1] = w0.y; Wc[2] = w0.z; Wc[3] = w0.w;
+                Wc[4] = w1.x; Wc[5] = w1.y; Wc[6] = w1.z; Wc[7] = w1.w;
+                Wc[8] = w2.x;
             }
             auto refresh = [&](int64_t t) {
                 if constexpr (OBJ == MMEE_OBJ_ENERGY) {
@@ -502,7 +521,7 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                 if constexpr (!DUMP && OBJ != MMEE_OBJ_EDP) {
                     const int s1c = slack1c - rt->Dc[d][0];
                     const int s2c = slack2c - rt->Dc[d][1];
-                    int acc = INT_MAX;
+                    int acc = INT_MAX, acc1 = INT_MAX, acc2 = INT_MAX;    // independent chains
                     fits = 0;
                     if constexpr (OBJ == MMEE_OBJ_ENERGY) {
                         int uc = sat_s32(xd - B);
@@ -514,8 +533,13 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                             int xc = __viaddmin_s32(uc, Gc[e], kRelCap);
                             xc = fit ? xc : kRelCap;
 #pragma unroll
-                            for (int s = 0; s < 9; ++s) acc = __viaddmin_s32(xc, Wc[s], acc);     // min(key_s - thr)
+                            for (int s = 0; s < 9; s += 3) {                                      // min(key_s - thr)
+                                acc = __viaddmin_s32(xc, Wc[s], acc);
+                                acc1 = __viaddmin_s32(xc, Wc[s + 1], acc1);
+                                acc2 = __viaddmin_s32(xc, Wc[s + 2], acc2);
+                            }
                         }
+                        acc = min(acc, min(acc1, acc2));
                     } else {
                         int uc[3];
 #pragma unroll
