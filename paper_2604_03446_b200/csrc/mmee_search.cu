@@ -110,9 +110,9 @@ __device__ __forceinline__ bool warp_insert(WarpTop* wt, int k, int64_t nk, uint
     return true;
 }
 
-// Threshold a lane compares keys against while it walks one task in ascending index order:
-// a key passes iff it can still enter the warp's list and is not above the CTA-wide bound G.
-// Strict against the list's last key when every index of the task lies above that entry's index.
+// Threshold for candidates whose indices are all >= first_idx: a key passes iff it can still enter
+// the warp's list and is not above the CTA-wide bound G.  Strict against the list's last key
+// when first_idx lies above that entry's index (a tie could then not displace it).
 __device__ __forceinline__ int64_t lane_threshold(const WarpTop* wt, const CtaShared* cs, int k, uint64_t task_first_idx) {
     int64_t thr = cs->G + 1;                       // G <= INT64_MAX - 1 always
     if (wt->count == k) {
@@ -199,8 +199,8 @@ template <int OBJ>
 __device__ __noinline__ int64_t slow_row(WarpTop* wt, CtaShared* cs, long long* global_g, int k, int lane, bool f,
                                          int64_t x, int64_t xe, const int64_t* wptr, const int64_t* qptr,
                                          int64_t p0, int64_t p1, int64_t p2,
-                                         uint64_t row_first_idx, uint64_t task_first_idx) {
-    int64_t thr = lane_threshold(wt, cs, k, task_first_idx);
+                                         uint64_t row_first_idx) {
+    int64_t thr = lane_threshold(wt, cs, k, row_first_idx);
     for (int s = 0; s < 9; ++s) {
         const int64_t pp = s < 3 ? p0 : (s < 6 ? p1 : p2);
         const int64_t key = candidate_key<OBJ>(x, xe, wptr[2 * s], pp, qptr[2 * s]);
@@ -212,7 +212,7 @@ __device__ __noinline__ int64_t slow_row(WarpTop* wt, CtaShared* cs, long long* 
             const int64_t lk = __shfl_sync(kFull, key, leader);
             const uint64_t li = __shfl_sync(kFull, row_first_idx + (uint64_t)s, leader);
             warp_insert(wt, k, lk, li, lane);
-            thr = lane_threshold(wt, cs, k, task_first_idx);
+            thr = lane_threshold(wt, cs, k, row_first_idx);
             pend = (lane == leader) ? false : (pend && key < thr);
         }
     }
@@ -224,12 +224,40 @@ __device__ __noinline__ int64_t slow_row(WarpTop* wt, CtaShared* cs, long long* 
         }
     }
     __syncwarp();
-    return lane_threshold(wt, cs, k, task_first_idx);
+    return thr;
 }
 
 // ------------------------------------------------------------------------------------------------
 // table construction
 // ------------------------------------------------------------------------------------------------
+
+// Tables of a tiling that cannot fit at all are filled with constants under which no row fits,
+// so that lanes whose task lies in such a tiling (they keep step with their warp) read defined data.
+__device__ __forceinline__ void fill_dead_order_item(OrderTab* ot, int item) {
+    const int l = item % 5;
+    if (item < 10) {
+        int64_t* s1 = item < 5 ? ot->A1 : ot->B1;
+        int64_t* s2 = item < 5 ? ot->A2 : ot->B2;
+        int64_t (*g)[2] = item < 5 ? ot->gA : ot->gB;
+        int64_t (*e)[2] = item < 5 ? ot->eA : ot->eB;
+        s1[l] = s2[l] = 0;
+        g[l][0] = g[l][1] = e[l][0] = e[l][1] = 0;
+    } else if (item < 15) {
+        ot->C1[l] = 0;
+        ot->rc[l] = 0;
+    } else if (item < 25) {
+        for (int v = 0; v < 2; ++v) {
+            int64_t* r = item < 20 ? ot->rt[v].D[l] : ot->rt[v].E[l];
+            int32_t* c = item < 20 ? ot->rt[v].Dc[l] : ot->rt[v].Ec[l];
+            r[0] = r[1] = (int64_t)kSizeCap; r[2] = r[3] = 0;
+            c[0] = c[1] = kSizeCap; c[2] = c[3] = 0;
+        }
+    } else {
+        ot->gCr = ot->eCr = 0;
+    }
+}
+
+__device__ __forceinline__ void fill_dead_tiling_item(struct TilingTab* tb, int item);
 
 // One thread per (tiling slot, order, item): the monomials of one operand at one level.
 template <int OBJ>
@@ -315,6 +343,15 @@ __device__ __forceinline__ void build_tiling_item(const Plan& p, TilingTab* tb, 
     }
 }
 
+__device__ __forceinline__ void fill_dead_tiling_item(TilingTab* tb, int item) {
+    if (item < 18) {
+        const int s = item >> 1, rc = item & 1;
+        tb->W[s][rc] = tb->CB[s][rc] = tb->QU[s][rc] = 0;
+    } else {
+        tb->C1w[item - 18] = 0;
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // the search kernel
 // ------------------------------------------------------------------------------------------------
@@ -378,12 +415,12 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                 const uint32_t e = it % kOrderItems;
                 const uint32_t so = it / kOrderItems;
                 const uint32_t slot = so / n_orders, os = so % n_orders;
-                if (!ttabs[slot].live) continue;
+                if (!ttabs[slot].live) { fill_dead_order_item(&otabs[slot * n_orders + os], (int)e); continue; }
                 build_order_item<OBJ>(p, ttabs[slot].b, p.order_id[os], &otabs[slot * n_orders + os], (int)e);
             } else {
                 const uint32_t j = it - order_items;
                 const uint32_t slot = j / kTilingItems;
-                if (!ttabs[slot].live) continue;
+                if (!ttabs[slot].live) { fill_dead_tiling_item(&ttabs[slot], (int)(j - slot * kTilingItems)); continue; }
                 build_tiling_item(p, &ttabs[slot], (int)(j - slot * kTilingItems));
             }
         }
@@ -392,7 +429,7 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
             // threshold-relative stationary-pair terms (see "32-bit differential keys")
             TilingTab* tb = &ttabs[tid >> 1];
             const int rc = tid & 1;
-            if (tb->live) {
+            {
                 int64_t m = tb->W[0][rc];
                 for (int s = 1; s < 9; ++s) m = tb->W[s][rc] < m ? tb->W[s][rc] : m;
                 tb->wmin[rc] = m;
@@ -474,7 +511,21 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                 if (seen < cs->G) atomicMin(&cs->G, seen);
             }
             __syncwarp();
-            int64_t thr = lane_threshold(wt, cs, k, task_first_idx);
+            // Threshold state of this lane: T1 = the non-strict threshold (a key passes iff key < T1);
+            // for a group whose first index lies above `ti`, the index of the list's last entry, the
+            // threshold is T1 - delta (ties with that entry cannot displace it).
+            int64_t T1;
+            uint64_t ti;
+            int delta;
+            auto load_threshold = [&]() {
+                const int64_t g1 = cs->G + 1;                 // G <= INT64_MAX - 1 always
+                T1 = g1; ti = UINT64_MAX; delta = 0;
+                if (wt->count == k) {
+                    const int64_t tk1 = wt->key[k - 1] + 1;
+                    if (tk1 <= g1) { T1 = tk1; delta = 1; ti = wt->idx[k - 1]; }
+                }
+            };
+            load_threshold();
             uint32_t rows = 0;
 
             // threshold-relative forms (see "32-bit differential keys"); refreshed when thr moves
@@ -499,7 +550,7 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                     for (int s = 0; s < 9; ++s) Qc[s] = sat_s32(Q[s] + P[s / 3] - t);
                 }
             };
-            refresh(thr);
+            refresh(T1);
             int E1c[5], E2c[5], Gc[5];
 #pragma unroll
             for (int e = 0; e < 5; ++e) {
@@ -560,8 +611,11 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                             acc = min(acc, fit ? racc : INT_MAX);
                         }
                     }
-                    hit_any = acc < 0;
+                    const uint64_t group_first_idx = task_first_idx + (uint64_t)(d * 45);
+                    hit_any = acc < (group_first_idx > ti ? -delta : 0);      // no overflow at acc = INT_MAX
                 } else {
+                    const uint64_t group_first_idx = task_first_idx + (uint64_t)(d * 45);
+                    const int64_t thr = T1 - (group_first_idx > ti ? delta : 0);
                     hit_any = 0; fits = 0;
 #pragma unroll
                     for (int e = 0; e < 5; ++e) {
@@ -591,15 +645,17 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                         const bool fit = (rt->E[e][0] <= s1) && (rt->E[e][1] <= s2);
                         const int64_t x = xd + rt->E[e][2];
                         const int64_t xe = (OBJ == MMEE_OBJ_EDP) ? xed + rt->E[e][3] : 0;
+                        const uint64_t row_first_idx = task_first_idx + (uint64_t)((d * 5 + e) * 9);
+                        const int64_t thr_row = lane_threshold(wt, cs, k, row_first_idx);
                         bool below = false;
                         for (int s = 0; s < 9; ++s)
-                            below |= candidate_key<OBJ>(x, xe, wptr[2 * s], P[s / 3], qptr[2 * s]) < thr;
-                        if (__any_sync(kFull, fit && below)) {
-                            thr = slow_row<OBJ>(wt, cs, &scratch->G, k, lane, fit, x, xe, wptr, qptr, P[0], P[1], P[2],
-                                                task_first_idx + (uint64_t)((d * 5 + e) * 9), task_first_idx);
-                        }
+                            below |= candidate_key<OBJ>(x, xe, wptr[2 * s], P[s / 3], qptr[2 * s]) < thr_row;
+                        if (__any_sync(kFull, fit && below))
+                            slow_row<OBJ>(wt, cs, &scratch->G, k, lane, fit, x, xe, wptr, qptr, P[0], P[1], P[2],
+                                          row_first_idx);
                     }
-                    refresh(thr);
+                    load_threshold();
+                    refresh(T1);
                 }
             }
             my_rows += rows;
