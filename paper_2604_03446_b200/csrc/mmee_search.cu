@@ -27,7 +27,8 @@ namespace mmee {
 namespace {
 
 constexpr unsigned kFull = 0xffffffffu;
-constexpr int kRelCap = (1 << 30) - 1;     // largest threshold-relative row term (see below)
+constexpr int kRelCap = (1 << 30) - 1;     // cap of a running threshold-relative sum (see below)
+constexpr int kTermCap = 1 << 29;          // cap of each non-negative addend of such a sum
 constexpr int kSizeCap = (1 << 30) - 1;    // buffer sizes saturate here; the capacity is smaller
 
 // ------------------------------------------------------------------------------------------------
@@ -42,7 +43,7 @@ constexpr int kSizeCap = (1 << 30) - 1;    // buffer sizes saturate here; the ca
 struct alignas(16) RowTab {
     int64_t D[5][4];        // per level of D: x1, x2, g, e
     int64_t E[5][4];        // per level of E: x1, x2, g, e
-    int32_t Dc[5][4];       // x1, x2 saturated to kSizeCap, g saturated to kRelCap + 1, unused
+    int32_t Dc[5][4];       // x1, x2 saturated to kSizeCap, g saturated to kTermCap, unused
     int32_t Ec[5][4];
 };
 
@@ -61,7 +62,7 @@ constexpr int kOrderItems = 26;
 // Per tiling: array-level terms by stationary pair and recompute flag.
 struct alignas(16) TilingTab {
     uint32_t b[8];
-    int32_t Wc[2][12];      // W[s][rc] - wmin[rc], saturated to kRelCap + 1 (entries 9..11 unused)
+    int32_t Wc[2][12];      // W[s][rc] - wmin[rc], saturated to kTermCap (entries 9..11 unused)
     int64_t W[9][2];        // energy of buffer<->PE traffic, MACs and softmax, in quanta
     int64_t CB[9][2];       // fused compute time in words (cycles * words per cycle)
     int64_t QU[9][2];       // unfused Op2 compute time in words, by s (sm2 = s % 3)
@@ -175,15 +176,16 @@ __device__ __forceinline__ void row_test(const int64_t (&k)[9], int64_t thr, int
 // bits, and keeps the minimum over the group of five rows; a negative minimum sends the warp to
 // the exact 64-bit insertion path, which re-evaluates the rows in full.
 //
-// Energy: key = x + W[s].  With wmin = min_s W[s], B = thr - wmin, x' = x - B and W' = W - wmin >= 0:
-// key < thr  <=>  x' + W' < 0, and x' = u + v with u = (task and D-level terms) - B per group and
-// v = the E-level term >= 0.  u is saturated to [-2^31, 2^30 - 1], v and W' to [0, 2^30], u + v is
-// capped at 2^30 - 1 again: no 32-bit sum can overflow.  Saturation only ever lowers v and W' and
-// raises u only when u < -2^31, so: if a candidate of a row truly passes, the saturated sum of the
-// row's candidate with W' = 0 is negative (the row is flagged); a flagged row that holds no passing
-// candidate is possible only when u < -2^30 while v >= 2^30, and costs one visit of the exact path.
+// Energy: key = x + W[s].  With wmin = min_s W[s], B = thr - wmin and W' = W - wmin >= 0:
+// key < thr  <=>  u + vD + vE + W' < 0, where u = (task-level terms) - B and vD, vE >= 0 are the D- and
+// E-level terms.  u is saturated to [-2^31, 2^30 - 1], each of vD, vE, W' to [0, 2^29], and every
+// running sum is capped at 2^30 - 1: no 32-bit sum can overflow.  Saturation only lowers the
+// non-negative addends and raises u only when u < -2^31, where the saturated sum is at most
+// -2^31 + 3 * 2^29 < 0.  Hence, if a candidate of a row truly passes, the saturated sum of the row's
+// candidate with W' = 0 is negative and the row is flagged; a flagged row without a passing
+// candidate needs u < -2^29 next to a saturated addend, and costs one visit of the exact path.
 // Latency: key = max(x + P, Q + P) and max(a, b) < thr <=> a - thr < 0 and b - thr < 0; the same
-// saturation is applied to x + P - thr = u + v.
+// saturation is applied to x + P - thr = u + vD + vE.
 // Capacity (Eq. 4): sizes are saturated to kSizeCap, which is above every admissible capacity, so
 // "size <= slack" keeps its truth value in 32 bits.
 __device__ __forceinline__ int sat_s32(int64_t v) {
@@ -297,7 +299,7 @@ __device__ __forceinline__ void build_order_item(const Plan& p, const uint32_t* 
         int32_t* uc = x == OP_D ? u->Dc[l] : u->Ec[l];
 #pragma unroll
         for (int i = 0; i < 3; ++i) {
-            const int64_t lim = i < 2 ? (int64_t)kSizeCap : (int64_t)kRelCap + 1;
+            const int64_t lim = i < 2 ? (int64_t)kSizeCap : (int64_t)kTermCap;
             fc[i] = (int32_t)(fr[i] < lim ? fr[i] : lim);
             uc[i] = (int32_t)(ur[i] < lim ? ur[i] : lim);
         }
@@ -435,7 +437,7 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                 tb->wmin[rc] = m;
                 for (int s = 0; s < 9; ++s) {
                     const int64_t wd = tb->W[s][rc] - m;
-                    tb->Wc[rc][s] = wd > (int64_t)(kRelCap + 1) ? (kRelCap + 1) : (int32_t)wd;
+                    tb->Wc[rc][s] = wd > (int64_t)kTermCap ? kTermCap : (int32_t)wd;
                 }
             }
         }
@@ -540,12 +542,19 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                 Wc[4] = w1.x; Wc[5] = w1.y; Wc[6] = w1.z; Wc[7] = w1.w;
                 Wc[8] = w2.x;
             }
+            int ut[3] = {0, 0, 0};      // saturated task-level part of key - thr
             auto refresh = [&](int64_t t) {
                 if constexpr (OBJ == MMEE_OBJ_ENERGY) {
                     B = t - wmin;
+                    const int u = sat_s32(x0 - B);
+                    ut[0] = u < kRelCap ? u : kRelCap;
                 } else if constexpr (OBJ == MMEE_OBJ_LATENCY) {
 #pragma unroll
-                    for (int j = 0; j < 3; ++j) PmT[j] = P[j] - t;
+                    for (int j = 0; j < 3; ++j) {
+                        PmT[j] = P[j] - t;
+                        const int u = sat_s32(x0 + PmT[j]);
+                        ut[j] = u < kRelCap ? u : kRelCap;
+                    }
 #pragma unroll
                     for (int s = 0; s < 9; ++s) Qc[s] = sat_s32(Q[s] + P[s / 3] - t);
                 }
@@ -562,21 +571,17 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
 
 #pragma unroll 1
             for (int d = 0; d < 5; ++d) {
-                const int64_t s1 = slack1 - rt->D[d][0];
-                const int64_t s2 = slack2 - rt->D[d][1];
-                const int64_t xd = x0 + rt->D[d][2];
-                const int64_t xed = (OBJ == MMEE_OBJ_EDP) ? xe0 + rt->D[d][3] : 0;
                 // Five rows (levels of E) are evaluated branch-free; one vote decides whether any
                 // lane of the warp has to enter the insertion path for this group.
                 unsigned hit_any, fits;
                 if constexpr (!DUMP && OBJ != MMEE_OBJ_EDP) {
-                    const int s1c = slack1c - rt->Dc[d][0];
-                    const int s2c = slack2c - rt->Dc[d][1];
+                    const int4 dc = *reinterpret_cast<const int4*>(rt->Dc[d]);
+                    const int s1c = slack1c - dc.x;
+                    const int s2c = slack2c - dc.y;
                     int acc = INT_MAX, acc1 = INT_MAX, acc2 = INT_MAX;    // independent chains
                     fits = 0;
                     if constexpr (OBJ == MMEE_OBJ_ENERGY) {
-                        int uc = sat_s32(xd - B);
-                        uc = uc < kRelCap ? uc : kRelCap;
+                        const int uc = __viaddmin_s32(ut[0], dc.z, kRelCap);
 #pragma unroll
                         for (int e = 0; e < 5; ++e) {
                             const unsigned fit = (unsigned)(E1c[e] <= s1c) & (unsigned)(E2c[e] <= s2c);   // Eq. (4)
@@ -594,10 +599,7 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                     } else {
                         int uc[3];
 #pragma unroll
-                        for (int j = 0; j < 3; ++j) {
-                            uc[j] = sat_s32(xd + PmT[j]);
-                            uc[j] = uc[j] < kRelCap ? uc[j] : kRelCap;
-                        }
+                        for (int j = 0; j < 3; ++j) uc[j] = __viaddmin_s32(ut[j], dc.z, kRelCap);
 #pragma unroll
                         for (int e = 0; e < 5; ++e) {
                             const unsigned fit = (unsigned)(E1c[e] <= s1c) & (unsigned)(E2c[e] <= s2c);   // Eq. (4)
@@ -614,6 +616,10 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                     const uint64_t group_first_idx = task_first_idx + (uint64_t)(d * 45);
                     hit_any = acc < (group_first_idx > ti ? -delta : 0);      // no overflow at acc = INT_MAX
                 } else {
+                    const int64_t s1 = slack1 - rt->D[d][0];
+                    const int64_t s2 = slack2 - rt->D[d][1];
+                    const int64_t xd = x0 + rt->D[d][2];
+                    const int64_t xed = (OBJ == MMEE_OBJ_EDP) ? xe0 + rt->D[d][3] : 0;
                     const uint64_t group_first_idx = task_first_idx + (uint64_t)(d * 45);
                     const int64_t thr = T1 - (group_first_idx > ti ? delta : 0);
                     hit_any = 0; fits = 0;
@@ -639,7 +645,11 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                 }
                 rows += fits;
                 if (__any_sync(kFull, hit_any != 0u)) {
-                    // rare: find the rows that passed and let the warp insert their candidates
+                    // rare: find the rows that passed, exactly, and let the warp insert their candidates
+                    const int64_t s1 = slack1 - rt->D[d][0];
+                    const int64_t s2 = slack2 - rt->D[d][1];
+                    const int64_t xd = x0 + rt->D[d][2];
+                    const int64_t xed = (OBJ == MMEE_OBJ_EDP) ? xe0 + rt->D[d][3] : 0;
 #pragma unroll 1
                     for (int e = 0; e < 5; ++e) {
                         const bool fit = (rt->E[e][0] <= s1) && (rt->E[e][1] <= s2);
