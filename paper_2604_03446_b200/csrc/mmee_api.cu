@@ -28,13 +28,13 @@ using namespace mmee;
 int choose_shape(const Plan& p, int device, LaunchShape* shape) {
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return MMEE_ERR_CUDA;
-    const uint32_t rounds = 8;
-    shape->range_tasks = rounds * kSearchThreads;
+    const uint32_t rounds = 9;
+    shape->range_tasks = rounds * kWorkerThreads;
     shape->slots = (shape->range_tasks - 1) / p.tasks_per_tiling + 2;
     size_t smem = search_smem_bytes(p, shape->slots);
     // Many small tilings per range need many table slots: shrink the range until they fit.
-    while (smem > 96 * 1024 && shape->range_tasks > kSearchThreads) {
-        shape->range_tasks -= kSearchThreads;
+    while (smem > 96 * 1024 && shape->range_tasks > kWorkerThreads) {
+        shape->range_tasks -= kWorkerThreads;
         shape->slots = (shape->range_tasks - 1) / p.tasks_per_tiling + 2;
         smem = search_smem_bytes(p, shape->slots);
     }

@@ -27,6 +27,8 @@ namespace mmee {
 namespace {
 
 constexpr unsigned kFull = 0xffffffffu;
+constexpr size_t kPlanBytes = (sizeof(Plan) + 15) / 16 * 16;
+static_assert(sizeof(Plan) % 4 == 0, "the plan is copied word by word");
 constexpr int kRelCap = (1 << 30) - 1;     // cap of a running threshold-relative sum (see below)
 constexpr int kTermCap = 1 << 29;          // cap of each non-negative addend of such a sum
 constexpr int kSizeCap = (1 << 30) - 1;    // buffer sizes saturate here; the capacity is smaller
@@ -57,7 +59,7 @@ struct alignas(16) OrderTab {
     uint32_t pad;
     RowTab rt[2];                                 // 0 fused, 1 unfused
 };
-constexpr int kOrderItems = 26;
+// 26 items per order: 5 levels each of A, B, C, D, E and the unfused C read-back
 
 // Per tiling: array-level terms by stationary pair and recompute flag.
 struct alignas(16) TilingTab {
@@ -75,7 +77,7 @@ struct alignas(16) TilingTab {
 static_assert(offsetof(TilingTab, Wc) % 16 == 0 && sizeof(int32_t[12]) % 16 == 0, "Wc rows are read as int4");
 static_assert(offsetof(RowTab, Ec) % 16 == 0 && offsetof(OrderTab, rt) % 16 == 0 && sizeof(RowTab) % 16 == 0,
               "Ec rows are read as int4");
-constexpr int kTilingItems = 21;    // 9 stationary pairs x 2 recompute flags, 3 unfused Op1 terms
+// 21 items per tiling: 9 stationary pairs x 2 recompute flags, 3 unfused Op1 terms
 
 struct alignas(16) WarpTop {
     int64_t key[MMEE_MAX_TOPK];
@@ -87,7 +89,7 @@ struct alignas(16) WarpTop {
 struct alignas(16) CtaShared {
     long long G;             // upper bound on the final k-th smallest key (any full list's last key)
     unsigned long long feasible_rows;
-    unsigned long long range_begin;
+    unsigned long long range_begin[2];       // first task of the range whose tables sit in buffer 0 / 1
 };
 
 __device__ __forceinline__ bool pair_less(int64_t ka, uint64_t ia, int64_t kb, uint64_t ib) {
@@ -360,24 +362,33 @@ __device__ __forceinline__ void fill_dead_tiling_item(TilingTab* tb, int item) {
 
 template <int OBJ, bool DUMP>
 __global__ void __launch_bounds__(kSearchThreads, 2)
-search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* __restrict__ scratch,
+search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Scratch* __restrict__ scratch,
               int64_t* __restrict__ dump) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    CtaShared* cs = reinterpret_cast<CtaShared*>(smem_raw);
-    WarpTop* wtops = reinterpret_cast<WarpTop*>(smem_raw + sizeof(CtaShared));
-    TilingTab* ttabs = reinterpret_cast<TilingTab*>(wtops + kSearchThreads / 32);
-    OrderTab* otabs = reinterpret_cast<OrderTab*>(ttabs + shape.slots);
+    // The plan is copied to shared memory: lanes index its tables (query vectors, divisor lists,
+    // block lists) with different indices, which the constant bank would serialise.
+    Plan* plan_sm = reinterpret_cast<Plan*>(smem_raw);
+    for (unsigned i = threadIdx.x; i < sizeof(Plan) / 4; i += kSearchThreads)
+        reinterpret_cast<uint32_t*>(plan_sm)[i] = reinterpret_cast<const uint32_t*>(&plan_arg)[i];
+    const Plan& p = *plan_sm;
+    CtaShared* cs = reinterpret_cast<CtaShared*>(smem_raw + kPlanBytes);
+    WarpTop* wtops = reinterpret_cast<WarpTop*>(smem_raw + kPlanBytes + sizeof(CtaShared));
+    TilingTab* ttabs_all = reinterpret_cast<TilingTab*>(wtops + kSearchThreads / 32);
+    OrderTab* otabs_all = reinterpret_cast<OrderTab*>(ttabs_all + 2 * shape.slots);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int k = (int)p.topk;
     WarpTop* wt = &wtops[warp];
+    // The last warp builds the tables of the next range while the other warps walk the tasks of
+    // the current one (two table buffers); one barrier per range separates the two.
+    const bool builder = warp == kWorkerWarps;
 
     if (tid == 0) {
         cs->G = scratch->G;
         cs->feasible_rows = 0;
     }
     if (lane == 0) wt->count = 0;
-    __syncthreads();
+    __syncthreads();      // the shared copy of the plan is complete
 
     const uint32_t tpt = p.tasks_per_tiling;
     const uint64_t task_begin = p.t_begin * tpt, task_end = p.t_end * tpt;
@@ -386,52 +397,54 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
     const uint32_t n_orders = p.n_orders;
     unsigned long long my_rows = 0;
 
-    while (true) {
-        if (tid == 0) {
-            // Ranges are visited in a stride-permuted order (stride coprime to their number), so that
-            // the first pull of every CTA samples the whole index space and the pruning bound G is
-            // near its final value from the start.
-            const unsigned long long got = atomicAdd(&scratch->next_task, 1ull);
-            cs->range_begin = got < shape.n_ranges
-                                  ? task_begin + ((got * shape.range_stride) % shape.n_ranges) * shape.range_tasks
-                                  : task_end;
-            // exchange the pruning bound with the other CTAs
-            const long long mine = cs->G;
-            const long long theirs = atomicMin(&scratch->G, mine);
-            if (theirs < mine) atomicMin(&cs->G, theirs);
-        }
-        __syncthreads();
-        const uint64_t r0 = cs->range_begin;
-        if (r0 >= task_end) break;
+    // Builder: pull the next range and build its tables into buffer `buf`.  Ranges are visited in a
+    // stride-permuted order (stride coprime to their number), so that the first pull of every CTA
+    // samples the whole index space and the pruning bound G is near its final value from the start.
+    auto build_next = [&](int buf) {
+        unsigned long long got = 0;
+        if (lane == 0) got = atomicAdd(&scratch->next_task, 1ull);
+        got = __shfl_sync(kFull, got, 0);
+        const uint64_t r0 = got < shape.n_ranges
+                                ? task_begin + ((got * shape.range_stride) % shape.n_ranges) * shape.range_tasks
+                                : task_end;
+        if (lane == 0) cs->range_begin[buf] = r0;
+        if (r0 >= task_end) return;
         const uint64_t r1 = (r0 + shape.range_tasks < task_end) ? r0 + shape.range_tasks : task_end;
         const uint64_t t_first = r0 / tpt, t_last = (r1 - 1) / tpt;
         const uint32_t n_slots = (uint32_t)(t_last - t_first + 1);
-
-        // ---- tables of the tilings this range touches
-        if (tid < (int)n_slots) build_tiling_head(p, t_first + tid, &ttabs[tid]);
-        __syncthreads();
-        const uint32_t order_items = n_slots * n_orders * kOrderItems;
-        const uint32_t items = order_items + n_slots * kTilingItems;
-        for (uint32_t it = tid; it < items; it += kSearchThreads) {
-            if (it < order_items) {
-                const uint32_t e = it % kOrderItems;
-                const uint32_t so = it / kOrderItems;
+        TilingTab* ttabs = ttabs_all + buf * shape.slots;
+        OrderTab* otabs = otabs_all + (size_t)buf * shape.slots * n_orders;
+        for (uint32_t sl = lane; sl < n_slots; sl += 32) build_tiling_head(p, t_first + sl, &ttabs[sl]);
+        __syncwarp();
+        // Items are visited kind by kind, so that the 32 lanes always run the same code path.
+        const uint32_t n_so = n_slots * n_orders;
+        auto order_pass = [&](uint32_t first_item, uint32_t n_items) {
+            for (uint32_t it = lane; it < n_so * n_items; it += 32) {
+                const uint32_t so = it / n_items, e = first_item + it % n_items;
                 const uint32_t slot = so / n_orders, os = so % n_orders;
-                if (!ttabs[slot].live) { fill_dead_order_item(&otabs[slot * n_orders + os], (int)e); continue; }
-                build_order_item<OBJ>(p, ttabs[slot].b, p.order_id[os], &otabs[slot * n_orders + os], (int)e);
-            } else {
-                const uint32_t j = it - order_items;
-                const uint32_t slot = j / kTilingItems;
-                if (!ttabs[slot].live) { fill_dead_tiling_item(&ttabs[slot], (int)(j - slot * kTilingItems)); continue; }
-                build_tiling_item(p, &ttabs[slot], (int)(j - slot * kTilingItems));
+                if (!ttabs[slot].live) { fill_dead_order_item(&otabs[so], (int)e); continue; }
+                build_order_item<OBJ>(p, ttabs[slot].b, p.order_id[os], &otabs[so], (int)e);
             }
-        }
-        __syncthreads();
-        if (OBJ == MMEE_OBJ_ENERGY && tid < (int)(2 * n_slots)) {
+        };
+        order_pass(0, 10);      // A, B
+        order_pass(10, 5);      // C
+        order_pass(15, 10);     // D, E
+        order_pass(25, 1);      // C read-back (unfused)
+        auto tiling_pass = [&](uint32_t first_item, uint32_t n_items) {
+            for (uint32_t it = lane; it < n_slots * n_items; it += 32) {
+                const uint32_t slot = it / n_items, e = first_item + it % n_items;
+                if (!ttabs[slot].live) { fill_dead_tiling_item(&ttabs[slot], (int)e); continue; }
+                build_tiling_item(p, &ttabs[slot], (int)e);
+            }
+        };
+        tiling_pass(0, 18);     // stationary pairs x recompute flag
+        tiling_pass(18, 3);     // unfused Op1 compute words
+        __syncwarp();
+        if (OBJ == MMEE_OBJ_ENERGY) {
             // threshold-relative stationary-pair terms (see "32-bit differential keys")
-            TilingTab* tb = &ttabs[tid >> 1];
-            const int rc = tid & 1;
-            {
+            for (uint32_t j = lane; j < 2 * n_slots; j += 32) {
+                TilingTab* tb = &ttabs[j >> 1];
+                const int rc = (int)(j & 1);
                 int64_t m = tb->W[0][rc];
                 for (int s = 1; s < 9; ++s) m = tb->W[s][rc] < m ? tb->W[s][rc] : m;
                 tb->wmin[rc] = m;
@@ -441,12 +454,26 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
                 }
             }
         }
-        __syncthreads();
+    };
+
+    if (builder) build_next(0);
+    __syncthreads();
+
+    for (int iter = 0;; ++iter) {
+        const int buf = iter & 1;
+        const uint64_t r0 = cs->range_begin[buf];
+        if (r0 >= task_end) break;
+        if (builder) build_next(buf ^ 1);
+        if (!builder) {
+        const uint64_t r1 = (r0 + shape.range_tasks < task_end) ? r0 + shape.range_tasks : task_end;
+        const uint64_t t_first = r0 / tpt;
+        const TilingTab* ttabs = ttabs_all + buf * shape.slots;
+        const OrderTab* otabs = otabs_all + (size_t)buf * shape.slots * n_orders;
 
         // ---- tasks
         const uint32_t w_first = (uint32_t)(r0 - t_first * tpt);      // task of r0 inside its tiling
         const uint32_t n_range = (uint32_t)(r1 - r0);
-        for (uint32_t off = 0; off < n_range; off += kSearchThreads) {
+        for (uint32_t off = 0; off < n_range; off += kWorkerThreads) {
             const bool valid = off + tid < n_range;
             const uint32_t o = valid ? off + tid : n_range - 1;
             const uint32_t wa = w_first + o;
@@ -670,7 +697,8 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
             }
             my_rows += rows;
         }
-        __syncthreads();      // tables are rebuilt at the top of the next range
+        }   // workers
+        __syncthreads();      // this buffer is rebuilt during the next range
     }
 
     // ---- feasible count
@@ -680,7 +708,7 @@ search_kernel(const __grid_constant__ Plan p, const LaunchShape shape, Scratch* 
 
     // ---- merge the warps' lists into warp 0's, then publish this CTA's partial list
     if (warp == 0) {
-        for (int w2 = 1; w2 < kSearchThreads / 32; ++w2) {
+        for (int w2 = 1; w2 < kWorkerWarps; ++w2) {
             const WarpTop* src = &wtops[w2];
             const int n = src->count;
             for (int j = 0; j < n; ++j)
@@ -788,8 +816,8 @@ cudaError_t occupancy_t(int* blocks_per_sm, size_t smem) {
 }  // namespace
 
 size_t search_smem_bytes(const Plan& p, uint32_t slots) {
-    return sizeof(CtaShared) + (kSearchThreads / 32) * sizeof(WarpTop) + slots * sizeof(TilingTab) +
-           (size_t)slots * p.n_orders * sizeof(OrderTab);
+    return kPlanBytes + sizeof(CtaShared) + (kSearchThreads / 32) * sizeof(WarpTop) + 2 * slots * sizeof(TilingTab) +
+           2 * (size_t)slots * p.n_orders * sizeof(OrderTab);
 }
 
 cudaError_t search_occupancy(const Plan& p, size_t smem, int* blocks_per_sm) {

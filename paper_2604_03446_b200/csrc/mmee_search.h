@@ -9,6 +9,8 @@
 namespace mmee {
 
 constexpr int kSearchThreads = 256;
+constexpr int kWorkerWarps = kSearchThreads / 32 - 1;     // the last warp builds tables
+constexpr int kWorkerThreads = kWorkerWarps * 32;
 
 // One CTA's k best (key, idx) pairs, best first.
 struct Partial {
@@ -30,7 +32,7 @@ struct Scratch {
 
 struct LaunchShape {
     uint32_t grid;          // persistent CTAs
-    uint32_t range_tasks;   // tasks a CTA takes per pull (multiple of kSearchThreads)
+    uint32_t range_tasks;   // tasks a CTA takes per pull (multiple of kWorkerThreads)
     uint32_t slots;         // tilings one range can touch
     uint32_t smem_bytes;
     uint64_t n_ranges;      // ranges of the searched task interval
