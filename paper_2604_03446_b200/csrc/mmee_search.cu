@@ -535,11 +535,9 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                 Q[s] = qptr[2 * s];
             }
             const uint64_t task_first_idx = tq * kCandPerTask;
-            if (lane == 0) {
-                const long long seen = *reinterpret_cast<volatile long long*>(&scratch->G);
-                if (seen < cs->G) atomicMin(&cs->G, seen);
-            }
-            __syncwarp();
+            // The other CTAs' pruning bound: the load is issued here and consumed at the end of the
+            // task, so that its latency is covered by the task's own work.
+            const long long g_seen = (lane == 0) ? *reinterpret_cast<volatile long long*>(&scratch->G) : 0;
             // Threshold state of this lane: T1 = the non-strict threshold (a key passes iff key < T1);
             // for a group whose first index lies above `ti`, the index of the list's last entry, the
             // threshold is T1 - delta (ties with that entry cannot displace it).
@@ -605,10 +603,13 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                     const int4 dc = *reinterpret_cast<const int4*>(rt->Dc[d]);
                     const int s1c = slack1c - dc.x;
                     const int s2c = slack2c - dc.y;
-                    int acc = INT_MAX, acc1 = INT_MAX, acc2 = INT_MAX;    // independent chains
+                    int acc = INT_MAX;
                     fits = 0;
                     if constexpr (OBJ == MMEE_OBJ_ENERGY) {
                         const int uc = __viaddmin_s32(ut[0], dc.z, kRelCap);
+                        int accs[9];          // one chain per stationary pair: nine independent chains
+#pragma unroll
+                        for (int s = 0; s < 9; ++s) accs[s] = INT_MAX;
 #pragma unroll
                         for (int e = 0; e < 5; ++e) {
                             const unsigned fit = (unsigned)(E1c[e] <= s1c) & (unsigned)(E2c[e] <= s2c);   // Eq. (4)
@@ -616,13 +617,10 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                             int xc = __viaddmin_s32(uc, Gc[e], kRelCap);
                             xc = fit ? xc : kRelCap;
 #pragma unroll
-                            for (int s = 0; s < 9; s += 3) {                                      // min(key_s - thr)
-                                acc = __viaddmin_s32(xc, Wc[s], acc);
-                                acc1 = __viaddmin_s32(xc, Wc[s + 1], acc1);
-                                acc2 = __viaddmin_s32(xc, Wc[s + 2], acc2);
-                            }
+                            for (int s = 0; s < 9; ++s) accs[s] = __viaddmin_s32(xc, Wc[s], accs[s]);   // min(key_s - thr)
                         }
-                        acc = min(acc, min(acc1, acc2));
+                        acc = __vimin3_s32(__vimin3_s32(accs[0], accs[1], accs[2]), __vimin3_s32(accs[3], accs[4], accs[5]),
+                                           __vimin3_s32(accs[6], accs[7], accs[8]));
                     } else {
                         int uc[3];
 #pragma unroll
@@ -696,6 +694,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                 }
             }
             my_rows += rows;
+            if (lane == 0 && g_seen < cs->G) atomicMin(&cs->G, g_seen);
         }
         }   // workers
         __syncthreads();      // this buffer is rebuilt during the next range
