@@ -26,8 +26,10 @@ using namespace mmee;
 
 // Tasks a CTA pulls per visit of the global counter, and the tilings such a range can touch.
 int choose_shape(const Plan& p, int device, LaunchShape* shape) {
-    cudaDeviceProp prop;
-    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return MMEE_ERR_CUDA;
+    int sm_count = 0, smem_optin = 0;      // attribute queries: cudaGetDeviceProperties costs milliseconds
+    if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess)
+        return MMEE_ERR_CUDA;
     const uint32_t rounds = 9;
     shape->range_tasks = rounds * kWorkerThreads;
     shape->slots = (shape->range_tasks - 1) / p.tasks_per_tiling + 2;
@@ -38,12 +40,12 @@ int choose_shape(const Plan& p, int device, LaunchShape* shape) {
         shape->slots = (shape->range_tasks - 1) / p.tasks_per_tiling + 2;
         smem = search_smem_bytes(p, shape->slots);
     }
-    if (smem > (size_t)prop.sharedMemPerBlockOptin) return MMEE_ERR_RANGE;
+    if (smem > (size_t)smem_optin) return MMEE_ERR_RANGE;
     shape->smem_bytes = (uint32_t)smem;
     int per_sm = 0;
     if (search_occupancy(p, smem, &per_sm) != cudaSuccess || per_sm < 1) return MMEE_ERR_CUDA;
     if (per_sm > 2) per_sm = 2;
-    uint64_t grid = (uint64_t)prop.multiProcessorCount * (uint32_t)per_sm;
+    uint64_t grid = (uint64_t)sm_count * (uint32_t)per_sm;
     const uint64_t tasks = (p.t_end - p.t_begin) * p.tasks_per_tiling;
     const uint64_t ranges = (tasks + shape->range_tasks - 1) / shape->range_tasks;
     if (grid > ranges) grid = ranges ? ranges : 1;
