@@ -148,6 +148,33 @@ int mmee_search(mmee_handle_t* handle, void* cuda_stream, mmee_result_t* out_bes
 
 int mmee_destroy(mmee_handle_t* handle);
 
+/*
+ * mmee_search_static -- the same search as mmee_create + mmee_search + mmee_destroy, for callers
+ * that must not allocate device memory.  (The paper has no counterpart: this is an interface
+ * variant of the library, not a part of the method.)
+ *
+ * For whom: a process that has given the whole device to its own memory pool (a cudaMalloc from a
+ * library then fails), or a latency-critical loop that cannot afford the device-wide
+ * synchronisation of cudaMalloc / cudaFree.  This call makes no cudaMalloc, cudaFree or other
+ * allocating call.  Its scratch (work counter, pruning bound, one partial top-k list per CTA) is a
+ * fixed 135 200-byte array inside the library image, present on every device that loads the
+ * library for as long as the process lives.
+ *
+ *   workload, arch, objective : HOST, as for mmee_create; planned on the host at every call.
+ *   out_best, out_topk        : DEVICE, caller-owned, as for mmee_search (out_topk may be NULL).
+ * Asynchronous on `cuda_stream`.  The first call on a device looks up the array's device address
+ * (with that device current); make that first call before any stream capture begins.
+ * Limits: the array holds the partial lists of at most 512 persistent CTAs; a device whose launch
+ * shape needs more is refused with MMEE_ERR_RANGE.  Other errors as mmee_create / mmee_search.
+ * All calls on a device share the one array and it keeps the previous call's contents: the call
+ * clears the header itself, but two mmee_search_static calls that overlap on the GPU (for instance
+ * on different streams) race on it and give undefined results: serialise them.  Searches through
+ * handles use their own scratch and are not affected.
+ */
+int mmee_search_static(const mmee_workload_t* workload, const mmee_arch_t* arch,
+                       const mmee_objective_t* objective, void* cuda_stream,
+                       mmee_result_t* out_best, mmee_result_t* out_topk);
+
 /* Number of candidates / tilings / rows of the full space of the handle (HOST values). */
 uint64_t mmee_num_candidates(const mmee_handle_t* handle);
 uint64_t mmee_num_tilings(const mmee_handle_t* handle);

@@ -19,7 +19,7 @@ MAX_TOPK = 16
 NO_INDEX = 2 ** 64 - 1
 OK, ERR_ARG, ERR_OVERFLOW, ERR_QUANTUM, ERR_NO_FEASIBLE, ERR_CUDA, ERR_TIMEOUT, ERR_RANGE = range(8)
 
-EXPORTS = ("mmee_create", "mmee_search", "mmee_destroy", "mmee_num_candidates", "mmee_num_tilings",
+EXPORTS = ("mmee_create", "mmee_search", "mmee_destroy", "mmee_search_static", "mmee_num_candidates", "mmee_num_tilings",
            "mmee_num_rows", "mmee_strerror", "mmee_last_cuda_error", "mmee_eval", "mmee_dump_keys", "mmee_solve_host",
            "mmee_query_vector", "mmee_recompute_flag", "mmee_last_search_stats", "mmee_kernel_timing",
            "mmee_alu_peak")
@@ -97,6 +97,8 @@ def library():
     L.mmee_create.argtypes = [C.POINTER(Workload), C.POINTER(Arch), C.POINTER(Objective), C.POINTER(H)]
     L.mmee_search.argtypes = [H, C.c_void_p, C.c_void_p, C.c_void_p]
     L.mmee_destroy.argtypes = [H]
+    L.mmee_search_static.argtypes = [C.POINTER(Workload), C.POINTER(Arch), C.POINTER(Objective),
+                                     C.c_void_p, C.c_void_p, C.c_void_p]
     for name in ("mmee_num_candidates", "mmee_num_tilings", "mmee_num_rows"):
         getattr(L, name).argtypes = [H]
         getattr(L, name).restype = C.c_uint64
@@ -170,6 +172,16 @@ def mmee_search(handle, out_best, out_topk=None, stream=None) -> None:
     _check(library().mmee_search(handle, _stream_ptr(stream), C.c_void_p(out_best.data_ptr()),
                                  C.c_void_p(out_topk.data_ptr()) if out_topk is not None else None),
            "mmee_search")
+
+
+def mmee_search_static(workload: dict, arch: dict, objective: dict, out_best, out_topk=None, stream=None) -> None:
+    """Search without device allocation: plans on the host, uses the library's fixed scratch.
+    Asynchronous; out_best / out_topk are caller-owned uint8 CUDA tensors (result_buffer())."""
+    _check(library().mmee_search_static(_fill(Workload(), workload), _fill(Arch(), arch),
+                                        _fill(Objective(), objective), _stream_ptr(stream),
+                                        C.c_void_p(out_best.data_ptr()),
+                                        C.c_void_p(out_topk.data_ptr()) if out_topk is not None else None),
+           "mmee_search_static")
 
 
 def mmee_eval(handle, idx_begin: int, count: int, out, stream=None) -> None:
