@@ -39,8 +39,18 @@ ALG_OPS_PER_CANDIDATE = {0: 1.0 + 5.0 / 9.0, 1: 2.0 + 8.0 / 9.0, 2: 13.0 + 12.0 
 INT_LANES_PER_SM = 64          # 4 sub-partitions x 16 integer-ALU lanes
 
 
-def workload_config():
-    return mi.config2()
+WORKLOADS = {"tiny": mi.config1, "bert": mi.config2, "llama": mi.config3, "gqa": mi.config4}
+
+
+def workload_jobs(name):
+    """(workload name, [(problem, search), ...]): one step runs every listed search once.
+    The default, "bert", is the configuration the headline metric is quoted on; "sweep" is the
+    28-point sequence-length sweep (one energy search per point)."""
+    if name == "sweep":
+        pts = mi.config5()
+        return "sweep_s1k_to_64k", [(c, c["searches"][0]) for c in pts]
+    cfg = WORKLOADS[name]()
+    return cfg["name"], [(cfg, s) for s in cfg["searches"]]
 
 
 class ClockSampler:
@@ -86,10 +96,9 @@ class ClockSampler:
                     reasons=sorted(reasons), samples=len(sm))
 
 
-def cpu_baseline(cfg, budget_s: float = 12.0):
+def cpu_baseline(cfg, obj, budget_s: float = 12.0):
     """The oracle as it stands on the host cores, on a bounded tiling sub-range of the workload."""
     import oracle
-    obj = cfg["searches"][0]
     p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
     probe = max(1, min(p.T, 40))
     t0 = time.perf_counter()
@@ -111,8 +120,8 @@ def run_reference(args, rank):
     if rank != 0:
         return
     import oracle
-    cfg = workload_config()
-    obj = cfg["searches"][0]
+    wname, jobs = workload_jobs(args.workload)
+    cfg, obj = jobs[0]
     p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
     n_t = max(1, min(p.T, 24))
     stride = max(1, (p.T - n_t) // max(1, args.steps + args.warmup))
@@ -132,7 +141,7 @@ def run_reference(args, rank):
         impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
         warmup=args.warmup, ms_per_step=1e3 * t_total / args.steps, higher_is_better=True, scaling="weak",
         vs_baseline=None, dtype="int64", data="synthetic",
-        config=dict(workload=cfg["name"], note="CPU oracle on host cores; " + sample),
+        config=dict(workload=wname, note="CPU oracle on host cores; " + sample),
         cpu_baseline=dict(value=value, unit=UNIT, cores=oracle.threads_used(), kind="oracle", sample=sample),
         e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))))
 
@@ -144,6 +153,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="bert", choices=sorted(WORKLOADS) + ["sweep"])
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -163,9 +173,9 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    cfg = workload_config()
-    searches = cfg["searches"]
-    handles = [mm.mmee_create(cfg["workload"], cfg["arch"], s) for s in searches]
+    wname, jobs = workload_jobs(args.workload)
+    searches = [s for _, s in jobs]
+    handles = [mm.mmee_create(c["workload"], c["arch"], s) for c, s in jobs]
     for h in handles:
         mm.mmee_kernel_timing(h, True)
     outs = [(mm.result_buffer(1), mm.result_buffer(s["topk"])) for s in searches]
@@ -234,13 +244,13 @@ def main():
     e2e_steps = max(3, min(args.steps, 30))
     h2d = d2h = 0
     for _ in range(2):
-        for s in searches:
-            mm.mmee_solve_host(cfg["workload"], cfg["arch"], s)
+        for c, s in jobs:
+            mm.mmee_solve_host(c["workload"], c["arch"], s)
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
         h2d = d2h = 0
-        for s in searches:
-            _, _, a, b = mm.mmee_solve_host(cfg["workload"], cfg["arch"], s)
+        for c, s in jobs:
+            _, _, a, b = mm.mmee_solve_host(c["workload"], c["arch"], s)
             h2d += a
             d2h += b
     e2e_s = time.perf_counter() - t0
@@ -258,8 +268,9 @@ def main():
             sm = statistics.mean(k[i][0] for k in kernel_ms)
             fm = statistics.mean(k[i][1] for k in kernel_ms)
             ops = bests[i].n_feasible * ALG_OPS_PER_CANDIDATE[s["objective"]]
-            per_kernel.append(dict(kernel="search_kernel<%s>" % OBJ_NAMES[s["objective"]], avg_ms=sm,
-                                   finalize_avg_ms=fm, candidates=n, feasible=bests[i].n_feasible,
+            per_kernel.append(dict(kernel="search_kernel<%s>" % OBJ_NAMES[s["objective"]], problem=jobs[i][0]["name"],
+                                   avg_ms=sm, finalize_avg_ms=fm, candidates=n, feasible=bests[i].n_feasible,
+                                   pruned_fraction=1.0 - bests[i].n_feasible / n, time_to_optimum_ms=tto_ms[i],
                                    candidates_per_s=n / (sm * 1e-3), achieved_gops=ops / (sm * 1e-3) / 1e9))
         dom = max(per_kernel, key=lambda k: k["avg_ms"])
         sm_mhz = clocks.get("sm_mhz") or peaks[3]
@@ -276,7 +287,7 @@ def main():
             metric=METRIC, value=world * cand_per_step * args.steps / (total_ms * 1e-3), unit=UNIT,
             n_gpus=world, steps=args.steps, warmup=args.warmup, ms_per_step=total_ms / args.steps,
             higher_is_better=True, scaling="weak", vs_baseline=None, dtype="int64", data="synthetic",
-            config=dict(workload=cfg["name"], searches=[OBJ_NAMES[s["objective"]] for s in searches],
+            config=dict(workload=wname, searches=[OBJ_NAMES[s["objective"]] for s in searches],
                         candidates_per_step=cand_per_step, parallelism="replicas only",
                         l2="flushed between steps (256 MB write); the path reads no HBM-resident input",
                         grid=stats[0].grid, block=stats[0].block, smem_bytes=stats[0].smem_bytes),
@@ -287,7 +298,7 @@ def main():
             time_to_optimum_ms=tto_ms, device_time_to_optimum_ms=[k["avg_ms"] + k["finalize_avg_ms"] for k in per_kernel],
             kernels=per_kernel, roofline=roofline)
         if not args.no_cpu_baseline:
-            line["cpu_baseline"] = cpu_baseline(cfg)
+            line["cpu_baseline"] = cpu_baseline(*jobs[0])
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
