@@ -90,6 +90,7 @@ struct alignas(16) CtaShared {
     long long G;             // upper bound on the final k-th smallest key (any full list's last key)
     unsigned long long feasible_rows;
     unsigned long long range_begin[2];       // first task of the range whose tables sit in buffer 0 / 1
+    unsigned int cursor[2];                  // next unassigned task of that range, relative to its begin
 };
 
 __device__ __forceinline__ bool pair_less(int64_t ka, uint64_t ia, int64_t kb, uint64_t ib) {
@@ -407,7 +408,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
         const uint64_t r0 = got < shape.n_ranges
                                 ? task_begin + ((got * shape.range_stride) % shape.n_ranges) * shape.range_tasks
                                 : task_end;
-        if (lane == 0) cs->range_begin[buf] = r0;
+        if (lane == 0) { cs->range_begin[buf] = r0; cs->cursor[buf] = 0; }
         if (r0 >= task_end) return;
         const uint64_t r1 = (r0 + shape.range_tasks < task_end) ? r0 + shape.range_tasks : task_end;
         const uint64_t t_first = r0 / tpt, t_last = (r1 - 1) / tpt;
@@ -473,9 +474,15 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
         // ---- tasks
         const uint32_t w_first = (uint32_t)(r0 - t_first * tpt);      // task of r0 inside its tiling
         const uint32_t n_range = (uint32_t)(r1 - r0);
-        for (uint32_t off = 0; off < n_range; off += kWorkerThreads) {
-            const bool valid = off + tid < n_range;
-            const uint32_t o = valid ? off + tid : n_range - 1;
+        // Worker warps take 32 tasks at a time from a cursor in shared memory: warps whose tasks fall
+        // into pruned tilings come back sooner and take more.
+        while (true) {
+            uint32_t off = 0;
+            if (lane == 0) off = atomicAdd(&cs->cursor[buf], 32u);
+            off = __shfl_sync(kFull, off, 0);
+            if (off >= n_range) break;
+            const bool valid = off + lane < n_range;
+            const uint32_t o = valid ? off + lane : n_range - 1;
             const uint32_t wa = w_first + o;
             const uint32_t slot = wa / tpt;
             const uint32_t w = wa - slot * tpt;
