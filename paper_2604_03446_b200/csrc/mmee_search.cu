@@ -197,6 +197,46 @@ __device__ __forceinline__ int sat_s32(int64_t v) {
     return r;
 }
 
+// EDP filter for one row on the FP64 pipe: for each of the nine mappings energy = de + dW[s],
+// key ~ energy * max(dl[s/3], dQP[s]); max(a, b) * e <= t  <=>  a * e <= t and b * e <= t for e >= 0, so
+// each mapping is two multiplies and two compares combined in predicates (a double-precision max or
+// min would cost a compare and two selects each).  Returns 1 if the row fits and some product <= thr.
+__device__ __forceinline__ unsigned edp_row_test(double de, const double (&dl)[3], const double (&dW)[9],
+                                                 const double (&dQP)[9], double thr, unsigned fit) {
+    unsigned hit;
+#define MMEE_EDP_CAND(w, l, q)                                        \
+    "add.f64 e, %2, " w ";\n\t"                                       \
+    "mul.f64 a, e, " l ";\n\t"                                        \
+    "mul.f64 b, e, " q ";\n\t"                                        \
+    "setp.le.f64 r, a, %24;\n\t"                                      \
+    "setp.le.and.f64 r, b, %24, r;\n\t"                               \
+    "or.pred p, p, r;\n\t"
+    asm("{\n\t"
+        ".reg .pred p, r, f;\n\t"
+        ".reg .f64 e, a, b;\n\t"
+        "setp.ne.u32 p, 0, 0;\n\t"
+        MMEE_EDP_CAND("%6", "%3", "%15")
+        MMEE_EDP_CAND("%7", "%3", "%16")
+        MMEE_EDP_CAND("%8", "%3", "%17")
+        MMEE_EDP_CAND("%9", "%4", "%18")
+        MMEE_EDP_CAND("%10", "%4", "%19")
+        MMEE_EDP_CAND("%11", "%4", "%20")
+        MMEE_EDP_CAND("%12", "%5", "%21")
+        MMEE_EDP_CAND("%13", "%5", "%22")
+        MMEE_EDP_CAND("%14", "%5", "%23")
+        "setp.ne.u32 f, %1, 0;\n\t"
+        "and.pred p, p, f;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}"
+        : "=r"(hit)
+        : "r"(fit), "d"(de), "d"(dl[0]), "d"(dl[1]), "d"(dl[2]),
+          "d"(dW[0]), "d"(dW[1]), "d"(dW[2]), "d"(dW[3]), "d"(dW[4]), "d"(dW[5]), "d"(dW[6]), "d"(dW[7]), "d"(dW[8]),
+          "d"(dQP[0]), "d"(dQP[1]), "d"(dQP[2]), "d"(dQP[3]), "d"(dQP[4]), "d"(dQP[5]), "d"(dQP[6]), "d"(dQP[7]), "d"(dQP[8]),
+          "d"(thr));
+#undef MMEE_EDP_CAND
+    return hit;
+}
+
 // Rare path: some lane of the warp has a key below its threshold in this row.  Every lane
 // re-evaluates its nine candidates of the row from the shared tables and the warp inserts the
 // passing ones, one at a time, into its sorted list.
@@ -575,6 +615,14 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                 Wc[8] = w2.x;
             }
             int ut[3] = {0, 0, 0};      // saturated task-level part of key - thr
+            double dW[9], dQP[9], dthr = 0.0;
+            if constexpr (OBJ == MMEE_OBJ_EDP) {
+#pragma unroll
+                for (int s = 0; s < 9; ++s) {
+                    dW[s] = (double)W[s];
+                    dQP[s] = (double)(Q[s] + P[s / 3]);
+                }
+            }
             auto refresh = [&](int64_t t) {
                 if constexpr (OBJ == MMEE_OBJ_ENERGY) {
                     B = t - wmin;
@@ -589,6 +637,10 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                     }
 #pragma unroll
                     for (int s = 0; s < 9; ++s) Qc[s] = sat_s32(Q[s] + P[s / 3] - t);
+                } else {
+                    // EDP keys are bit patterns of positive doubles; anything from +inf up means "no bound yet"
+                    dthr = t >= 0x7ff0000000000000ll ? __longlong_as_double(0x7ff0000000000000ll)
+                                                     : __longlong_as_double(t) * (1.0 + 1e-14);
                 }
             };
             refresh(T1);
@@ -647,6 +699,31 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                     }
                     const uint64_t group_first_idx = task_first_idx + (uint64_t)(d * 45);
                     hit_any = acc < (group_first_idx > ti ? -delta : 0);      // no overflow at acc = INT_MAX
+                } else if constexpr (!DUMP && OBJ == MMEE_OBJ_EDP) {
+                    // The energy-delay product is not separable, so the filter is a double-precision
+                    // evaluation of every mapping on the FP64 pipe: energy and latency sums converted
+                    // once per row, then an add, two multiplies and two compares per mapping.  Each
+                    // approximate product is within a few 2^-53 of the exact key, so comparing against
+                    // the threshold widened by 1e-14 relative can flag a row needlessly but never miss
+                    // one; the exact 64-bit path below decides.
+                    const int4 dc = *reinterpret_cast<const int4*>(rt->Dc[d]);
+                    const int s1c = slack1c - dc.x;
+                    const int s2c = slack2c - dc.y;
+                    const int64_t xd = x0 + rt->D[d][2];
+                    const int64_t xed = xe0 + rt->D[d][3];
+                    fits = 0;
+                    hit_any = 0;
+#pragma unroll
+                    for (int e = 0; e < 5; ++e) {
+                        const unsigned fit = (unsigned)(E1c[e] <= s1c) & (unsigned)(E2c[e] <= s2c);       // Eq. (4)
+                        fits += fit;
+                        const int64_t x = xd + rt->E[e][2];
+                        const double de = (double)(xed + rt->E[e][3]);
+                        double dl[3];
+#pragma unroll
+                        for (int j = 0; j < 3; ++j) dl[j] = (double)(x + P[j]);
+                        hit_any |= edp_row_test(de, dl, dW, dQP, dthr, fit);
+                    }
                 } else {
                     const int64_t s1 = slack1 - rt->D[d][0];
                     const int64_t s2 = slack2 - rt->D[d][1];
