@@ -185,5 +185,33 @@ def simulate(bound, pi: int, beta) -> SimOut:
     return out
 
 
+class RowSymbols(C.Structure):
+    _fields_ = [("bs_q", C.c_uint8 * 5), ("da_q", C.c_uint8 * 5), ("tau", C.c_uint8 * 5),
+                ("recompute", C.c_uint8)]
+
+
+def row_symbolic(pi: int, beta) -> RowSymbols:
+    out = RowSymbols()
+    L = lib()
+    L.mo_row_symbolic.argtypes = [C.c_uint32, C.POINTER(C.c_uint32), C.POINTER(RowSymbols)]
+    rc = L.mo_row_symbolic(pi, (C.c_uint32 * 5)(*beta), out)
+    if rc:
+        raise OracleError(rc)
+    return out
+
+
+def symbolic_prune():
+    """(keep uint8[18750], kept per recompute group, rows per recompute group) -- Eq. (12) of Section VI-B."""
+    import numpy as np
+    keep = np.zeros(18750, dtype=np.uint8)
+    kept, total = (C.c_uint32 * 2)(), (C.c_uint32 * 2)()
+    L = lib()
+    L.mo_symbolic_prune.argtypes = [C.POINTER(C.c_uint8), C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]
+    rc = L.mo_symbolic_prune(keep.ctypes.data_as(C.POINTER(C.c_uint8)), kept, total)
+    if rc:
+        raise OracleError(rc)
+    return keep, list(kept), list(total)
+
+
 def threads_used() -> int:
     return lib().mo_threads_used()

@@ -499,6 +499,152 @@ int mo_search(const mo_problem* p, mo_record* out_topk, uint64_t* n_total, uint6
 }
 
 /* ------------------------------------------------------------------------------------------ */
+/* symbolic rows and offline pruning (Section VI-B)                                            */
+/* ------------------------------------------------------------------------------------------ */
+/*
+ * The same rules as in mo_eval, with "multiply by a bound" replaced by "add the bound to a set":
+ * a monomial in the loop bounds with exponents 0/1 is the set of bounds it contains (the query
+ * vector of Section V-E).
+ */
+static uint8_t sym_buffer(int x, int beta, const nest_t* n)
+{
+    uint8_t q = (uint8_t)((1u << (4 + OWN[x][0])) | (1u << (4 + OWN[x][1])));   /* the tile: both x_G */
+    for (int v = 4; v <= beta; ++v)
+        if (n->present[v] && is_own(x, n->lev[v])) q |= (uint8_t)(1u << n->lev[v]);
+    return q;
+}
+
+static uint8_t sym_dram_own_blocker(int x, int beta, uint8_t bs, const nest_t* n, const int eff[4])
+{
+    int blocker = 0;
+    for (int v = beta + 1; v <= 7; ++v) {
+        if (!n->present[v]) continue;
+        if (is_own(x, n->lev[v])) { blocker = v; break; }
+    }
+    if (!blocker) return bs;
+    uint8_t q = (uint8_t)(bs | (1u << n->lev[blocker]));
+    for (int u = blocker + 1; u <= 7; ++u)
+        if (n->present[u] && eff[n->lev[u]]) q |= (uint8_t)(1u << n->lev[u]);
+    return q;
+}
+
+int mo_row_symbolic(uint32_t pi, const uint32_t beta[5], mo_row_symbols* o)
+{
+    if (pi > 5 || !beta || !o) return MO_ERR_ARG;
+    for (int x = 0; x < 5; ++x) if (beta[x] < 3 || beta[x] > 7) return MO_ERR_ARG;
+    memset(o, 0, sizeof(*o));
+    nest_t fused;
+    memset(&fused, 0, sizeof(fused));
+    fused.lev[4] = LP_K;
+    fused.lev[5] = ORDERS[pi][2];
+    fused.lev[6] = ORDERS[pi][1];
+    fused.lev[7] = ORDERS[pi][0];
+    for (int v = 4; v <= 7; ++v) fused.present[v] = 1;
+    for (int x = 0; x < 5; ++x) {
+        o->bs_q[x] = sym_buffer(x, (int)beta[x], &fused);
+        o->tau[x] = beta[x] >= 4;
+    }
+    int c_blocker = 0, rc = 0;
+    for (int v = (int)beta[OPD_C] + 1; v <= 7; ++v)
+        if (fused.lev[v] == LP_I || fused.lev[v] == LP_L) { c_blocker = v; break; }
+    if (c_blocker)
+        for (int u = c_blocker + 1; u <= 7; ++u)
+            if (fused.lev[u] == LP_J) rc = 1;
+    o->recompute = (uint8_t)rc;
+    int eff_p[4] = {1, 1, 1, rc};
+    int eff_c[4] = {1, 0, 1, 1};
+    for (int x = 0; x < 5; ++x) {
+        if (x == OPD_C) continue;
+        int consumer = (x == OPD_D || x == OPD_E);
+        if (consumer && beta[x] == 3)
+            o->da_q[x] = (uint8_t)(o->bs_q[x] | (1u << LP_I) | (1u << LP_L) | (1u << LP_J));
+        else
+            o->da_q[x] = sym_dram_own_blocker(x, (int)beta[x], o->bs_q[x], &fused, consumer ? eff_c : eff_p);
+    }
+    return MO_OK;
+}
+
+/* A sum of monomials, each a set of bounds (all bounds are integers >= 1). */
+typedef struct { int n; uint8_t term[6]; } sym_sum;
+
+/* P >= Q for every assignment of the bounds if the terms of Q can be matched one-to-one into
+ * terms of P with term_Q a subset of term_P (a product over a superset of bounds >= 1 is not
+ * smaller).  This is the comparison "without specific tiling solutions" of Section VI-B. */
+static int match_terms(const sym_sum* p, const sym_sum* q, int qi, unsigned used)
+{
+    if (qi == q->n) return 1;
+    for (int i = 0; i < p->n; ++i) {
+        if (used & (1u << i)) continue;
+        if ((q->term[qi] & p->term[i]) != q->term[qi]) continue;
+        if (match_terms(p, q, qi + 1, used | (1u << i))) return 1;
+    }
+    return 0;
+}
+static int sum_ge(const sym_sum* p, const sym_sum* q) { return q->n <= p->n && match_terms(p, q, 0, 0); }
+/* "greater" in the paper's symbolic sense (i_G k_G < i_G k_G i_D): >= and not also <=. */
+static int sum_gt(const sym_sum* p, const sym_sum* q) { return sum_ge(p, q) && !sum_ge(q, p); }
+
+typedef struct { sym_sum bs1, bs2, da; int rc; } sym_row;
+
+static void sym_row_build(uint32_t pi, const uint32_t beta[5], sym_row* r)
+{
+    mo_row_symbols s;
+    mo_row_symbolic(pi, beta, &s);
+    r->rc = s.recompute;
+    /* Eq. (1), (2): retained operands of the other operator count */
+    r->bs1.n = 0; r->bs2.n = 0; r->da.n = 0;
+    r->bs1.term[r->bs1.n++] = s.bs_q[OPD_A]; r->bs1.term[r->bs1.n++] = s.bs_q[OPD_B];
+    r->bs1.term[r->bs1.n++] = s.bs_q[OPD_C];
+    if (s.tau[OPD_D]) r->bs1.term[r->bs1.n++] = s.bs_q[OPD_D];
+    if (s.tau[OPD_E]) r->bs1.term[r->bs1.n++] = s.bs_q[OPD_E];
+    r->bs2.term[r->bs2.n++] = s.bs_q[OPD_C]; r->bs2.term[r->bs2.n++] = s.bs_q[OPD_D];
+    r->bs2.term[r->bs2.n++] = s.bs_q[OPD_E];
+    if (s.tau[OPD_A]) r->bs2.term[r->bs2.n++] = s.bs_q[OPD_A];
+    if (s.tau[OPD_B]) r->bs2.term[r->bs2.n++] = s.bs_q[OPD_B];
+    r->da.term[r->da.n++] = s.da_q[OPD_A]; r->da.term[r->da.n++] = s.da_q[OPD_B];
+    r->da.term[r->da.n++] = s.da_q[OPD_D]; r->da.term[r->da.n++] = s.da_q[OPD_E];
+}
+
+/* BS = max(BS1, BS2) (Eq. 4): BS_v >= BS_u when both operator sums are >=; > when, in addition,
+ * one of them is >. */
+static int bs_ge(const sym_row* v, const sym_row* u) { return sum_ge(&v->bs1, &u->bs1) && sum_ge(&v->bs2, &u->bs2); }
+static int bs_gt(const sym_row* v, const sym_row* u)
+{
+    return bs_ge(v, u) && (sum_gt(&v->bs1, &u->bs1) || sum_gt(&v->bs2, &u->bs2));
+}
+
+int mo_symbolic_prune(uint8_t* keep, uint32_t kept_per_group[2], uint32_t rows_per_group[2])
+{
+    enum { NROWS = 18750 };
+    if (!keep || !kept_per_group || !rows_per_group) return MO_ERR_ARG;
+    sym_row* rows = (sym_row*)malloc(sizeof(sym_row) * NROWS);
+    if (!rows) return MO_ERR_ARG;
+    for (uint32_t r = 0; r < NROWS; ++r) {
+        uint32_t q = r % 3125u;
+        uint32_t beta[5] = {3 + q / 625u, 3 + (q / 125u) % 5u, 3 + (q / 25u) % 5u, 3 + (q / 5u) % 5u, 3 + q % 5u};
+        sym_row_build(r / 3125u, beta, &rows[r]);
+    }
+    kept_per_group[0] = kept_per_group[1] = rows_per_group[0] = rows_per_group[1] = 0;
+#pragma omp parallel for schedule(dynamic, 64)
+    for (int v = 0; v < NROWS; ++v) {
+        int pruned = 0;
+        for (int u = 0; u < NROWS && !pruned; ++u) {
+            if (u == v || rows[u].rc != rows[v].rc) continue;
+            /* Eq. (12): s_v is inferior to s_u */
+            if (bs_ge(&rows[v], &rows[u]) && sum_gt(&rows[v].da, &rows[u].da)) pruned = 1;
+            else if (bs_gt(&rows[v], &rows[u]) && sum_ge(&rows[v].da, &rows[u].da)) pruned = 1;
+        }
+        keep[v] = (uint8_t)!pruned;
+    }
+    for (int v = 0; v < NROWS; ++v) {
+        rows_per_group[rows[v].rc]++;
+        kept_per_group[rows[v].rc] += keep[v];
+    }
+    free(rows);
+    return MO_OK;
+}
+
+/* ------------------------------------------------------------------------------------------ */
 /* tile-granular simulator of the fused pseudo nested loop (Section IV)                        */
 /* ------------------------------------------------------------------------------------------ */
 /*

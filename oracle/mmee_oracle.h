@@ -117,6 +117,20 @@ int  mo_search(const mo_problem*, mo_record* out_topk, uint64_t* n_total, uint64
 int  mo_simulate(const uint32_t bound[8], uint32_t pi, const uint32_t beta[5], mo_sim_out* out);
 int  mo_threads_used(void);
 
+/* Symbolic form of one fused row (Section V-E): every BS_X / DA_X as the set of loop bounds it is the
+ * product of, bit d = x_D of loop d (i,k,l,j), bit 4+d = x_G.  da_q[OPD_C] = 0 (no DRAM traffic). */
+typedef struct {
+    uint8_t bs_q[5], da_q[5];
+    uint8_t tau[5];
+    uint8_t recompute;
+} mo_row_symbols;
+int  mo_row_symbolic(uint32_t pi, const uint32_t beta[5], mo_row_symbols* out);
+
+/* Offline symbolic pruning of the fused row space (Section VI-B, Eq. 12) over all six orders:
+ * keep[r] = 0 for rows that another row of the same recompute group dominates for every tiling.
+ * kept_per_group[g] / rows_per_group[g]: g = recompute flag.  18 750 rows. */
+int  mo_symbolic_prune(uint8_t* keep, uint32_t kept_per_group[2], uint32_t rows_per_group[2]);
+
 #ifdef __cplusplus
 }
 #endif

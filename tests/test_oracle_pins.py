@@ -282,3 +282,61 @@ def test_bad_inputs_are_rejected():
     with pytest.raises(oracle.OracleError) as e:
         oracle.make_problem(w, dict(a, e_gb_pj=6.3), mi.objective())
     assert e.value.code == oracle.ERR_QUANTUM
+
+
+# ---------------------------------------------------------------------------------------------------
+# Offline symbolic pruning (Section VI-B, Eq. 12)
+# ---------------------------------------------------------------------------------------------------
+
+def _row_levels(r):
+    q = r % 3125
+    return r // 3125, [3 + q // 625, 3 + (q // 125) % 5, 3 + (q // 25) % 5, 3 + (q // 5) % 5, 3 + q % 5]
+
+
+def test_symbolic_rows_are_the_monomials_the_model_evaluates():
+    """With eight distinct primes as bounds, the product over a row's symbolic set of bounds must
+    be the number the evaluation computes for that operand."""
+    p = _prime_problem(fuse_mask=mi.FUSE_FUSED)
+    t = tiling_index(p, PRIME_BOUNDS[4:])
+    rng = np.random.default_rng(5)
+    for r in rng.integers(0, 18750, size=1500):
+        pi, beta = _row_levels(int(r))
+        s = oracle.row_symbolic(pi, beta)
+        rec = oracle.evaluate(p, (t * p.R + int(r)) * 9)
+        assert s.recompute == rec.recompute
+        for x in range(5):
+            prod = lambda q: int(np.prod([b for d, b in enumerate(PRIME_BOUNDS) if q >> d & 1], dtype=object))
+            assert prod(s.bs_q[x]) == rec.bs_x[x]
+            if x != 2:
+                assert prod(s.da_q[x]) == rec.da_x[x]
+
+
+def test_symbolic_pruning_keeps_every_optimum_and_few_distinct_rows():
+    """Eq. (12): a pruned row is never strictly better than the best kept row, for any tiling,
+    stationary pair or objective (the optimality statement of Section VI-C); and the kept rows
+    collapse to a few dozen distinct symbolic rows per recompute group (the paper reports 58)."""
+    keep, kept, total = oracle.symbolic_prune()
+    assert total == [12500, 6250] and sum(total) == 18750
+    distinct = {0: set(), 1: set()}
+    for r in np.nonzero(keep)[0]:
+        pi, beta = _row_levels(int(r))
+        s = oracle.row_symbolic(pi, beta)
+        bs, da, tau = list(s.bs_q), list(s.da_q), list(s.tau)
+        bs1 = tuple(sorted(bs[:3] + [bs[x] for x in (3, 4) if tau[x]]))
+        bs2 = tuple(sorted(bs[2:] + [bs[x] for x in (0, 1) if tau[x]]))
+        distinct[s.recompute].add((bs1, bs2, tuple(sorted(da[:2] + da[3:]))))
+    assert (len(distinct[0]), len(distinct[1])) == (53, 37)
+    assert all(58 / 2 <= len(d) <= 58 * 2 for d in distinct.values())
+
+    for seed, objective in ((1, mi.OBJ_ENERGY), (2, mi.OBJ_LATENCY), (4, mi.OBJ_ENERGY), (8, mi.OBJ_LATENCY)):
+        cfg = mi.random_tiny_problem(seed)
+        obj = dict(cfg["searches"][0], objective=objective, topk=1, order_set=mi.ORD_ALL6,
+                   fuse_mask=mi.FUSE_FUSED)
+        p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
+        n_t = min(p.T, max(1, 2_000_000 // (p.R * 9)))
+        keys, feas = oracle.keys_range(p, 0, n_t * p.R * 9)
+        keys = keys.reshape(n_t, 18750, 9).astype(np.float64)
+        keys[~feas.reshape(n_t, 18750, 9).astype(bool)] = np.inf
+        per_tiling_all = keys.min(axis=(1, 2))
+        per_tiling_kept = keys[:, keep.astype(bool), :].min(axis=(1, 2))
+        assert np.array_equal(per_tiling_all, per_tiling_kept)
