@@ -92,6 +92,10 @@ typedef struct {
     uint32_t tiling_set;                     /* MMEE_TILE_*                                       */
     uint32_t order_set;                      /* MMEE_ORD_*                                        */
     uint32_t fuse_mask;                      /* OR of MMEE_FUSE_*, at least one bit               */
+    uint32_t row_pruning;                    /* 1: offline symbolic row pruning (Section VI-B); needs
+                                                topk = 1.  Rows that a lower-index row dominates for every
+                                                tiling are not evaluated: the optimum is unchanged, but
+                                                n_feasible then counts only the evaluated rows.        */
     uint64_t t_begin, t_end;                 /* tiling sub-range [t_begin,t_end); 0,0 = all       */
 } mmee_objective_t;
 
@@ -164,6 +168,7 @@ int mmee_destroy(mmee_handle_t* handle);
  *   out_best, out_topk        : DEVICE, caller-owned, as for mmee_search (out_topk may be NULL).
  * Asynchronous on `cuda_stream`.  The first call on a device looks up the array's device address
  * (with that device current); make that first call before any stream capture begins.
+ * objective.row_pruning must be 0 here (its kept-row list would need a device allocation).
  * Limits: the array holds the partial lists of at most 512 persistent CTAs; a device whose launch
  * shape needs more is refused with MMEE_ERR_RANGE.  Other errors as mmee_create / mmee_search.
  * All calls on a device share the one array and it keeps the previous call's contents: the call
@@ -223,6 +228,18 @@ int mmee_solve_host(const mmee_workload_t* workload, const mmee_arch_t* arch,
 int mmee_query_vector(uint32_t metric, uint32_t phi, uint32_t pi, uint32_t operand, uint32_t beta,
                       uint32_t recompute, uint8_t out_q[8]);
 
+/*
+ * mmee_row_pruning_keep -- HOST only, no device needed.  The rows of one tiling that survive the
+ * offline symbolic pruning (Section VI-B) for the order set and fusion modes of `objective`:
+ * out_keep[r] = 1 if row r is evaluated when objective.row_pruning = 1, else 0.  A row is dropped iff
+ * a row of the same fusion mode and recompute group with a lower index needs, for every tiling, no
+ * more buffer in either operator and no more DRAM traffic (Eq. 12 made safe for ties: the dropped row
+ * can then never be the lowest-index optimum).  out_keep: HOST, `capacity` bytes; *out_rows receives
+ * the number of rows R; MMEE_ERR_RANGE if capacity < R.
+ */
+int mmee_row_pruning_keep(const mmee_objective_t* objective, uint8_t* out_keep, uint32_t capacity,
+                          uint32_t* out_rows);
+
 /* HOST only: whether order `pi` with C buffered at level `beta_c` regenerates C (Section III-C). */
 int mmee_recompute_flag(uint32_t pi, uint32_t beta_c, uint32_t* out_flag);
 
@@ -237,6 +254,8 @@ typedef struct {
     uint32_t kernels_launched, grid, block, smem_bytes;
     uint64_t tasks;
     float    search_ms, finalize_ms;
+    uint32_t rows_per_tiling;                /* R                                                  */
+    uint32_t rows_evaluated_per_tiling;      /* R, or the rows that survive symbolic row pruning   */
 } mmee_launch_stats_t;
 int mmee_last_search_stats(const mmee_handle_t* handle, mmee_launch_stats_t* out);
 

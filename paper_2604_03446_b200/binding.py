@@ -21,7 +21,7 @@ OK, ERR_ARG, ERR_OVERFLOW, ERR_QUANTUM, ERR_NO_FEASIBLE, ERR_CUDA, ERR_TIMEOUT, 
 
 EXPORTS = ("mmee_create", "mmee_search", "mmee_destroy", "mmee_search_static", "mmee_num_candidates", "mmee_num_tilings",
            "mmee_num_rows", "mmee_strerror", "mmee_last_cuda_error", "mmee_eval", "mmee_dump_keys", "mmee_solve_host",
-           "mmee_query_vector", "mmee_recompute_flag", "mmee_last_search_stats", "mmee_kernel_timing",
+           "mmee_query_vector", "mmee_recompute_flag", "mmee_row_pruning_keep", "mmee_last_search_stats", "mmee_kernel_timing",
            "mmee_alu_peak")
 
 
@@ -41,7 +41,7 @@ class Arch(C.Structure):
 
 class Objective(C.Structure):
     _fields_ = [("objective", C.c_uint32), ("topk", C.c_uint32), ("tiling_set", C.c_uint32),
-                ("order_set", C.c_uint32), ("fuse_mask", C.c_uint32),
+                ("order_set", C.c_uint32), ("fuse_mask", C.c_uint32), ("row_pruning", C.c_uint32),
                 ("t_begin", C.c_uint64), ("t_end", C.c_uint64)]
 
 
@@ -62,7 +62,8 @@ class Result(C.Structure):
 class LaunchStats(C.Structure):
     _fields_ = [("kernels_launched", C.c_uint32), ("grid", C.c_uint32), ("block", C.c_uint32),
                 ("smem_bytes", C.c_uint32), ("tasks", C.c_uint64),
-                ("search_ms", C.c_float), ("finalize_ms", C.c_float)]
+                ("search_ms", C.c_float), ("finalize_ms", C.c_float),
+                ("rows_per_tiling", C.c_uint32), ("rows_evaluated_per_tiling", C.c_uint32)]
 
 
 RESULT_BYTES = C.sizeof(Result)
@@ -113,6 +114,8 @@ def library():
                                   C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
     L.mmee_query_vector.argtypes = [C.c_uint32] * 6 + [C.POINTER(C.c_uint8)]
     L.mmee_recompute_flag.argtypes = [C.c_uint32, C.c_uint32, C.POINTER(C.c_uint32)]
+    L.mmee_row_pruning_keep.argtypes = [C.POINTER(Objective), C.POINTER(C.c_uint8), C.c_uint32,
+                                        C.POINTER(C.c_uint32)]
     L.mmee_last_search_stats.argtypes = [H, C.POINTER(LaunchStats)]
     L.mmee_kernel_timing.argtypes = [H, C.c_int]
     L.mmee_alu_peak.argtypes = [C.POINTER(C.c_double)]
@@ -210,6 +213,15 @@ def mmee_query_vector(metric: int, phi: int, pi: int, operand: int, beta: int, r
     q = (C.c_uint8 * 8)()
     _check(library().mmee_query_vector(metric, phi, pi, operand, beta, recompute, q), "mmee_query_vector")
     return list(q)
+
+
+def mmee_row_pruning_keep(objective: dict):
+    """List of 0/1 per row of a tiling: the rows evaluated under objective.row_pruning = 1."""
+    rows = C.c_uint32()
+    buf = (C.c_uint8 * 26250)()
+    _check(library().mmee_row_pruning_keep(_fill(Objective(), objective), buf, 26250, C.byref(rows)),
+           "mmee_row_pruning_keep")
+    return list(buf[:rows.value])
 
 
 def mmee_recompute_flag(pi: int, beta_c: int) -> int:

@@ -8,7 +8,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmmee.so")
-SOURCES = ["mmee_plan.cu", "mmee_search.cu", "mmee_api.cu", "mmee_alu_peak.cu", "mmee_static.cu"]
+SOURCES = ["mmee_plan.cu", "mmee_search.cu", "mmee_api.cu", "mmee_alu_peak.cu", "mmee_static.cu", "mmee_prune.cu"]
 HEADERS = ["mmee_plan.h", "mmee_search.h", "mmee_eval.cuh", os.path.join("..", "..", "include", "mmee.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
               "-Xcompiler", "-fPIC", "-shared", "--expt-relaxed-constexpr"]

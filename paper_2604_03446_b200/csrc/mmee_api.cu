@@ -4,6 +4,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "mmee_search.h"
 
@@ -14,6 +15,8 @@ struct mmee_handle {
     mmee::Plan plan;
     mmee::LaunchShape shape;
     mmee::Scratch* scratch;      // device
+    mmee::PrunedTask* pruned;    // device, row pruning only
+    uint32_t kept_rows;          // rows of a tiling that survive pruning (all rows without it)
     int device;
     mmee_launch_stats_t last;
     bool timing;
@@ -25,19 +28,22 @@ namespace {
 using namespace mmee;
 
 // Tasks a CTA pulls per visit of the global counter, and the tilings such a range can touch.
-int choose_shape(const Plan& p, int device, LaunchShape* shape) {
+int choose_shape(const Plan& p, int device, uint32_t search_tpt, LaunchShape* shape) {
     int sm_count = 0, smem_optin = 0;      // attribute queries: cudaGetDeviceProperties costs milliseconds
     if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
         cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess)
         return MMEE_ERR_CUDA;
     const uint32_t rounds = 9;
     shape->range_tasks = rounds * kWorkerThreads;
-    shape->slots = (shape->range_tasks - 1) / p.tasks_per_tiling + 2;
+    shape->search_tpt = search_tpt;
+    shape->pad = 0;
+    shape->pruned = nullptr;
+    shape->slots = (shape->range_tasks - 1) / search_tpt + 2;
     size_t smem = search_smem_bytes(p, shape->slots);
     // Many small tilings per range need many table slots: shrink the range until they fit.
     while (smem > 96 * 1024 && shape->range_tasks > kWorkerThreads) {
         shape->range_tasks -= kWorkerThreads;
-        shape->slots = (shape->range_tasks - 1) / p.tasks_per_tiling + 2;
+        shape->slots = (shape->range_tasks - 1) / search_tpt + 2;
         smem = search_smem_bytes(p, shape->slots);
     }
     if (smem > (size_t)smem_optin) return MMEE_ERR_RANGE;
@@ -46,7 +52,7 @@ int choose_shape(const Plan& p, int device, LaunchShape* shape) {
     if (search_occupancy(p, smem, &per_sm) != cudaSuccess || per_sm < 1) return MMEE_ERR_CUDA;
     if (per_sm > 2) per_sm = 2;
     uint64_t grid = (uint64_t)sm_count * (uint32_t)per_sm;
-    const uint64_t tasks = (p.t_end - p.t_begin) * p.tasks_per_tiling;
+    const uint64_t tasks = (p.t_end - p.t_begin) * search_tpt;
     const uint64_t ranges = (tasks + shape->range_tasks - 1) / shape->range_tasks;
     if (grid > ranges) grid = ranges ? ranges : 1;
     shape->grid = (uint32_t)grid;
@@ -83,14 +89,37 @@ int mmee_create(const mmee_workload_t* workload, const mmee_arch_t* arch, const 
     int rc = build_plan(workload, arch, objective, &h->plan);
     if (rc) { delete h; return rc; }
     if (cudaGetDevice(&h->device) != cudaSuccess) { delete h; return MMEE_ERR_CUDA; }
-    rc = choose_shape(h->plan, h->device, &h->shape);
+    // Row pruning: the searched task space lists only the tasks that keep at least one row.
+    std::vector<PrunedTask> kept_tasks;
+    uint32_t search_tpt = h->plan.tasks_per_tiling;
+    h->kept_rows = h->plan.rows_per_tiling;
+    if (h->plan.row_pruning) {
+        kept_tasks.resize(h->plan.tasks_per_tiling);
+        uint32_t n = 0;
+        build_pruned_tasks(h->plan, kept_tasks.data(), &n, &h->kept_rows);
+        kept_tasks.resize(n);
+        search_tpt = n;
+    }
+    rc = choose_shape(h->plan, h->device, search_tpt, &h->shape);
     if (rc) { delete h; return rc; }
+    if (h->plan.row_pruning) {
+        const size_t bytes = kept_tasks.size() * sizeof(PrunedTask);
+        if (cudaMalloc(reinterpret_cast<void**>(&h->pruned), bytes) != cudaSuccess ||
+            cudaMemcpy(h->pruned, kept_tasks.data(), bytes, cudaMemcpyHostToDevice) != cudaSuccess) {
+            if (h->pruned) cudaFree(h->pruned);
+            delete h;
+            return MMEE_ERR_CUDA;
+        }
+        h->shape.pruned = h->pruned;
+    }
     if (cudaMalloc(reinterpret_cast<void**>(&h->scratch), scratch_bytes(h->shape.grid)) != cudaSuccess) {
+        if (h->pruned) cudaFree(h->pruned);
         delete h;
         return MMEE_ERR_CUDA;
     }
     if (launch_reset(h->scratch, 0) != cudaSuccess || cudaStreamSynchronize(0) != cudaSuccess) {
         cudaFree(h->scratch);
+        if (h->pruned) cudaFree(h->pruned);
         delete h;
         return MMEE_ERR_CUDA;
     }
@@ -111,7 +140,9 @@ int mmee_search(mmee_handle_t* h, void* cuda_stream, mmee_result_t* out_best, mm
     h->last.grid = h->shape.grid;
     h->last.block = kSearchThreads;
     h->last.smem_bytes = h->shape.smem_bytes;
-    h->last.tasks = (h->plan.t_end - h->plan.t_begin) * h->plan.tasks_per_tiling;
+    h->last.tasks = (h->plan.t_end - h->plan.t_begin) * h->shape.search_tpt;
+    h->last.rows_per_tiling = h->plan.rows_per_tiling;
+    h->last.rows_evaluated_per_tiling = h->kept_rows;
     return cuda_status(e);
 }
 
@@ -120,6 +151,7 @@ int mmee_destroy(mmee_handle_t* h) {
     cudaError_t e = cudaSuccess;
     if (h->timing) for (int i = 0; i < 3; ++i) cudaEventDestroy(h->ev[i]);
     if (h->scratch) e = cudaFree(h->scratch);
+    if (h->pruned) cudaFree(h->pruned);
     delete h;
     return cuda_status(e);
 }
@@ -152,7 +184,7 @@ int mmee_eval(mmee_handle_t* h, void* cuda_stream, uint64_t idx_begin, uint64_t 
 }
 
 int mmee_dump_keys(mmee_handle_t* h, void* cuda_stream, int64_t* out_keys) {
-    if (!h || !out_keys) return MMEE_ERR_ARG;
+    if (!h || !out_keys || h->plan.row_pruning) return MMEE_ERR_ARG;
     const uint64_t n = (h->plan.t_end - h->plan.t_begin) * (uint64_t)h->plan.rows_per_tiling * 9u;
     if (n > (1ull << 31)) return MMEE_ERR_RANGE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -202,6 +234,36 @@ int mmee_query_vector(uint32_t metric, uint32_t phi, uint32_t pi, uint32_t opera
         q = tables.da_unfused[pi][operand][beta - 3];
     }
     for (int d = 0; d < 8; ++d) out_q[d] = (uint8_t)((q >> d) & 1u);
+    return MMEE_OK;
+}
+
+int mmee_row_pruning_keep(const mmee_objective_t* objective, uint8_t* out_keep, uint32_t capacity,
+                          uint32_t* out_rows) {
+    if (!objective || !out_keep || !out_rows) return MMEE_ERR_ARG;
+    // the row space depends on the objective's order set and fusion modes only: plan a unit workload
+    const mmee_workload_t w = {1, 1, 1, 1, 1, 1, 1, 1};
+    mmee_arch_t a;
+    std::memset(&a, 0, sizeof(a));
+    a.pe_rows = a.pe_cols = a.n_arrays = 1;
+    a.gb_bytes = 16;
+    a.dram_words_per_cycle = 1;
+    a.energy_quantum_pj = 1.0;
+    mmee_objective_t o = *objective;
+    o.topk = 1;
+    o.row_pruning = 1;
+    o.t_begin = o.t_end = 0;
+    Plan plan;
+    const int rc = build_plan(&w, &a, &o, &plan);
+    if (rc) return rc;
+    *out_rows = plan.rows_per_tiling;
+    if (capacity < plan.rows_per_tiling) return MMEE_ERR_RANGE;
+    std::vector<PrunedTask> tasks(plan.tasks_per_tiling);
+    uint32_t n = 0, kept = 0;
+    build_pruned_tasks(plan, tasks.data(), &n, &kept);
+    std::memset(out_keep, 0, plan.rows_per_tiling);
+    for (uint32_t i = 0; i < n; ++i)
+        for (uint32_t de = 0; de < 25; ++de)
+            if (tasks[i].rows >> de & 1u) out_keep[tasks[i].task * 25u + de] = 1;
     return MMEE_OK;
 }
 

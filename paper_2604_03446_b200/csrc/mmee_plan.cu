@@ -141,6 +141,7 @@ int build_plan(const mmee_workload_t* w, const mmee_arch_t* a, const mmee_object
     if (o->objective > MMEE_OBJ_EDP) return MMEE_ERR_ARG;
     if (o->topk < 1) return MMEE_ERR_ARG;
     if (o->topk > MMEE_MAX_TOPK) return MMEE_ERR_RANGE;
+    if (o->row_pruning > 1 || (o->row_pruning && o->topk != 1)) return MMEE_ERR_ARG;
     if (o->tiling_set > MMEE_TILE_ALL_DIVISORS || o->order_set > MMEE_ORD_ALL6) return MMEE_ERR_ARG;
     if (!(o->fuse_mask & 7u) || (o->fuse_mask & ~7u)) return MMEE_ERR_ARG;
 
@@ -223,6 +224,7 @@ int build_plan(const mmee_workload_t* w, const mmee_arch_t* a, const mmee_object
     p->pe_cols = a->pe_cols;
     p->objective = o->objective;
     p->topk = o->topk;
+    p->row_pruning = o->row_pruning;
 
     // Largest key any mapping of this problem can have.  M bounds the MAC count with the largest
     // recomputation factor (j_D <= J); each of at most seven DRAM terms is <= I*K*L*J <= M, the

@@ -49,6 +49,7 @@ struct Plan {
     uint32_t has_rf;
     uint32_t bw, pe_rows, pe_cols;
     uint32_t objective, topk;
+    uint32_t row_pruning, reserved;
     double   quantum_pj;
     QueryTables q;
     uint32_t divs[4][MMEE_MAX_DIVISORS];
@@ -57,5 +58,9 @@ struct Plan {
 // Host planner (mmee_plan.cu).  Fills `plan`; returns an MMEE_* status.
 int build_plan(const mmee_workload_t* w, const mmee_arch_t* a, const mmee_objective_t* o, Plan* plan);
 void build_query_tables(QueryTables* q);
+
+// Tie-safe symbolic row pruning (mmee_prune.cu): keep[row] for every row of a tiling.
+struct PrunedTask { uint32_t task, rows; };     // task inside a tiling, 25-bit mask of kept rows
+int build_pruned_tasks(const Plan& plan, PrunedTask* out, uint32_t* n_out, uint32_t* kept_rows);
 
 }  // namespace mmee

@@ -27,6 +27,7 @@ namespace mmee {
 namespace {
 
 constexpr unsigned kFull = 0xffffffffu;
+constexpr int kModeSearch = 0, kModeDump = 1, kModePrune = 2;
 constexpr size_t kPlanBytes = (sizeof(Plan) + 15) / 16 * 16;
 static_assert(sizeof(Plan) % 4 == 0, "the plan is copied word by word");
 constexpr int kRelCap = (1 << 30) - 1;     // cap of a running threshold-relative sum (see below)
@@ -401,10 +402,12 @@ __device__ __forceinline__ void fill_dead_tiling_item(TilingTab* tb, int item) {
 // the search kernel
 // ------------------------------------------------------------------------------------------------
 
-template <int OBJ, bool DUMP>
+template <int OBJ, int MODE>
 __global__ void __launch_bounds__(kSearchThreads, 2)
 search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Scratch* __restrict__ scratch,
               int64_t* __restrict__ dump) {
+    constexpr bool DUMP = MODE == kModeDump;        // store every key instead of reducing
+    constexpr bool PRUNE = MODE == kModePrune;      // visit only the rows kept by symbolic pruning
     extern __shared__ __align__(16) unsigned char smem_raw[];
     // The plan is copied to shared memory: lanes index its tables (query vectors, divisor lists,
     // block lists) with different indices, which the constant bank would serialise.
@@ -431,7 +434,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
     if (lane == 0) wt->count = 0;
     __syncthreads();      // the shared copy of the plan is complete
 
-    const uint32_t tpt = p.tasks_per_tiling;
+    const uint32_t tpt = shape.search_tpt;          // tasks per tiling in the searched task space
     const uint64_t task_begin = p.t_begin * tpt, task_end = p.t_end * tpt;
     const uint64_t dump_origin = task_begin * kCandPerTask;
     const int64_t cap = p.cap_words;
@@ -525,8 +528,16 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
             const uint32_t o = valid ? off + lane : n_range - 1;
             const uint32_t wa = w_first + o;
             const uint32_t slot = wa / tpt;
-            const uint32_t w = wa - slot * tpt;
-            const uint64_t tq = r0 + o;
+            const uint32_t wc = wa - slot * tpt;
+            // With row pruning the searched task space lists only the tasks that still hold a kept
+            // row; `kept` is the 25-bit mask of those rows.
+            uint32_t w = wc, kept = 0x1ffffffu;
+            if constexpr (PRUNE) {
+                const PrunedTask pt = shape.pruned[wc];
+                w = pt.task;
+                kept = pt.rows;
+            }
+            const uint64_t tq = PRUNE ? (t_first + slot) * (uint64_t)p.tasks_per_tiling + w : r0 + o;
             const TilingTab* tb = &ttabs[slot];
             const bool live = valid && tb->live;
             if (DUMP && valid && !tb->live) {
@@ -655,6 +666,9 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
 
 #pragma unroll 1
             for (int d = 0; d < 5; ++d) {
+                if constexpr (PRUNE) {
+                    if (!__any_sync(kFull, live && ((kept >> (d * 5)) & 31u))) continue;
+                }
                 // Five rows (levels of E) are evaluated branch-free; one vote decides whether any
                 // lane of the warp has to enter the insertion path for this group.
                 unsigned hit_any, fits;
@@ -671,7 +685,8 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                         for (int s = 0; s < 9; ++s) accs[s] = INT_MAX;
 #pragma unroll
                         for (int e = 0; e < 5; ++e) {
-                            const unsigned fit = (unsigned)(E1c[e] <= s1c) & (unsigned)(E2c[e] <= s2c);   // Eq. (4)
+                            unsigned fit = (unsigned)(E1c[e] <= s1c) & (unsigned)(E2c[e] <= s2c);         // Eq. (4)
+                            if constexpr (PRUNE) fit &= kept >> (d * 5 + e);
                             fits += fit;
                             int xc = __viaddmin_s32(uc, Gc[e], kRelCap);
                             xc = fit ? xc : kRelCap;
@@ -686,7 +701,8 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                         for (int j = 0; j < 3; ++j) uc[j] = __viaddmin_s32(ut[j], dc.z, kRelCap);
 #pragma unroll
                         for (int e = 0; e < 5; ++e) {
-                            const unsigned fit = (unsigned)(E1c[e] <= s1c) & (unsigned)(E2c[e] <= s2c);   // Eq. (4)
+                            unsigned fit = (unsigned)(E1c[e] <= s1c) & (unsigned)(E2c[e] <= s2c);         // Eq. (4)
+                            if constexpr (PRUNE) fit &= kept >> (d * 5 + e);
                             fits += fit;
                             int a[3];
 #pragma unroll
@@ -715,7 +731,8 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                     hit_any = 0;
 #pragma unroll
                     for (int e = 0; e < 5; ++e) {
-                        const unsigned fit = (unsigned)(E1c[e] <= s1c) & (unsigned)(E2c[e] <= s2c);       // Eq. (4)
+                        unsigned fit = (unsigned)(E1c[e] <= s1c) & (unsigned)(E2c[e] <= s2c);             // Eq. (4)
+                        if constexpr (PRUNE) fit &= kept >> (d * 5 + e);
                         fits += fit;
                         const int64_t x = xd + rt->E[e][2];
                         const double de = (double)(xed + rt->E[e][3]);
@@ -761,7 +778,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                     const int64_t xed = (OBJ == MMEE_OBJ_EDP) ? xe0 + rt->D[d][3] : 0;
 #pragma unroll 1
                     for (int e = 0; e < 5; ++e) {
-                        const bool fit = (rt->E[e][0] <= s1) && (rt->E[e][1] <= s2);
+                        const bool fit = (rt->E[e][0] <= s1) && (rt->E[e][1] <= s2) && ((kept >> (d * 5 + e)) & 1u);
                         const int64_t x = xd + rt->E[e][2];
                         const int64_t xe = (OBJ == MMEE_OBJ_EDP) ? xed + rt->E[e][3] : 0;
                         const uint64_t row_first_idx = task_first_idx + (uint64_t)((d * 5 + e) * 9);
@@ -880,20 +897,20 @@ __global__ void eval_kernel(const __grid_constant__ Plan p, uint64_t idx_begin, 
     }
 }
 
-template <int OBJ, bool DUMP>
+template <int OBJ, int MODE>
 cudaError_t launch_search_t(const Plan& p, const LaunchShape& shape, Scratch* scratch, int64_t* dump, cudaStream_t st) {
-    cudaError_t e = cudaFuncSetAttribute(search_kernel<OBJ, DUMP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(search_kernel<OBJ, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)shape.smem_bytes);
     if (e != cudaSuccess) return e;
-    search_kernel<OBJ, DUMP><<<shape.grid, kSearchThreads, shape.smem_bytes, st>>>(p, shape, scratch, dump);
+    search_kernel<OBJ, MODE><<<shape.grid, kSearchThreads, shape.smem_bytes, st>>>(p, shape, scratch, dump);
     return cudaGetLastError();
 }
 
-template <int OBJ, bool DUMP>
+template <int OBJ, int MODE>
 cudaError_t occupancy_t(int* blocks_per_sm, size_t smem) {
-    cudaError_t e = cudaFuncSetAttribute(search_kernel<OBJ, DUMP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(search_kernel<OBJ, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, search_kernel<OBJ, DUMP>, kSearchThreads, smem);
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, search_kernel<OBJ, MODE>, kSearchThreads, smem);
 }
 
 }  // namespace
@@ -905,24 +922,31 @@ size_t search_smem_bytes(const Plan& p, uint32_t slots) {
 
 cudaError_t search_occupancy(const Plan& p, size_t smem, int* blocks_per_sm) {
     switch (p.objective) {
-        case MMEE_OBJ_ENERGY: return occupancy_t<MMEE_OBJ_ENERGY, false>(blocks_per_sm, smem);
-        case MMEE_OBJ_LATENCY: return occupancy_t<MMEE_OBJ_LATENCY, false>(blocks_per_sm, smem);
-        default: return occupancy_t<MMEE_OBJ_EDP, false>(blocks_per_sm, smem);
+        case MMEE_OBJ_ENERGY: return occupancy_t<MMEE_OBJ_ENERGY, kModeSearch>(blocks_per_sm, smem);
+        case MMEE_OBJ_LATENCY: return occupancy_t<MMEE_OBJ_LATENCY, kModeSearch>(blocks_per_sm, smem);
+        default: return occupancy_t<MMEE_OBJ_EDP, kModeSearch>(blocks_per_sm, smem);
     }
 }
 
 cudaError_t launch_search(const Plan& p, const LaunchShape& shape, Scratch* scratch, int64_t* dump, cudaStream_t st) {
     if (dump) {
         switch (p.objective) {
-            case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, true>(p, shape, scratch, dump, st);
-            case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, true>(p, shape, scratch, dump, st);
-            default: return launch_search_t<MMEE_OBJ_EDP, true>(p, shape, scratch, dump, st);
+            case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, kModeDump>(p, shape, scratch, dump, st);
+            case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, kModeDump>(p, shape, scratch, dump, st);
+            default: return launch_search_t<MMEE_OBJ_EDP, kModeDump>(p, shape, scratch, dump, st);
+        }
+    }
+    if (shape.pruned) {
+        switch (p.objective) {
+            case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, kModePrune>(p, shape, scratch, nullptr, st);
+            case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, kModePrune>(p, shape, scratch, nullptr, st);
+            default: return launch_search_t<MMEE_OBJ_EDP, kModePrune>(p, shape, scratch, nullptr, st);
         }
     }
     switch (p.objective) {
-        case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, false>(p, shape, scratch, nullptr, st);
-        case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, false>(p, shape, scratch, nullptr, st);
-        default: return launch_search_t<MMEE_OBJ_EDP, false>(p, shape, scratch, nullptr, st);
+        case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, kModeSearch>(p, shape, scratch, nullptr, st);
+        case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, kModeSearch>(p, shape, scratch, nullptr, st);
+        default: return launch_search_t<MMEE_OBJ_EDP, kModeSearch>(p, shape, scratch, nullptr, st);
     }
 }
 

@@ -35,6 +35,9 @@ struct LaunchShape {
     uint32_t range_tasks;   // tasks a CTA takes per pull (multiple of kWorkerThreads)
     uint32_t slots;         // tilings one range can touch
     uint32_t smem_bytes;
+    uint32_t search_tpt;    // tasks per tiling in the searched task space (fewer with row pruning)
+    uint32_t pad;
+    const PrunedTask* pruned;   // device: the kept tasks of a tiling (row pruning), else null
     uint64_t n_ranges;      // ranges of the searched task interval
     uint64_t range_stride;  // ranges are visited as (i * range_stride) mod n_ranges; coprime to n_ranges
 };

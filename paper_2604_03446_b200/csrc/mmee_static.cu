@@ -49,6 +49,9 @@ int static_shape(const Plan& p, int device, LaunchShape* shape) {
         cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess)
         return MMEE_ERR_CUDA;
     shape->range_tasks = 9 * kWorkerThreads;
+    shape->search_tpt = p.tasks_per_tiling;
+    shape->pad = 0;
+    shape->pruned = nullptr;
     shape->slots = (shape->range_tasks - 1) / p.tasks_per_tiling + 2;
     size_t smem = search_smem_bytes(p, shape->slots);
     while (smem > 96 * 1024 && shape->range_tasks > (uint32_t)kWorkerThreads) {
@@ -88,6 +91,7 @@ extern "C" int mmee_search_static(const mmee_workload_t* workload, const mmee_ar
     Plan plan;
     int rc = build_plan(workload, arch, objective, &plan);      // host only
     if (rc) return rc;
+    if (plan.row_pruning) return MMEE_ERR_ARG;      // the kept-task list would need a device allocation
     int device = 0;
     if (cudaGetDevice(&device) != cudaSuccess) return MMEE_ERR_CUDA;
     LaunchShape shape;

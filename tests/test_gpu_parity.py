@@ -267,3 +267,50 @@ def test_search_on_a_side_stream():
         st.synchronize()
     got = mm.read_results(best, 1)[0]
     assert got.idx == (want.topk[0].idx if want.topk else mm.NO_INDEX)
+
+
+@pytest.mark.parametrize("seed", TINY_SEEDS)
+def test_row_pruning_keeps_the_optimum(seed):
+    """Offline symbolic row pruning (Section VI-B) in its tie-safe form: the optimum record of the
+    pruned search is the oracle's optimum of the full space, index included, for every objective."""
+    cfg = mi.random_tiny_problem(seed)
+    for objective in (mi.OBJ_ENERGY, mi.OBJ_LATENCY, mi.OBJ_EDP):
+        obj = shrink(cfg, dict(cfg["searches"][0], objective=objective, topk=1), 6_000_000)
+        p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
+        want = oracle.search(p)
+        best = mm.result_buffer(1)
+        with Handle(cfg, dict(obj, row_pruning=1)) as h:
+            mm.mmee_search(h, best, None)
+            torch.cuda.synchronize()
+            stats = mm.mmee_last_search_stats(h)
+        got = mm.read_results(best, 1)[0]
+        assert stats.rows_evaluated_per_tiling < stats.rows_per_tiling
+        if want.topk:
+            assert_same_record(got, want.topk[0], "seed %d objective %d" % (seed, objective))
+        else:
+            assert got.idx == mm.NO_INDEX and got.status == mm.ERR_NO_FEASIBLE
+
+
+def test_row_pruning_on_the_benchmark_workloads():
+    for path in _golden_files():
+        with open(path) as f:
+            gold = json.load(f)
+        if "sweep" in gold["name"] and not gold["name"].endswith("s1024"):
+            continue
+        cfg = dict(name=gold["name"], workload=gold["workload"], arch=gold["arch"])
+        for s in gold["searches"]:
+            obj = dict(s["objective"], topk=1, row_pruning=1)
+            best = mm.result_buffer(1)
+            with Handle(cfg, obj) as h:
+                mm.mmee_search(h, best, None)
+                torch.cuda.synchronize()
+            got = mm.read_results(best, 1)[0]
+            o = s["topk"][0]
+            assert got.idx == o["idx"] and got.e_key == o["e_key"] and got.l_key == o["l_key"] and list(got.n) == o["n"]
+
+
+def test_row_pruning_needs_a_single_optimum():
+    cfg = mi.config1()
+    with pytest.raises(mm.MmeeError) as e:
+        mm.mmee_create(cfg["workload"], cfg["arch"], dict(cfg["searches"][0], topk=2, row_pruning=1))
+    assert e.value.code == mm.ERR_ARG

@@ -112,3 +112,28 @@ def test_without_a_gpu_create_fails_loudly():
     with pytest.raises(mm.MmeeError) as e:
         mm.mmee_create(mi.workload(1, 1, 1, 8, 8, 4, 4), mi.arch_tiny(), mi.objective())
     assert e.value.code == mm.ERR_CUDA
+
+
+def test_tie_safe_row_pruning_never_drops_a_lowest_index_optimum():
+    """The planner's symbolic row pruning (Section VI-B, Eq. 12 with a lower-index dominator): for
+    every tiling and objective of small problems, the (key, idx)-smallest feasible mapping over the
+    kept rows is the (key, idx)-smallest over all rows."""
+    import numpy as np
+    full = np.array(mm.mmee_row_pruning_keep(mi.objective()), dtype=bool)
+    assert (full.size, int(full.sum()), int(full[:18750].sum())) == (26250, 204, 100)
+    assert int(np.array(mm.mmee_row_pruning_keep(mi.config1()["searches"][0])).sum()) == 56
+    for seed in (1, 2, 3, 5, 8, 11):
+        cfg = mi.random_tiny_problem(seed)
+        for objective in (mi.OBJ_ENERGY, mi.OBJ_LATENCY, mi.OBJ_EDP):
+            obj = dict(cfg["searches"][0], objective=objective, topk=1)
+            keep = np.array(mm.mmee_row_pruning_keep(obj), dtype=bool)
+            p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
+            assert keep.size == p.R
+            n_t = min(p.T, max(1, 1_500_000 // (p.R * 9)))
+            keys, feas = oracle.keys_range(p, 0, n_t * p.R * 9)
+            keys = np.where(feas.astype(bool), keys, np.iinfo(np.int64).max).reshape(n_t, p.R, 9)
+            flat_all = keys.reshape(n_t, -1)
+            masked = np.where(keep[None, :, None], keys, np.iinfo(np.int64).max).reshape(n_t, -1)
+            # argmin returns the first (lowest-index) minimum
+            assert np.array_equal(flat_all.argmin(axis=1), masked.argmin(axis=1))
+            assert np.array_equal(flat_all.min(axis=1), masked.min(axis=1))
