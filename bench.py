@@ -242,6 +242,26 @@ def main():
             samples.append(1e3 * (time.perf_counter() - t0))
         tto_ms.append(statistics.median(samples))
 
+    # offline symbolic row pruning (single-optimum searches only): same optimum, fewer rows evaluated
+    pruning = []
+    for i, (c, s) in enumerate(jobs):
+        if s["topk"] != 1:
+            continue
+        hp = mm.mmee_create(c["workload"], c["arch"], dict(s, row_pruning=1))
+        mm.mmee_kernel_timing(hp, True)
+        bp = mm.result_buffer(1)
+        ms = []
+        for _ in range(13):
+            mm.mmee_search(hp, bp, None)
+            torch.cuda.synchronize()
+            ms.append(mm.mmee_last_search_stats(hp).search_ms)
+        st = mm.mmee_last_search_stats(hp)
+        got = mm.read_results(bp, 1)[0]
+        pruning.append(dict(problem=c["name"], objective=OBJ_NAMES[s["objective"]],
+                            rows=st.rows_per_tiling, rows_kept=st.rows_evaluated_per_tiling,
+                            kernel_ms=statistics.median(ms[3:]), same_optimum=bool(got.idx == bests[i].idx)))
+        mm.mmee_destroy(hp)
+
     # end to end through the host-buffer entry point: plan, launch, copy back, every step
     e2e_steps = max(3, min(args.steps, 30))
     h2d = d2h = 0
@@ -298,7 +318,7 @@ def main():
                      d2h_bytes_per_step=d2h, ms_per_step=1e3 * e2e_s / e2e_steps,
                      note="mmee_solve_host: plan + launch + result copy to host buffers, host wall clock"),
             time_to_optimum_ms=tto_ms, device_time_to_optimum_ms=[k["avg_ms"] + k["finalize_avg_ms"] for k in per_kernel],
-            kernels=per_kernel, roofline=roofline)
+            kernels=per_kernel, roofline=roofline, row_pruning=pruning)
         if not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(*jobs[0])
         print(json.dumps(line))
