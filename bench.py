@@ -51,6 +51,12 @@ def workload_jobs(name):
     if name == "sweep":
         pts = mi.config5()
         return "sweep_s1k_to_64k", [(c, c["searches"][0]) for c in pts]
+    if name == "ffn":
+        pts = mi.ffn_dram_sweep_configs()
+        return "ffn_gpt3_dram_vs_buffer", [(c, c["searches"][0]) for c in pts]
+    if name == "beyond":
+        pts = mi.beyond_attention_configs()
+        return "two_gemm_and_conv_chains", [(c, c["searches"][0]) for c in pts]
     cfg = WORKLOADS[name]()
     return cfg["name"], [(cfg, s) for s in cfg["searches"]]
 
@@ -155,7 +161,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="bert", choices=sorted(WORKLOADS) + ["sweep"])
+    ap.add_argument("--workload", default="bert", choices=sorted(WORKLOADS) + ["sweep", "ffn", "beyond"])
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -259,7 +265,9 @@ def main():
         got = mm.read_results(bp, 1)[0]
         pruning.append(dict(problem=c["name"], objective=OBJ_NAMES[s["objective"]],
                             rows=st.rows_per_tiling, rows_kept=st.rows_evaluated_per_tiling,
-                            kernel_ms=statistics.median(ms[3:]), same_optimum=bool(got.idx == bests[i].idx)))
+                            kernel_ms=statistics.median(ms[3:]), same_optimum=bool(got.idx == bests[i].idx),
+                            optimum=dict(idx=got.idx, bs_words=got.bs, dram_words=got.n[0],
+                                         energy_pj=got.energy_pj, latency_cycles=got.latency_cycles)))
         mm.mmee_destroy(hp)
 
     # end to end through the host-buffer entry point: plan, launch, copy back, every step

@@ -113,6 +113,53 @@ def all_configs():
     return [config1(), config2(), config3(), config4()] + config5()
 
 
+# --- beyond attention: two GEMMs and convolution chains (Section VII-J), buffer-size sweeps ------
+
+def two_gemm(I, K, L, J, word_bytes=2):
+    """C = A(I x K) * B(K x L), E = C * D(L x J) as a single-instance workload."""
+    return workload(1, 1, 1, I, L, K, J, word_bytes)
+
+
+def conv_chain(hw, c_in, c_mid, c_out, k1):
+    """Two convolutions as GEMMs via im2col: a k1 x k1 convolution over hw pixels followed by a 1 x 1
+    convolution.  I = pixels, K = c_in * k1^2, L = c_mid, J = c_out."""
+    return two_gemm(hw, c_in * k1 * k1, c_mid, c_out)
+
+
+def arch_dram_only(gb_bytes, pe=32):
+    """Cost coefficients that make the energy key the DRAM traffic in words: the objective of the
+    DRAM-access-versus-buffer-size studies (Section VII-C)."""
+    return arch(pe, pe, 1, gb_bytes, 0, 1, 1.0, 0.0, 0.0, 0.0, c_softmax=0.0, energy_quantum_pj=1.0)
+
+
+def beyond_attention_configs():
+    """The four non-attention chains of the paper's applicability table, on its first accelerator."""
+    shapes = [("mlp_768_64_384_64", two_gemm(768, 64, 384, 64)),
+              ("ffn_2048_768_3072_768", two_gemm(2048, 768, 3072, 768)),
+              ("conv_chain_cc1", conv_chain(112 * 112, 64, 192, 128, 3)),
+              ("conv_chain_cc2", conv_chain(56 * 56, 64, 64, 64, 1))]
+    return [dict(name=n, workload=w, arch=arch_accel1(),
+                 searches=[objective(OBJ_ENERGY, 1, fuse_mask=FUSE_FUSED)]) for n, w in shapes]
+
+
+FFN_SWEEP_BUFFER_BYTES = tuple(64 * KiB << i for i in range(0, 10))      # 64 KB .. 32 MB
+
+
+def ffn_dram_sweep_configs():
+    """Fused feed-forward GEMMs of GPT-3-6.7B (32k x 4k x 16k and 32k x 16k x 4k, Section VII-C):
+    the least DRAM traffic at each buffer size; 40 560 tilings x 18 750 rows x 9 mappings each."""
+    w = two_gemm(32768, 4096, 16384, 4096)
+    return [dict(name="ffn_gpt3_dram_%dKB" % (b // KiB), workload=w, arch=arch_dram_only(b),
+                 searches=[objective(OBJ_ENERGY, 1, fuse_mask=FUSE_FUSED)]) for b in FFN_SWEEP_BUFFER_BYTES]
+
+
+def golden_configs():
+    """Workloads whose exhaustive-search answers are stored under tests/golden/."""
+    extra = [c for c in beyond_attention_configs() if c["name"] in ("mlp_768_64_384_64", "conv_chain_cc2")]
+    sweep = [c for c in ffn_dram_sweep_configs() if c["name"] in ("ffn_gpt3_dram_1024KB",)]
+    return all_configs() + extra + sweep
+
+
 # --- seeded tiny problems for exhaustive parity ----------------------------------------------
 
 def random_tiny_problem(seed: int):

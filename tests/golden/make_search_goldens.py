@@ -4,7 +4,7 @@ multi-minute CPU enumeration inside the test run.
 
 Calls only the CPU oracle and the input module.  Usage (from the repo root):
     python tests/golden/make_search_goldens.py [--threads N] [name-substring ...]
-A full run over all 32 workloads enumerates about 8e10 mappings (tens of minutes on 8 cores).
+A full run over all 35 workloads enumerates about 9e10 mappings (about an hour on 8 cores).
 """
 import argparse
 import json
@@ -35,7 +35,7 @@ def main():
     ap.add_argument("--threads", type=int, default=0)
     ap.add_argument("names", nargs="*")
     args = ap.parse_args()
-    for cfg in mi.all_configs():
+    for cfg in mi.golden_configs():
         if args.names and not any(s in cfg["name"] for s in args.names):
             continue
         path = os.path.join(HERE, "search_%s.json" % cfg["name"])
