@@ -314,3 +314,40 @@ def test_row_pruning_needs_a_single_optimum():
     with pytest.raises(mm.MmeeError) as e:
         mm.mmee_create(cfg["workload"], cfg["arch"], dict(cfg["searches"][0], topk=2, row_pruning=1))
     assert e.value.code == mm.ERR_ARG
+
+
+def test_two_gemm_and_conv_chain_shapes_sampled():
+    """Non-attention chains with ragged divisor lists (Section VII-J): sampled mappings field by field."""
+    rng = np.random.default_rng(23)
+    for cfg in mi.beyond_attention_configs():
+        obj = cfg["searches"][0]
+        p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
+        with Handle(cfg, obj) as h:
+            assert mm.mmee_num_candidates(h) == p.N
+            for s in [0, p.N - 32] + [int(v) for v in rng.integers(0, p.N - 32, size=12)]:
+                buf = mm.result_buffer(32)
+                mm.mmee_eval(h, s, 32, buf)
+                torch.cuda.synchronize()
+                for g, o in zip(mm.read_results(buf, 32), oracle.evaluate_range(p, s, 32)):
+                    assert_same_record(g, o, "%s idx %d" % (cfg["name"], o.idx))
+
+
+def test_dram_traffic_against_buffer_size_is_a_staircase():
+    """Fused feed-forward GEMMs, least DRAM traffic per buffer size (Section VII-C): 7.605e8 x 9
+    mappings per search; traffic never rises with a larger buffer, never falls below the compulsory
+    |A| + |B| + |D| + |E|, and the optimum is a real mapping that fits (re-evaluated by the oracle)."""
+    pts = mi.ffn_dram_sweep_configs()
+    last = None
+    for cfg in pts[::3]:
+        obj = cfg["searches"][0]
+        best, _, _ = gpu_search(cfg, obj)
+        assert best.n_total == 760500000 * 9 and best.status == mm.OK
+        p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
+        o = oracle.evaluate(p, best.idx)
+        assert_same_record(best, o, cfg["name"])
+        assert o.feasible and o.e_key == o.n[0]
+        I, K, L, J = [int(v) for v in p.dim]
+        assert o.n[0] >= I * K + K * L + L * J + I * J
+        if last is not None:
+            assert o.n[0] <= last
+        last = o.n[0]
