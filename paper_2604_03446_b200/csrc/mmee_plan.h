@@ -49,7 +49,8 @@ struct Plan {
     uint32_t has_rf;
     uint32_t bw, pe_rows, pe_cols;
     uint32_t objective, topk;
-    uint32_t row_pruning, reserved;
+    uint32_t row_pruning;
+    uint32_t rel_shift;           // energy: threshold-relative keys are kept in units of 2^rel_shift quanta
     double   quantum_pj;
     QueryTables q;
     uint32_t divs[4][MMEE_MAX_DIVISORS];

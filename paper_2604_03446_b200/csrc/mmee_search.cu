@@ -188,6 +188,10 @@ __device__ __forceinline__ void row_test(const int64_t (&k)[9], int64_t thr, int
 // -2^31 + 3 * 2^29 < 0.  Hence, if a candidate of a row truly passes, the saturated sum of the row's
 // candidate with W' = 0 is negative and the row is flagged; a flagged row without a passing
 // candidate needs u < -2^29 next to a saturated addend, and costs one visit of the exact path.
+// So that addends do not saturate on large problems, all energy terms are kept in units of 2^rel_shift
+// quanta, rounded down (the plan picks the shift from the largest possible DRAM term); rounding down
+// can only lower a sum, so a passing candidate still yields a negative sum, and the rows flagged
+// needlessly are those within 3 * 2^rel_shift quanta above the threshold.
 // Latency: key = max(x + P, Q + P) and max(a, b) < thr <=> a - thr < 0 and b - thr < 0; the same
 // saturation is applied to x + P - thr = u + vD + vE.
 // Capacity (Eq. 4): sizes are saturated to kSizeCap, which is above every admissible capacity, so
@@ -343,9 +347,12 @@ __device__ __forceinline__ void build_order_item(const Plan& p, const uint32_t* 
         int32_t* uc = x == OP_D ? u->Dc[l] : u->Ec[l];
 #pragma unroll
         for (int i = 0; i < 3; ++i) {
+            // sizes saturate; the DRAM term is kept in units of 2^rel_shift (rounded down), then saturated
             const int64_t lim = i < 2 ? (int64_t)kSizeCap : (int64_t)kTermCap;
-            fc[i] = (int32_t)(fr[i] < lim ? fr[i] : lim);
-            uc[i] = (int32_t)(ur[i] < lim ? ur[i] : lim);
+            const int64_t fv = i < 2 ? fr[i] : (fr[i] >> p.rel_shift);
+            const int64_t uv = i < 2 ? ur[i] : (ur[i] >> p.rel_shift);
+            fc[i] = (int32_t)(fv < lim ? fv : lim);
+            uc[i] = (int32_t)(uv < lim ? uv : lim);
         }
         fc[3] = 0;
         uc[3] = 0;
@@ -494,7 +501,8 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                 tb->wmin[rc] = m;
                 for (int s = 0; s < 9; ++s) {
                     const int64_t wd = tb->W[s][rc] - m;
-                    tb->Wc[rc][s] = wd > (int64_t)kTermCap ? kTermCap : (int32_t)wd;
+                    const int64_t ws = wd >> p.rel_shift;
+                    tb->Wc[rc][s] = ws > (int64_t)kTermCap ? kTermCap : (int32_t)ws;
                 }
             }
         }
@@ -636,9 +644,13 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
             }
             auto refresh = [&](int64_t t) {
                 if constexpr (OBJ == MMEE_OBJ_ENERGY) {
+                    // ut[0]: against the non-strict threshold t; ut[1]: against t - delta (ties excluded).
+                    // Rounding every term down to a multiple of 2^rel_shift can only lower the sum.
                     B = t - wmin;
-                    const int u = sat_s32(x0 - B);
-                    ut[0] = u < kRelCap ? u : kRelCap;
+                    const int u0 = sat_s32((x0 - B) >> p.rel_shift);
+                    const int u1 = sat_s32((x0 - B + delta) >> p.rel_shift);
+                    ut[0] = u0 < kRelCap ? u0 : kRelCap;
+                    ut[1] = u1 < kRelCap ? u1 : kRelCap;
                 } else if constexpr (OBJ == MMEE_OBJ_LATENCY) {
 #pragma unroll
                     for (int j = 0; j < 3; ++j) {
@@ -679,7 +691,8 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                     int acc = INT_MAX;
                     fits = 0;
                     if constexpr (OBJ == MMEE_OBJ_ENERGY) {
-                        const int uc = __viaddmin_s32(ut[0], dc.z, kRelCap);
+                        const uint64_t group_first_idx = task_first_idx + (uint64_t)(d * 45);
+                        const int uc = __viaddmin_s32(group_first_idx > ti ? ut[1] : ut[0], dc.z, kRelCap);
                         int accs[9];          // one chain per stationary pair: nine independent chains
 #pragma unroll
                         for (int s = 0; s < 9; ++s) accs[s] = INT_MAX;
@@ -713,8 +726,12 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                             acc = min(acc, fit ? racc : INT_MAX);
                         }
                     }
-                    const uint64_t group_first_idx = task_first_idx + (uint64_t)(d * 45);
-                    hit_any = acc < (group_first_idx > ti ? -delta : 0);      // no overflow at acc = INT_MAX
+                    if constexpr (OBJ == MMEE_OBJ_ENERGY) {
+                        hit_any = acc < 0;
+                    } else {
+                        const uint64_t group_first_idx = task_first_idx + (uint64_t)(d * 45);
+                        hit_any = acc < (group_first_idx > ti ? -delta : 0);  // no overflow at acc = INT_MAX
+                    }
                 } else if constexpr (!DUMP && OBJ == MMEE_OBJ_EDP) {
                     // The energy-delay product is not separable, so the filter is a double-precision
                     // evaluation of every mapping on the FP64 pipe: energy and latency sums converted
