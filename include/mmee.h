@@ -246,7 +246,7 @@ int mmee_recompute_flag(uint32_t pi, uint32_t beta_c, uint32_t* out_flag);
 /*
  * mmee_last_search_stats -- HOST counters of the most recent mmee_search on the handle, valid
  * after the stream has been synchronised: kernels launched by that call, persistent CTAs,
- * threads per CTA, dynamic shared memory per CTA, tasks (groups of 225 consecutive mappings) and,
+ * threads per CTA, dynamic shared memory per CTA, tasks (groups of 1125 consecutive mappings) and,
  * when mmee_kernel_timing is on, the device time of the search kernel and of the finalize kernel
  * in milliseconds (CUDA events recorded on the search's stream; -1 when timing is off).
  */

@@ -33,7 +33,7 @@ int choose_shape(const Plan& p, int device, uint32_t search_tpt, LaunchShape* sh
     if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
         cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess)
         return MMEE_ERR_CUDA;
-    const uint32_t rounds = 9;
+    const uint32_t rounds = 2;      // each task is 1125 mappings
     shape->range_tasks = rounds * kWorkerThreads;
     shape->search_tpt = search_tpt;
     shape->pad = 0;
@@ -262,8 +262,8 @@ int mmee_row_pruning_keep(const mmee_objective_t* objective, uint8_t* out_keep, 
     build_pruned_tasks(plan, tasks.data(), &n, &kept);
     std::memset(out_keep, 0, plan.rows_per_tiling);
     for (uint32_t i = 0; i < n; ++i)
-        for (uint32_t de = 0; de < 25; ++de)
-            if (tasks[i].rows >> de & 1u) out_keep[tasks[i].task * 25u + de] = 1;
+        for (uint32_t r = 0; r < 125; ++r)
+            if (tasks[i].rows[r / 25u] >> (r % 25u) & 1u) out_keep[tasks[i].task * 125u + r] = 1;
     return MMEE_OK;
 }
 

@@ -92,27 +92,26 @@ __device__ __forceinline__ void tiling_bounds(const Plan& p, uint64_t t64, uint3
     }
 }
 
-// Task index inside a tiling -> (block, levels of A, B, C).  Rows of a task: levels of D, E.
+// Task index inside a tiling -> (block, outer levels).  A task is 125 consecutive rows: a fused
+// task fixes the levels of A and B and walks those of C, D, E; an unfused task (C always at L3)
+// fixes the level of A and walks those of B, D, E.
 struct TaskChoice {
     uint32_t block, phi, order_slot, order;
-    uint32_t la, lb, lc;        // beta - 3
+    uint32_t la, lb;            // beta - 3; lb is not used by an unfused task
 };
 
 __device__ __forceinline__ TaskChoice decode_task(const Plan& p, uint32_t w) {
     TaskChoice c;
     if (w < p.fused_tasks) {
-        c.block = w / 125u;
-        const uint32_t rem = w - c.block * 125u;
-        c.la = rem / 25u;
-        c.lb = (rem / 5u) % 5u;
-        c.lc = rem % 5u;
-    } else {
-        const uint32_t u = w - p.fused_tasks;
-        c.block = p.n_fused_blocks + u / 25u;
-        const uint32_t rem = u % 25u;
+        c.block = w / 25u;
+        const uint32_t rem = w - c.block * 25u;
         c.la = rem / 5u;
         c.lb = rem % 5u;
-        c.lc = 0;
+    } else {
+        const uint32_t u = w - p.fused_tasks;
+        c.block = p.n_fused_blocks + u / 5u;
+        c.la = u % 5u;
+        c.lb = 0;
     }
     c.phi = p.block_phi[c.block];
     c.order_slot = p.block_order_slot[c.block];
@@ -128,9 +127,9 @@ __device__ inline void evaluate_candidate(const Plan& p, uint64_t idx, mmee_resu
     const uint64_t t = idx / per_t;
     const uint32_t rem = (uint32_t)(idx - t * per_t);
     const uint32_t row = rem / 9u, s = rem % 9u;
-    const uint32_t w = row / 25u, de = row % 25u;
+    const uint32_t w = row / 125u, mid = (row % 125u) / 25u, de = row % 25u;
     const TaskChoice c = decode_task(p, w);
-    const uint32_t lv[5] = {c.la, c.lb, c.lc, de / 5u, de % 5u};
+    const uint32_t lv[5] = {c.la, c.phi == 0 ? c.lb : mid, c.phi == 0 ? mid : 0u, de / 5u, de % 5u};
     const int sm1 = (int)(s / 3u), sm2 = (int)(s % 3u);
 
     uint32_t b[8];
@@ -147,7 +146,7 @@ __device__ inline void evaluate_candidate(const Plan& p, uint64_t idx, mmee_resu
 
     const QueryTables& q = p.q;
     const bool fused = c.phi == 0;
-    const uint32_t rc = fused ? q.recompute[c.order][c.lc] : 0u;
+    const uint32_t rc = fused ? q.recompute[c.order][lv[OP_C]] : 0u;
 
     int64_t bs[5], da[5];
     for (int x = 0; x < 5; ++x) {

@@ -189,8 +189,8 @@ int build_plan(const mmee_workload_t* w, const mmee_arch_t* a, const mmee_object
             if (phi == 0) ++p->n_fused_blocks;
         }
     }
-    p->fused_tasks = p->n_fused_blocks * 125u;
-    p->tasks_per_tiling = p->fused_tasks + (p->n_blocks - p->n_fused_blocks) * 25u;
+    p->fused_tasks = p->n_fused_blocks * 25u;
+    p->tasks_per_tiling = p->fused_tasks + (p->n_blocks - p->n_fused_blocks) * 5u;
     p->rows_per_tiling = p->tasks_per_tiling * (uint32_t)kRowsPerTask;
     if (p->n_tilings > UINT64_MAX / ((uint64_t)p->rows_per_tiling * 9u)) return MMEE_ERR_OVERFLOW;
 

@@ -8,8 +8,8 @@ namespace mmee {
 
 constexpr int kMaxOrders = 6;
 constexpr int kMaxBlocks = 18;     // (fusion mode, order) pairs
-constexpr int kRowsPerTask = 25;   // levels of D and E
-constexpr int kCandPerTask = 225;  // rows x 9 stationary pairs
+constexpr int kRowsPerTask = 125;   // one middle level (C when fused, B when unfused) x levels of D and E
+constexpr int kCandPerTask = 1125;  // rows x 9 stationary pairs
 constexpr int64_t kInfKey = INT64_MAX;
 
 // Operand / loop numbering shared by host planner and kernels.
@@ -33,11 +33,11 @@ struct Plan {
     uint32_t order_id[kMaxOrders];
     uint32_t n_blocks;            // (phi, order) blocks in row order, fused first
     uint32_t n_fused_blocks;
-    uint32_t fused_tasks;         // n_fused_blocks * 125
+    uint32_t fused_tasks;         // n_fused_blocks * 25
     uint8_t  block_phi[kMaxBlocks];
     uint8_t  block_order_slot[kMaxBlocks];   // position of the block's order in order_id[]
-    uint32_t tasks_per_tiling;    // fused_tasks + 25 per unfused block
-    uint32_t rows_per_tiling;     // R = 25 * tasks_per_tiling
+    uint32_t tasks_per_tiling;    // fused_tasks + 5 per unfused block
+    uint32_t rows_per_tiling;     // R = 125 * tasks_per_tiling
     uint64_t n_tilings;           // T
     uint64_t t_begin, t_end;
     int64_t  cap_words;
@@ -61,7 +61,7 @@ int build_plan(const mmee_workload_t* w, const mmee_arch_t* a, const mmee_object
 void build_query_tables(QueryTables* q);
 
 // Tie-safe symbolic row pruning (mmee_prune.cu): keep[row] for every row of a tiling.
-struct PrunedTask { uint32_t task, rows; };     // task inside a tiling, 25-bit mask of kept rows
+struct PrunedTask { uint32_t task, rows[5]; };  // task inside a tiling; per middle level the 25-bit mask of kept rows
 int build_pruned_tasks(const Plan& plan, PrunedTask* out, uint32_t* n_out, uint32_t* kept_rows);
 
 }  // namespace mmee

@@ -105,15 +105,24 @@ void build_row_keep(const Plan& p, std::vector<uint8_t>* keep) {
     std::map<Signature, int> ids;
     std::vector<Signature> sigs;
     std::vector<uint32_t> first_row;                      // lowest row index with this signature
-    for (uint32_t w = 0; w < p.tasks_per_tiling; ++w) {
-        uint32_t block, la, lb, lc;
-        if (w < p.fused_tasks) { block = w / 125u; const uint32_t r = w % 125u; la = r / 25u; lb = (r / 5u) % 5u; lc = r % 5u; }
-        else { const uint32_t u = w - p.fused_tasks; block = p.n_fused_blocks + u / 25u; const uint32_t r = u % 25u; la = r / 5u; lb = r % 5u; lc = 0; }
+    // rows in index order: fused r = o*3125 + lA*625 + lB*125 + lC*25 + lD*5 + lE, then per unfused
+    // mode o*625 + lA*125 + lB*25 + lD*5 + lE
+    const uint32_t fused_rows = p.n_fused_blocks * 3125u;
+    for (uint32_t row = 0; row < R; ++row) {
+        uint32_t block, lv[5];
+        if (row < fused_rows) {
+            block = row / 3125u;
+            const uint32_t r = row % 3125u;
+            lv[0] = r / 625u; lv[1] = (r / 125u) % 5u; lv[2] = (r / 25u) % 5u; lv[3] = (r / 5u) % 5u; lv[4] = r % 5u;
+        } else {
+            const uint32_t u = row - fused_rows;
+            block = p.n_fused_blocks + u / 625u;
+            const uint32_t r = u % 625u;
+            lv[0] = r / 125u; lv[1] = (r / 25u) % 5u; lv[2] = 0; lv[3] = (r / 5u) % 5u; lv[4] = r % 5u;
+        }
         const uint32_t phi = p.block_phi[block], order = p.order_id[p.block_order_slot[block]];
-        for (uint32_t de = 0; de < 25; ++de) {
-            const uint32_t lv[5] = {la, lb, lc, de / 5u, de % 5u};
+        {
             const Signature s = signature_of(p.q, phi, order, lv);
-            const uint32_t row = w * 25u + de;
             auto it = ids.find(s);
             if (it == ids.end()) {
                 it = ids.emplace(s, (int)sigs.size()).first;
@@ -135,17 +144,18 @@ void build_row_keep(const Plan& p, std::vector<uint8_t>* keep) {
 
 }  // namespace
 
-// The tasks (25 rows each) that still hold a kept row, in task order, with their kept-row masks.
+// The tasks (125 rows each) that still hold a kept row, in task order, with their kept-row masks.
 // `out` has room for tasks_per_tiling entries.
 int build_pruned_tasks(const Plan& p, PrunedTask* out, uint32_t* n_out, uint32_t* kept_rows) {
     std::vector<uint8_t> keep;
     build_row_keep(p, &keep);
     uint32_t n = 0, rows = 0;
     for (uint32_t w = 0; w < p.tasks_per_tiling; ++w) {
-        uint32_t mask = 0;
-        for (uint32_t de = 0; de < 25; ++de)
-            if (keep[w * 25u + de]) { mask |= 1u << de; ++rows; }
-        if (mask) { out[n].task = w; out[n].rows = mask; ++n; }
+        PrunedTask t = {w, {0, 0, 0, 0, 0}};
+        uint32_t any = 0;
+        for (uint32_t r = 0; r < 125; ++r)
+            if (keep[w * 125u + r]) { t.rows[r / 25u] |= 1u << (r % 25u); ++rows; any = 1; }
+        if (any) out[n++] = t;
     }
     *n_out = n;
     *kept_rows = rows;

@@ -538,12 +538,14 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
             const uint32_t slot = wa / tpt;
             const uint32_t wc = wa - slot * tpt;
             // With row pruning the searched task space lists only the tasks that still hold a kept
-            // row; `kept` is the 25-bit mask of those rows.
-            uint32_t w = wc, kept = 0x1ffffffu;
+            // row; kept_rows[m] is the 25-bit mask of those rows at middle level m.
+            uint32_t w = wc;
+            uint32_t kept_rows[5] = {0x1ffffffu, 0x1ffffffu, 0x1ffffffu, 0x1ffffffu, 0x1ffffffu};
             if constexpr (PRUNE) {
                 const PrunedTask pt = shape.pruned[wc];
                 w = pt.task;
-                kept = pt.rows;
+#pragma unroll
+                for (int m = 0; m < 5; ++m) kept_rows[m] = pt.rows[m];
             }
             const uint64_t tq = PRUNE ? (t_first + slot) * (uint64_t)p.tasks_per_tiling + w : r0 + o;
             const TilingTab* tb = &ttabs[slot];
@@ -557,49 +559,8 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
             const OrderTab* ot = &otabs[slot * n_orders + c.order_slot];
             const bool fused = c.phi == 0;
             const RowTab* rt = &ot->rt[fused ? 0 : 1];
-            // Tables of a tiling that cannot fit are never built: a lane whose task lies in such a
-            // tiling must not index with what it reads from them.
-            const uint32_t rc = (fused && live) ? (ot->rc[c.lc] & 1u) : 0u;
-            const int64_t a1 = ot->A1[c.la], b1 = ot->B1[c.lb], c1 = ot->C1[c.lc];
-            const int64_t a2 = fused ? ot->A2[c.la] : 0, b2 = fused ? ot->B2[c.lb] : 0;
-            // Eq. (1)/(2): a retained operand (level >= L4) of the other operator keeps its space.
-            // A lane without a live task gets a negative slack, so that none of its rows fits.
-            const int64_t slack1 = live ? cap - (a1 + b1 + c1) : -1;
-            const int64_t slack2 = live ? cap - (c1 + a2 + b2) : -1;
-            const int64_t gab = ot->gA[c.la][rc] + ot->gB[c.lb][rc];
-
-            int64_t x0, xe0 = 0, P[3], Q[9], W[9];
-            const int64_t* wptr = &tb->W[0][rc];
-            const int64_t* qptr;
-            if constexpr (OBJ == MMEE_OBJ_ENERGY) {
-                const int64_t extra = p.c_dram_gb * (tb->cw + (c.phi == 2 ? tb->smx : 0));
-                x0 = fused ? gab : gab + ot->gCr + extra;
-                P[0] = P[1] = P[2] = 0;
-                qptr = wptr;
-            } else {
-                const int64_t pass = (c.phi == 2) ? tb->smx : 0;
-                if (fused) {
-                    x0 = gab;
-                    P[0] = P[1] = P[2] = 0;
-                    qptr = &tb->CB[0][rc];
-                } else {
-                    // unfused latency: max(DA1, C1) + softmax pass + max(DA2, C2)
-                    x0 = ot->gCr;
-                    const int64_t da1 = gab + tb->cw;
-#pragma unroll
-                    for (int m = 0; m < 3; ++m) P[m] = (da1 > tb->C1w[m] ? da1 : tb->C1w[m]) + pass;
-                    qptr = &tb->QU[0][0];
-                }
-                if constexpr (OBJ == MMEE_OBJ_EDP) {
-                    const int64_t eab = ot->eA[c.la][rc] + ot->eB[c.lb][rc];
-                    xe0 = fused ? eab : eab + ot->eCr + p.c_dram_gb * (tb->cw + pass);
-                }
-            }
-#pragma unroll
-            for (int s = 0; s < 9; ++s) {
-                W[s] = wptr[2 * s];
-                Q[s] = qptr[2 * s];
-            }
+            const int64_t a1 = ot->A1[c.la];
+            const int64_t a2 = fused ? ot->A2[c.la] : 0;
             const uint64_t task_first_idx = tq * kCandPerTask;
             // The other CTAs' pruning bound: the load is issued here and consumed at the end of the
             // task, so that its latency is covered by the task's own work.
@@ -620,7 +581,67 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
             };
             load_threshold();
             uint32_t rows = 0;
+            int E1c[5], E2c[5], Gc[5];
+#pragma unroll
+            for (int e = 0; e < 5; ++e) {
+                const int4 v = *reinterpret_cast<const int4*>(rt->Ec[e]);
+                E1c[e] = v.x; E2c[e] = v.y; Gc[e] = v.z;
+            }
 
+            // Middle loop of the task: the level of C for a fused task, of B for an unfused one.
+#pragma unroll 1
+            for (int m = 0; m < 5; ++m) {
+            uint32_t kept = 0x1ffffffu;
+            if constexpr (PRUNE) {
+                kept = kept_rows[m];
+                if (!__any_sync(kFull, live && kept)) continue;
+            }
+            const uint32_t lb = fused ? c.lb : (uint32_t)m;
+            const uint32_t lc = fused ? (uint32_t)m : 0u;
+            const uint64_t mid_first_idx = task_first_idx + (uint64_t)(m * 225);
+            // Tables of a tiling that cannot fit are never built: a lane whose task lies in such a
+            // tiling must not index with what it reads from them.
+            const uint32_t rc = (fused && live) ? (ot->rc[lc] & 1u) : 0u;
+            const int64_t b1 = ot->B1[lb], c1 = ot->C1[lc];
+            const int64_t b2 = fused ? ot->B2[lb] : 0;
+            // Eq. (1)/(2): a retained operand (level >= L4) of the other operator keeps its space.
+            // A lane without a live task gets a negative slack, so that none of its rows fits.
+            const int64_t slack1 = live ? cap - (a1 + b1 + c1) : -1;
+            const int64_t slack2 = live ? cap - (c1 + a2 + b2) : -1;
+            const int64_t gab = ot->gA[c.la][rc] + ot->gB[lb][rc];
+
+            int64_t x0, xe0 = 0, P[3], Q[9], W[9];
+            const int64_t* wptr = &tb->W[0][rc];
+            const int64_t* qptr;
+            if constexpr (OBJ == MMEE_OBJ_ENERGY) {
+                const int64_t extra = p.c_dram_gb * (tb->cw + (c.phi == 2 ? tb->smx : 0));
+                x0 = fused ? gab : gab + ot->gCr + extra;
+                P[0] = P[1] = P[2] = 0;
+                qptr = wptr;
+            } else {
+                const int64_t pass = (c.phi == 2) ? tb->smx : 0;
+                if (fused) {
+                    x0 = gab;
+                    P[0] = P[1] = P[2] = 0;
+                    qptr = &tb->CB[0][rc];
+                } else {
+                    // unfused latency: max(DA1, C1) + softmax pass + max(DA2, C2)
+                    x0 = ot->gCr;
+                    const int64_t da1 = gab + tb->cw;
+#pragma unroll
+                    for (int j = 0; j < 3; ++j) P[j] = (da1 > tb->C1w[j] ? da1 : tb->C1w[j]) + pass;
+                    qptr = &tb->QU[0][0];
+                }
+                if constexpr (OBJ == MMEE_OBJ_EDP) {
+                    const int64_t eab = ot->eA[c.la][rc] + ot->eB[lb][rc];
+                    xe0 = fused ? eab : eab + ot->eCr + p.c_dram_gb * (tb->cw + pass);
+                }
+            }
+#pragma unroll
+            for (int s = 0; s < 9; ++s) {
+                W[s] = wptr[2 * s];
+                Q[s] = qptr[2 * s];
+            }
             // threshold-relative forms (see "32-bit differential keys"); refreshed when thr moves
             int64_t wmin = 0;
             int Wc[9], Qc[9];
@@ -667,12 +688,6 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                 }
             };
             refresh(T1);
-            int E1c[5], E2c[5], Gc[5];
-#pragma unroll
-            for (int e = 0; e < 5; ++e) {
-                const int4 v = *reinterpret_cast<const int4*>(rt->Ec[e]);
-                E1c[e] = v.x; E2c[e] = v.y; Gc[e] = v.z;
-            }
             const int slack1c = slack1 < 0 ? -1 : (int)slack1;      // slack <= capacity < 2^30
             const int slack2c = slack2 < 0 ? -1 : (int)slack2;
 
@@ -691,7 +706,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                     int acc = INT_MAX;
                     fits = 0;
                     if constexpr (OBJ == MMEE_OBJ_ENERGY) {
-                        const uint64_t group_first_idx = task_first_idx + (uint64_t)(d * 45);
+                        const uint64_t group_first_idx = mid_first_idx + (uint64_t)(d * 45);
                         const int uc = __viaddmin_s32(group_first_idx > ti ? ut[1] : ut[0], dc.z, kRelCap);
                         int accs[9];          // one chain per stationary pair: nine independent chains
 #pragma unroll
@@ -729,7 +744,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                     if constexpr (OBJ == MMEE_OBJ_ENERGY) {
                         hit_any = acc < 0;
                     } else {
-                        const uint64_t group_first_idx = task_first_idx + (uint64_t)(d * 45);
+                        const uint64_t group_first_idx = mid_first_idx + (uint64_t)(d * 45);
                         hit_any = acc < (group_first_idx > ti ? -delta : 0);  // no overflow at acc = INT_MAX
                     }
                 } else if constexpr (!DUMP && OBJ == MMEE_OBJ_EDP) {
@@ -763,7 +778,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                     const int64_t s2 = slack2 - rt->D[d][1];
                     const int64_t xd = x0 + rt->D[d][2];
                     const int64_t xed = (OBJ == MMEE_OBJ_EDP) ? xe0 + rt->D[d][3] : 0;
-                    const uint64_t group_first_idx = task_first_idx + (uint64_t)(d * 45);
+                    const uint64_t group_first_idx = mid_first_idx + (uint64_t)(d * 45);
                     const int64_t thr = T1 - (group_first_idx > ti ? delta : 0);
                     hit_any = 0; fits = 0;
 #pragma unroll
@@ -781,7 +796,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                             if (valid) {
 #pragma unroll
                                 for (int s = 0; s < 9; ++s)
-                                    dump[task_first_idx - dump_origin + (d * 5 + e) * 9 + s] = fit ? key[s] : kInfKey;
+                                    dump[mid_first_idx - dump_origin + (d * 5 + e) * 9 + s] = fit ? key[s] : kInfKey;
                             }
                         }
                     }
@@ -798,7 +813,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                         const bool fit = (rt->E[e][0] <= s1) && (rt->E[e][1] <= s2) && ((kept >> (d * 5 + e)) & 1u);
                         const int64_t x = xd + rt->E[e][2];
                         const int64_t xe = (OBJ == MMEE_OBJ_EDP) ? xed + rt->E[e][3] : 0;
-                        const uint64_t row_first_idx = task_first_idx + (uint64_t)((d * 5 + e) * 9);
+                        const uint64_t row_first_idx = mid_first_idx + (uint64_t)((d * 5 + e) * 9);
                         const int64_t thr_row = lane_threshold(wt, cs, k, row_first_idx);
                         bool below = false;
                         for (int s = 0; s < 9; ++s)
@@ -811,6 +826,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                     refresh(T1);
                 }
             }
+            }   // middle loop
             my_rows += rows;
             if (lane == 0 && g_seen < cs->G) atomicMin(&cs->G, g_seen);
         }
