@@ -33,7 +33,8 @@ int choose_shape(const Plan& p, int device, uint32_t search_tpt, LaunchShape* sh
     if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
         cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess)
         return MMEE_ERR_CUDA;
-    const uint32_t rounds = 2;      // each task is 1125 mappings
+    // A task is 1125 mappings (225 with row pruning, where the searched units are single middle levels).
+    const uint32_t rounds = p.row_pruning ? 9 : 3;
     shape->range_tasks = rounds * kWorkerThreads;
     shape->search_tpt = search_tpt;
     shape->pad = 0;
@@ -94,7 +95,7 @@ int mmee_create(const mmee_workload_t* workload, const mmee_arch_t* arch, const 
     uint32_t search_tpt = h->plan.tasks_per_tiling;
     h->kept_rows = h->plan.rows_per_tiling;
     if (h->plan.row_pruning) {
-        kept_tasks.resize(h->plan.tasks_per_tiling);
+        kept_tasks.resize(5 * (size_t)h->plan.tasks_per_tiling);
         uint32_t n = 0;
         build_pruned_tasks(h->plan, kept_tasks.data(), &n, &h->kept_rows);
         kept_tasks.resize(n);
@@ -257,13 +258,13 @@ int mmee_row_pruning_keep(const mmee_objective_t* objective, uint8_t* out_keep, 
     if (rc) return rc;
     *out_rows = plan.rows_per_tiling;
     if (capacity < plan.rows_per_tiling) return MMEE_ERR_RANGE;
-    std::vector<PrunedTask> tasks(plan.tasks_per_tiling);
+    std::vector<PrunedTask> tasks(5 * (size_t)plan.tasks_per_tiling);
     uint32_t n = 0, kept = 0;
     build_pruned_tasks(plan, tasks.data(), &n, &kept);
     std::memset(out_keep, 0, plan.rows_per_tiling);
     for (uint32_t i = 0; i < n; ++i)
-        for (uint32_t r = 0; r < 125; ++r)
-            if (tasks[i].rows[r / 25u] >> (r % 25u) & 1u) out_keep[tasks[i].task * 125u + r] = 1;
+        for (uint32_t de = 0; de < 25; ++de)
+            if (tasks[i].rows >> de & 1u) out_keep[tasks[i].task * 125u + tasks[i].mid * 25u + de] = 1;
     return MMEE_OK;
 }
 

@@ -61,7 +61,7 @@ int build_plan(const mmee_workload_t* w, const mmee_arch_t* a, const mmee_object
 void build_query_tables(QueryTables* q);
 
 // Tie-safe symbolic row pruning (mmee_prune.cu): keep[row] for every row of a tiling.
-struct PrunedTask { uint32_t task, rows[5]; };  // task inside a tiling; per middle level the 25-bit mask of kept rows
+struct PrunedTask { uint32_t task, mid, rows, pad; };   // task inside a tiling, middle level, 25-bit mask of kept rows
 int build_pruned_tasks(const Plan& plan, PrunedTask* out, uint32_t* n_out, uint32_t* kept_rows);
 
 }  // namespace mmee

@@ -144,18 +144,19 @@ void build_row_keep(const Plan& p, std::vector<uint8_t>* keep) {
 
 }  // namespace
 
-// The tasks (125 rows each) that still hold a kept row, in task order, with their kept-row masks.
-// `out` has room for tasks_per_tiling entries.
+// The (task, middle level) groups of 25 rows that still hold a kept row, in index order, with their
+// kept-row masks.  `out` has room for 5 * tasks_per_tiling entries.
 int build_pruned_tasks(const Plan& p, PrunedTask* out, uint32_t* n_out, uint32_t* kept_rows) {
     std::vector<uint8_t> keep;
     build_row_keep(p, &keep);
     uint32_t n = 0, rows = 0;
     for (uint32_t w = 0; w < p.tasks_per_tiling; ++w) {
-        PrunedTask t = {w, {0, 0, 0, 0, 0}};
-        uint32_t any = 0;
-        for (uint32_t r = 0; r < 125; ++r)
-            if (keep[w * 125u + r]) { t.rows[r / 25u] |= 1u << (r % 25u); ++rows; any = 1; }
-        if (any) out[n++] = t;
+        for (uint32_t m = 0; m < 5; ++m) {
+            PrunedTask t = {w, m, 0, 0};
+            for (uint32_t de = 0; de < 25; ++de)
+                if (keep[w * 125u + m * 25u + de]) { t.rows |= 1u << de; ++rows; }
+            if (t.rows) out[n++] = t;
+        }
     }
     *n_out = n;
     *kept_rows = rows;

@@ -538,14 +538,13 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
             const uint32_t slot = wa / tpt;
             const uint32_t wc = wa - slot * tpt;
             // With row pruning the searched task space lists only the tasks that still hold a kept
-            // row; kept_rows[m] is the 25-bit mask of those rows at middle level m.
-            uint32_t w = wc;
-            uint32_t kept_rows[5] = {0x1ffffffu, 0x1ffffffu, 0x1ffffffu, 0x1ffffffu, 0x1ffffffu};
+            // row: each searched unit is one middle level (kept_mid) of a task, `kept` the mask of its rows.
+            uint32_t w = wc, kept = 0x1ffffffu, kept_mid = 0;
             if constexpr (PRUNE) {
                 const PrunedTask pt = shape.pruned[wc];
                 w = pt.task;
-#pragma unroll
-                for (int m = 0; m < 5; ++m) kept_rows[m] = pt.rows[m];
+                kept_mid = pt.mid;
+                kept = pt.rows;
             }
             const uint64_t tq = PRUNE ? (t_first + slot) * (uint64_t)p.tasks_per_tiling + w : r0 + o;
             const TilingTab* tb = &ttabs[slot];
@@ -590,12 +589,8 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
 
             // Middle loop of the task: the level of C for a fused task, of B for an unfused one.
 #pragma unroll 1
-            for (int m = 0; m < 5; ++m) {
-            uint32_t kept = 0x1ffffffu;
-            if constexpr (PRUNE) {
-                kept = kept_rows[m];
-                if (!__any_sync(kFull, live && kept)) continue;
-            }
+            for (int mi = 0; mi < (PRUNE ? 1 : 5); ++mi) {
+            const int m = PRUNE ? (int)kept_mid : mi;
             const uint32_t lb = fused ? c.lb : (uint32_t)m;
             const uint32_t lc = fused ? (uint32_t)m : 0u;
             const uint64_t mid_first_idx = task_first_idx + (uint64_t)(m * 225);

@@ -48,7 +48,7 @@ int static_shape(const Plan& p, int device, LaunchShape* shape) {
     if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
         cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess)
         return MMEE_ERR_CUDA;
-    shape->range_tasks = 2 * kWorkerThreads;
+    shape->range_tasks = 3 * kWorkerThreads;
     shape->search_tpt = p.tasks_per_tiling;
     shape->pad = 0;
     shape->pruned = nullptr;
