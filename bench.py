@@ -39,6 +39,9 @@ OBJ_NAMES = {0: "energy", 1: "latency", 2: "edp"}
 # conversions, four 64-bit adds and the capacity test (15).
 ALG_OPS_PER_CANDIDATE = {0: 1.0 + 5.0 / 9.0, 1: 2.0 + 8.0 / 9.0, 2: 6.0 + 15.0 / 9.0}
 INT_LANES_PER_SM = 64          # 4 sub-partitions x 16 integer-ALU lanes
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the exhaustive search kernels on the BERT workload,
+# from the ncu capture summarised under profiles/ (energy, latency); None for other workloads.
+NCU_DRAM_BYTES_PER_LAUNCH = {"bert": {0: 92160, 1: 91648}}
 
 
 WORKLOADS = {"tiny": mi.config1, "bert": mi.config2, "llama": mi.config3, "gqa": mi.config4}
@@ -298,7 +301,8 @@ def main():
             sm = statistics.mean(k[i][0] for k in kernel_ms)
             fm = statistics.mean(k[i][1] for k in kernel_ms)
             ops = bests[i].n_feasible * ALG_OPS_PER_CANDIDATE[s["objective"]]
-            per_kernel.append(dict(kernel="search_kernel<%s>" % OBJ_NAMES[s["objective"]], problem=jobs[i][0]["name"],
+            per_kernel.append(dict(kernel="search_kernel<%s>" % OBJ_NAMES[s["objective"]], objective=s["objective"],
+                                   problem=jobs[i][0]["name"],
                                    avg_ms=sm, finalize_avg_ms=fm, candidates=n, feasible=bests[i].n_feasible,
                                    pruned_fraction=1.0 - bests[i].n_feasible / n, time_to_optimum_ms=tto_ms[i],
                                    candidates_per_s=n / (sm * 1e-3), achieved_gops=ops / (sm * 1e-3) / 1e9))
@@ -307,7 +311,8 @@ def main():
         n_sm = torch.cuda.get_device_properties(local_rank).multi_processor_count
         peak = n_sm * INT_LANES_PER_SM * sm_mhz * 1e6 / 1e9
         roofline = dict(bound="alu", kernel=dom["kernel"], achieved=dom["achieved_gops"], peak=peak,
-                        unit="Gop/s (32-bit integer instructions)", frac=dom["achieved_gops"] / peak, traffic=None,
+                        unit="Gop/s (32-bit integer instructions)", frac=dom["achieved_gops"] / peak,
+                        traffic=NCU_DRAM_BYTES_PER_LAUNCH.get(args.workload, {}).get(dom["objective"]),
                         peak_source="%d SMs x %d integer-ALU lanes x %.0f MHz (clock sampled during the run)" %
                                     (n_sm, INT_LANES_PER_SM, sm_mhz),
                         measured_rates_gops=dict(logic=peaks[0], add_logic=peaks[1], key_mix=peaks[2],
