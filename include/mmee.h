@@ -41,6 +41,8 @@ extern "C" {
 #define MMEE_OBJ_ENERGY   0u   /* energy-driven search (Section VII-D)                         */
 #define MMEE_OBJ_LATENCY  1u   /* latency-driven search                                         */
 #define MMEE_OBJ_EDP      2u   /* energy-delay product (Section VII-K)                          */
+#define MMEE_OBJ_ENERGY_LCAP   3u   /* least energy among mappings with l_key <= key_cap          */
+#define MMEE_OBJ_LATENCY_ECAP  4u   /* least latency among mappings with e_key <= key_cap         */
 /* tiling_set */
 #define MMEE_TILE_POW2          0u   /* only power-of-two tile extents                          */
 #define MMEE_TILE_ALL_DIVISORS  1u   /* every integer factorisation (Section VI-A)              */
@@ -97,6 +99,8 @@ typedef struct {
                                                 tiling are not evaluated: the optimum is unchanged, but
                                                 n_feasible then counts only the evaluated rows.        */
     uint64_t t_begin, t_end;                 /* tiling sub-range [t_begin,t_end); 0,0 = all       */
+    int64_t  key_cap;                        /* MMEE_OBJ_*CAP: bound on the other key (energy in quanta,
+                                                latency in words); ignored otherwise                   */
 } mmee_objective_t;
 
 /* One fully evaluated mapping.  Counts are per instance. */
@@ -217,6 +221,21 @@ int mmee_dump_keys(mmee_handle_t* handle, void* cuda_stream, int64_t* out_keys);
 int mmee_solve_host(const mmee_workload_t* workload, const mmee_arch_t* arch,
                     const mmee_objective_t* objective, mmee_result_t* out_best,
                     mmee_result_t* out_topk, uint64_t* h2d_bytes, uint64_t* d2h_bytes);
+
+/*
+ * mmee_pareto_front -- the energy-latency trade-off of the whole mapping space (Section VII-E): every
+ * pair (e_key, l_key) of a feasible mapping that no other feasible mapping improves in one key without
+ * losing in the other, by increasing energy / decreasing latency, each with the lowest-index mapping
+ * that attains it.  Computed by alternating capped searches on the device (least energy under a latency
+ * bound, then least latency at that energy): two searches per point.  objective.objective, .topk,
+ * .row_pruning and .key_cap are ignored.  Synchronous.
+ *   out_points : HOST, `capacity` records; *n_points receives the number of points of the front, also
+ *                when it exceeds capacity (then MMEE_ERR_RANGE is returned and the first `capacity`
+ *                points are valid).
+ */
+int mmee_pareto_front(const mmee_workload_t* workload, const mmee_arch_t* arch,
+                      const mmee_objective_t* objective, mmee_result_t* out_points, uint32_t capacity,
+                      uint32_t* n_points);
 
 /*
  * mmee_query_vector -- HOST only, no device needed.  The query vector q in {0,1}^8 over

@@ -10,7 +10,7 @@ from __future__ import annotations
 
 import random
 
-OBJ_ENERGY, OBJ_LATENCY, OBJ_EDP = 0, 1, 2
+OBJ_ENERGY, OBJ_LATENCY, OBJ_EDP, OBJ_ENERGY_LCAP, OBJ_LATENCY_ECAP = 0, 1, 2, 3, 4
 TILE_POW2, TILE_ALL_DIVISORS = 0, 1
 ORD_NORECOMP2, ORD_ALL6 = 0, 1
 FUSE_FUSED, FUSE_SOFTMAX_IN_OP1, FUSE_SEPARATE = 1, 2, 4
@@ -34,9 +34,9 @@ def arch(pe_rows, pe_cols, n_arrays, gb_bytes, rf_bytes, dram_words_per_cycle,
 
 
 def objective(objective=OBJ_ENERGY, topk=1, tiling_set=TILE_ALL_DIVISORS, order_set=ORD_ALL6,
-              fuse_mask=FUSE_ALL, t_begin=0, t_end=0, row_pruning=0):
+              fuse_mask=FUSE_ALL, t_begin=0, t_end=0, row_pruning=0, key_cap=0):
     return dict(objective=objective, topk=topk, tiling_set=tiling_set, order_set=order_set,
-                fuse_mask=fuse_mask, row_pruning=row_pruning, t_begin=t_begin, t_end=t_end)
+                fuse_mask=fuse_mask, row_pruning=row_pruning, t_begin=t_begin, t_end=t_end, key_cap=key_cap)
 
 
 # --- accelerators -----------------------------------------------------------------------------

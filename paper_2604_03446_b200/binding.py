@@ -11,7 +11,7 @@ import os
 
 from . import build as _build
 
-OBJ_ENERGY, OBJ_LATENCY, OBJ_EDP = 0, 1, 2
+OBJ_ENERGY, OBJ_LATENCY, OBJ_EDP, OBJ_ENERGY_LCAP, OBJ_LATENCY_ECAP = 0, 1, 2, 3, 4
 TILE_POW2, TILE_ALL_DIVISORS = 0, 1
 ORD_NORECOMP2, ORD_ALL6 = 0, 1
 FUSE_FUSED, FUSE_SOFTMAX_IN_OP1, FUSE_SEPARATE = 1, 2, 4
@@ -20,7 +20,7 @@ NO_INDEX = 2 ** 64 - 1
 OK, ERR_ARG, ERR_OVERFLOW, ERR_QUANTUM, ERR_NO_FEASIBLE, ERR_CUDA, ERR_TIMEOUT, ERR_RANGE = range(8)
 
 EXPORTS = ("mmee_create", "mmee_search", "mmee_destroy", "mmee_search_static", "mmee_num_candidates", "mmee_num_tilings",
-           "mmee_num_rows", "mmee_strerror", "mmee_last_cuda_error", "mmee_eval", "mmee_dump_keys", "mmee_solve_host",
+           "mmee_num_rows", "mmee_strerror", "mmee_last_cuda_error", "mmee_eval", "mmee_dump_keys", "mmee_solve_host", "mmee_pareto_front",
            "mmee_query_vector", "mmee_recompute_flag", "mmee_row_pruning_keep", "mmee_last_search_stats", "mmee_kernel_timing",
            "mmee_alu_peak")
 
@@ -42,7 +42,7 @@ class Arch(C.Structure):
 class Objective(C.Structure):
     _fields_ = [("objective", C.c_uint32), ("topk", C.c_uint32), ("tiling_set", C.c_uint32),
                 ("order_set", C.c_uint32), ("fuse_mask", C.c_uint32), ("row_pruning", C.c_uint32),
-                ("t_begin", C.c_uint64), ("t_end", C.c_uint64)]
+                ("t_begin", C.c_uint64), ("t_end", C.c_uint64), ("key_cap", C.c_int64)]
 
 
 class Result(C.Structure):
@@ -112,6 +112,8 @@ def library():
     L.mmee_solve_host.argtypes = [C.POINTER(Workload), C.POINTER(Arch), C.POINTER(Objective),
                                   C.POINTER(Result), C.POINTER(Result),
                                   C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
+    L.mmee_pareto_front.argtypes = [C.POINTER(Workload), C.POINTER(Arch), C.POINTER(Objective),
+                                    C.POINTER(Result), C.c_uint32, C.POINTER(C.c_uint32)]
     L.mmee_query_vector.argtypes = [C.c_uint32] * 6 + [C.POINTER(C.c_uint8)]
     L.mmee_recompute_flag.argtypes = [C.c_uint32, C.c_uint32, C.POINTER(C.c_uint32)]
     L.mmee_row_pruning_keep.argtypes = [C.POINTER(Objective), C.POINTER(C.c_uint8), C.c_uint32,
@@ -207,6 +209,16 @@ def mmee_solve_host(workload: dict, arch: dict, objective: dict):
                                      _fill(Objective(), objective), C.byref(best), topk,
                                      C.byref(h2d), C.byref(d2h)), "mmee_solve_host")
     return best, list(topk), h2d.value, d2h.value
+
+
+def mmee_pareto_front(workload: dict, arch: dict, objective: dict, capacity: int = 256):
+    """Energy-latency Pareto front of the whole mapping space: list of Result, by increasing energy."""
+    pts = (Result * capacity)()
+    n = C.c_uint32()
+    _check(library().mmee_pareto_front(_fill(Workload(), workload), _fill(Arch(), arch),
+                                       _fill(Objective(), objective), pts, capacity, C.byref(n)),
+           "mmee_pareto_front")
+    return list(pts[:n.value])
 
 
 def mmee_query_vector(metric: int, phi: int, pi: int, operand: int, beta: int, recompute: int = 0):

@@ -219,6 +219,47 @@ int mmee_solve_host(const mmee_workload_t* workload, const mmee_arch_t* arch, co
     return rc ? rc : rc2;
 }
 
+int mmee_pareto_front(const mmee_workload_t* workload, const mmee_arch_t* arch, const mmee_objective_t* objective,
+                      mmee_result_t* out_points, uint32_t capacity, uint32_t* n_points) {
+    if (!objective || !n_points || (!out_points && capacity)) return MMEE_ERR_ARG;
+    *n_points = 0;
+    mmee_objective_t oe = *objective, ol = *objective;
+    oe.objective = MMEE_OBJ_ENERGY_LCAP;  oe.topk = 1; oe.row_pruning = 0; oe.key_cap = INT64_MAX - 1;
+    ol.objective = MMEE_OBJ_LATENCY_ECAP; ol.topk = 1; ol.row_pruning = 0; ol.key_cap = INT64_MAX - 1;
+    mmee_handle_t *he = nullptr, *hl = nullptr;
+    int rc = mmee_create(workload, arch, &oe, &he);
+    if (rc) return rc;
+    rc = mmee_create(workload, arch, &ol, &hl);
+    if (rc) { mmee_destroy(he); return rc; }
+    mmee_result_t* dev = nullptr;
+    if (cudaMalloc(reinterpret_cast<void**>(&dev), sizeof(mmee_result_t)) != cudaSuccess) rc = MMEE_ERR_CUDA;
+    mmee_result_t r;
+    int64_t latency_cap = INT64_MAX - 1;
+    uint32_t n = 0;
+    while (rc == MMEE_OK) {
+        // least energy among the mappings that are still faster than the previous point
+        he->plan.key_cap = latency_cap;
+        if ((rc = mmee_search(he, nullptr, dev, nullptr))) break;
+        if ((rc = cuda_status(cudaMemcpy(&r, dev, sizeof(r), cudaMemcpyDeviceToHost)))) break;
+        if (r.idx == MMEE_NO_INDEX) break;                       // nothing faster is left
+        // the fastest mapping at that energy: the point of the front, with its lowest index
+        hl->plan.key_cap = r.e_key;
+        if ((rc = mmee_search(hl, nullptr, dev, nullptr))) break;
+        if ((rc = cuda_status(cudaMemcpy(&r, dev, sizeof(r), cudaMemcpyDeviceToHost)))) break;
+        if (r.idx == MMEE_NO_INDEX) { rc = MMEE_ERR_CUDA; break; }   // cannot happen: the previous optimum qualifies
+        if (n < capacity) out_points[n] = r;
+        ++n;
+        if (r.l_key == 0) break;
+        latency_cap = r.l_key - 1;
+    }
+    if (dev) cudaFree(dev);
+    mmee_destroy(he);
+    mmee_destroy(hl);
+    *n_points = n;
+    if (rc == MMEE_OK && n > capacity) rc = MMEE_ERR_RANGE;
+    return rc;
+}
+
 int mmee_query_vector(uint32_t metric, uint32_t phi, uint32_t pi, uint32_t operand, uint32_t beta,
                       uint32_t recompute, uint8_t out_q[8]) {
     if (!out_q || metric > 1 || phi > 2 || pi > 5 || operand > 4 || beta < 3 || beta > 7 || recompute > 1)

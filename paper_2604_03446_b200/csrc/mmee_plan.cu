@@ -138,7 +138,8 @@ int build_plan(const mmee_workload_t* w, const mmee_arch_t* a, const mmee_object
     if (!w->batch || !w->q_heads || !w->kv_heads || (w->q_heads % w->kv_heads)) return MMEE_ERR_ARG;
     if (!w->seq_q || !w->seq_kv || !w->d_qk || !w->d_v || !w->word_bytes) return MMEE_ERR_ARG;
     if (!a->pe_rows || !a->pe_cols || !a->n_arrays || !a->dram_words_per_cycle) return MMEE_ERR_ARG;
-    if (o->objective > MMEE_OBJ_EDP) return MMEE_ERR_ARG;
+    if (o->objective > MMEE_OBJ_LATENCY_ECAP) return MMEE_ERR_ARG;
+    if (o->objective >= MMEE_OBJ_ENERGY_LCAP && o->key_cap < 0) return MMEE_ERR_ARG;
     if (o->topk < 1) return MMEE_ERR_ARG;
     if (o->topk > MMEE_MAX_TOPK) return MMEE_ERR_RANGE;
     if (o->row_pruning > 1 || (o->row_pruning && o->topk != 1)) return MMEE_ERR_ARG;
@@ -225,6 +226,7 @@ int build_plan(const mmee_workload_t* w, const mmee_arch_t* a, const mmee_object
     p->objective = o->objective;
     p->topk = o->topk;
     p->row_pruning = o->row_pruning;
+    p->key_cap = o->key_cap;
 
     // Largest key any mapping of this problem can have.  M bounds the MAC count with the largest
     // recomputation factor (j_D <= J); each of at most seven DRAM terms is <= I*K*L*J <= M, the

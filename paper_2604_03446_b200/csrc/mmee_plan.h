@@ -50,6 +50,7 @@ struct Plan {
     uint32_t bw, pe_rows, pe_cols;
     uint32_t objective, topk;
     uint32_t row_pruning;
+    int64_t  key_cap;             // capped objectives: bound on the other key
     uint32_t rel_shift;           // energy: threshold-relative keys are kept in units of 2^rel_shift quanta
     double   quantum_pj;
     QueryTables q;

@@ -130,8 +130,12 @@ __device__ __forceinline__ int64_t lane_threshold(const WarpTop* wt, const CtaSh
 
 __device__ __forceinline__ int64_t dbits(double v) { return __double_as_longlong(v); }
 
+// x: row sum of the objective's primary side (energy-scaled for the energy objective, DRAM words for
+// the others); xe: energy-scaled row sum (objectives that need both sides); w, p, q: stationary-pair
+// terms; cap: bound on the other key for the capped objectives (a violating mapping gets kInfKey,
+// which never passes a threshold).
 template <int OBJ>
-__device__ __forceinline__ int64_t candidate_key(int64_t x, int64_t xe, int64_t w, int64_t p, int64_t q) {
+__device__ __forceinline__ int64_t candidate_key(int64_t x, int64_t xe, int64_t w, int64_t p, int64_t q, int64_t cap) {
     if constexpr (OBJ == MMEE_OBJ_ENERGY) {
         return x + w;
     } else if constexpr (OBJ == MMEE_OBJ_LATENCY) {
@@ -139,7 +143,9 @@ __device__ __forceinline__ int64_t candidate_key(int64_t x, int64_t xe, int64_t 
     } else {
         const int64_t e = xe + w;
         const int64_t l = p + (x > q ? x : q);
-        return dbits(__dmul_rn((double)e, (double)l));
+        if constexpr (OBJ == MMEE_OBJ_EDP) return dbits(__dmul_rn((double)e, (double)l));
+        else if constexpr (OBJ == MMEE_OBJ_ENERGY_LCAP) return l <= cap ? e : kInfKey;
+        else return e <= cap ? l : kInfKey;
     }
 }
 
@@ -248,12 +254,12 @@ __device__ __forceinline__ unsigned edp_row_test(double de, const double (&dl)[3
 template <int OBJ>
 __device__ __noinline__ int64_t slow_row(WarpTop* wt, CtaShared* cs, long long* global_g, int k, int lane, bool f,
                                          int64_t x, int64_t xe, const int64_t* wptr, const int64_t* qptr,
-                                         int64_t p0, int64_t p1, int64_t p2,
+                                         int64_t p0, int64_t p1, int64_t p2, int64_t cap,
                                          uint64_t row_first_idx) {
     int64_t thr = lane_threshold(wt, cs, k, row_first_idx);
     for (int s = 0; s < 9; ++s) {
         const int64_t pp = s < 3 ? p0 : (s < 6 ? p1 : p2);
-        const int64_t key = candidate_key<OBJ>(x, xe, wptr[2 * s], pp, qptr[2 * s]);
+        const int64_t key = candidate_key<OBJ>(x, xe, wptr[2 * s], pp, qptr[2 * s], cap);
         bool pend = f && key < thr;
         while (true) {
             const unsigned m = __ballot_sync(kFull, pend);
@@ -328,7 +334,7 @@ __device__ __forceinline__ void build_order_item(const Plan& p, const uint32_t* 
         s2[l] = l ? bs : 0;                            // retained (tau = 1) from L4 upwards
         g[l][0] = scale * v0;
         g[l][1] = scale * v1;
-        if (OBJ == MMEE_OBJ_EDP) { e[l][0] = escale * v0; e[l][1] = escale * v1; }
+        if (OBJ >= MMEE_OBJ_EDP) { e[l][0] = escale * v0; e[l][1] = escale * v1; }
     } else if (item < 15) {                            // C
         ot->C1[l] = monomial(q.bs[order][OP_C][l], b);
         ot->rc[l] = q.recompute[order][l];
@@ -627,7 +633,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                     for (int j = 0; j < 3; ++j) P[j] = (da1 > tb->C1w[j] ? da1 : tb->C1w[j]) + pass;
                     qptr = &tb->QU[0][0];
                 }
-                if constexpr (OBJ == MMEE_OBJ_EDP) {
+                if constexpr (OBJ >= MMEE_OBJ_EDP) {
                     const int64_t eab = ot->eA[c.la][rc] + ot->eB[lb][rc];
                     xe0 = fused ? eab : eab + ot->eCr + p.c_dram_gb * (tb->cw + pass);
                 }
@@ -676,7 +682,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                     }
 #pragma unroll
                     for (int s = 0; s < 9; ++s) Qc[s] = sat_s32(Q[s] + P[s / 3] - t);
-                } else {
+                } else if constexpr (OBJ == MMEE_OBJ_EDP) {
                     // EDP keys are bit patterns of positive doubles; anything from +inf up means "no bound yet"
                     dthr = t >= 0x7ff0000000000000ll ? __longlong_as_double(0x7ff0000000000000ll)
                                                      : __longlong_as_double(t) * (1.0 + 1e-14);
@@ -694,7 +700,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                 // Five rows (levels of E) are evaluated branch-free; one vote decides whether any
                 // lane of the warp has to enter the insertion path for this group.
                 unsigned hit_any, fits;
-                if constexpr (!DUMP && OBJ != MMEE_OBJ_EDP) {
+                if constexpr (!DUMP && OBJ <= MMEE_OBJ_LATENCY) {
                     const int4 dc = *reinterpret_cast<const int4*>(rt->Dc[d]);
                     const int s1c = slack1c - dc.x;
                     const int s2c = slack2c - dc.y;
@@ -772,17 +778,17 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                     const int64_t s1 = slack1 - rt->D[d][0];
                     const int64_t s2 = slack2 - rt->D[d][1];
                     const int64_t xd = x0 + rt->D[d][2];
-                    const int64_t xed = (OBJ == MMEE_OBJ_EDP) ? xe0 + rt->D[d][3] : 0;
+                    const int64_t xed = (OBJ >= MMEE_OBJ_EDP) ? xe0 + rt->D[d][3] : 0;
                     const uint64_t group_first_idx = mid_first_idx + (uint64_t)(d * 45);
                     const int64_t thr = T1 - (group_first_idx > ti ? delta : 0);
                     hit_any = 0; fits = 0;
 #pragma unroll
                     for (int e = 0; e < 5; ++e) {
                         const int64_t x = xd + rt->E[e][2];
-                        const int64_t xe = (OBJ == MMEE_OBJ_EDP) ? xed + rt->E[e][3] : 0;
+                        const int64_t xe = (OBJ >= MMEE_OBJ_EDP) ? xed + rt->E[e][3] : 0;
                         int64_t key[9];
 #pragma unroll
-                        for (int s = 0; s < 9; ++s) key[s] = candidate_key<OBJ>(x, xe, W[s], P[s / 3], Q[s]);
+                        for (int s = 0; s < 9; ++s) key[s] = candidate_key<OBJ>(x, xe, W[s], P[s / 3], Q[s], p.key_cap);
                         unsigned fit, hit;
                         row_test(key, thr, rt->E[e][0], s1, rt->E[e][1], s2, fit, hit);
                         fits += fit;
@@ -802,19 +808,19 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                     const int64_t s1 = slack1 - rt->D[d][0];
                     const int64_t s2 = slack2 - rt->D[d][1];
                     const int64_t xd = x0 + rt->D[d][2];
-                    const int64_t xed = (OBJ == MMEE_OBJ_EDP) ? xe0 + rt->D[d][3] : 0;
+                    const int64_t xed = (OBJ >= MMEE_OBJ_EDP) ? xe0 + rt->D[d][3] : 0;
 #pragma unroll 1
                     for (int e = 0; e < 5; ++e) {
                         const bool fit = (rt->E[e][0] <= s1) && (rt->E[e][1] <= s2) && ((kept >> (d * 5 + e)) & 1u);
                         const int64_t x = xd + rt->E[e][2];
-                        const int64_t xe = (OBJ == MMEE_OBJ_EDP) ? xed + rt->E[e][3] : 0;
+                        const int64_t xe = (OBJ >= MMEE_OBJ_EDP) ? xed + rt->E[e][3] : 0;
                         const uint64_t row_first_idx = mid_first_idx + (uint64_t)((d * 5 + e) * 9);
                         const int64_t thr_row = lane_threshold(wt, cs, k, row_first_idx);
                         bool below = false;
                         for (int s = 0; s < 9; ++s)
-                            below |= candidate_key<OBJ>(x, xe, wptr[2 * s], P[s / 3], qptr[2 * s]) < thr_row;
+                            below |= candidate_key<OBJ>(x, xe, wptr[2 * s], P[s / 3], qptr[2 * s], p.key_cap) < thr_row;
                         if (__any_sync(kFull, fit && below))
-                            slow_row<OBJ>(wt, cs, &scratch->G, k, lane, fit, x, xe, wptr, qptr, P[0], P[1], P[2],
+                            slow_row<OBJ>(wt, cs, &scratch->G, k, lane, fit, x, xe, wptr, qptr, P[0], P[1], P[2], p.key_cap,
                                           row_first_idx);
                     }
                     load_threshold();
@@ -952,7 +958,9 @@ cudaError_t search_occupancy(const Plan& p, size_t smem, int* blocks_per_sm) {
     switch (p.objective) {
         case MMEE_OBJ_ENERGY: return occupancy_t<MMEE_OBJ_ENERGY, kModeSearch>(blocks_per_sm, smem);
         case MMEE_OBJ_LATENCY: return occupancy_t<MMEE_OBJ_LATENCY, kModeSearch>(blocks_per_sm, smem);
-        default: return occupancy_t<MMEE_OBJ_EDP, kModeSearch>(blocks_per_sm, smem);
+        case MMEE_OBJ_EDP: return occupancy_t<MMEE_OBJ_EDP, kModeSearch>(blocks_per_sm, smem);
+        case MMEE_OBJ_ENERGY_LCAP: return occupancy_t<MMEE_OBJ_ENERGY_LCAP, kModeSearch>(blocks_per_sm, smem);
+        default: return occupancy_t<MMEE_OBJ_LATENCY_ECAP, kModeSearch>(blocks_per_sm, smem);
     }
 }
 
@@ -961,20 +969,26 @@ cudaError_t launch_search(const Plan& p, const LaunchShape& shape, Scratch* scra
         switch (p.objective) {
             case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, kModeDump>(p, shape, scratch, dump, st);
             case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, kModeDump>(p, shape, scratch, dump, st);
-            default: return launch_search_t<MMEE_OBJ_EDP, kModeDump>(p, shape, scratch, dump, st);
+            case MMEE_OBJ_EDP: return launch_search_t<MMEE_OBJ_EDP, kModeDump>(p, shape, scratch, dump, st);
+            case MMEE_OBJ_ENERGY_LCAP: return launch_search_t<MMEE_OBJ_ENERGY_LCAP, kModeDump>(p, shape, scratch, dump, st);
+            default: return launch_search_t<MMEE_OBJ_LATENCY_ECAP, kModeDump>(p, shape, scratch, dump, st);
         }
     }
     if (shape.pruned) {
         switch (p.objective) {
             case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, kModePrune>(p, shape, scratch, nullptr, st);
             case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, kModePrune>(p, shape, scratch, nullptr, st);
-            default: return launch_search_t<MMEE_OBJ_EDP, kModePrune>(p, shape, scratch, nullptr, st);
+            case MMEE_OBJ_EDP: return launch_search_t<MMEE_OBJ_EDP, kModePrune>(p, shape, scratch, nullptr, st);
+            case MMEE_OBJ_ENERGY_LCAP: return launch_search_t<MMEE_OBJ_ENERGY_LCAP, kModePrune>(p, shape, scratch, nullptr, st);
+            default: return launch_search_t<MMEE_OBJ_LATENCY_ECAP, kModePrune>(p, shape, scratch, nullptr, st);
         }
     }
     switch (p.objective) {
         case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, kModeSearch>(p, shape, scratch, nullptr, st);
         case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, kModeSearch>(p, shape, scratch, nullptr, st);
-        default: return launch_search_t<MMEE_OBJ_EDP, kModeSearch>(p, shape, scratch, nullptr, st);
+        case MMEE_OBJ_EDP: return launch_search_t<MMEE_OBJ_EDP, kModeSearch>(p, shape, scratch, nullptr, st);
+        case MMEE_OBJ_ENERGY_LCAP: return launch_search_t<MMEE_OBJ_ENERGY_LCAP, kModeSearch>(p, shape, scratch, nullptr, st);
+        default: return launch_search_t<MMEE_OBJ_LATENCY_ECAP, kModeSearch>(p, shape, scratch, nullptr, st);
     }
 }
 

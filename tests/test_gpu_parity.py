@@ -351,3 +351,59 @@ def test_dram_traffic_against_buffer_size_is_a_staircase():
         if last is not None:
             assert o.n[0] <= last
         last = o.n[0]
+
+
+def _all_keys(cfg, base_obj, limit):
+    """(e_key, l_key, feasible, idx) of every candidate of the (possibly range-limited) problem."""
+    oe = shrink(cfg, dict(base_obj, objective=mi.OBJ_ENERGY, topk=1), limit)
+    ol = dict(oe, objective=mi.OBJ_LATENCY)
+    pe = oracle.make_problem(cfg["workload"], cfg["arch"], oe)
+    pl = oracle.make_problem(cfg["workload"], cfg["arch"], ol)
+    begin, count = pe.t_begin * pe.R * 9, (pe.t_end - pe.t_begin) * pe.R * 9
+    ek, feas = oracle.keys_range(pe, begin, count)
+    lk, _ = oracle.keys_range(pl, begin, count)
+    return oe, ek, lk, feas.astype(bool), np.arange(begin, begin + count, dtype=np.int64)
+
+
+def _brute_force_front(ek, lk, feas, idx):
+    order = np.lexsort((idx[feas], lk[feas], ek[feas]))
+    e, l, i = ek[feas][order], lk[feas][order], idx[feas][order]
+    front, best_l = [], None
+    for a, b, c in zip(e, l, i):
+        if best_l is None or b < best_l:
+            front.append((int(a), int(b), int(c)))
+            best_l = b
+    return front
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3, 5, 7, 9])
+def test_energy_latency_pareto_front(seed):
+    """The front of Section VII-E by alternating capped searches, against a brute-force sweep over
+    every candidate's (energy, latency) pair from the oracle; each point with its lowest index."""
+    cfg = mi.random_tiny_problem(seed)
+    base = dict(cfg["searches"][0], row_pruning=0)
+    obj, ek, lk, feas, idx = _all_keys(cfg, base, 3_000_000)
+    want = _brute_force_front(ek, lk, feas, idx)
+    got = mm.mmee_pareto_front(cfg["workload"], cfg["arch"], obj)
+    assert [(r.e_key, r.l_key, r.idx) for r in got] == want
+    p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
+    for r in got:
+        assert_same_record(r, oracle.evaluate(p, r.idx), "front point %d" % r.idx)
+
+
+def test_capped_searches_match_brute_force():
+    cfg = mi.random_tiny_problem(4)
+    obj, ek, lk, feas, idx = _all_keys(cfg, cfg["searches"][0], 3_000_000)
+    for cap_q in (0.1, 0.5, 0.9):
+        lcap = int(np.quantile(lk[feas], cap_q))
+        ok = feas & (lk <= lcap)
+        order = np.lexsort((idx[ok], ek[ok]))
+        best, _, _ = gpu_search(cfg, dict(obj, objective=mi.OBJ_ENERGY_LCAP, key_cap=lcap))
+        assert (best.e_key, best.idx) == (int(ek[ok][order[0]]), int(idx[ok][order[0]])) and best.l_key <= lcap
+        ecap = int(np.quantile(ek[feas], cap_q))
+        ok = feas & (ek <= ecap)
+        order = np.lexsort((idx[ok], lk[ok]))
+        best, _, _ = gpu_search(cfg, dict(obj, objective=mi.OBJ_LATENCY_ECAP, key_cap=ecap))
+        assert (best.l_key, best.idx) == (int(lk[ok][order[0]]), int(idx[ok][order[0]])) and best.e_key <= ecap
+    best, _, _ = gpu_search(cfg, dict(obj, objective=mi.OBJ_ENERGY_LCAP, key_cap=int(lk[feas].min()) - 1))
+    assert best.idx == mm.NO_INDEX and best.status == mm.ERR_NO_FEASIBLE
