@@ -1,19 +1,21 @@
 // The search kernels: exhaustive evaluation of every mapping, capacity pruning, top-k.
 //
-// Work decomposition.  A "task" is one (tiling, fusion mode, order, levels of A, B, C) choice; its
-// 25 rows are the levels of D and E and each row has 9 stationary pairs, so a task is 225
-// consecutive candidate indices: idx = task*225 + row*9 + s.  One thread owns one task at a time
-// and walks it in ascending index order.
+// Work decomposition.  A "task" is one (tiling, fusion mode, order, levels of A and B) choice: 1125
+// consecutive candidate indices, idx = task*1125 + mid*225 + row*9 + s, where mid is the level of C
+// (of B for an unfused task), the 25 rows are the levels of D and E and s is the stationary pair.
+// One thread owns one task at a time and walks it in ascending index order.
 //
 // The cost of a mapping is separable over operands (Section V-B/V-C: BS and DA are sums of
 // per-operand monomials; Section V-D: energy is linear in the access counts), so the query-matrix
 // product exp(Q . ln B) (Eq. 11) is evaluated once per (tiling, order, operand, level) into small
 // shared-memory tables -- each entry an exact integer monomial already multiplied by its energy
-// coefficient -- and a candidate's key is a handful of adds of table entries.  Nothing per
-// candidate ever touches global memory.
+// coefficient -- and a candidate's key is a short sum of table entries.  The row loop evaluates
+// every candidate's key relative to the current top-k threshold in saturated 32-bit arithmetic
+// (one fused add-min per candidate for energy); exact 64-bit keys are formed only for rows that
+// can enter the list.  Nothing per candidate ever touches global memory.
 //
-// CTAs are persistent and pull ranges of tasks from a global counter; per range they rebuild the
-// tables of the (at most a few) tilings the range touches.
+// CTAs are persistent and pull ranges of tasks from a global counter.  Seven warps walk tasks while
+// the eighth builds the tables of the next range into a second buffer.
 #include <cuda_runtime.h>
 
 #include <climits>
