@@ -67,6 +67,7 @@ struct alignas(16) OrderTab {
 // Per tiling: array-level terms by stationary pair and recompute flag.
 struct alignas(16) TilingTab {
     uint32_t b[8];
+    int64_t half[2][16];    // products of every subset of the four x_D bounds / of the four x_G bounds
     int32_t Wc[2][12];      // W[s][rc] - wmin[rc], saturated to kTermCap (entries 9..11 unused)
     int64_t W[9][2];        // energy of buffer<->PE traffic, MACs and softmax, in quanta
     int64_t CB[9][2];       // fused compute time in words (cycles * words per cycle)
@@ -319,15 +320,18 @@ __device__ __forceinline__ void fill_dead_tiling_item(struct TilingTab* tb, int 
 
 // One thread per (tiling slot, order, item): the monomials of one operand at one level.
 template <int OBJ>
-__device__ __forceinline__ void build_order_item(const Plan& p, const uint32_t* b, uint32_t order, OrderTab* ot, int item) {
+__device__ __forceinline__ void build_order_item(const Plan& p, const TilingTab* tb, uint32_t order, OrderTab* ot, int item) {
     const QueryTables& q = p.q;
+    // exp(q . ln b) (Eq. 8) as the product of two subset products: bits 0-3 of a query vector select
+    // x_D bounds, bits 4-7 x_G bounds
+    auto monomial = [tb](uint32_t qv) { return tb->half[0][qv & 15u] * tb->half[1][qv >> 4]; };
     const int64_t scale = (OBJ == MMEE_OBJ_ENERGY) ? p.c_dram_gb : 1;
     const int64_t escale = p.c_dram_gb;
     const int l = item % 5;
     if (item < 10) {                                   // A, B
         const int x = item < 5 ? OP_A : OP_B;
-        const int64_t bs = monomial(q.bs[order][x][l], b);
-        const int64_t v0 = monomial(q.da[order][x][l][0], b), v1 = monomial(q.da[order][x][l][1], b);
+        const int64_t bs = monomial(q.bs[order][x][l]);
+        const int64_t v0 = monomial(q.da[order][x][l][0]), v1 = monomial(q.da[order][x][l][1]);
         int64_t* s1 = x == OP_A ? ot->A1 : ot->B1;
         int64_t* s2 = x == OP_A ? ot->A2 : ot->B2;
         int64_t (*g)[2] = x == OP_A ? ot->gA : ot->gB;
@@ -338,13 +342,13 @@ __device__ __forceinline__ void build_order_item(const Plan& p, const uint32_t* 
         g[l][1] = scale * v1;
         if (OBJ >= MMEE_OBJ_EDP) { e[l][0] = escale * v0; e[l][1] = escale * v1; }
     } else if (item < 15) {                            // C
-        ot->C1[l] = monomial(q.bs[order][OP_C][l], b);
+        ot->C1[l] = monomial(q.bs[order][OP_C][l]);
         ot->rc[l] = q.recompute[order][l];
     } else if (item < 25) {                            // D, E
         const int x = item < 20 ? OP_D : OP_E;
-        const int64_t bs = monomial(q.bs[order][x][l], b);
-        const int64_t vf = monomial(q.da[order][x][l][0], b);
-        const int64_t vu = monomial(q.da_unfused[order][x][l], b);
+        const int64_t bs = monomial(q.bs[order][x][l]);
+        const int64_t vf = monomial(q.da[order][x][l][0]);
+        const int64_t vu = monomial(q.da_unfused[order][x][l]);
         RowTab* f = &ot->rt[0];
         RowTab* u = &ot->rt[1];
         int64_t* fr = x == OP_D ? f->D[l] : f->E[l];
@@ -365,7 +369,7 @@ __device__ __forceinline__ void build_order_item(const Plan& p, const uint32_t* 
         fc[3] = 0;
         uc[3] = 0;
     } else {
-        const int64_t v = monomial(q.da_unfused[order][OP_C][0], b);
+        const int64_t v = monomial(q.da_unfused[order][OP_C][0]);
         ot->gCr = scale * v;
         ot->eCr = escale * v;
     }
@@ -475,6 +479,17 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
         OrderTab* otabs = otabs_all + (size_t)buf * shape.slots * n_orders;
         for (uint32_t sl = lane; sl < n_slots; sl += 32) build_tiling_head(p, t_first + sl, &ttabs[sl]);
         __syncwarp();
+        // subset products of the bounds: one lane per (slot, half, subset)
+        for (uint32_t it = lane; it < n_slots * 32u; it += 32) {
+            TilingTab* tb = &ttabs[it >> 5];
+            const uint32_t h = (it >> 4) & 1u, m = it & 15u;
+            int64_t v = 1;
+#pragma unroll
+            for (int d = 0; d < 4; ++d)
+                if (m >> d & 1u) v *= (int64_t)tb->b[h * 4 + d];
+            tb->half[h][m] = v;
+        }
+        __syncwarp();
         // Items are visited kind by kind, so that the 32 lanes always run the same code path.
         const uint32_t n_so = n_slots * n_orders;
         auto order_pass = [&](uint32_t first_item, uint32_t n_items) {
@@ -482,7 +497,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                 const uint32_t so = it / n_items, e = first_item + it % n_items;
                 const uint32_t slot = so / n_orders, os = so % n_orders;
                 if (!ttabs[slot].live) { fill_dead_order_item(&otabs[so], (int)e); continue; }
-                build_order_item<OBJ>(p, ttabs[slot].b, p.order_id[os], &otabs[so], (int)e);
+                build_order_item<OBJ>(p, &ttabs[slot], p.order_id[os], &otabs[so], (int)e);
             }
         };
         order_pass(0, 10);      // A, B
