@@ -407,3 +407,32 @@ def test_capped_searches_match_brute_force():
         assert (best.l_key, best.idx) == (int(lk[ok][order[0]]), int(idx[ok][order[0]])) and best.e_key <= ecap
     best, _, _ = gpu_search(cfg, dict(obj, objective=mi.OBJ_ENERGY_LCAP, key_cap=int(lk[feas].min()) - 1))
     assert best.idx == mm.NO_INDEX and best.status == mm.ERR_NO_FEASIBLE
+
+
+def test_largest_divisor_list_and_ragged_dims():
+    """A dimension with exactly the maximum number of divisors (7560 = 2^3 3^3 5 7 has 64), others
+    ragged: sub-range searches at both ends of the tiling space, all three objectives."""
+    cfg = dict(name="divisors64", workload=mi.workload(1, 1, 1, 7560, 30, 6, 6, 2),
+               arch=mi.arch(4, 8, 2, 8192, 64, 6, 120.0, 4.0, 1.0, 0.5, c_softmax=3.0, energy_quantum_pj=0.5))
+    base = mi.objective(mi.OBJ_ENERGY, 5)
+    p = oracle.make_problem(cfg["workload"], cfg["arch"], base)
+    assert list(p.ndiv) == [64, 4, 8, 4] and p.T == 8192
+    for objective, (lo, hi) in ((mi.OBJ_ENERGY, (0, 9)), (mi.OBJ_LATENCY, (4000, 4007)), (mi.OBJ_EDP, (8185, 8192))):
+        check_search(cfg, dict(base, objective=objective, t_begin=lo, t_end=hi))
+
+
+@pytest.mark.parametrize("seed", range(13, 41))
+def test_more_random_problems_keys_and_optimum(seed):
+    """Wider seed range: every candidate key through the search kernel's own path, and the top-5."""
+    cfg = mi.random_tiny_problem(seed)
+    obj = shrink(cfg, dict(cfg["searches"][0], topk=5), 1_500_000)
+    p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
+    begin, count = p.t_begin * p.R * 9, (p.t_end - p.t_begin) * p.R * 9
+    keys, feas = oracle.keys_range(p, begin, count)
+    want = np.where(feas.astype(bool), keys, np.iinfo(np.int64).max)
+    out = torch.full((count,), -7, dtype=torch.int64, device="cuda")
+    with Handle(cfg, obj) as h:
+        mm.mmee_dump_keys(h, out)
+        torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy(), want)
+    check_search(cfg, obj)
