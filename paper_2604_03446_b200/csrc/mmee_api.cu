@@ -43,7 +43,7 @@ int choose_shape(const Plan& p, int device, uint32_t search_tpt, LaunchShape* sh
     size_t smem = search_smem_bytes(p, shape->slots);
     // Many small tilings per range need many table slots: shrink the range until they fit.
     // (Worker warps take 32 tasks at a time, so a range may be as short as one warp's share.)
-    while (smem > 96 * 1024 && shape->range_tasks > 32) {
+    while (smem > 110 * 1024 && shape->range_tasks > 32) {
         shape->range_tasks -= shape->range_tasks > kWorkerThreads ? kWorkerThreads : 32;
         shape->slots = (shape->range_tasks - 1) / search_tpt + 2;
         smem = search_smem_bytes(p, shape->slots);

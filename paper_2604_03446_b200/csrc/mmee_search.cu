@@ -33,7 +33,7 @@ constexpr int kModeSearch = 0, kModeDump = 1, kModePrune = 2;
 constexpr size_t kPlanBytes = (sizeof(Plan) + 15) / 16 * 16;
 static_assert(sizeof(Plan) % 4 == 0, "the plan is copied word by word");
 constexpr int kRelCap = (1 << 30) - 1;     // cap of a running threshold-relative sum (see below)
-constexpr int kTermCap = 1 << 29;          // cap of each non-negative addend of such a sum
+constexpr int kTermCap = 1 << 28;          // cap of each non-negative addend of such a sum (at most six of them)
 constexpr int kSizeCap = (1 << 30) - 1;    // buffer sizes saturate here; the capacity is smaller
 
 // ------------------------------------------------------------------------------------------------
@@ -60,8 +60,16 @@ struct alignas(16) OrderTab {
     int64_t gCr, eCr;                             // unfused: C read back by Op2
     uint32_t rc[5];
     uint32_t pad;
+    // 32-bit forms for the threshold-relative walk: per level x1 = size, x2 = size if retained,
+    // g[recompute] = DRAM term in relative units; sizes saturated to kSizeCap, terms to kTermCap
+    int32_t Ac[5][4];
+    int32_t Bc[5][4];
+    int32_t Cc[5][2];                             // size, recompute flag
+    int32_t gXc[2];                               // energy: C round trip (+ softmax pass) of an unfused task, phi = 1, 2
     RowTab rt[2];                                 // 0 fused, 1 unfused
 };
+static_assert(offsetof(OrderTab, Ac) % 16 == 0 && offsetof(OrderTab, Bc) % 16 == 0 && offsetof(OrderTab, Cc) % 8 == 0,
+              "Ac / Bc rows are read as int4, Cc rows as int2");
 // 26 items per order: 5 levels each of A, B, C, D, E and the unfused C read-back
 
 // Per tiling: array-level terms by stationary pair and recompute flag.
@@ -75,10 +83,13 @@ struct alignas(16) TilingTab {
     int64_t C1w[3];         // unfused Op1 compute time in words, by sm1
     int64_t cw, smx;        // C write-back words (I*L); separate softmax pass words (2*I*L)
     int64_t wmin[2];        // min over the stationary pairs of W[.][rc]
+    int64_t qmin[3];        // min over the stationary pairs of CB[.][0], CB[.][1], QU[.][0]
+    int32_t Qrel[3][12];    // CB[s][0], CB[s][1], QU[s][0] minus that minimum, saturated to kTermCap
     int32_t live;           // smallest possible buffer need of this tiling fits
     int32_t pad[3];
 };
-static_assert(offsetof(TilingTab, Wc) % 16 == 0 && sizeof(int32_t[12]) % 16 == 0, "Wc rows are read as int4");
+static_assert(offsetof(TilingTab, Wc) % 16 == 0 && offsetof(TilingTab, Qrel) % 16 == 0 && sizeof(int32_t[12]) % 16 == 0,
+              "Wc and Qrel rows are read as int4");
 static_assert(offsetof(RowTab, Ec) % 16 == 0 && offsetof(OrderTab, rt) % 16 == 0 && sizeof(RowTab) % 16 == 0,
               "Ec rows are read as int4");
 // 21 items per tiling: 9 stationary pairs x 2 recompute flags, 3 unfused Op1 terms
@@ -301,9 +312,12 @@ __device__ __forceinline__ void fill_dead_order_item(OrderTab* ot, int item) {
         int64_t (*e)[2] = item < 5 ? ot->eA : ot->eB;
         s1[l] = s2[l] = 0;
         g[l][0] = g[l][1] = e[l][0] = e[l][1] = 0;
+        int32_t* c = item < 5 ? ot->Ac[l] : ot->Bc[l];
+        c[0] = c[1] = kSizeCap; c[2] = c[3] = 0;
     } else if (item < 15) {
         ot->C1[l] = 0;
         ot->rc[l] = 0;
+        ot->Cc[l][0] = kSizeCap; ot->Cc[l][1] = 0;
     } else if (item < 25) {
         for (int v = 0; v < 2; ++v) {
             int64_t* r = item < 20 ? ot->rt[v].D[l] : ot->rt[v].E[l];
@@ -313,6 +327,7 @@ __device__ __forceinline__ void fill_dead_order_item(OrderTab* ot, int item) {
         }
     } else {
         ot->gCr = ot->eCr = 0;
+        ot->gXc[0] = ot->gXc[1] = 0;
     }
 }
 
@@ -328,6 +343,10 @@ __device__ __forceinline__ void build_order_item(const Plan& p, const TilingTab*
     const int64_t scale = (OBJ == MMEE_OBJ_ENERGY) ? p.c_dram_gb : 1;
     const int64_t escale = p.c_dram_gb;
     const int l = item % 5;
+    // 32-bit forms: a size saturates at kSizeCap (above every admissible capacity); a DRAM term is kept in
+    // units of 2^rel_shift, rounded down, and saturates at kTermCap
+    auto size32 = [](int64_t v) { return (int32_t)(v < (int64_t)kSizeCap ? v : (int64_t)kSizeCap); };
+    auto term32 = [&p](int64_t v) { const int64_t u = v >> p.rel_shift; return (int32_t)(u < (int64_t)kTermCap ? u : (int64_t)kTermCap); };
     if (item < 10) {                                   // A, B
         const int x = item < 5 ? OP_A : OP_B;
         const int64_t bs = monomial(q.bs[order][x][l]);
@@ -341,9 +360,17 @@ __device__ __forceinline__ void build_order_item(const Plan& p, const TilingTab*
         g[l][0] = scale * v0;
         g[l][1] = scale * v1;
         if (OBJ >= MMEE_OBJ_EDP) { e[l][0] = escale * v0; e[l][1] = escale * v1; }
+        int32_t* c = x == OP_A ? ot->Ac[l] : ot->Bc[l];
+        c[0] = size32(bs);
+        c[1] = l ? size32(bs) : 0;
+        c[2] = term32(scale * v0);
+        c[3] = term32(scale * v1);
     } else if (item < 15) {                            // C
-        ot->C1[l] = monomial(q.bs[order][OP_C][l]);
+        const int64_t bs = monomial(q.bs[order][OP_C][l]);
+        ot->C1[l] = bs;
         ot->rc[l] = q.recompute[order][l];
+        ot->Cc[l][0] = size32(bs);
+        ot->Cc[l][1] = (int32_t)q.recompute[order][l];
     } else if (item < 25) {                            // D, E
         const int x = item < 20 ? OP_D : OP_E;
         const int64_t bs = monomial(q.bs[order][x][l]);
@@ -372,6 +399,9 @@ __device__ __forceinline__ void build_order_item(const Plan& p, const TilingTab*
         const int64_t v = monomial(q.da_unfused[order][OP_C][0]);
         ot->gCr = scale * v;
         ot->eCr = escale * v;
+        // energy of an unfused task's C round trip: read-back, write, and the separate softmax pass of phi = 2
+        ot->gXc[0] = term32(p.c_dram_gb * (v + tb->cw));
+        ot->gXc[1] = term32(p.c_dram_gb * (v + tb->cw + tb->smx));
     }
 }
 
@@ -418,6 +448,401 @@ __device__ __forceinline__ void fill_dead_tiling_item(TilingTab* tb, int item) {
 }
 
 // ------------------------------------------------------------------------------------------------
+// walking one task
+// ------------------------------------------------------------------------------------------------
+
+// Threshold of one lane: a key passes iff key < T1; for candidates whose index lies above `ti`,
+// the index of the list's last entry, the threshold is T1 - delta (a tie could not displace it).
+struct LaneThreshold {
+    int64_t T1;
+    uint64_t ti;
+    int delta;
+};
+
+__device__ __forceinline__ LaneThreshold load_threshold(const WarpTop* wt, const CtaShared* cs, int k) {
+    LaneThreshold t;
+    const int64_t g1 = cs->G + 1;                 // G <= INT64_MAX - 1 always
+    t.T1 = g1; t.ti = UINT64_MAX; t.delta = 0;
+    if (wt->count == k) {
+        const int64_t tk1 = wt->key[k - 1] + 1;
+        if (tk1 <= g1) { t.T1 = tk1; t.delta = 1; t.ti = wt->idx[k - 1]; }
+    }
+    return t;
+}
+
+// Exact 64-bit terms of one (task, middle level): the middle level m is the level of C for a fused
+// task and of B for an unfused one.
+struct MidExact {
+    int64_t slack1, slack2;     // capacity left for the D and E terms in Op1's / Op2's buffer need (Eq. 1, 2)
+    int64_t x0, xe0;            // task-level part of the row sum: the objective's primary side / the energy side
+    int64_t P[3];               // unfused latency: Op1 stage and softmax pass, by sm1
+    const int64_t* wptr;        // W[s][rc], stride 2
+    const int64_t* qptr;        // compute words by s, stride 2
+};
+
+template <int OBJ>
+__device__ __forceinline__ MidExact mid_exact(const Plan& p, const TilingTab* tb, const OrderTab* ot, uint32_t phi,
+                                              uint32_t la, uint32_t lb_task, int m, bool live) {
+    MidExact r;
+    const bool fused = phi == 0;
+    const uint32_t lb = fused ? lb_task : (uint32_t)m;
+    const uint32_t lc = fused ? (uint32_t)m : 0u;
+    // Tables of a tiling that cannot fit are filled with constants: a lane whose task lies in such
+    // a tiling must not index with what it reads from them.
+    const uint32_t rc = (fused && live) ? (ot->rc[lc] & 1u) : 0u;
+    const int64_t a1 = ot->A1[la], b1 = ot->B1[lb], c1 = ot->C1[lc];
+    const int64_t a2 = fused ? ot->A2[la] : 0, b2 = fused ? ot->B2[lb] : 0;
+    // Eq. (1)/(2): a retained operand (level >= L4) of the other operator keeps its space.
+    // A lane without a live task gets a negative slack, so that none of its rows fits.
+    r.slack1 = live ? p.cap_words - (a1 + b1 + c1) : -1;
+    r.slack2 = live ? p.cap_words - (c1 + a2 + b2) : -1;
+    const int64_t gab = ot->gA[la][rc] + ot->gB[lb][rc];
+    r.wptr = &tb->W[0][rc];
+    r.xe0 = 0;
+    if constexpr (OBJ == MMEE_OBJ_ENERGY) {
+        const int64_t extra = p.c_dram_gb * (tb->cw + (phi == 2 ? tb->smx : 0));
+        r.x0 = fused ? gab : gab + ot->gCr + extra;
+        r.P[0] = r.P[1] = r.P[2] = 0;
+        r.qptr = r.wptr;
+    } else {
+        const int64_t pass = (phi == 2) ? tb->smx : 0;
+        if (fused) {
+            r.x0 = gab;
+            r.P[0] = r.P[1] = r.P[2] = 0;
+            r.qptr = &tb->CB[0][rc];
+        } else {
+            // unfused latency: max(DA1, C1) + softmax pass + max(DA2, C2)
+            r.x0 = ot->gCr;
+            const int64_t da1 = gab + tb->cw;
+#pragma unroll
+            for (int j = 0; j < 3; ++j) r.P[j] = (da1 > tb->C1w[j] ? da1 : tb->C1w[j]) + pass;
+            r.qptr = &tb->QU[0][0];
+        }
+        if constexpr (OBJ >= MMEE_OBJ_EDP) {
+            const int64_t eab = ot->eA[la][rc] + ot->eB[lb][rc];
+            r.xe0 = fused ? eab : eab + ot->eCr + p.c_dram_gb * (tb->cw + pass);
+        }
+    }
+    return r;
+}
+
+// Rare path: the filter flagged group d (five rows, the levels of E) of middle level m for some lane.
+// Every lane finds its rows that hold a passing candidate, exactly, and the warp inserts them.
+template <int OBJ>
+__device__ __noinline__ void exact_group(const Plan& p, const TilingTab* tb, const OrderTab* ot, uint32_t phi, uint32_t la,
+                                         uint32_t lb_task, int m, int d, bool live, uint32_t kept,
+                                         uint64_t task_first_idx, WarpTop* wt, CtaShared* cs, long long* global_g, int k,
+                                         int lane) {
+    const MidExact me = mid_exact<OBJ>(p, tb, ot, phi, la, lb_task, m, live);
+    const RowTab* rt = &ot->rt[phi == 0 ? 0 : 1];
+    const int64_t s1 = me.slack1 - rt->D[d][0];
+    const int64_t s2 = me.slack2 - rt->D[d][1];
+    const int64_t xd = me.x0 + rt->D[d][2];
+    const int64_t xed = (OBJ >= MMEE_OBJ_EDP) ? me.xe0 + rt->D[d][3] : 0;
+#pragma unroll 1
+    for (int e = 0; e < 5; ++e) {
+        const bool fit = (rt->E[e][0] <= s1) && (rt->E[e][1] <= s2) && ((kept >> (d * 5 + e)) & 1u);
+        const int64_t x = xd + rt->E[e][2];
+        const int64_t xe = (OBJ >= MMEE_OBJ_EDP) ? xed + rt->E[e][3] : 0;
+        const uint64_t row_first_idx = task_first_idx + (uint64_t)(m * 225 + (d * 5 + e) * 9);
+        const int64_t thr_row = lane_threshold(wt, cs, k, row_first_idx);
+        bool below = false;
+        for (int s = 0; s < 9; ++s)
+            below |= candidate_key<OBJ>(x, xe, me.wptr[2 * s], me.P[s / 3], me.qptr[2 * s], p.key_cap) < thr_row;
+        if (__any_sync(kFull, fit && below))
+            slow_row<OBJ>(wt, cs, global_g, k, lane, fit, x, xe, me.wptr, me.qptr, me.P[0], me.P[1], me.P[2], p.key_cap,
+                          row_first_idx);
+    }
+}
+
+// The walk in 64-bit keys: the energy-delay product (double-precision filter, see edp_row_test),
+// the capped objectives and the key dump.  Returns the number of rows that fit.
+template <int OBJ, bool DUMP, bool PRUNE>
+__device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingTab* tb, const OrderTab* ot,
+                                                    const TaskChoice& c, bool live, bool valid, uint32_t kept,
+                                                    uint32_t kept_mid, uint64_t task_first_idx, WarpTop* wt,
+                                                    CtaShared* cs, long long* global_g, int k, int lane,
+                                                    int64_t* __restrict__ dump, uint64_t dump_origin) {
+    const RowTab* rt = &ot->rt[c.phi == 0 ? 0 : 1];
+    LaneThreshold th = load_threshold(wt, cs, k);
+    uint32_t rows = 0;
+    int E1c[5], E2c[5];
+#pragma unroll
+    for (int e = 0; e < 5; ++e) {
+        const int4 v = *reinterpret_cast<const int4*>(rt->Ec[e]);
+        E1c[e] = v.x; E2c[e] = v.y;
+    }
+#pragma unroll 1
+    for (int mi = 0; mi < (PRUNE ? 1 : 5); ++mi) {
+        const int m = PRUNE ? (int)kept_mid : mi;
+        const uint64_t mid_first_idx = task_first_idx + (uint64_t)(m * 225);
+        const MidExact me = mid_exact<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, live);
+        int64_t W[9], Q[9];
+#pragma unroll
+        for (int s = 0; s < 9; ++s) {
+            W[s] = me.wptr[2 * s];
+            Q[s] = me.qptr[2 * s];
+        }
+        double dW[9], dQP[9], dthr = 0.0;
+        if constexpr (OBJ == MMEE_OBJ_EDP) {
+#pragma unroll
+            for (int s = 0; s < 9; ++s) {
+                dW[s] = (double)W[s];
+                dQP[s] = (double)(Q[s] + me.P[s / 3]);
+            }
+        }
+        auto refresh = [&]() {
+            if constexpr (OBJ == MMEE_OBJ_EDP) {
+                // EDP keys are bit patterns of positive doubles; anything from +inf up means "no bound yet"
+                dthr = th.T1 >= 0x7ff0000000000000ll ? __longlong_as_double(0x7ff0000000000000ll)
+                                                    : __longlong_as_double(th.T1) * (1.0 + 1e-14);
+            }
+        };
+        refresh();
+        const int slack1c = me.slack1 < 0 ? -1 : (int)me.slack1;      // slack <= capacity < 2^30
+        const int slack2c = me.slack2 < 0 ? -1 : (int)me.slack2;
+
+#pragma unroll 1
+        for (int d = 0; d < 5; ++d) {
+            if constexpr (PRUNE) {
+                if (!__any_sync(kFull, live && ((kept >> (d * 5)) & 31u))) continue;
+            }
+            unsigned hit_any = 0, fits = 0;
+            if constexpr (!DUMP && OBJ == MMEE_OBJ_EDP) {
+                // The energy-delay product is not separable, so the filter is a double-precision
+                // evaluation of every mapping on the FP64 pipe: energy and latency sums converted
+                // once per row, then an add, two multiplies and two compares per mapping.  Each
+                // approximate product is within a few 2^-53 of the exact key, so comparing against
+                // the threshold widened by 1e-14 relative can flag a row needlessly but never miss
+                // one; the exact path decides.
+                const int4 dc = *reinterpret_cast<const int4*>(rt->Dc[d]);
+                const int s1c = slack1c - dc.x;
+                const int s2c = slack2c - dc.y;
+                const int64_t xd = me.x0 + rt->D[d][2];
+                const int64_t xed = me.xe0 + rt->D[d][3];
+#pragma unroll
+                for (int e = 0; e < 5; ++e) {
+                    unsigned fit = (unsigned)(E1c[e] <= s1c) & (unsigned)(E2c[e] <= s2c);             // Eq. (4)
+                    if constexpr (PRUNE) fit &= kept >> (d * 5 + e);
+                    fits += fit;
+                    const int64_t x = xd + rt->E[e][2];
+                    const double de = (double)(xed + rt->E[e][3]);
+                    double dl[3];
+#pragma unroll
+                    for (int j = 0; j < 3; ++j) dl[j] = (double)(x + me.P[j]);
+                    hit_any |= edp_row_test(de, dl, dW, dQP, dthr, fit);
+                }
+            } else {
+                const int64_t s1 = me.slack1 - rt->D[d][0];
+                const int64_t s2 = me.slack2 - rt->D[d][1];
+                const int64_t xd = me.x0 + rt->D[d][2];
+                const int64_t xed = (OBJ >= MMEE_OBJ_EDP) ? me.xe0 + rt->D[d][3] : 0;
+                const uint64_t group_first_idx = mid_first_idx + (uint64_t)(d * 45);
+                const int64_t thr = th.T1 - (group_first_idx > th.ti ? th.delta : 0);
+#pragma unroll
+                for (int e = 0; e < 5; ++e) {
+                    const int64_t x = xd + rt->E[e][2];
+                    const int64_t xe = (OBJ >= MMEE_OBJ_EDP) ? xed + rt->E[e][3] : 0;
+                    int64_t key[9];
+#pragma unroll
+                    for (int s = 0; s < 9; ++s) key[s] = candidate_key<OBJ>(x, xe, W[s], me.P[s / 3], Q[s], p.key_cap);
+                    unsigned fit, hit;
+                    row_test(key, thr, rt->E[e][0], s1, rt->E[e][1], s2, fit, hit);
+                    if constexpr (PRUNE) { fit &= kept >> (d * 5 + e); hit &= fit; }
+                    fits += fit;
+                    hit_any |= hit;
+                    if (DUMP) {
+                        if (valid) {
+#pragma unroll
+                            for (int s = 0; s < 9; ++s)
+                                dump[mid_first_idx - dump_origin + (d * 5 + e) * 9 + s] = fit ? key[s] : kInfKey;
+                        }
+                    }
+                }
+            }
+            rows += fits;
+            if (__any_sync(kFull, hit_any != 0u)) {
+                exact_group<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, k, lane);
+                th = load_threshold(wt, cs, k);
+                refresh();
+            }
+        }
+    }
+    return rows;
+}
+
+// The walk in 32-bit threshold-relative keys (see "32-bit differential keys"): energy and latency
+// objectives.  Everything a middle level, a group or a row needs is a 32-bit table entry or a
+// register; 64-bit arithmetic is left to the places where the threshold enters (once per task and
+// after each visit of the exact path).  Returns the number of rows that fit.
+template <int OBJ, bool PRUNE>
+__device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const TilingTab* tb, const OrderTab* ot,
+                                                       const TaskChoice& c, bool live, uint32_t kept, uint32_t kept_mid,
+                                                       uint64_t task_first_idx, WarpTop* wt, CtaShared* cs,
+                                                       long long* global_g, int k, int lane) {
+    const bool fused = c.phi == 0;
+    const RowTab* rt = &ot->rt[fused ? 0 : 1];
+    int E1c[5], E2c[5], Gc[5];
+#pragma unroll
+    for (int e = 0; e < 5; ++e) {
+        const int4 v = *reinterpret_cast<const int4*>(rt->Ec[e]);
+        E1c[e] = v.x; E2c[e] = v.y; Gc[e] = v.z;
+    }
+    const int4 av = *reinterpret_cast<const int4*>(ot->Ac[c.la]);
+    const int a1c = av.x, a2c = fused ? av.y : 0;
+    const int capc = (int)p.cap_words;
+    const int gxc = (OBJ == MMEE_OBJ_ENERGY && !fused) ? ot->gXc[c.phi == 2 ? 1 : 0] : 0;
+    auto rel32 = [](int64_t v) { const int r = sat_s32(v); return r < kRelCap ? r : kRelCap; };
+
+    // Threshold state.  Energy: base[rc] = (terms of A and of the C round trip) - ceil((T1 - wmin[rc]) / 2^rel_shift).
+    // Latency, fused task: ua2[rc] = DRAM words of A and B - T1, qo2[rc] = least compute words - T1.
+    int base[2] = {0, 0}, ua2[2] = {0, 0}, qo2[2] = {0, 0};
+    int64_t T1 = 0;
+    int delta = 0, strict_from = INT_MAX;
+    auto rebase = [&]() {
+        const LaneThreshold th = load_threshold(wt, cs, k);
+        T1 = th.T1;
+        delta = th.delta;
+        // first candidate of the task, by position, whose index lies above the list's last entry
+        strict_from = th.ti < task_first_idx ? 0
+                      : (th.ti - task_first_idx >= (uint64_t)kCandPerTask ? INT_MAX : (int)(th.ti - task_first_idx) + 1);
+        if constexpr (OBJ == MMEE_OBJ_ENERGY) {
+#pragma unroll
+            for (int rc = 0; rc < 2; ++rc) {
+                const int64_t bs = ((T1 - tb->wmin[rc] - 1) >> p.rel_shift) + 1;      // ceiling of the quotient
+                const int64_t bl = bs > (int64_t)INT_MAX ? (int64_t)INT_MAX : (bs < -(int64_t)kTermCap ? -(int64_t)kTermCap : bs);
+                const int t = (rc ? av.w : av.z) + gxc - (int)bl;
+                base[rc] = t < kRelCap ? t : kRelCap;
+            }
+        } else {
+            if (fused) {
+#pragma unroll
+                for (int rc = 0; rc < 2; ++rc) {
+                    ua2[rc] = rel32(ot->gA[c.la][rc] + ot->gB[c.lb][rc] - T1);
+                    qo2[rc] = rel32(tb->qmin[rc] - T1);
+                }
+            }
+        }
+    };
+    rebase();
+
+    uint32_t rows = 0;
+#pragma unroll 1
+    for (int mi = 0; mi < (PRUNE ? 1 : 5); ++mi) {
+        const int m = PRUNE ? (int)kept_mid : mi;
+        const int4 bv = *reinterpret_cast<const int4*>(ot->Bc[fused ? c.lb : (uint32_t)m]);
+        const int2 cv = *reinterpret_cast<const int2*>(ot->Cc[fused ? m : 0]);
+        // (a lane without a live task may read the constant tables of a tiling that cannot fit)
+        const uint32_t rc = (fused && live) ? ((uint32_t)cv.y & 1u) : 0u;
+        // Eq. (1)/(2) in saturated 32-bit sizes: a retained operand of the other operator keeps its space
+        int y1 = __viaddmin_s32(a1c, bv.x, kSizeCap);
+        y1 = __viaddmin_s32(y1, cv.x, kSizeCap);
+        int y2 = __viaddmin_s32(a2c, fused ? bv.y : 0, kSizeCap);
+        y2 = __viaddmin_s32(y2, cv.x, kSizeCap);
+        const int slack1c = live ? capc - y1 : -1;       // a lane without a live task: none of its rows fits
+        const int slack2c = live ? capc - y2 : -1;
+
+        int u = 0, Wc[9], ua[3], Qc[9];
+        if constexpr (OBJ == MMEE_OBJ_ENERGY) {
+            const int4* wc4 = reinterpret_cast<const int4*>(tb->Wc[rc]);
+            const int4 w0 = wc4[0], w1 = wc4[1], w2 = wc4[2];
+            Wc[0] = w0.x; Wc[1] = w0.y; Wc[2] = w0.z; Wc[3] = w0.w;
+            Wc[4] = w1.x; Wc[5] = w1.y; Wc[6] = w1.z; Wc[7] = w1.w;
+            Wc[8] = w2.x;
+        }
+        // the part of the set-up that depends on the threshold: redone after a visit of the exact path
+        auto mid_setup = [&]() {
+            if constexpr (OBJ == MMEE_OBJ_ENERGY) {
+                u = __viaddmin_s32(base[rc], rc ? bv.w : bv.z, kRelCap);
+            } else {
+                int qo[3];
+                const int32_t* qrel;
+                if (fused) {
+                    ua[0] = ua[1] = ua[2] = ua2[rc];
+                    qo[0] = qo[1] = qo[2] = qo2[rc];
+                    qrel = tb->Qrel[rc];
+                } else {
+                    // unfused latency: max(DA1, C1) + softmax pass + max(DA2, C2); the first two terms are
+                    // fixed by (level of A, level of B = m, sm1)
+                    const int64_t da1 = ot->gA[c.la][0] + ot->gB[m][0] + tb->cw;
+                    const int64_t pass = c.phi == 2 ? tb->smx : 0;
+#pragma unroll
+                    for (int j = 0; j < 3; ++j) {
+                        const int64_t c1w = tb->C1w[j];
+                        const int64_t pj = (da1 > c1w ? da1 : c1w) + pass - T1;
+                        ua[j] = rel32(ot->gCr + pj);
+                        qo[j] = rel32(tb->qmin[2] + pj);
+                    }
+                    qrel = tb->Qrel[2];
+                }
+                const int4* q4 = reinterpret_cast<const int4*>(qrel);
+                const int4 q0 = q4[0], q1 = q4[1], q2 = q4[2];
+                Qc[0] = q0.x + qo[0]; Qc[1] = q0.y + qo[0]; Qc[2] = q0.z + qo[0];
+                Qc[3] = q0.w + qo[1]; Qc[4] = q1.x + qo[1]; Qc[5] = q1.y + qo[1];
+                Qc[6] = q1.z + qo[2]; Qc[7] = q1.w + qo[2]; Qc[8] = q2.x + qo[2];
+            }
+        };
+        mid_setup();
+
+#pragma unroll 1
+        for (int d = 0; d < 5; ++d) {
+            if constexpr (PRUNE) {
+                if (!__any_sync(kFull, live && ((kept >> (d * 5)) & 31u))) continue;
+            }
+            // Five rows (levels of E) are evaluated branch-free; one vote decides whether any lane of the
+            // warp has to enter the exact path for this group.
+            const int4 dc = *reinterpret_cast<const int4*>(rt->Dc[d]);
+            const int s1c = slack1c - dc.x;
+            const int s2c = slack2c - dc.y;
+            const uint32_t kd = kept >> (d * 5);
+            int a0 = INT_MAX, a1 = INT_MAX, a2 = INT_MAX;
+            bool hit;
+            if constexpr (OBJ == MMEE_OBJ_ENERGY) {
+                const int uc = __viaddmin_s32(u, dc.z, kRelCap);
+#pragma unroll
+                for (int e = 0; e < 5; ++e) {
+                    bool fit = (E1c[e] <= s1c) & (E2c[e] <= s2c);                                   // Eq. (4)
+                    if constexpr (PRUNE) fit = fit & ((kd >> e) & 1u);
+                    rows += fit;
+                    const int xc = uc + Gc[e];
+                    if (fit) {                                   // one fused add-min per mapping: min(key_s - thr)
+                        a0 = __viaddmin_s32(xc, Wc[0], a0); a1 = __viaddmin_s32(xc, Wc[1], a1); a2 = __viaddmin_s32(xc, Wc[2], a2);
+                        a0 = __viaddmin_s32(xc, Wc[3], a0); a1 = __viaddmin_s32(xc, Wc[4], a1); a2 = __viaddmin_s32(xc, Wc[5], a2);
+                        a0 = __viaddmin_s32(xc, Wc[6], a0); a1 = __viaddmin_s32(xc, Wc[7], a1); a2 = __viaddmin_s32(xc, Wc[8], a2);
+                    }
+                }
+                hit = __vimin3_s32(a0, a1, a2) < 0;
+            } else {
+                int uc[3];
+#pragma unroll
+                for (int j = 0; j < 3; ++j) uc[j] = __viaddmin_s32(ua[j], dc.z, kRelCap);
+#pragma unroll
+                for (int e = 0; e < 5; ++e) {
+                    bool fit = (E1c[e] <= s1c) & (E2c[e] <= s2c);                                   // Eq. (4)
+                    if constexpr (PRUNE) fit = fit & ((kd >> e) & 1u);
+                    rows += fit;
+                    int v[9];                                    // one fused add-max per mapping: key_s - thr
+#pragma unroll
+                    for (int s = 0; s < 9; ++s) v[s] = __viaddmax_s32(uc[s / 3], Gc[e], Qc[s]);
+                    if (fit) {
+                        a0 = __vimin3_s32(a0, v[0], v[1]); a1 = __vimin3_s32(a1, v[2], v[3]); a2 = __vimin3_s32(a2, v[4], v[5]);
+                        a0 = __vimin3_s32(a0, v[6], v[7]); a1 = min(a1, v[8]);
+                    }
+                }
+                // ties with the list's last entry cannot displace it from a higher index
+                hit = __vimin3_s32(a0, a1, a2) < ((m * 225 + d * 45) >= strict_from ? -delta : 0);
+            }
+            if (__any_sync(kFull, hit)) {
+                exact_group<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, k, lane);
+                rebase();
+                mid_setup();
+            }
+        }
+    }
+    return rows;
+}
+
+// ------------------------------------------------------------------------------------------------
 // the search kernel
 // ------------------------------------------------------------------------------------------------
 
@@ -456,7 +881,6 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
     const uint32_t tpt = shape.search_tpt;          // tasks per tiling in the searched task space
     const uint64_t task_begin = p.t_begin * tpt, task_end = p.t_end * tpt;
     const uint64_t dump_origin = task_begin * kCandPerTask;
-    const int64_t cap = p.cap_words;
     const uint32_t n_orders = p.n_orders;
     unsigned long long my_rows = 0;
 
@@ -514,6 +938,22 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
         tiling_pass(0, 18);     // stationary pairs x recompute flag
         tiling_pass(18, 3);     // unfused Op1 compute words
         __syncwarp();
+        if (OBJ == MMEE_OBJ_LATENCY) {
+            // compute words relative to their minimum over the stationary pairs: fused without and with
+            // recomputation, and Op2 of an unfused task
+            for (uint32_t j = lane; j < 3 * n_slots; j += 32) {
+                TilingTab* tb = &ttabs[j / 3];
+                const int v = (int)(j % 3);
+                const int64_t* src = v < 2 ? &tb->CB[0][v] : &tb->QU[0][0];
+                int64_t m = src[0];
+                for (int s = 1; s < 9; ++s) m = src[2 * s] < m ? src[2 * s] : m;
+                tb->qmin[v] = m;
+                for (int s = 0; s < 9; ++s) {
+                    const int64_t qd = src[2 * s] - m;
+                    tb->Qrel[v][s] = qd > (int64_t)kTermCap ? kTermCap : (int32_t)qd;
+                }
+            }
+        }
         if (OBJ == MMEE_OBJ_ENERGY) {
             // threshold-relative stationary-pair terms (see "32-bit differential keys")
             for (uint32_t j = lane; j < 2 * n_slots; j += 32) {
@@ -579,273 +1019,17 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
 
             const TaskChoice c = decode_task(p, w);
             const OrderTab* ot = &otabs[slot * n_orders + c.order_slot];
-            const bool fused = c.phi == 0;
-            const RowTab* rt = &ot->rt[fused ? 0 : 1];
-            const int64_t a1 = ot->A1[c.la];
-            const int64_t a2 = fused ? ot->A2[c.la] : 0;
             const uint64_t task_first_idx = tq * kCandPerTask;
             // The other CTAs' pruning bound: the load is issued here and consumed at the end of the
             // task, so that its latency is covered by the task's own work.
             const long long g_seen = (lane == 0) ? *reinterpret_cast<volatile long long*>(&scratch->G) : 0;
-            // Threshold state of this lane: T1 = the non-strict threshold (a key passes iff key < T1);
-            // for a group whose first index lies above `ti`, the index of the list's last entry, the
-            // threshold is T1 - delta (ties with that entry cannot displace it).
-            int64_t T1;
-            uint64_t ti;
-            int delta;
-            auto load_threshold = [&]() {
-                const int64_t g1 = cs->G + 1;                 // G <= INT64_MAX - 1 always
-                T1 = g1; ti = UINT64_MAX; delta = 0;
-                if (wt->count == k) {
-                    const int64_t tk1 = wt->key[k - 1] + 1;
-                    if (tk1 <= g1) { T1 = tk1; delta = 1; ti = wt->idx[k - 1]; }
-                }
-            };
-            load_threshold();
-            uint32_t rows = 0;
-            int E1c[5], E2c[5], Gc[5];
-#pragma unroll
-            for (int e = 0; e < 5; ++e) {
-                const int4 v = *reinterpret_cast<const int4*>(rt->Ec[e]);
-                E1c[e] = v.x; E2c[e] = v.y; Gc[e] = v.z;
-            }
-
-            // Middle loop of the task: the level of C for a fused task, of B for an unfused one.
-#pragma unroll 1
-            for (int mi = 0; mi < (PRUNE ? 1 : 5); ++mi) {
-            const int m = PRUNE ? (int)kept_mid : mi;
-            const uint32_t lb = fused ? c.lb : (uint32_t)m;
-            const uint32_t lc = fused ? (uint32_t)m : 0u;
-            const uint64_t mid_first_idx = task_first_idx + (uint64_t)(m * 225);
-            // Tables of a tiling that cannot fit are never built: a lane whose task lies in such a
-            // tiling must not index with what it reads from them.
-            const uint32_t rc = (fused && live) ? (ot->rc[lc] & 1u) : 0u;
-            const int64_t b1 = ot->B1[lb], c1 = ot->C1[lc];
-            const int64_t b2 = fused ? ot->B2[lb] : 0;
-            // Eq. (1)/(2): a retained operand (level >= L4) of the other operator keeps its space.
-            // A lane without a live task gets a negative slack, so that none of its rows fits.
-            const int64_t slack1 = live ? cap - (a1 + b1 + c1) : -1;
-            const int64_t slack2 = live ? cap - (c1 + a2 + b2) : -1;
-            const int64_t gab = ot->gA[c.la][rc] + ot->gB[lb][rc];
-
-            int64_t x0, xe0 = 0, P[3], Q[9], W[9];
-            const int64_t* wptr = &tb->W[0][rc];
-            const int64_t* qptr;
-            if constexpr (OBJ == MMEE_OBJ_ENERGY) {
-                const int64_t extra = p.c_dram_gb * (tb->cw + (c.phi == 2 ? tb->smx : 0));
-                x0 = fused ? gab : gab + ot->gCr + extra;
-                P[0] = P[1] = P[2] = 0;
-                qptr = wptr;
+            if constexpr (!DUMP && OBJ <= MMEE_OBJ_LATENCY) {
+                my_rows += walk_task_relative<OBJ, PRUNE>(p, tb, ot, c, live, kept, kept_mid, task_first_idx, wt, cs,
+                                                          &scratch->G, k, lane);
             } else {
-                const int64_t pass = (c.phi == 2) ? tb->smx : 0;
-                if (fused) {
-                    x0 = gab;
-                    P[0] = P[1] = P[2] = 0;
-                    qptr = &tb->CB[0][rc];
-                } else {
-                    // unfused latency: max(DA1, C1) + softmax pass + max(DA2, C2)
-                    x0 = ot->gCr;
-                    const int64_t da1 = gab + tb->cw;
-#pragma unroll
-                    for (int j = 0; j < 3; ++j) P[j] = (da1 > tb->C1w[j] ? da1 : tb->C1w[j]) + pass;
-                    qptr = &tb->QU[0][0];
-                }
-                if constexpr (OBJ >= MMEE_OBJ_EDP) {
-                    const int64_t eab = ot->eA[c.la][rc] + ot->eB[lb][rc];
-                    xe0 = fused ? eab : eab + ot->eCr + p.c_dram_gb * (tb->cw + pass);
-                }
+                my_rows += walk_task_exact<OBJ, DUMP, PRUNE>(p, tb, ot, c, live, valid, kept, kept_mid, task_first_idx, wt,
+                                                             cs, &scratch->G, k, lane, dump, dump_origin);
             }
-#pragma unroll
-            for (int s = 0; s < 9; ++s) {
-                W[s] = wptr[2 * s];
-                Q[s] = qptr[2 * s];
-            }
-            // threshold-relative forms (see "32-bit differential keys"); refreshed when thr moves
-            int64_t wmin = 0;
-            int Wc[9], Qc[9];
-            int64_t B = 0, PmT[3];
-            if constexpr (OBJ == MMEE_OBJ_ENERGY) {
-                wmin = tb->wmin[rc];
-                const int4* wc4 = reinterpret_cast<const int4*>(tb->Wc[rc]);
-                const int4 w0 = wc4[0], w1 = wc4[1], w2 = wc4[2];
-                Wc[0] = w0.x; Wc[1] = w0.y; Wc[2] = w0.z; Wc[3] = w0.w;
-                Wc[4] = w1.x; Wc[5] = w1.y; Wc[6] = w1.z; Wc[7] = w1.w;
-                Wc[8] = w2.x;
-            }
-            int ut[3] = {0, 0, 0};      // saturated task-level part of key - thr
-            double dW[9], dQP[9], dthr = 0.0;
-            if constexpr (OBJ == MMEE_OBJ_EDP) {
-#pragma unroll
-                for (int s = 0; s < 9; ++s) {
-                    dW[s] = (double)W[s];
-                    dQP[s] = (double)(Q[s] + P[s / 3]);
-                }
-            }
-            auto refresh = [&](int64_t t) {
-                if constexpr (OBJ == MMEE_OBJ_ENERGY) {
-                    // ut[0]: against the non-strict threshold t; ut[1]: against t - delta (ties excluded).
-                    // Rounding every term down to a multiple of 2^rel_shift can only lower the sum.
-                    B = t - wmin;
-                    const int u0 = sat_s32((x0 - B) >> p.rel_shift);
-                    const int u1 = sat_s32((x0 - B + delta) >> p.rel_shift);
-                    ut[0] = u0 < kRelCap ? u0 : kRelCap;
-                    ut[1] = u1 < kRelCap ? u1 : kRelCap;
-                } else if constexpr (OBJ == MMEE_OBJ_LATENCY) {
-#pragma unroll
-                    for (int j = 0; j < 3; ++j) {
-                        PmT[j] = P[j] - t;
-                        const int u = sat_s32(x0 + PmT[j]);
-                        ut[j] = u < kRelCap ? u : kRelCap;
-                    }
-#pragma unroll
-                    for (int s = 0; s < 9; ++s) Qc[s] = sat_s32(Q[s] + P[s / 3] - t);
-                } else if constexpr (OBJ == MMEE_OBJ_EDP) {
-                    // EDP keys are bit patterns of positive doubles; anything from +inf up means "no bound yet"
-                    dthr = t >= 0x7ff0000000000000ll ? __longlong_as_double(0x7ff0000000000000ll)
-                                                     : __longlong_as_double(t) * (1.0 + 1e-14);
-                }
-            };
-            refresh(T1);
-            const int slack1c = slack1 < 0 ? -1 : (int)slack1;      // slack <= capacity < 2^30
-            const int slack2c = slack2 < 0 ? -1 : (int)slack2;
-
-#pragma unroll 1
-            for (int d = 0; d < 5; ++d) {
-                if constexpr (PRUNE) {
-                    if (!__any_sync(kFull, live && ((kept >> (d * 5)) & 31u))) continue;
-                }
-                // Five rows (levels of E) are evaluated branch-free; one vote decides whether any
-                // lane of the warp has to enter the insertion path for this group.
-                unsigned hit_any, fits;
-                if constexpr (!DUMP && OBJ <= MMEE_OBJ_LATENCY) {
-                    const int4 dc = *reinterpret_cast<const int4*>(rt->Dc[d]);
-                    const int s1c = slack1c - dc.x;
-                    const int s2c = slack2c - dc.y;
-                    int acc = INT_MAX;
-                    fits = 0;
-                    if constexpr (OBJ == MMEE_OBJ_ENERGY) {
-                        const uint64_t group_first_idx = mid_first_idx + (uint64_t)(d * 45);
-                        const int uc = __viaddmin_s32(group_first_idx > ti ? ut[1] : ut[0], dc.z, kRelCap);
-                        int accs[9];          // one chain per stationary pair: nine independent chains
-#pragma unroll
-                        for (int s = 0; s < 9; ++s) accs[s] = INT_MAX;
-#pragma unroll
-                        for (int e = 0; e < 5; ++e) {
-                            unsigned fit = (unsigned)(E1c[e] <= s1c) & (unsigned)(E2c[e] <= s2c);         // Eq. (4)
-                            if constexpr (PRUNE) fit &= kept >> (d * 5 + e);
-                            fits += fit;
-                            int xc = __viaddmin_s32(uc, Gc[e], kRelCap);
-                            xc = fit ? xc : kRelCap;
-#pragma unroll
-                            for (int s = 0; s < 9; ++s) accs[s] = __viaddmin_s32(xc, Wc[s], accs[s]);   // min(key_s - thr)
-                        }
-                        acc = __vimin3_s32(__vimin3_s32(accs[0], accs[1], accs[2]), __vimin3_s32(accs[3], accs[4], accs[5]),
-                                           __vimin3_s32(accs[6], accs[7], accs[8]));
-                    } else {
-                        int uc[3];
-#pragma unroll
-                        for (int j = 0; j < 3; ++j) uc[j] = __viaddmin_s32(ut[j], dc.z, kRelCap);
-#pragma unroll
-                        for (int e = 0; e < 5; ++e) {
-                            unsigned fit = (unsigned)(E1c[e] <= s1c) & (unsigned)(E2c[e] <= s2c);         // Eq. (4)
-                            if constexpr (PRUNE) fit &= kept >> (d * 5 + e);
-                            fits += fit;
-                            int a[3];
-#pragma unroll
-                            for (int j = 0; j < 3; ++j) a[j] = __viaddmin_s32(uc[j], Gc[e], kRelCap);
-                            int racc = INT_MAX;
-#pragma unroll
-                            for (int s = 0; s < 9; ++s) racc = min(racc, max(a[s / 3], Qc[s]));   // min(key_s - thr)
-                            acc = min(acc, fit ? racc : INT_MAX);
-                        }
-                    }
-                    if constexpr (OBJ == MMEE_OBJ_ENERGY) {
-                        hit_any = acc < 0;
-                    } else {
-                        const uint64_t group_first_idx = mid_first_idx + (uint64_t)(d * 45);
-                        hit_any = acc < (group_first_idx > ti ? -delta : 0);  // no overflow at acc = INT_MAX
-                    }
-                } else if constexpr (!DUMP && OBJ == MMEE_OBJ_EDP) {
-                    // The energy-delay product is not separable, so the filter is a double-precision
-                    // evaluation of every mapping on the FP64 pipe: energy and latency sums converted
-                    // once per row, then an add, two multiplies and two compares per mapping.  Each
-                    // approximate product is within a few 2^-53 of the exact key, so comparing against
-                    // the threshold widened by 1e-14 relative can flag a row needlessly but never miss
-                    // one; the exact 64-bit path below decides.
-                    const int4 dc = *reinterpret_cast<const int4*>(rt->Dc[d]);
-                    const int s1c = slack1c - dc.x;
-                    const int s2c = slack2c - dc.y;
-                    const int64_t xd = x0 + rt->D[d][2];
-                    const int64_t xed = xe0 + rt->D[d][3];
-                    fits = 0;
-                    hit_any = 0;
-#pragma unroll
-                    for (int e = 0; e < 5; ++e) {
-                        unsigned fit = (unsigned)(E1c[e] <= s1c) & (unsigned)(E2c[e] <= s2c);             // Eq. (4)
-                        if constexpr (PRUNE) fit &= kept >> (d * 5 + e);
-                        fits += fit;
-                        const int64_t x = xd + rt->E[e][2];
-                        const double de = (double)(xed + rt->E[e][3]);
-                        double dl[3];
-#pragma unroll
-                        for (int j = 0; j < 3; ++j) dl[j] = (double)(x + P[j]);
-                        hit_any |= edp_row_test(de, dl, dW, dQP, dthr, fit);
-                    }
-                } else {
-                    const int64_t s1 = slack1 - rt->D[d][0];
-                    const int64_t s2 = slack2 - rt->D[d][1];
-                    const int64_t xd = x0 + rt->D[d][2];
-                    const int64_t xed = (OBJ >= MMEE_OBJ_EDP) ? xe0 + rt->D[d][3] : 0;
-                    const uint64_t group_first_idx = mid_first_idx + (uint64_t)(d * 45);
-                    const int64_t thr = T1 - (group_first_idx > ti ? delta : 0);
-                    hit_any = 0; fits = 0;
-#pragma unroll
-                    for (int e = 0; e < 5; ++e) {
-                        const int64_t x = xd + rt->E[e][2];
-                        const int64_t xe = (OBJ >= MMEE_OBJ_EDP) ? xed + rt->E[e][3] : 0;
-                        int64_t key[9];
-#pragma unroll
-                        for (int s = 0; s < 9; ++s) key[s] = candidate_key<OBJ>(x, xe, W[s], P[s / 3], Q[s], p.key_cap);
-                        unsigned fit, hit;
-                        row_test(key, thr, rt->E[e][0], s1, rt->E[e][1], s2, fit, hit);
-                        fits += fit;
-                        hit_any |= hit;
-                        if (DUMP) {
-                            if (valid) {
-#pragma unroll
-                                for (int s = 0; s < 9; ++s)
-                                    dump[mid_first_idx - dump_origin + (d * 5 + e) * 9 + s] = fit ? key[s] : kInfKey;
-                            }
-                        }
-                    }
-                }
-                rows += fits;
-                if (__any_sync(kFull, hit_any != 0u)) {
-                    // rare: find the rows that passed, exactly, and let the warp insert their candidates
-                    const int64_t s1 = slack1 - rt->D[d][0];
-                    const int64_t s2 = slack2 - rt->D[d][1];
-                    const int64_t xd = x0 + rt->D[d][2];
-                    const int64_t xed = (OBJ >= MMEE_OBJ_EDP) ? xe0 + rt->D[d][3] : 0;
-#pragma unroll 1
-                    for (int e = 0; e < 5; ++e) {
-                        const bool fit = (rt->E[e][0] <= s1) && (rt->E[e][1] <= s2) && ((kept >> (d * 5 + e)) & 1u);
-                        const int64_t x = xd + rt->E[e][2];
-                        const int64_t xe = (OBJ >= MMEE_OBJ_EDP) ? xed + rt->E[e][3] : 0;
-                        const uint64_t row_first_idx = mid_first_idx + (uint64_t)((d * 5 + e) * 9);
-                        const int64_t thr_row = lane_threshold(wt, cs, k, row_first_idx);
-                        bool below = false;
-                        for (int s = 0; s < 9; ++s)
-                            below |= candidate_key<OBJ>(x, xe, wptr[2 * s], P[s / 3], qptr[2 * s], p.key_cap) < thr_row;
-                        if (__any_sync(kFull, fit && below))
-                            slow_row<OBJ>(wt, cs, &scratch->G, k, lane, fit, x, xe, wptr, qptr, P[0], P[1], P[2], p.key_cap,
-                                          row_first_idx);
-                    }
-                    load_threshold();
-                    refresh(T1);
-                }
-            }
-            }   // middle loop
-            my_rows += rows;
             if (lane == 0 && g_seen < cs->G) atomicMin(&cs->G, g_seen);
         }
         }   // workers

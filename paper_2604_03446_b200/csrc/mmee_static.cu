@@ -54,7 +54,7 @@ int static_shape(const Plan& p, int device, LaunchShape* shape) {
     shape->pruned = nullptr;
     shape->slots = (shape->range_tasks - 1) / p.tasks_per_tiling + 2;
     size_t smem = search_smem_bytes(p, shape->slots);
-    while (smem > 96 * 1024 && shape->range_tasks > 32) {
+    while (smem > 110 * 1024 && shape->range_tasks > 32) {
         shape->range_tasks -= shape->range_tasks > (uint32_t)kWorkerThreads ? kWorkerThreads : 32;
         shape->slots = (shape->range_tasks - 1) / p.tasks_per_tiling + 2;
         smem = search_smem_bytes(p, shape->slots);
