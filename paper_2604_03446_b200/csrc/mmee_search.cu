@@ -682,11 +682,13 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
                                                        long long* global_g, int k, int lane) {
     const bool fused = c.phi == 0;
     const RowTab* rt = &ot->rt[fused ? 0 : 1];
-    int E1c[5], E2c[5], Gc[5];
+    // Row-side terms of E.  Its buffer need while Op1 runs is its size when retained (level >= L4 of a
+    // fused task) and 0 otherwise, so that only the size itself has to be kept.
+    int E2c[5], Gc[5];
 #pragma unroll
     for (int e = 0; e < 5; ++e) {
         const int4 v = *reinterpret_cast<const int4*>(rt->Ec[e]);
-        E1c[e] = v.x; E2c[e] = v.y; Gc[e] = v.z;
+        E2c[e] = v.y; Gc[e] = v.z;
     }
     const int4 av = *reinterpret_cast<const int4*>(ot->Ac[c.la]);
     const int a1c = av.x, a2c = fused ? av.y : 0;
@@ -694,9 +696,11 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
     const int gxc = (OBJ == MMEE_OBJ_ENERGY && !fused) ? ot->gXc[c.phi == 2 ? 1 : 0] : 0;
     auto rel32 = [](int64_t v) { const int r = sat_s32(v); return r < kRelCap ? r : kRelCap; };
 
-    // Threshold state.  Energy: base[rc] = (terms of A and of the C round trip) - ceil((T1 - wmin[rc]) / 2^rel_shift).
+    // Threshold state.  Energy: base[rc] = (terms of A and of the C round trip) - ceil((T1 - wmin[rc]) / 2^rel_shift),
+    // base_strict[rc] the same against T1 - delta.  (Most terms are multiples of the unit, so that a tie with the
+    // list's last entry is told from a better key even in coarse units.)
     // Latency, fused task: ua2[rc] = DRAM words of A and B - T1, qo2[rc] = least compute words - T1.
-    int base[2] = {0, 0}, ua2[2] = {0, 0}, qo2[2] = {0, 0};
+    int base[2] = {0, 0}, base_strict[2] = {0, 0}, ua2[2] = {0, 0}, qo2[2] = {0, 0};
     int64_t T1 = 0;
     int delta = 0, strict_from = INT_MAX;
     auto rebase = [&]() {
@@ -709,10 +713,14 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
         if constexpr (OBJ == MMEE_OBJ_ENERGY) {
 #pragma unroll
             for (int rc = 0; rc < 2; ++rc) {
-                const int64_t bs = ((T1 - tb->wmin[rc] - 1) >> p.rel_shift) + 1;      // ceiling of the quotient
-                const int64_t bl = bs > (int64_t)INT_MAX ? (int64_t)INT_MAX : (bs < -(int64_t)kTermCap ? -(int64_t)kTermCap : bs);
-                const int t = (rc ? av.w : av.z) + gxc - (int)bl;
-                base[rc] = t < kRelCap ? t : kRelCap;
+#pragma unroll
+                for (int st = 0; st < 2; ++st) {
+                    const int64_t b64 = T1 - (st ? delta : 0) - tb->wmin[rc];
+                    const int64_t bs = ((b64 - 1) >> p.rel_shift) + 1;                // ceiling of the quotient
+                    const int64_t bl = bs > (int64_t)INT_MAX ? (int64_t)INT_MAX : (bs < -(int64_t)kTermCap ? -(int64_t)kTermCap : bs);
+                    const int t = (rc ? av.w : av.z) + gxc - (int)bl;
+                    (st ? base_strict : base)[rc] = t < kRelCap ? t : kRelCap;
+                }
             }
         } else {
             if (fused) {
@@ -742,7 +750,7 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
         const int slack1c = live ? capc - y1 : -1;       // a lane without a live task: none of its rows fits
         const int slack2c = live ? capc - y2 : -1;
 
-        int u = 0, Wc[9], ua[3], Qc[9];
+        int u = 0, u_strict = 0, Wc[9], ua[3], Qc[9];
         if constexpr (OBJ == MMEE_OBJ_ENERGY) {
             const int4* wc4 = reinterpret_cast<const int4*>(tb->Wc[rc]);
             const int4 w0 = wc4[0], w1 = wc4[1], w2 = wc4[2];
@@ -754,6 +762,7 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
         auto mid_setup = [&]() {
             if constexpr (OBJ == MMEE_OBJ_ENERGY) {
                 u = __viaddmin_s32(base[rc], rc ? bv.w : bv.z, kRelCap);
+                u_strict = __viaddmin_s32(base_strict[rc], rc ? bv.w : bv.z, kRelCap);
             } else {
                 int qo[3];
                 const int32_t* qrel;
@@ -784,7 +793,7 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
         };
         mid_setup();
 
-#pragma unroll 1
+#pragma unroll
         for (int d = 0; d < 5; ++d) {
             if constexpr (PRUNE) {
                 if (!__any_sync(kFull, live && ((kept >> (d * 5)) & 31u))) continue;
@@ -794,22 +803,26 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
             const int4 dc = *reinterpret_cast<const int4*>(rt->Dc[d]);
             const int s1c = slack1c - dc.x;
             const int s2c = slack2c - dc.y;
+            // Eq. (4) for the five levels of E: at L3, and in an unfused task, E takes no space while Op1
+            // runs (size <= s2c, given s1c >= 0); retained, it must fit beside both operators' operands
+            const int lim_l3 = s1c >= 0 ? s2c : -1;
+            const int lim_retained = fused ? min(s1c, s2c) : lim_l3;
             const uint32_t kd = kept >> (d * 5);
             int a0 = INT_MAX, a1 = INT_MAX, a2 = INT_MAX;
             bool hit;
             if constexpr (OBJ == MMEE_OBJ_ENERGY) {
-                const int uc = __viaddmin_s32(u, dc.z, kRelCap);
+                // ties with the list's last entry cannot displace it from a higher index
+                const int uc = __viaddmin_s32((m * 225 + d * 45) >= strict_from ? u_strict : u, dc.z, kRelCap);
 #pragma unroll
                 for (int e = 0; e < 5; ++e) {
-                    bool fit = (E1c[e] <= s1c) & (E2c[e] <= s2c);                                   // Eq. (4)
+                    bool fit = E2c[e] <= (e == 0 ? lim_l3 : lim_retained);
                     if constexpr (PRUNE) fit = fit & ((kd >> e) & 1u);
                     rows += fit;
-                    const int xc = uc + Gc[e];
-                    if (fit) {                                   // one fused add-min per mapping: min(key_s - thr)
-                        a0 = __viaddmin_s32(xc, Wc[0], a0); a1 = __viaddmin_s32(xc, Wc[1], a1); a2 = __viaddmin_s32(xc, Wc[2], a2);
-                        a0 = __viaddmin_s32(xc, Wc[3], a0); a1 = __viaddmin_s32(xc, Wc[4], a1); a2 = __viaddmin_s32(xc, Wc[5], a2);
-                        a0 = __viaddmin_s32(xc, Wc[6], a0); a1 = __viaddmin_s32(xc, Wc[7], a1); a2 = __viaddmin_s32(xc, Wc[8], a2);
-                    }
+                    const int xc = fit ? uc + Gc[e] : kRelCap;
+                    // one fused add-min per mapping: min(key_s - thr)
+                    a0 = __viaddmin_s32(xc, Wc[0], a0); a1 = __viaddmin_s32(xc, Wc[1], a1); a2 = __viaddmin_s32(xc, Wc[2], a2);
+                    a0 = __viaddmin_s32(xc, Wc[3], a0); a1 = __viaddmin_s32(xc, Wc[4], a1); a2 = __viaddmin_s32(xc, Wc[5], a2);
+                    a0 = __viaddmin_s32(xc, Wc[6], a0); a1 = __viaddmin_s32(xc, Wc[7], a1); a2 = __viaddmin_s32(xc, Wc[8], a2);
                 }
                 hit = __vimin3_s32(a0, a1, a2) < 0;
             } else {
@@ -818,7 +831,7 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
                 for (int j = 0; j < 3; ++j) uc[j] = __viaddmin_s32(ua[j], dc.z, kRelCap);
 #pragma unroll
                 for (int e = 0; e < 5; ++e) {
-                    bool fit = (E1c[e] <= s1c) & (E2c[e] <= s2c);                                   // Eq. (4)
+                    bool fit = E2c[e] <= (e == 0 ? lim_l3 : lim_retained);
                     if constexpr (PRUNE) fit = fit & ((kd >> e) & 1u);
                     rows += fit;
                     int v[9];                                    // one fused add-max per mapping: key_s - thr
