@@ -240,6 +240,7 @@ int build_plan(const mmee_workload_t* w, const mmee_arch_t* a, const mmee_object
     // Scale of the 32-bit threshold-relative energy keys: the largest DRAM term of any mapping,
     // c_dram_gb * I*K*L*J, must fit below 2^28 after the shift.
     p->rel_shift = 0;
+    p->unit = 1;
     if (p->objective == MMEE_OBJ_ENERGY) {
         long double biggest = (long double)dims[0] * dims[1] * dims[2] * dims[3] * (long double)p->c_dram_gb;
         while (biggest >= 268435456.0L) { biggest /= 2.0L; ++p->rel_shift; }

@@ -52,6 +52,8 @@ struct Plan {
     uint32_t row_pruning;
     int64_t  key_cap;             // capped objectives: bound on the other key
     uint32_t rel_shift;           // energy: threshold-relative keys are kept in units of 2^rel_shift quanta
+    int32_t  unit;                // the constant 1, as a run-time value: x * unit + y is issued as an integer
+                                  // multiply-add, which the FMA pipe executes beside the integer ALU pipe
     double   quantum_pj;
     QueryTables q;
     uint32_t divs[4][MMEE_MAX_DIVISORS];

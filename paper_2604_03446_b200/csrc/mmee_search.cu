@@ -33,8 +33,10 @@ constexpr int kModeSearch = 0, kModeDump = 1, kModePrune = 2;
 constexpr size_t kPlanBytes = (sizeof(Plan) + 15) / 16 * 16;
 static_assert(sizeof(Plan) % 4 == 0, "the plan is copied word by word");
 constexpr int kRelCap = (1 << 30) - 1;     // cap of a running threshold-relative sum (see below)
-constexpr int kTermCap = 1 << 28;          // cap of each non-negative addend of such a sum (at most six of them)
+constexpr int kTermCap = (1 << 28) - 1;    // cap of each non-negative addend of such a sum (at most six of them)
 constexpr int kSizeCap = (1 << 30) - 1;    // buffer sizes saturate here; the capacity is smaller
+constexpr int kUnfit = 1 << 30;            // added to the keys of a row that does not fit; also the lower clamp of a row sum
+constexpr int kRowCap = (1 << 29) - 1;     // upper cap of a row sum: kRowCap + 2 * kTermCap + kUnfit < 2^31
 
 // ------------------------------------------------------------------------------------------------
 // shared-memory tables
@@ -216,6 +218,19 @@ __device__ __forceinline__ void row_test(const int64_t (&k)[9], int64_t thr, int
 // saturation is applied to x + P - thr = u + vD + vE.
 // Capacity (Eq. 4): sizes are saturated to kSizeCap, which is above every admissible capacity, so
 // "size <= slack" keeps its truth value in 32 bits.
+// Integer multiply-add and arithmetic shift as single PTX instructions, opaque to the optimiser: the row
+// loops use them to keep additions on the FMA pipe and sign masks out of compare-and-select form.
+__device__ __forceinline__ int imad(int a, int b, int c) {
+    int r;
+    asm("mad.lo.s32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+    return r;
+}
+__device__ __forceinline__ int sign_mask(int a) {       // -1 if a < 0, else 0
+    int r;
+    asm("shr.s32 %0, %1, 31;" : "=r"(r) : "r"(a));
+    return r;
+}
+
 __device__ __forceinline__ int sat_s32(int64_t v) {
     int r;
     asm("cvt.sat.s32.s64 %0, %1;" : "=r"(r) : "l"(v));
@@ -693,8 +708,13 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
     const int4 av = *reinterpret_cast<const int4*>(ot->Ac[c.la]);
     const int a1c = av.x, a2c = fused ? av.y : 0;
     const int capc = (int)p.cap_words;
+    // Additions that need no saturation are written x * one + y: an integer multiply-add runs on the FMA
+    // pipe, which is otherwise idle, instead of the integer ALU pipe that bounds this kernel.
+    const int one = p.unit, minus_one = -p.unit;
     const int gxc = (OBJ == MMEE_OBJ_ENERGY && !fused) ? ot->gXc[c.phi == 2 ? 1 : 0] : 0;
-    auto rel32 = [](int64_t v) { const int r = sat_s32(v); return r < kRelCap ? r : kRelCap; };
+    // task-level part of key - thr, clamped to [-kUnfit, kRowCap]: clamping from below keeps the sign of every
+    // sum that follows (at most 4 * kTermCap < kUnfit is added), clamping from above only lowers
+    auto rel32 = [](int64_t v) { const int r = sat_s32(v); return max(min(r, kRowCap), -kUnfit); };
 
     // Threshold state.  Energy: base[rc] = (terms of A and of the C round trip) - ceil((T1 - wmin[rc]) / 2^rel_shift),
     // base_strict[rc] the same against T1 - delta.  (Most terms are multiples of the unit, so that a tie with the
@@ -719,7 +739,7 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
                     const int64_t bs = ((b64 - 1) >> p.rel_shift) + 1;                // ceiling of the quotient
                     const int64_t bl = bs > (int64_t)INT_MAX ? (int64_t)INT_MAX : (bs < -(int64_t)kTermCap ? -(int64_t)kTermCap : bs);
                     const int t = (rc ? av.w : av.z) + gxc - (int)bl;
-                    (st ? base_strict : base)[rc] = t < kRelCap ? t : kRelCap;
+                    (st ? base_strict : base)[rc] = max(min(t, kRowCap), -kUnfit);
                 }
             }
         } else {
@@ -734,7 +754,8 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
     };
     rebase();
 
-    uint32_t rows = 0;
+    int unfit = 0;          // minus the number of visited rows that do not fit
+    uint32_t groups = 0;
 #pragma unroll 1
     for (int mi = 0; mi < (PRUNE ? 1 : 5); ++mi) {
         const int m = PRUNE ? (int)kept_mid : mi;
@@ -747,8 +768,8 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
         y1 = __viaddmin_s32(y1, cv.x, kSizeCap);
         int y2 = __viaddmin_s32(a2c, fused ? bv.y : 0, kSizeCap);
         y2 = __viaddmin_s32(y2, cv.x, kSizeCap);
-        const int slack1c = live ? capc - y1 : -1;       // a lane without a live task: none of its rows fits
-        const int slack2c = live ? capc - y2 : -1;
+        const int slack1c = live ? max(capc - y1, -1) : -1;       // a lane without a live task: none of its rows fits
+        const int slack2c = live ? max(capc - y2, -1) : -1;
 
         int u = 0, u_strict = 0, Wc[9], ua[3], Qc[9];
         if constexpr (OBJ == MMEE_OBJ_ENERGY) {
@@ -761,8 +782,8 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
         // the part of the set-up that depends on the threshold: redone after a visit of the exact path
         auto mid_setup = [&]() {
             if constexpr (OBJ == MMEE_OBJ_ENERGY) {
-                u = __viaddmin_s32(base[rc], rc ? bv.w : bv.z, kRelCap);
-                u_strict = __viaddmin_s32(base_strict[rc], rc ? bv.w : bv.z, kRelCap);
+                u = __viaddmin_s32(base[rc], rc ? bv.w : bv.z, kRowCap);
+                u_strict = __viaddmin_s32(base_strict[rc], rc ? bv.w : bv.z, kRowCap);
             } else {
                 int qo[3];
                 const int32_t* qrel;
@@ -800,6 +821,7 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
             }
             // Five rows (levels of E) are evaluated branch-free; one vote decides whether any lane of the
             // warp has to enter the exact path for this group.
+            ++groups;
             const int4 dc = *reinterpret_cast<const int4*>(rt->Dc[d]);
             const int s1c = slack1c - dc.x;
             const int s2c = slack2c - dc.y;
@@ -812,13 +834,15 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
             bool hit;
             if constexpr (OBJ == MMEE_OBJ_ENERGY) {
                 // ties with the list's last entry cannot displace it from a higher index
-                const int uc = __viaddmin_s32((m * 225 + d * 45) >= strict_from ? u_strict : u, dc.z, kRelCap);
+                const int uc = __viaddmin_s32((m * 225 + d * 45) >= strict_from ? u_strict : u, dc.z, kRowCap);
 #pragma unroll
                 for (int e = 0; e < 5; ++e) {
-                    bool fit = E2c[e] <= (e == 0 ? lim_l3 : lim_retained);
-                    if constexpr (PRUNE) fit = fit & ((kd >> e) & 1u);
-                    rows += fit;
-                    const int xc = fit ? uc + Gc[e] : kRelCap;
+                    // t = -1 if the row does not fit (Eq. 4), else 0; such a row's keys are moved up by kUnfit,
+                    // which makes them non-negative
+                    int t = sign_mask(imad(E2c[e], minus_one, e == 0 ? lim_l3 : lim_retained));
+                    if constexpr (PRUNE) t |= (int)((kd >> e) & 1u) - 1;
+                    unfit = imad(t, one, unfit);
+                    const int xc = imad(t, -kUnfit, imad(uc, one, Gc[e]));
                     // one fused add-min per mapping: min(key_s - thr)
                     a0 = __viaddmin_s32(xc, Wc[0], a0); a1 = __viaddmin_s32(xc, Wc[1], a1); a2 = __viaddmin_s32(xc, Wc[2], a2);
                     a0 = __viaddmin_s32(xc, Wc[3], a0); a1 = __viaddmin_s32(xc, Wc[4], a1); a2 = __viaddmin_s32(xc, Wc[5], a2);
@@ -828,19 +852,18 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
             } else {
                 int uc[3];
 #pragma unroll
-                for (int j = 0; j < 3; ++j) uc[j] = __viaddmin_s32(ua[j], dc.z, kRelCap);
+                for (int j = 0; j < 3; ++j) uc[j] = __viaddmin_s32(ua[j], dc.z, kRowCap);
 #pragma unroll
                 for (int e = 0; e < 5; ++e) {
-                    bool fit = E2c[e] <= (e == 0 ? lim_l3 : lim_retained);
-                    if constexpr (PRUNE) fit = fit & ((kd >> e) & 1u);
-                    rows += fit;
+                    int t = sign_mask(imad(E2c[e], minus_one, e == 0 ? lim_l3 : lim_retained));      // -1: the row does not fit
+                    if constexpr (PRUNE) t |= (int)((kd >> e) & 1u) - 1;
+                    unfit = imad(t, one, unfit);
+                    const int ge = imad(t, -kUnfit, Gc[e]);
                     int v[9];                                    // one fused add-max per mapping: key_s - thr
 #pragma unroll
-                    for (int s = 0; s < 9; ++s) v[s] = __viaddmax_s32(uc[s / 3], Gc[e], Qc[s]);
-                    if (fit) {
-                        a0 = __vimin3_s32(a0, v[0], v[1]); a1 = __vimin3_s32(a1, v[2], v[3]); a2 = __vimin3_s32(a2, v[4], v[5]);
-                        a0 = __vimin3_s32(a0, v[6], v[7]); a1 = min(a1, v[8]);
-                    }
+                    for (int s = 0; s < 9; ++s) v[s] = __viaddmax_s32(uc[s / 3], ge, Qc[s]);
+                    a0 = __vimin3_s32(a0, v[0], v[1]); a1 = __vimin3_s32(a1, v[2], v[3]); a2 = __vimin3_s32(a2, v[4], v[5]);
+                    a0 = __vimin3_s32(a0, v[6], v[7]); a1 = min(a1, v[8]);
                 }
                 // ties with the list's last entry cannot displace it from a higher index
                 hit = __vimin3_s32(a0, a1, a2) < ((m * 225 + d * 45) >= strict_from ? -delta : 0);
@@ -852,7 +875,7 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
             }
         }
     }
-    return rows;
+    return (uint32_t)((int)(groups * 5u) + unfit);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -992,7 +1015,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
         const uint64_t r0 = cs->range_begin[buf];
         if (r0 >= task_end) break;
         if (builder) build_next(buf ^ 1);
-        if (!builder) {
+        {       // every warp walks tasks; the builder warp joins once the next range's tables are done
         const uint64_t r1 = (r0 + shape.range_tasks < task_end) ? r0 + shape.range_tasks : task_end;
         const uint64_t t_first = r0 / tpt;
         const TilingTab* ttabs = ttabs_all + buf * shape.slots;
@@ -1056,7 +1079,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
 
     // ---- merge the warps' lists into warp 0's, then publish this CTA's partial list
     if (warp == 0) {
-        for (int w2 = 1; w2 < kWorkerWarps; ++w2) {
+        for (int w2 = 1; w2 < kSearchThreads / 32; ++w2) {
             const WarpTop* src = &wtops[w2];
             const int n = src->count;
             for (int j = 0; j < n; ++j)
