@@ -20,6 +20,7 @@
 
 #include <climits>
 #include <cstddef>
+#include <type_traits>
 
 #include "mmee_eval.cuh"
 #include "mmee_search.h"
@@ -923,24 +924,32 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
     // Builder: pull the next range and build its tables into buffer `buf`.  Ranges are visited in a
     // stride-permuted order (stride coprime to their number), so that the first pull of every CTA
     // samples the whole index space and the pruning bound G is near its final value from the start.
-    auto build_next = [&](int buf) {
-        unsigned long long got = 0;
-        if (lane == 0) got = atomicAdd(&scratch->next_task, 1ull);
-        got = __shfl_sync(kFull, got, 0);
-        const uint64_t r0 = got < shape.n_ranges
-                                ? task_begin + ((got * shape.range_stride) % shape.n_ranges) * shape.range_tasks
-                                : task_end;
-        if (lane == 0) { cs->range_begin[buf] = r0; cs->cursor[buf] = 0; }
+    // `coop` (a std::bool_constant): the whole CTA builds together (the first range, when there is nothing to walk
+    // yet) instead of the builder warp alone.
+    auto build_next = [&](int buf, auto coop) {
+        constexpr bool COOP = decltype(coop)::value;
+        const uint32_t first = COOP ? (uint32_t)tid : (uint32_t)lane;
+        const uint32_t step = COOP ? (uint32_t)kSearchThreads : 32u;
+        auto sync = [] { if constexpr (COOP) __syncthreads(); else __syncwarp(); };
+        if (first == 0) {
+            const unsigned long long got = atomicAdd(&scratch->next_task, 1ull);
+            cs->range_begin[buf] = got < shape.n_ranges
+                                       ? task_begin + ((got * shape.range_stride) % shape.n_ranges) * shape.range_tasks
+                                       : task_end;
+            cs->cursor[buf] = 0;
+        }
+        sync();
+        const uint64_t r0 = cs->range_begin[buf];
         if (r0 >= task_end) return;
         const uint64_t r1 = (r0 + shape.range_tasks < task_end) ? r0 + shape.range_tasks : task_end;
         const uint64_t t_first = r0 / tpt, t_last = (r1 - 1) / tpt;
         const uint32_t n_slots = (uint32_t)(t_last - t_first + 1);
         TilingTab* ttabs = ttabs_all + buf * shape.slots;
         OrderTab* otabs = otabs_all + (size_t)buf * shape.slots * n_orders;
-        for (uint32_t sl = lane; sl < n_slots; sl += 32) build_tiling_head(p, t_first + sl, &ttabs[sl]);
-        __syncwarp();
+        for (uint32_t sl = first; sl < n_slots; sl += step) build_tiling_head(p, t_first + sl, &ttabs[sl]);
+        sync();
         // subset products of the bounds: one lane per (slot, half, subset)
-        for (uint32_t it = lane; it < n_slots * 32u; it += 32) {
+        for (uint32_t it = first; it < n_slots * 32u; it += step) {
             TilingTab* tb = &ttabs[it >> 5];
             const uint32_t h = (it >> 4) & 1u, m = it & 15u;
             int64_t v = 1;
@@ -949,11 +958,11 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                 if (m >> d & 1u) v *= (int64_t)tb->b[h * 4 + d];
             tb->half[h][m] = v;
         }
-        __syncwarp();
+        sync();
         // Items are visited kind by kind, so that the 32 lanes always run the same code path.
         const uint32_t n_so = n_slots * n_orders;
         auto order_pass = [&](uint32_t first_item, uint32_t n_items) {
-            for (uint32_t it = lane; it < n_so * n_items; it += 32) {
+            for (uint32_t it = first; it < n_so * n_items; it += step) {
                 const uint32_t so = it / n_items, e = first_item + it % n_items;
                 const uint32_t slot = so / n_orders, os = so % n_orders;
                 if (!ttabs[slot].live) { fill_dead_order_item(&otabs[so], (int)e); continue; }
@@ -965,7 +974,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
         order_pass(15, 10);     // D, E
         order_pass(25, 1);      // C read-back (unfused)
         auto tiling_pass = [&](uint32_t first_item, uint32_t n_items) {
-            for (uint32_t it = lane; it < n_slots * n_items; it += 32) {
+            for (uint32_t it = first; it < n_slots * n_items; it += step) {
                 const uint32_t slot = it / n_items, e = first_item + it % n_items;
                 if (!ttabs[slot].live) { fill_dead_tiling_item(&ttabs[slot], (int)e); continue; }
                 build_tiling_item(p, &ttabs[slot], (int)e);
@@ -973,11 +982,11 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
         };
         tiling_pass(0, 18);     // stationary pairs x recompute flag
         tiling_pass(18, 3);     // unfused Op1 compute words
-        __syncwarp();
+        sync();
         if (OBJ == MMEE_OBJ_LATENCY) {
             // compute words relative to their minimum over the stationary pairs: fused without and with
             // recomputation, and Op2 of an unfused task
-            for (uint32_t j = lane; j < 3 * n_slots; j += 32) {
+            for (uint32_t j = first; j < 3 * n_slots; j += step) {
                 TilingTab* tb = &ttabs[j / 3];
                 const int v = (int)(j % 3);
                 const int64_t* src = v < 2 ? &tb->CB[0][v] : &tb->QU[0][0];
@@ -992,7 +1001,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
         }
         if (OBJ == MMEE_OBJ_ENERGY) {
             // threshold-relative stationary-pair terms (see "32-bit differential keys")
-            for (uint32_t j = lane; j < 2 * n_slots; j += 32) {
+            for (uint32_t j = first; j < 2 * n_slots; j += step) {
                 TilingTab* tb = &ttabs[j >> 1];
                 const int rc = (int)(j & 1);
                 int64_t m = tb->W[0][rc];
@@ -1007,14 +1016,14 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
         }
     };
 
-    if (builder) build_next(0);
+    build_next(0, std::true_type{});
     __syncthreads();
 
     for (int iter = 0;; ++iter) {
         const int buf = iter & 1;
         const uint64_t r0 = cs->range_begin[buf];
         if (r0 >= task_end) break;
-        if (builder) build_next(buf ^ 1);
+        if (builder) build_next(buf ^ 1, std::false_type{});
         {       // every warp walks tasks; the builder warp joins once the next range's tables are done
         const uint64_t r1 = (r0 + shape.range_tasks < task_end) ? r0 + shape.range_tasks : task_end;
         const uint64_t t_first = r0 / tpt;
