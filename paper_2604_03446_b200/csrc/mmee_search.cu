@@ -571,6 +571,54 @@ __device__ __noinline__ void exact_group(const Plan& p, const TilingTab* tb, con
     }
 }
 
+// The same for a single optimum (k = 1), without the insertion loop: every lane finds the best of its 45
+// candidates (ascending index, so the first of equal keys stays), the warp reduces those to the smallest
+// (key, idx) pair, and one lane replaces the list's entry if that pair precedes it.
+template <int OBJ>
+__device__ __noinline__ void exact_group_single(const Plan& p, const TilingTab* tb, const OrderTab* ot, uint32_t phi,
+                                                uint32_t la, uint32_t lb_task, int m, int d, bool live, uint32_t kept,
+                                                uint64_t task_first_idx, WarpTop* wt, CtaShared* cs, long long* global_g,
+                                                int lane) {
+    const MidExact me = mid_exact<OBJ>(p, tb, ot, phi, la, lb_task, m, live);
+    const RowTab* rt = &ot->rt[phi == 0 ? 0 : 1];
+    const int64_t s1 = me.slack1 - rt->D[d][0];
+    const int64_t s2 = me.slack2 - rt->D[d][1];
+    const int64_t xd = me.x0 + rt->D[d][2];
+    const int64_t xed = (OBJ >= MMEE_OBJ_EDP) ? me.xe0 + rt->D[d][3] : 0;
+    int64_t best = kInfKey;
+    uint32_t best_pos = 0;
+#pragma unroll 1
+    for (int e = 0; e < 5; ++e) {
+        const bool fit = (rt->E[e][0] <= s1) && (rt->E[e][1] <= s2) && ((kept >> (d * 5 + e)) & 1u);
+        const int64_t x = xd + rt->E[e][2];
+        const int64_t xe = (OBJ >= MMEE_OBJ_EDP) ? xed + rt->E[e][3] : 0;
+#pragma unroll
+        for (int s = 0; s < 9; ++s) {
+            const int64_t key = candidate_key<OBJ>(x, xe, me.wptr[2 * s], me.P[s / 3], me.qptr[2 * s], p.key_cap);
+            if (fit && key < best) { best = key; best_pos = (uint32_t)(e * 9 + s); }
+        }
+    }
+    uint64_t best_idx = task_first_idx + (uint64_t)(m * 225 + d * 45) + best_pos;
+    // a key above the CTA-wide bound cannot be the optimum; an infeasible or capped-out lane holds kInfKey > G
+    if (best > cs->G) { best = kInfKey; best_idx = UINT64_MAX; }
+#pragma unroll
+    for (int off = 16; off; off >>= 1) {
+        const int64_t ok = __shfl_xor_sync(kFull, best, off);
+        const uint64_t oi = __shfl_xor_sync(kFull, best_idx, off);
+        if (pair_less(ok, oi, best, best_idx)) { best = ok; best_idx = oi; }
+    }
+    if (lane == 0 && best != kInfKey && (wt->count == 0 || pair_less(best, best_idx, wt->key[0], wt->idx[0]))) {
+        wt->key[0] = best;
+        wt->idx[0] = best_idx;
+        wt->count = 1;
+        if (best < cs->G) {
+            atomicMin(&cs->G, (long long)best);
+            atomicMin(global_g, (long long)best);       // other CTAs pick it up at their next task
+        }
+    }
+    __syncwarp();
+}
+
 // The walk in 64-bit keys: the energy-delay product (double-precision filter, see edp_row_test),
 // the capped objectives and the key dump.  Returns the number of rows that fit.
 template <int OBJ, bool DUMP, bool PRUNE>
@@ -678,7 +726,8 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
             }
             rows += fits;
             if (__any_sync(kFull, hit_any != 0u)) {
-                exact_group<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, k, lane);
+                if (k == 1) exact_group_single<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, lane);
+                else exact_group<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, k, lane);
                 th = load_threshold(wt, cs, k);
                 refresh();
             }
@@ -870,7 +919,8 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
                 hit = __vimin3_s32(a0, a1, a2) < ((m * 225 + d * 45) >= strict_from ? -delta : 0);
             }
             if (__any_sync(kFull, hit)) {
-                exact_group<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, k, lane);
+                if (k == 1) exact_group_single<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, lane);
+                else exact_group<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, k, lane);
                 rebase();
                 mid_setup();
             }
