@@ -32,12 +32,14 @@ OBJ_NAMES = {0: "energy", 1: "latency", 2: "edp"}
 
 # Algorithmic integer work per mapping in the hoisted separable form of the model, counted in
 # thread-level 32-bit integer instructions.  Energy: one fused add-min per mapping (its key relative
-# to the threshold) plus, per row of 9 mappings, two capacity compares, the feasible count, the row
-# term and the feasibility select (5).  Latency: max + min per mapping plus 8 per row.  EDP (not
-# separable) is evaluated in double precision on the FP64 pipe, which has the same 64 lanes per SM:
-# add, two multiplies, two compares and a predicate OR per mapping (6) plus, per row, four
-# conversions, four 64-bit adds and the capacity test (15).
-ALG_OPS_PER_CANDIDATE = {0: 1.0 + 5.0 / 9.0, 1: 2.0 + 8.0 / 9.0, 2: 6.0 + 15.0 / 9.0}
+# to the threshold) plus, per row of 9 mappings, the row add, the capacity difference, its sign mask,
+# the masking multiply-add and the feasible count (5).  Latency: one fused add-max per mapping and
+# five 3-/2-input mins per row (14), plus the capacity difference, its sign mask, the masking
+# multiply-add and the feasible count (4).  EDP (not separable) is evaluated in double precision on
+# the FP64 pipe, which has the same 64 lanes per SM: add, two multiplies, two compares and a
+# predicate OR per mapping (6) plus, per row, four conversions, four 64-bit adds and the capacity
+# test (15).
+ALG_OPS_PER_CANDIDATE = {0: 1.0 + 5.0 / 9.0, 1: 2.0, 2: 6.0 + 15.0 / 9.0}
 INT_LANES_PER_SM = 64          # 4 sub-partitions x 16 integer-ALU lanes
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the exhaustive search kernels on the BERT workload,
 # from the ncu capture summarised under profiles/ (energy, latency); None for other workloads.
