@@ -11,11 +11,13 @@
 // shared-memory tables -- each entry an exact integer monomial already multiplied by its energy
 // coefficient -- and a candidate's key is a short sum of table entries.  The row loop evaluates
 // every candidate's key relative to the current top-k threshold in saturated 32-bit arithmetic
-// (one fused add-min per candidate for energy); exact 64-bit keys are formed only for rows that
-// can enter the list.  Nothing per candidate ever touches global memory.
+// (one fused add-min per candidate for energy, one fused add-max for latency); exact 64-bit keys
+// are formed only for groups of rows that can enter the list.  Nothing per candidate ever touches
+// global memory.
 //
-// CTAs are persistent and pull ranges of tasks from a global counter.  Seven warps walk tasks while
-// the eighth builds the tables of the next range into a second buffer.
+// CTAs are persistent and pull ranges of tasks from a global counter.  All warps build the tables
+// of a CTA's first range together; after that seven warps walk tasks while the eighth builds the
+// tables of the next range into a second buffer and then joins them.
 #include <cuda_runtime.h>
 
 #include <climits>
@@ -33,7 +35,6 @@ constexpr unsigned kFull = 0xffffffffu;
 constexpr int kModeSearch = 0, kModeDump = 1, kModePrune = 2;
 constexpr size_t kPlanBytes = (sizeof(Plan) + 15) / 16 * 16;
 static_assert(sizeof(Plan) % 4 == 0, "the plan is copied word by word");
-constexpr int kRelCap = (1 << 30) - 1;     // cap of a running threshold-relative sum (see below)
 constexpr int kTermCap = (1 << 28) - 1;    // cap of each non-negative addend of such a sum (at most six of them)
 constexpr int kSizeCap = (1 << 30) - 1;    // buffer sizes saturate here; the capacity is smaller
 constexpr int kUnfit = 1 << 30;            // added to the keys of a row that does not fit; also the lower clamp of a row sum
@@ -198,27 +199,29 @@ __device__ __forceinline__ void row_test(const int64_t (&k)[9], int64_t thr, int
 // ------------------------------------------------------------------------------------------------
 // 32-bit differential keys
 // ------------------------------------------------------------------------------------------------
-// Whether a candidate enters the top-k depends only on the sign of key - thr.  The row loop
-// therefore evaluates every candidate's key RELATIVE to the current threshold, saturated to 32
-// bits, and keeps the minimum over the group of five rows; a negative minimum sends the warp to
-// the exact 64-bit insertion path, which re-evaluates the rows in full.
+// Whether a candidate enters the top-k depends only on the sign of key - thr.  The row loops
+// therefore evaluate every candidate's key RELATIVE to the lane's current threshold, in saturated
+// 32-bit arithmetic, and keep the minimum over a group of five rows; a negative minimum sends the
+// warp to the exact 64-bit path, which re-evaluates the group in full.  The filter may flag a group
+// needlessly; it must never miss a candidate that passes.
 //
 // Energy: key = x + W[s].  With wmin = min_s W[s], B = thr - wmin and W' = W - wmin >= 0:
-// key < thr  <=>  u + vD + vE + W' < 0, where u = (task-level terms) - B and vD, vE >= 0 are the D- and
-// E-level terms.  u is saturated to [-2^31, 2^30 - 1], each of vD, vE, W' to [0, 2^29], and every
-// running sum is capped at 2^30 - 1: no 32-bit sum can overflow.  Saturation only lowers the
-// non-negative addends and raises u only when u < -2^31, where the saturated sum is at most
-// -2^31 + 3 * 2^29 < 0.  Hence, if a candidate of a row truly passes, the saturated sum of the row's
-// candidate with W' = 0 is negative and the row is flagged; a flagged row without a passing
-// candidate needs u < -2^29 next to a saturated addend, and costs one visit of the exact path.
-// So that addends do not saturate on large problems, all energy terms are kept in units of 2^rel_shift
-// quanta, rounded down (the plan picks the shift from the largest possible DRAM term); rounding down
-// can only lower a sum, so a passing candidate still yields a negative sum, and the rows flagged
-// needlessly are those within 3 * 2^rel_shift quanta above the threshold.
-// Latency: key = max(x + P, Q + P) and max(a, b) < thr <=> a - thr < 0 and b - thr < 0; the same
-// saturation is applied to x + P - thr = u + vD + vE.
+// key < thr  <=>  (gA + gX - B) + gB + vD + vE + W' < 0, the g / v terms being the DRAM energies of the
+// operands at their levels (gX: the C round trip of an unfused task).  All terms are kept in units of
+// 2^rel_shift quanta (the plan picks the shift from the largest possible DRAM term): every addend is
+// rounded down and capped at kTermCap, B is rounded up, so that the 32-bit sum is never above the
+// true one.  The task-level part (gA + gX - ceil(B / unit)) is clamped to [-kUnfit, kRowCap]; at most
+// four addends of at most kTermCap follow, 4 * kTermCap < kUnfit, so a sum that was clamped from below
+// stays negative (the group is flagged, which is the safe side), and no 32-bit sum overflows:
+// kRowCap + 2 * kTermCap + kUnfit < 2^31.  Most terms are multiples of the unit, so that a tie with
+// the list's last entry is still told from a better key: groups whose indices lie above that entry
+// use the threshold thr - 1.
+// Latency: key = P + max(x, Q[s]) (P: the Op1 stage of an unfused task, else 0), and
+// max(a, b) < thr  <=>  a - thr < 0 and b - thr < 0.  a = (x0 + P - thr) + vD + vE with the same
+// clamping; b = (Q[s] - qmin) + (qmin + P - thr), the first part a table entry capped at kTermCap.
 // Capacity (Eq. 4): sizes are saturated to kSizeCap, which is above every admissible capacity, so
-// "size <= slack" keeps its truth value in 32 bits.
+// "size <= slack" keeps its truth value in 32 bits.  A row that does not fit has kUnfit added to its
+// keys, which makes them non-negative whatever the threshold.
 // Integer multiply-add and arithmetic shift as single PTX instructions, opaque to the optimiser: the row
 // loops use them to keep additions on the FMA pipe and sign masks out of compare-and-select form.
 __device__ __forceinline__ int imad(int a, int b, int c) {
