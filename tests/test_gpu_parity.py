@@ -134,6 +134,34 @@ def test_search_matches_the_oracle_on_tiny_problems(seed, k):
         check_search(cfg, obj)
 
 
+@pytest.mark.parametrize("seed", TINY_SEEDS[:6])
+@pytest.mark.parametrize("log2_quantum", [-12, -24])
+def test_energy_search_in_coarse_relative_units(seed, log2_quantum):
+    """The energy walk keeps threshold-relative keys in units of 2^rel_shift quanta once the largest DRAM term
+    leaves 28 bits.  A small energy quantum (a power of two, so that every energy stays an integer multiple)
+    drives small problems into that regime and, at 2^-24 pJ, into saturated stationary-pair terms; the top-16,
+    the optimum and the feasible count must still be the oracle's."""
+    cfg = mi.random_tiny_problem(seed)
+    arch = dict(cfg["arch"], energy_quantum_pj=2.0 ** log2_quantum)
+    cfg = dict(cfg, arch=arch)
+    for k in (1, 16):
+        obj = shrink(cfg, dict(cfg["searches"][0], objective=mi.OBJ_ENERGY, topk=k), 6_000_000)
+        check_search(cfg, obj)
+
+
+@pytest.mark.parametrize("seed", TINY_SEEDS[:6])
+def test_search_with_the_largest_admissible_buffer(seed):
+    """Capacities just below 2^30 words (the documented maximum): no size saturates below the capacity, every
+    mapping fits, and the 32-bit capacity arithmetic of the walk must not overflow."""
+    cfg = mi.random_tiny_problem(seed)
+    wb = cfg["workload"]["word_bytes"]
+    cfg = dict(cfg, arch=dict(cfg["arch"], gb_bytes=((1 << 30) - 2) * wb))
+    for objective in (mi.OBJ_ENERGY, mi.OBJ_LATENCY):
+        obj = shrink(cfg, dict(cfg["searches"][0], objective=objective, topk=4), 4_000_000)
+        best, _ = check_search(cfg, obj)
+        assert best.n_feasible == best.n_total
+
+
 def test_config1_full_search():
     cfg = mi.config1()
     best, _ = check_search(cfg, cfg["searches"][0])
