@@ -821,7 +821,10 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
         y1 = __viaddmin_s32(y1, cv.x, kSizeCap);
         int y2 = __viaddmin_s32(a2c, fused ? bv.y : 0, kSizeCap);
         y2 = __viaddmin_s32(y2, cv.x, kSizeCap);
-        const int slack1c = live ? max(capc - y1, -1) : -1;       // a lane without a live task: none of its rows fits
+        // (a lane without a live task: none of its rows fits.)  D and E of an unfused task take no space while
+        // Op1 runs: its first slack only has to be non-negative, and is made large so that min(s1, s2) = s2 below.
+        const int room1 = capc - y1;
+        const int slack1c = live ? (fused ? max(room1, -1) : (room1 >= 0 ? kSizeCap : -1)) : -1;
         const int slack2c = live ? max(capc - y2, -1) : -1;
 
         int u = 0, u_strict = 0, Wc[9], ua[3], Qc[9];
@@ -860,9 +863,9 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
                 }
                 const int4* q4 = reinterpret_cast<const int4*>(qrel);
                 const int4 q0 = q4[0], q1 = q4[1], q2 = q4[2];
-                Qc[0] = q0.x + qo[0]; Qc[1] = q0.y + qo[0]; Qc[2] = q0.z + qo[0];
-                Qc[3] = q0.w + qo[1]; Qc[4] = q1.x + qo[1]; Qc[5] = q1.y + qo[1];
-                Qc[6] = q1.z + qo[2]; Qc[7] = q1.w + qo[2]; Qc[8] = q2.x + qo[2];
+                Qc[0] = imad(qo[0], one, q0.x); Qc[1] = imad(qo[0], one, q0.y); Qc[2] = imad(qo[0], one, q0.z);
+                Qc[3] = imad(qo[1], one, q0.w); Qc[4] = imad(qo[1], one, q1.x); Qc[5] = imad(qo[1], one, q1.y);
+                Qc[6] = imad(qo[2], one, q1.z); Qc[7] = imad(qo[2], one, q1.w); Qc[8] = imad(qo[2], one, q2.x);
             }
         };
         mid_setup();
@@ -874,14 +877,14 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
             }
             // Five rows (levels of E) are evaluated branch-free; one vote decides whether any lane of the
             // warp has to enter the exact path for this group.
-            ++groups;
+            if constexpr (PRUNE) ++groups;
             const int4 dc = *reinterpret_cast<const int4*>(rt->Dc[d]);
-            const int s1c = slack1c - dc.x;
-            const int s2c = slack2c - dc.y;
+            const int s1c = imad(dc.x, minus_one, slack1c);
+            const int s2c = imad(dc.y, minus_one, slack2c);
             // Eq. (4) for the five levels of E: at L3, and in an unfused task, E takes no space while Op1
             // runs (size <= s2c, given s1c >= 0); retained, it must fit beside both operators' operands
             const int lim_l3 = s1c >= 0 ? s2c : -1;
-            const int lim_retained = fused ? min(s1c, s2c) : lim_l3;
+            const int lim_retained = min(s1c, s2c);
             const uint32_t kd = kept >> (d * 5);
             int a0 = INT_MAX, a1 = INT_MAX, a2 = INT_MAX;
             bool hit;
@@ -929,6 +932,7 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
             }
         }
     }
+    if constexpr (!PRUNE) groups = 25;
     return (uint32_t)((int)(groups * 5u) + unfit);
 }
 
