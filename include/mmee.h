@@ -101,6 +101,11 @@ typedef struct {
     uint64_t t_begin, t_end;                 /* tiling sub-range [t_begin,t_end); 0,0 = all       */
     int64_t  key_cap;                        /* MMEE_OBJ_*CAP: bound on the other key (energy in quanta,
                                                 latency in words); ignored otherwise                   */
+    uint32_t stationary_mask;                /* bit 3*sm1+sm2 set: the array offers that stationary pair
+                                                (Section VII-K: a fixed array offers one, a reconfigurable
+                                                one several); 0 = all nine.  A mapping with another pair
+                                                is outside the space: never selected, not in n_feasible */
+    uint32_t reserved;                       /* 0 */
 } mmee_objective_t;
 
 /* One fully evaluated mapping.  Counts are per instance. */
@@ -123,7 +128,7 @@ typedef struct {
     double   energy_pj;                      /* e_key * quantum * instances                       */
     double   latency_cycles;                 /* l_key / words_per_cycle * ceil(instances/n_arrays) */
     uint64_t n_total;                        /* candidates of the searched range (in out_best)    */
-    uint64_t n_feasible;                     /* of which fit the buffer (in out_best)             */
+    uint64_t n_feasible;                     /* of which fit the buffer, with an offered stationary pair (in out_best) */
 } mmee_result_t;
 
 typedef struct mmee_handle mmee_handle_t;
@@ -236,6 +241,22 @@ int mmee_solve_host(const mmee_workload_t* workload, const mmee_arch_t* arch,
 int mmee_pareto_front(const mmee_workload_t* workload, const mmee_arch_t* arch,
                       const mmee_objective_t* objective, mmee_result_t* out_points, uint32_t capacity,
                       uint32_t* n_points);
+
+/*
+ * mmee_search_shapes -- reconfigurable PE arrays (Section VII-K): the same search on each of several logical
+ * array shapes (the stationary modes the array can switch between are objective.stationary_mask), one device
+ * search per shape, and the shape whose optimum has the least key.  arch.pe_rows / pe_cols are replaced by each
+ * shape in turn; everything else is as given.  Synchronous.
+ *   shapes      : HOST, n_shapes pairs (rows, cols), each >= 1.
+ *   out_per_shape : HOST, n_shapes records: the optimum on that shape (idx = MMEE_NO_INDEX, status
+ *                   MMEE_ERR_NO_FEASIBLE when nothing fits; n_total / n_feasible of that search).
+ *   out_best_shape : HOST, index of the shape with the least key (the objective's; the first of equal ones),
+ *                    UINT32_MAX when no shape has a feasible mapping.
+ * objective.topk and .row_pruning are ignored (one optimum per shape, exhaustive).
+ */
+int mmee_search_shapes(const mmee_workload_t* workload, const mmee_arch_t* arch,
+                       const mmee_objective_t* objective, const uint32_t* shapes, uint32_t n_shapes,
+                       mmee_result_t* out_per_shape, uint32_t* out_best_shape);
 
 /*
  * mmee_query_vector -- HOST only, no device needed.  The query vector q in {0,1}^8 over

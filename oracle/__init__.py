@@ -40,7 +40,7 @@ class Arch(C.Structure):
 
 class Objective(C.Structure):
     _fields_ = [("objective", C.c_uint32), ("topk", C.c_uint32), ("tiling_set", C.c_uint32),
-                ("order_set", C.c_uint32), ("fuse_mask", C.c_uint32),
+                ("order_set", C.c_uint32), ("fuse_mask", C.c_uint32), ("stationary_mask", C.c_uint32),
                 ("t_begin", C.c_uint64), ("t_end", C.c_uint64)]
 
 
@@ -54,7 +54,8 @@ class Problem(C.Structure):
                 ("cq_mac", C.c_int64), ("cq_sfu", C.c_int64), ("quantum_pj", C.c_double),
                 ("has_rf", C.c_int), ("cap_words", C.c_uint64),
                 ("pe_rows", C.c_uint32), ("pe_cols", C.c_uint32), ("n_arrays", C.c_uint32),
-                ("bw", C.c_uint32), ("objective", C.c_uint32), ("topk", C.c_uint32)]
+                ("bw", C.c_uint32), ("objective", C.c_uint32), ("topk", C.c_uint32),
+                ("stationary_mask", C.c_uint32)]
 
 
 class Record(C.Structure):

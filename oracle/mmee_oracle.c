@@ -69,6 +69,7 @@ int mo_problem_init(const mo_workload* w, const mo_arch* a, const mo_objective* 
     if (o->objective > MO_OBJ_EDP || o->topk < 1 || o->topk > MO_MAX_TOPK) return MO_ERR_ARG;
     if (o->tiling_set > MO_TILE_ALL_DIVISORS || o->order_set > MO_ORD_ALL6) return MO_ERR_ARG;
     if ((o->fuse_mask & 7u) == 0 || (o->fuse_mask & ~7u)) return MO_ERR_ARG;
+    if (o->stationary_mask & ~0x1ffu) return MO_ERR_ARG;
 
     /* Heads are independent instances (Section V, "we omit the head dimension"); the g query
      * heads that share one K/V head are stacked along I, so K and V are loaded once per group. */
@@ -124,6 +125,7 @@ int mo_problem_init(const mo_workload* w, const mo_arch* a, const mo_objective* 
     p->pe_rows = a->pe_rows; p->pe_cols = a->pe_cols; p->n_arrays = a->n_arrays;
     p->bw = a->dram_words_per_cycle;
     p->objective = o->objective; p->topk = o->topk;
+    p->stationary_mask = o->stationary_mask ? o->stationary_mask : 0x1ffu;
 
     /* Worst-case key bound.  With M = I*L*J*(K+1) >= the largest MAC count (recomputation factor
      * at most J): every DRAM term is at most I*K*L*J <= M and there are at most 7 of them; array
@@ -379,7 +381,8 @@ int mo_eval(const mo_problem* p, uint64_t idx, mo_record* o)
     o->n[3] = (int64_t)n_mac;  o->n[4] = (int64_t)n_sfu;
     o->e_key = (int64_t)e_key; o->l_key = (int64_t)l_key;
     o->recompute = (uint32_t)rc_flag;
-    o->feasible = bsmax <= (i128)p->cap_words;
+    /* in the space iff it fits the buffer (Eq. 4) and the array offers its stationary pair (Section VII-K) */
+    o->feasible = bsmax <= (i128)p->cap_words && ((p->stationary_mask >> (3u * o->sm[0] + o->sm[1])) & 1u);
 
     volatile double ek = (double)o->e_key, lk = (double)o->l_key;   /* one IEEE multiply, no FMA */
     o->edp_key = ek * lk;

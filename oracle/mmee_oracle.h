@@ -51,6 +51,8 @@ typedef struct {
 
 typedef struct {
     uint32_t objective, topk, tiling_set, order_set, fuse_mask;
+    uint32_t stationary_mask;              /* bit 3*sm1+sm2 set: that stationary pair is in the space; 0 = all nine
+                                              (a reconfigurable array offers several, a fixed one a single pair) */
     uint64_t t_begin, t_end;
 } mo_objective;
 
@@ -72,6 +74,7 @@ typedef struct {
     uint64_t cap_words;                    /* floor(gb_bytes / word_bytes)          */
     uint32_t pe_rows, pe_cols, n_arrays, bw;
     uint32_t objective, topk;
+    uint32_t stationary_mask;              /* never 0 */
 } mo_problem;
 
 typedef struct {
@@ -108,7 +111,7 @@ int  mo_problem_init(const mo_workload*, const mo_arch*, const mo_objective*, mo
 int  mo_eval(const mo_problem*, uint64_t idx, mo_record* out);
 int  mo_eval_range(const mo_problem*, uint64_t begin, uint64_t count, mo_record* out);
 /* key as the search orders it: int64 for energy/latency, IEEE bits of the product for EDP;
- * feasible[i] = 1 iff the candidate fits the global buffer. */
+ * feasible[i] = 1 iff the candidate fits the global buffer and its stationary pair is in the space. */
 int  mo_keys_range(const mo_problem*, uint64_t begin, uint64_t count, int64_t* keys, uint8_t* feasible);
 /* k smallest (key, idx) among feasible candidates of tilings [t_begin, t_end); out_topk has topk
  * entries, unused ones carry idx = UINT64_MAX.  n_threads <= 0: all cores. */

@@ -20,7 +20,7 @@ NO_INDEX = 2 ** 64 - 1
 OK, ERR_ARG, ERR_OVERFLOW, ERR_QUANTUM, ERR_NO_FEASIBLE, ERR_CUDA, ERR_TIMEOUT, ERR_RANGE = range(8)
 
 EXPORTS = ("mmee_create", "mmee_search", "mmee_destroy", "mmee_search_static", "mmee_num_candidates", "mmee_num_tilings",
-           "mmee_num_rows", "mmee_strerror", "mmee_last_cuda_error", "mmee_eval", "mmee_dump_keys", "mmee_solve_host", "mmee_pareto_front",
+           "mmee_num_rows", "mmee_strerror", "mmee_last_cuda_error", "mmee_eval", "mmee_dump_keys", "mmee_solve_host", "mmee_pareto_front", "mmee_search_shapes",
            "mmee_query_vector", "mmee_recompute_flag", "mmee_row_pruning_keep", "mmee_last_search_stats", "mmee_kernel_timing",
            "mmee_alu_peak")
 
@@ -42,7 +42,8 @@ class Arch(C.Structure):
 class Objective(C.Structure):
     _fields_ = [("objective", C.c_uint32), ("topk", C.c_uint32), ("tiling_set", C.c_uint32),
                 ("order_set", C.c_uint32), ("fuse_mask", C.c_uint32), ("row_pruning", C.c_uint32),
-                ("t_begin", C.c_uint64), ("t_end", C.c_uint64), ("key_cap", C.c_int64)]
+                ("t_begin", C.c_uint64), ("t_end", C.c_uint64), ("key_cap", C.c_int64),
+                ("stationary_mask", C.c_uint32), ("reserved", C.c_uint32)]
 
 
 class Result(C.Structure):
@@ -114,6 +115,8 @@ def library():
                                   C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
     L.mmee_pareto_front.argtypes = [C.POINTER(Workload), C.POINTER(Arch), C.POINTER(Objective),
                                     C.POINTER(Result), C.c_uint32, C.POINTER(C.c_uint32)]
+    L.mmee_search_shapes.argtypes = [C.POINTER(Workload), C.POINTER(Arch), C.POINTER(Objective),
+                                     C.POINTER(C.c_uint32), C.c_uint32, C.POINTER(Result), C.POINTER(C.c_uint32)]
     L.mmee_query_vector.argtypes = [C.c_uint32] * 6 + [C.POINTER(C.c_uint8)]
     L.mmee_recompute_flag.argtypes = [C.c_uint32, C.c_uint32, C.POINTER(C.c_uint32)]
     L.mmee_row_pruning_keep.argtypes = [C.POINTER(Objective), C.POINTER(C.c_uint8), C.c_uint32,
@@ -219,6 +222,17 @@ def mmee_pareto_front(workload: dict, arch: dict, objective: dict, capacity: int
                                        _fill(Objective(), objective), pts, capacity, C.byref(n)),
            "mmee_pareto_front")
     return list(pts[:n.value])
+
+
+def mmee_search_shapes(workload: dict, arch: dict, objective: dict, shapes):
+    """One search per logical array shape (rows, cols): (list of Result per shape, index of the best shape or None)."""
+    n = len(shapes)
+    flat = (C.c_uint32 * (2 * n))(*[v for rc in shapes for v in rc])
+    out = (Result * n)()
+    best = C.c_uint32()
+    _check(library().mmee_search_shapes(_fill(Workload(), workload), _fill(Arch(), arch), _fill(Objective(), objective),
+                                        flat, n, out, C.byref(best)), "mmee_search_shapes")
+    return list(out), (None if best.value == 2 ** 32 - 1 else best.value)
 
 
 def mmee_query_vector(metric: int, phi: int, pi: int, operand: int, beta: int, recompute: int = 0):

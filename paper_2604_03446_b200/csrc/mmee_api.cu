@@ -261,6 +261,45 @@ int mmee_pareto_front(const mmee_workload_t* workload, const mmee_arch_t* arch, 
     return rc;
 }
 
+int mmee_search_shapes(const mmee_workload_t* workload, const mmee_arch_t* arch, const mmee_objective_t* objective,
+                       const uint32_t* shapes, uint32_t n_shapes, mmee_result_t* out_per_shape,
+                       uint32_t* out_best_shape) {
+    if (!arch || !objective || !shapes || !n_shapes || !out_per_shape || !out_best_shape) return MMEE_ERR_ARG;
+    *out_best_shape = UINT32_MAX;
+    mmee_objective_t o = *objective;
+    o.topk = 1;
+    o.row_pruning = 0;
+    mmee_result_t* dev = nullptr;
+    if (cudaMalloc(reinterpret_cast<void**>(&dev), sizeof(mmee_result_t)) != cudaSuccess) return MMEE_ERR_CUDA;
+    int rc = MMEE_OK;
+    bool have = false;
+    int64_t best_key = 0;
+    for (uint32_t i = 0; i < n_shapes && rc == MMEE_OK; ++i) {
+        mmee_arch_t a = *arch;
+        a.pe_rows = shapes[2 * i];
+        a.pe_cols = shapes[2 * i + 1];
+        mmee_handle_t* h = nullptr;
+        if ((rc = mmee_create(workload, &a, &o, &h))) break;
+        rc = mmee_search(h, nullptr, dev, nullptr);
+        if (rc == MMEE_OK)
+            rc = cuda_status(cudaMemcpy(&out_per_shape[i], dev, sizeof(mmee_result_t), cudaMemcpyDeviceToHost));
+        const int rc2 = mmee_destroy(h);
+        if (rc == MMEE_OK) rc = rc2;
+        if (rc != MMEE_OK || out_per_shape[i].idx == MMEE_NO_INDEX) continue;
+        const mmee_result_t& r = out_per_shape[i];
+        // the key the search ordered by: energy, latency, or the bit pattern of the positive EDP product
+        int64_t key;
+        switch (o.objective) {
+            case MMEE_OBJ_ENERGY: case MMEE_OBJ_ENERGY_LCAP: key = r.e_key; break;
+            case MMEE_OBJ_LATENCY: case MMEE_OBJ_LATENCY_ECAP: key = r.l_key; break;
+            default: std::memcpy(&key, &r.edp_key, sizeof(key)); break;
+        }
+        if (!have || key < best_key) { have = true; best_key = key; *out_best_shape = i; }
+    }
+    cudaFree(dev);
+    return rc;
+}
+
 int mmee_query_vector(uint32_t metric, uint32_t phi, uint32_t pi, uint32_t operand, uint32_t beta,
                       uint32_t recompute, uint8_t out_q[8]) {
     if (!out_q || metric > 1 || phi > 2 || pi > 5 || operand > 4 || beta < 3 || beta > 7 || recompute > 1)

@@ -191,7 +191,7 @@ __device__ inline void evaluate_candidate(const Plan& p, uint64_t idx, mmee_resu
     o.n[0] = n_dram; o.n[1] = n_gb; o.n[2] = n_rf; o.n[3] = n_mac; o.n[4] = n_sfu;
     o.e_key = e_key; o.l_key = l_key;
     o.recompute = (uint8_t)rc;
-    o.feasible = (uint8_t)(o.bs <= p.cap_words);
+    o.feasible = (uint8_t)(o.bs <= p.cap_words && ((p.sm_mask >> s) & 1u));
     o.edp_key = __dmul_rn((double)e_key, (double)l_key);
     o.energy_pj = __dmul_rn(__dmul_rn((double)e_key, p.quantum_pj), (double)p.instances);
     const uint32_t waves = (p.instances + p.n_arrays - 1) / p.n_arrays;

@@ -50,6 +50,7 @@ struct Plan {
     uint32_t bw, pe_rows, pe_cols;
     uint32_t objective, topk;
     uint32_t row_pruning;
+    uint32_t sm_mask, n_sm;       // stationary pairs in the space (bit s = 3*sm1+sm2; never 0) and their number
     int64_t  key_cap;             // capped objectives: bound on the other key
     uint32_t rel_shift;           // energy: threshold-relative keys are kept in units of 2^rel_shift quanta
     int32_t  unit;                // the constant 1, as a run-time value: x * unit + y is issued as an integer

@@ -287,13 +287,13 @@ __device__ __forceinline__ unsigned edp_row_test(double de, const double (&dl)[3
 template <int OBJ>
 __device__ __noinline__ int64_t slow_row(WarpTop* wt, CtaShared* cs, long long* global_g, int k, int lane, bool f,
                                          int64_t x, int64_t xe, const int64_t* wptr, const int64_t* qptr,
-                                         int64_t p0, int64_t p1, int64_t p2, int64_t cap,
+                                         int64_t p0, int64_t p1, int64_t p2, int64_t cap, uint32_t sm_mask,
                                          uint64_t row_first_idx) {
     int64_t thr = lane_threshold(wt, cs, k, row_first_idx);
     for (int s = 0; s < 9; ++s) {
         const int64_t pp = s < 3 ? p0 : (s < 6 ? p1 : p2);
         const int64_t key = candidate_key<OBJ>(x, xe, wptr[2 * s], pp, qptr[2 * s], cap);
-        bool pend = f && key < thr;
+        bool pend = f && ((sm_mask >> s) & 1u) && key < thr;
         while (true) {
             const unsigned m = __ballot_sync(kFull, pend);
             if (!m) break;
@@ -567,10 +567,11 @@ __device__ __noinline__ void exact_group(const Plan& p, const TilingTab* tb, con
         const int64_t thr_row = lane_threshold(wt, cs, k, row_first_idx);
         bool below = false;
         for (int s = 0; s < 9; ++s)
-            below |= candidate_key<OBJ>(x, xe, me.wptr[2 * s], me.P[s / 3], me.qptr[2 * s], p.key_cap) < thr_row;
+            below |= ((p.sm_mask >> s) & 1u) &&
+                     candidate_key<OBJ>(x, xe, me.wptr[2 * s], me.P[s / 3], me.qptr[2 * s], p.key_cap) < thr_row;
         if (__any_sync(kFull, fit && below))
             slow_row<OBJ>(wt, cs, global_g, k, lane, fit, x, xe, me.wptr, me.qptr, me.P[0], me.P[1], me.P[2], p.key_cap,
-                          row_first_idx);
+                          p.sm_mask, row_first_idx);
     }
 }
 
@@ -598,7 +599,7 @@ __device__ __noinline__ void exact_group_single(const Plan& p, const TilingTab* 
 #pragma unroll
         for (int s = 0; s < 9; ++s) {
             const int64_t key = candidate_key<OBJ>(x, xe, me.wptr[2 * s], me.P[s / 3], me.qptr[2 * s], p.key_cap);
-            if (fit && key < best) { best = key; best_pos = (uint32_t)(e * 9 + s); }
+            if (fit && ((p.sm_mask >> s) & 1u) && key < best) { best = key; best_pos = (uint32_t)(e * 9 + s); }
         }
     }
     uint64_t best_idx = task_first_idx + (uint64_t)(m * 225 + d * 45) + best_pos;
@@ -654,7 +655,8 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
         if constexpr (OBJ == MMEE_OBJ_EDP) {
 #pragma unroll
             for (int s = 0; s < 9; ++s) {
-                dW[s] = (double)W[s];
+                // (a pair the array does not offer: infinite energy, flagged at most while no bound exists yet)
+                dW[s] = ((p.sm_mask >> s) & 1u) ? (double)W[s] : __longlong_as_double(0x7ff0000000000000ll);
                 dQP[s] = (double)(Q[s] + me.P[s / 3]);
             }
         }
@@ -712,7 +714,8 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
                     const int64_t xe = (OBJ >= MMEE_OBJ_EDP) ? xed + rt->E[e][3] : 0;
                     int64_t key[9];
 #pragma unroll
-                    for (int s = 0; s < 9; ++s) key[s] = candidate_key<OBJ>(x, xe, W[s], me.P[s / 3], Q[s], p.key_cap);
+                    for (int s = 0; s < 9; ++s)
+                        key[s] = ((p.sm_mask >> s) & 1u) ? candidate_key<OBJ>(x, xe, W[s], me.P[s / 3], Q[s], p.key_cap) : kInfKey;
                     unsigned fit, hit;
                     row_test(key, thr, rt->E[e][0], s1, rt->E[e][1], s2, fit, hit);
                     if constexpr (PRUNE) { fit &= kept >> (d * 5 + e); hit &= fit; }
@@ -866,6 +869,11 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
                 Qc[0] = imad(qo[0], one, q0.x); Qc[1] = imad(qo[0], one, q0.y); Qc[2] = imad(qo[0], one, q0.z);
                 Qc[3] = imad(qo[1], one, q0.w); Qc[4] = imad(qo[1], one, q1.x); Qc[5] = imad(qo[1], one, q1.y);
                 Qc[6] = imad(qo[2], one, q1.z); Qc[7] = imad(qo[2], one, q1.w); Qc[8] = imad(qo[2], one, q2.x);
+                if (p.sm_mask != 0x1ffu) {       // a stationary pair the array does not offer never passes
+#pragma unroll
+                    for (int s = 0; s < 9; ++s)
+                        if (!((p.sm_mask >> s) & 1u)) Qc[s] = kRowCap;
+                }
             }
         };
         mid_setup();
@@ -1047,12 +1055,13 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                 TilingTab* tb = &ttabs[j / 3];
                 const int v = (int)(j % 3);
                 const int64_t* src = v < 2 ? &tb->CB[0][v] : &tb->QU[0][0];
-                int64_t m = src[0];
-                for (int s = 1; s < 9; ++s) m = src[2 * s] < m ? src[2 * s] : m;
+                int64_t m = kInfKey;       // over the stationary pairs the array offers (never none)
+                for (int s = 0; s < 9; ++s)
+                    if ((p.sm_mask >> s) & 1u) m = src[2 * s] < m ? src[2 * s] : m;
                 tb->qmin[v] = m;
                 for (int s = 0; s < 9; ++s) {
                     const int64_t qd = src[2 * s] - m;
-                    tb->Qrel[v][s] = qd > (int64_t)kTermCap ? kTermCap : (int32_t)qd;
+                    tb->Qrel[v][s] = (qd > (int64_t)kTermCap || !((p.sm_mask >> s) & 1u)) ? kTermCap : (int32_t)qd;
                 }
             }
         }
@@ -1061,13 +1070,16 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
             for (uint32_t j = first; j < 2 * n_slots; j += step) {
                 TilingTab* tb = &ttabs[j >> 1];
                 const int rc = (int)(j & 1);
-                int64_t m = tb->W[0][rc];
-                for (int s = 1; s < 9; ++s) m = tb->W[s][rc] < m ? tb->W[s][rc] : m;
+                // The minimum runs over the stationary pairs the array offers (never none).  A pair it does not
+                // offer gets the largest term: the row's minimum over s is then still that of an offered pair.
+                int64_t m = kInfKey;
+                for (int s = 0; s < 9; ++s)
+                    if ((p.sm_mask >> s) & 1u) m = tb->W[s][rc] < m ? tb->W[s][rc] : m;
                 tb->wmin[rc] = m;
                 for (int s = 0; s < 9; ++s) {
                     const int64_t wd = tb->W[s][rc] - m;
                     const int64_t ws = wd >> p.rel_shift;
-                    tb->Wc[rc][s] = ws > (int64_t)kTermCap ? kTermCap : (int32_t)ws;
+                    tb->Wc[rc][s] = (ws > (int64_t)kTermCap || !((p.sm_mask >> s) & 1u)) ? kTermCap : (int32_t)ws;
                 }
             }
         }
@@ -1190,7 +1202,7 @@ finalize_kernel(const __grid_constant__ Plan p, Scratch* __restrict__ scratch, i
         }
         const int found = wt->count;
         const uint64_t n_total = (p.t_end - p.t_begin) * (uint64_t)p.rows_per_tiling * 9u;
-        const uint64_t n_feasible = scratch->feasible_rows * 9ull;
+        const uint64_t n_feasible = scratch->feasible_rows * (uint64_t)p.n_sm;
         if (lane < k) {
             mmee_result_t r;
             if (lane < found) {

@@ -162,6 +162,64 @@ def test_search_with_the_largest_admissible_buffer(seed):
         assert best.n_feasible == best.n_total
 
 
+@pytest.mark.parametrize("seed", TINY_SEEDS[:8])
+def test_search_over_a_subset_of_stationary_pairs(seed):
+    """Arrays that offer only some stationary pairs (Section VII-K): every objective, k = 1 and 16, masks from a
+    single pair to eight of nine; optimum, top-k, records and the feasible count against the oracle."""
+    cfg = mi.random_tiny_problem(seed)
+    masks = [1 << (seed % 9), 0x1ff ^ (1 << ((3 * seed) % 9)), (0x0a5 << (seed % 2)) & 0x1ff, 0x007, 0x049]
+    for i, mask in enumerate(masks):
+        objective = (mi.OBJ_ENERGY, mi.OBJ_LATENCY, mi.OBJ_EDP)[(seed + i) % 3]
+        for k in (1, 16):
+            obj = shrink(cfg, dict(cfg["searches"][0], objective=objective, topk=k, stationary_mask=mask), 4_000_000)
+            _, found = check_search(cfg, obj)
+            assert all((mask >> (3 * r.sm[0] + r.sm[1])) & 1 for r in found)
+
+
+def test_every_key_with_a_stationary_mask():
+    """The key dump under a mask: INT64_MAX for the pairs the array does not offer, the oracle's key elsewhere."""
+    cfg = mi.random_tiny_problem(4)
+    for objective, mask in ((mi.OBJ_ENERGY, 0x124), (mi.OBJ_LATENCY, 0x00f), (mi.OBJ_EDP, 0x180)):
+        obj = shrink(cfg, dict(cfg["searches"][0], objective=objective, stationary_mask=mask), 2_000_000)
+        p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
+        begin, count = p.t_begin * p.R * 9, (p.t_end - p.t_begin) * p.R * 9
+        keys, feas = oracle.keys_range(p, begin, count)
+        want = np.where(feas.astype(bool), keys, np.iinfo(np.int64).max)
+        got = torch.empty(count, dtype=torch.int64, device="cuda")
+        with Handle(cfg, obj) as h:
+            mm.mmee_dump_keys(h, got)
+            torch.cuda.synchronize()
+        assert np.array_equal(got.cpu().numpy(), want)
+
+
+def test_search_shapes_picks_the_best_logical_array():
+    """Reconfigurable array shapes (Section VII-K): one search per shape, each equal to the oracle's search on that
+    shape, and the index of the shape with the least key; for the four designs of the paper's comparison
+    (fixed pair on one shape, free pairs, free shape, both) more freedom is never worse."""
+    cfg = mi.random_tiny_problem(6)
+    shapes = [(4, 4), (2, 8), (8, 2), (1, 16), (16, 1)]
+    best_key = {}
+    for name, mask, shp in (("fixed", 0x001, shapes[:1]), ("flow", 0x1ff, shapes[:1]),
+                            ("shape", 0x001, shapes), ("shape_flow", 0x1ff, shapes)):
+        obj = shrink(cfg, dict(cfg["searches"][0], objective=mi.OBJ_EDP, topk=1, stationary_mask=mask), 3_000_000)
+        per_shape, best = mm.mmee_search_shapes(cfg["workload"], cfg["arch"], obj, shp)
+        want = []
+        for (r, c), got in zip(shp, per_shape):
+            arch = dict(cfg["arch"], pe_rows=r, pe_cols=c)
+            res = oracle.search(oracle.make_problem(cfg["workload"], arch, obj))
+            assert got.n_feasible == res.n_feasible
+            if res.topk:
+                assert_same_record(got, res.topk[0], name)
+                want.append(res.topk[0].edp_key)
+            else:
+                assert got.idx == mm.NO_INDEX
+                want.append(float("inf"))
+        assert best == (None if min(want) == float("inf") else want.index(min(want)))
+        best_key[name] = min(want)
+    assert best_key["shape_flow"] <= best_key["shape"] <= best_key["fixed"]
+    assert best_key["shape_flow"] <= best_key["flow"] <= best_key["fixed"]
+
+
 def test_config1_full_search():
     cfg = mi.config1()
     best, _ = check_search(cfg, cfg["searches"][0])

@@ -83,7 +83,8 @@ def test_argument_errors_come_before_any_device_call():
         assert e.value.code == mm.ERR_ARG
     for bad_o, code in ((dict(o, fuse_mask=0), mm.ERR_ARG), (dict(o, topk=0), mm.ERR_ARG),
                         (dict(o, topk=17), mm.ERR_RANGE), (dict(o, objective=5), mm.ERR_ARG), (dict(o, objective=3, key_cap=-1), mm.ERR_ARG),
-                        (dict(o, t_begin=5, t_end=2), mm.ERR_ARG)):
+                        (dict(o, t_begin=5, t_end=2), mm.ERR_ARG), (dict(o, stationary_mask=0x200), mm.ERR_ARG),
+                        (dict(o, reserved=1), mm.ERR_ARG)):
         with pytest.raises(mm.MmeeError) as e:
             mm.mmee_create(w, a, bad_o)
         assert e.value.code == code

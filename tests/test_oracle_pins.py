@@ -236,6 +236,37 @@ def test_search_is_the_sorted_prefix_of_all_keys():
         assert [(r.idx) for r in oracle.search(p, threads=1).topk] == [g[1] for g in got]
 
 
+def test_stationary_mask_only_removes_mappings_from_the_space():
+    """Section VII-K: an array that offers only some stationary pairs.  The model of a mapping does not change
+    (same keys, same records); mappings with another pair leave the space, and the search is the sorted prefix of
+    what remains.  A fixed weight-stationary array (pair 0 alone) can be no better than one that may switch."""
+    cfg = mi.random_tiny_problem(3)
+    base = dict(cfg["searches"][0], objective=mi.OBJ_EDP, topk=8)
+    p_all = oracle.make_problem(cfg["workload"], cfg["arch"], base)
+    begin, count = 0, min(p_all.N, 2_000_000) // (p_all.R * 9) * p_all.R * 9
+    base.update(t_begin=0, t_end=count // (p_all.R * 9))
+    p_all = oracle.make_problem(cfg["workload"], cfg["arch"], base)
+    keys_all, feas_all = oracle.keys_range(p_all, begin, count)
+    idx = np.arange(begin, begin + count, dtype=np.uint64)
+    best = {}
+    for mask in (0x001, 0x1ff, 0x0a4, 0x111):
+        p = oracle.make_problem(cfg["workload"], cfg["arch"], dict(base, stationary_mask=mask))
+        keys, feas = oracle.keys_range(p, begin, count)
+        assert (keys == keys_all).all()
+        allowed = ((mask >> (idx % 9).astype(np.int64)) & 1).astype(bool)
+        assert (feas.astype(bool) == (feas_all.astype(bool) & allowed)).all()
+        keep = feas.astype(bool)
+        order = np.lexsort((idx[keep], keys[keep]))[:8]
+        res = oracle.search(p, threads=2)
+        assert [r.idx for r in res.topk] == [int(idx[keep][i]) for i in order]
+        assert res.n_feasible == int(keep.sum())
+        assert all((mask >> (3 * r.sm[0] + r.sm[1])) & 1 for r in res.topk)
+        best[mask] = res.topk[0].edp_key if res.topk else float("inf")
+    assert best[0x1ff] <= min(best.values()) and best[0x001] >= best[0x111] >= best[0x1ff]
+    with pytest.raises(oracle.OracleError):
+        oracle.make_problem(cfg["workload"], cfg["arch"], dict(base, stationary_mask=0x200))
+
+
 def test_edp_key_is_one_ieee_product():
     p = _prime_problem(objective=mi.OBJ_EDP)
     for idx in (0, 12345, p.N - 1):
