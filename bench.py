@@ -28,7 +28,7 @@ import mmee_inputs as mi  # noqa: E402
 
 METRIC = "candidate mappings evaluated/sec"
 UNIT = "candidates/s"
-OBJ_NAMES = {0: "energy", 1: "latency", 2: "edp"}
+OBJ_NAMES = {0: "energy", 1: "latency", 2: "edp", 3: "energy_lcap", 4: "latency_ecap"}
 
 # Algorithmic integer work per mapping in the hoisted separable form of the model, counted in
 # thread-level 32-bit integer instructions.  Energy: one fused add-min per mapping (its key relative
@@ -62,6 +62,9 @@ def workload_jobs(name):
     if name == "beyond":
         pts = mi.beyond_attention_configs()
         return "two_gemm_and_conv_chains", [(c, c["searches"][0]) for c in pts]
+    if name == "reconfig":
+        cfg, _ = mi.reconfigurable_array_designs()
+        return "reconfigurable_arrays_" + cfg["name"], [(cfg, cfg["searches"][0])]
     cfg = WORKLOADS[name]()
     return cfg["name"], [(cfg, s) for s in cfg["searches"]]
 
@@ -159,6 +162,33 @@ def run_reference(args, rank):
         e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))))
 
 
+def run_reconfig(args):
+    """EDP-driven search over the four array designs of the reconfigurable-array comparison: one search per
+    logical shape through mmee_search_shapes, host wall clock per design."""
+    import torch
+    import paper_2604_03446_b200 as mm
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    cfg, designs = mi.reconfigurable_array_designs()
+    out, total_ms, total_cand = [], 0.0, 0
+    for name, mask, shapes in designs:
+        obj = dict(cfg["searches"][0], stationary_mask=mask)
+        mm.mmee_search_shapes(cfg["workload"], cfg["arch"], obj, shapes)          # warm-up
+        t0 = time.perf_counter()
+        per_shape, best = mm.mmee_search_shapes(cfg["workload"], cfg["arch"], obj, shapes)
+        ms = 1e3 * (time.perf_counter() - t0)
+        r = per_shape[best]
+        total_ms += ms
+        total_cand += sum(p.n_total for p in per_shape)
+        out.append(dict(design=name, shapes=len(shapes), best_shape=list(shapes[best]), edp_key=r.edp_key,
+                        energy_pj=r.energy_pj, latency_cycles=r.latency_cycles, sm=list(r.sm), idx=r.idx, ms=ms))
+    print(json.dumps(dict(metric=METRIC, value=total_cand / (total_ms * 1e-3), unit=UNIT, n_gpus=1, steps=1, warmup=1,
+                          ms_per_step=total_ms, higher_is_better=True, scaling="weak", vs_baseline=None,
+                          dtype="f64", data="synthetic",
+                          config=dict(workload="reconfigurable_arrays_" + cfg["name"],
+                                      note="host wall clock of mmee_search_shapes (plan + search + copy per shape)"),
+                          designs=out)))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -166,7 +196,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="bert", choices=sorted(WORKLOADS) + ["sweep", "ffn", "beyond"])
+    ap.add_argument("--workload", default="bert", choices=sorted(WORKLOADS) + ["sweep", "ffn", "beyond", "reconfig"])
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -176,6 +206,10 @@ def main():
 
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.workload == "reconfig":
+        if rank == 0:
+            run_reconfig(args)
         return
 
     import torch

@@ -34,9 +34,10 @@ def arch(pe_rows, pe_cols, n_arrays, gb_bytes, rf_bytes, dram_words_per_cycle,
 
 
 def objective(objective=OBJ_ENERGY, topk=1, tiling_set=TILE_ALL_DIVISORS, order_set=ORD_ALL6,
-              fuse_mask=FUSE_ALL, t_begin=0, t_end=0, row_pruning=0, key_cap=0):
+              fuse_mask=FUSE_ALL, t_begin=0, t_end=0, row_pruning=0, key_cap=0, stationary_mask=0):
     return dict(objective=objective, topk=topk, tiling_set=tiling_set, order_set=order_set,
-                fuse_mask=fuse_mask, row_pruning=row_pruning, t_begin=t_begin, t_end=t_end, key_cap=key_cap)
+                fuse_mask=fuse_mask, row_pruning=row_pruning, t_begin=t_begin, t_end=t_end, key_cap=key_cap,
+                stationary_mask=stationary_mask)
 
 
 # --- accelerators -----------------------------------------------------------------------------
@@ -151,6 +152,22 @@ def ffn_dram_sweep_configs():
     w = two_gemm(32768, 4096, 16384, 4096)
     return [dict(name="ffn_gpt3_dram_%dKB" % (b // KiB), workload=w, arch=arch_dram_only(b),
                  searches=[objective(OBJ_ENERGY, 1, fuse_mask=FUSE_FUSED)]) for b in FFN_SWEEP_BUFFER_BYTES]
+
+
+SM_WS_WS, SM_ALL = 0x001, 0x1ff      # stationary-pair masks: weight-stationary for both operators; all nine
+
+
+def reconfigurable_array_designs(seq=512, d=64):
+    """The four array designs of the paper's reconfigurable-array comparison (Section VII-K) for one
+    BERT-Base-shaped head on its first accelerator, EDP-driven: fixed 32x32 weight-stationary array; free
+    stationary modes on 32x32; free logical shape (every power-of-two rows x cols with 1024 PEs) under weight
+    stationary; both.  Each entry: (name, stationary mask, list of (rows, cols))."""
+    shapes = [(1 << a, 1024 >> a) for a in range(11)]
+    cfg = dict(name="bert_base_s%d_accel1" % seq, workload=workload(1, 12, 12, seq, seq, d, d), arch=arch_accel1(),
+               searches=[objective(OBJ_EDP, 1, fuse_mask=FUSE_FUSED)])
+    designs = [("fixed_32x32_ws", SM_WS_WS, [(32, 32)]), ("ideal_flow_32x32", SM_ALL, [(32, 32)]),
+               ("ideal_shape_ws", SM_WS_WS, shapes), ("ideal_shape_and_flow", SM_ALL, shapes)]
+    return cfg, designs
 
 
 def golden_configs():
