@@ -339,7 +339,8 @@ def main():
             ops = bests[i].n_feasible * ALG_OPS_PER_CANDIDATE[s["objective"]]
             per_kernel.append(dict(kernel="search_kernel<%s>" % OBJ_NAMES[s["objective"]], objective=s["objective"],
                                    problem=jobs[i][0]["name"],
-                                   avg_ms=sm, finalize_avg_ms=fm, candidates=n, feasible=bests[i].n_feasible,
+                                   avg_ms=sm, median_ms=statistics.median(k[i][0] for k in kernel_ms),
+                                   max_ms=max(k[i][0] for k in kernel_ms), finalize_avg_ms=fm, candidates=n, feasible=bests[i].n_feasible,
                                    pruned_fraction=1.0 - bests[i].n_feasible / n, time_to_optimum_ms=tto_ms[i],
                                    candidates_per_s=n / (sm * 1e-3), achieved_gops=ops / (sm * 1e-3) / 1e9))
         dom = max(per_kernel, key=lambda k: k["avg_ms"])
