@@ -240,12 +240,13 @@ int build_plan(const mmee_workload_t* w, const mmee_arch_t* a, const mmee_object
     const long double limit = 4611686018427387904.0L;     // 2^62
     if (emax >= limit || lmax >= limit) return MMEE_ERR_OVERFLOW;
 
-    // Scale of the 32-bit threshold-relative energy keys: the largest DRAM term of any mapping,
-    // c_dram_gb * I*K*L*J, must fit below 2^28 after the shift.
+    // Scale of the 32-bit threshold-relative keys of the energy and latency walks: the largest DRAM term of any
+    // mapping, I*K*L*J words (times c_dram_gb quanta for energy), must fit below 2^28 after the shift.
     p->rel_shift = 0;
     p->unit = 1;
-    if (p->objective == MMEE_OBJ_ENERGY) {
-        long double biggest = (long double)dims[0] * dims[1] * dims[2] * dims[3] * (long double)p->c_dram_gb;
+    if (p->objective == MMEE_OBJ_ENERGY || p->objective == MMEE_OBJ_LATENCY) {
+        long double biggest = (long double)dims[0] * dims[1] * dims[2] * dims[3] *
+                              (p->objective == MMEE_OBJ_ENERGY ? (long double)p->c_dram_gb : 1.0L);
         while (biggest >= 268435456.0L) { biggest /= 2.0L; ++p->rel_shift; }
     }
 

@@ -552,6 +552,9 @@ __device__ __noinline__ void exact_group(const Plan& p, const TilingTab* tb, con
                                          uint32_t lb_task, int m, int d, bool live, uint32_t kept,
                                          uint64_t task_first_idx, WarpTop* wt, CtaShared* cs, long long* global_g, int k,
                                          int lane) {
+    // The other CTAs' bound, read afresh: a lane that visits this path with a stale threshold would come back for
+    // every group.  The load is consumed at the end of the visit, before the caller renews its threshold.
+    const long long g_now = (lane == 0) ? *reinterpret_cast<volatile long long*>(global_g) : 0;
     const MidExact me = mid_exact<OBJ>(p, tb, ot, phi, la, lb_task, m, live);
     const RowTab* rt = &ot->rt[phi == 0 ? 0 : 1];
     const int64_t s1 = me.slack1 - rt->D[d][0];
@@ -573,6 +576,8 @@ __device__ __noinline__ void exact_group(const Plan& p, const TilingTab* tb, con
             slow_row<OBJ>(wt, cs, global_g, k, lane, fit, x, xe, me.wptr, me.qptr, me.P[0], me.P[1], me.P[2], p.key_cap,
                           p.sm_mask, row_first_idx);
     }
+    if (lane == 0 && g_now < cs->G) atomicMin(&cs->G, g_now);
+    __syncwarp();
 }
 
 // The same for a single optimum (k = 1), without the insertion loop: every lane finds the best of its 45
@@ -583,6 +588,9 @@ __device__ __noinline__ void exact_group_single(const Plan& p, const TilingTab* 
                                                 uint32_t la, uint32_t lb_task, int m, int d, bool live, uint32_t kept,
                                                 uint64_t task_first_idx, WarpTop* wt, CtaShared* cs, long long* global_g,
                                                 int lane) {
+    // The other CTAs' bound, read afresh: a lane that visits this path with a stale threshold would come back for
+    // every group.  The load is consumed at the end of the visit, before the caller renews its threshold.
+    const long long g_now = (lane == 0) ? *reinterpret_cast<volatile long long*>(global_g) : 0;
     const MidExact me = mid_exact<OBJ>(p, tb, ot, phi, la, lb_task, m, live);
     const RowTab* rt = &ot->rt[phi == 0 ? 0 : 1];
     const int64_t s1 = me.slack1 - rt->D[d][0];
@@ -620,6 +628,7 @@ __device__ __noinline__ void exact_group_single(const Plan& p, const TilingTab* 
             atomicMin(global_g, (long long)best);       // other CTAs pick it up at their next task
         }
     }
+    if (lane == 0 && g_now < cs->G) atomicMin(&cs->G, g_now);
     __syncwarp();
 }
 
@@ -772,43 +781,38 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
     // sum that follows (at most 4 * kTermCap < kUnfit is added), clamping from above only lowers
     auto rel32 = [](int64_t v) { const int r = sat_s32(v); return max(min(r, kRowCap), -kUnfit); };
 
-    // Threshold state.  Energy: base[rc] = (terms of A and of the C round trip) - ceil((T1 - wmin[rc]) / 2^rel_shift),
-    // base_strict[rc] the same against T1 - delta.  (Most terms are multiples of the unit, so that a tie with the
-    // list's last entry is told from a better key even in coarse units.)
-    // Latency, fused task: ua2[rc] = DRAM words of A and B - T1, qo2[rc] = least compute words - T1.
-    int base[2] = {0, 0}, base_strict[2] = {0, 0}, ua2[2] = {0, 0}, qo2[2] = {0, 0};
-    int64_t T1 = 0;
-    int delta = 0, strict_from = INT_MAX;
-    auto rebase = [&]() {
+    // Threshold state, set at the start of the task and after each visit of the exact path.  `next_pos` is the
+    // position in the task of the first candidate still to be walked: if its index lies above the list's last
+    // entry, so do all that follow, a tie cannot displace that entry, and the threshold is T1 - delta.  (Most
+    // terms are multiples of the unit, so that a tie is told from a better key even in coarse units.)
+    // Energy: base[rc] = (terms of A and of the C round trip) - ceil((thr - wmin[rc]) / 2^rel_shift).
+    // Latency, fused task: ua2[rc] = DRAM words of A and B - thr, qo2[rc] = least compute words - thr, in units
+    // of 2^rel_shift words rounded down.
+    int base[2] = {0, 0}, ua2[2] = {0, 0}, qo2[2] = {0, 0};
+    int64_t thr = 0;
+    auto rebase = [&](int next_pos) {
         const LaneThreshold th = load_threshold(wt, cs, k);
-        T1 = th.T1;
-        delta = th.delta;
-        // first candidate of the task, by position, whose index lies above the list's last entry
-        strict_from = th.ti < task_first_idx ? 0
-                      : (th.ti - task_first_idx >= (uint64_t)kCandPerTask ? INT_MAX : (int)(th.ti - task_first_idx) + 1);
+        thr = th.T1 - ((task_first_idx + (uint64_t)next_pos > th.ti) ? th.delta : 0);
         if constexpr (OBJ == MMEE_OBJ_ENERGY) {
 #pragma unroll
             for (int rc = 0; rc < 2; ++rc) {
-#pragma unroll
-                for (int st = 0; st < 2; ++st) {
-                    const int64_t b64 = T1 - (st ? delta : 0) - tb->wmin[rc];
-                    const int64_t bs = ((b64 - 1) >> p.rel_shift) + 1;                // ceiling of the quotient
-                    const int64_t bl = bs > (int64_t)INT_MAX ? (int64_t)INT_MAX : (bs < -(int64_t)kTermCap ? -(int64_t)kTermCap : bs);
-                    const int t = (rc ? av.w : av.z) + gxc - (int)bl;
-                    (st ? base_strict : base)[rc] = max(min(t, kRowCap), -kUnfit);
-                }
+                const int64_t b64 = thr - tb->wmin[rc];
+                const int64_t bs = ((b64 - 1) >> p.rel_shift) + 1;                // ceiling of the quotient
+                const int64_t bl = bs > (int64_t)INT_MAX ? (int64_t)INT_MAX : (bs < -(int64_t)kTermCap ? -(int64_t)kTermCap : bs);
+                const int t = (rc ? av.w : av.z) + gxc - (int)bl;
+                base[rc] = max(min(t, kRowCap), -kUnfit);
             }
         } else {
             if (fused) {
 #pragma unroll
                 for (int rc = 0; rc < 2; ++rc) {
-                    ua2[rc] = rel32(ot->gA[c.la][rc] + ot->gB[c.lb][rc] - T1);
-                    qo2[rc] = rel32(tb->qmin[rc] - T1);
+                    ua2[rc] = rel32((ot->gA[c.la][rc] + ot->gB[c.lb][rc] - thr) >> p.rel_shift);
+                    qo2[rc] = rel32((tb->qmin[rc] - thr) >> p.rel_shift);
                 }
             }
         }
     };
-    rebase();
+    rebase(0);
 
     int unfit = 0;          // minus the number of visited rows that do not fit
     uint32_t groups = 0;
@@ -830,7 +834,7 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
         const int slack1c = live ? (fused ? max(room1, -1) : (room1 >= 0 ? kSizeCap : -1)) : -1;
         const int slack2c = live ? max(capc - y2, -1) : -1;
 
-        int u = 0, u_strict = 0, Wc[9], ua[3], Qc[9];
+        int u = 0, Wc[9], ua[3], Qc[9];
         if constexpr (OBJ == MMEE_OBJ_ENERGY) {
             const int4* wc4 = reinterpret_cast<const int4*>(tb->Wc[rc]);
             const int4 w0 = wc4[0], w1 = wc4[1], w2 = wc4[2];
@@ -842,7 +846,6 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
         auto mid_setup = [&]() {
             if constexpr (OBJ == MMEE_OBJ_ENERGY) {
                 u = __viaddmin_s32(base[rc], rc ? bv.w : bv.z, kRowCap);
-                u_strict = __viaddmin_s32(base_strict[rc], rc ? bv.w : bv.z, kRowCap);
             } else {
                 int qo[3];
                 const int32_t* qrel;
@@ -858,9 +861,9 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
 #pragma unroll
                     for (int j = 0; j < 3; ++j) {
                         const int64_t c1w = tb->C1w[j];
-                        const int64_t pj = (da1 > c1w ? da1 : c1w) + pass - T1;
-                        ua[j] = rel32(ot->gCr + pj);
-                        qo[j] = rel32(tb->qmin[2] + pj);
+                        const int64_t pj = (da1 > c1w ? da1 : c1w) + pass - thr;
+                        ua[j] = rel32((ot->gCr + pj) >> p.rel_shift);
+                        qo[j] = rel32((tb->qmin[2] + pj) >> p.rel_shift);
                     }
                     qrel = tb->Qrel[2];
                 }
@@ -897,8 +900,7 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
             int a0 = INT_MAX, a1 = INT_MAX, a2 = INT_MAX;
             bool hit;
             if constexpr (OBJ == MMEE_OBJ_ENERGY) {
-                // ties with the list's last entry cannot displace it from a higher index
-                const int uc = __viaddmin_s32((m * 225 + d * 45) >= strict_from ? u_strict : u, dc.z, kRowCap);
+                const int uc = __viaddmin_s32(u, dc.z, kRowCap);
 #pragma unroll
                 for (int e = 0; e < 5; ++e) {
                     // t = -1 if the row does not fit (Eq. 4), else 0; such a row's keys are moved up by kUnfit,
@@ -929,13 +931,12 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
                     a0 = __vimin3_s32(a0, v[0], v[1]); a1 = __vimin3_s32(a1, v[2], v[3]); a2 = __vimin3_s32(a2, v[4], v[5]);
                     a0 = __vimin3_s32(a0, v[6], v[7]); a1 = min(a1, v[8]);
                 }
-                // ties with the list's last entry cannot displace it from a higher index
-                hit = __vimin3_s32(a0, a1, a2) < ((m * 225 + d * 45) >= strict_from ? -delta : 0);
+                hit = __vimin3_s32(a0, a1, a2) < 0;
             }
             if (__any_sync(kFull, hit)) {
                 if (k == 1) exact_group_single<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, lane);
                 else exact_group<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, k, lane);
-                rebase();
+                rebase(m * 225 + d * 45 + 45);
                 mid_setup();
             }
         }
@@ -1061,7 +1062,8 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                 tb->qmin[v] = m;
                 for (int s = 0; s < 9; ++s) {
                     const int64_t qd = src[2 * s] - m;
-                    tb->Qrel[v][s] = (qd > (int64_t)kTermCap || !((p.sm_mask >> s) & 1u)) ? kTermCap : (int32_t)qd;
+                    const int64_t qs = qd >> p.rel_shift;
+                    tb->Qrel[v][s] = (qs > (int64_t)kTermCap || !((p.sm_mask >> s) & 1u)) ? kTermCap : (int32_t)qs;
                 }
             }
         }
