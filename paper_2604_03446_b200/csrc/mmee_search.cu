@@ -88,7 +88,7 @@ struct alignas(16) TilingTab {
     int64_t cw, smx;        // C write-back words (I*L); separate softmax pass words (2*I*L)
     int64_t wmin[2];        // min over the stationary pairs of W[.][rc]
     int64_t qmin[3];        // min over the stationary pairs of CB[.][0], CB[.][1], QU[.][0]
-    int32_t Qrel[3][12];    // CB[s][0], CB[s][1], QU[s][0] minus that minimum, saturated to kTermCap
+    int32_t Qrel[3][12];    // CB[s][0], CB[s][1], QU[s][0] minus that minimum, saturated to kTermCap (kUnfit: pair not offered)
     int32_t live;           // smallest possible buffer need of this tiling fits
     int32_t pad[3];
 };
@@ -872,11 +872,6 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
                 Qc[0] = imad(qo[0], one, q0.x); Qc[1] = imad(qo[0], one, q0.y); Qc[2] = imad(qo[0], one, q0.z);
                 Qc[3] = imad(qo[1], one, q0.w); Qc[4] = imad(qo[1], one, q1.x); Qc[5] = imad(qo[1], one, q1.y);
                 Qc[6] = imad(qo[2], one, q1.z); Qc[7] = imad(qo[2], one, q1.w); Qc[8] = imad(qo[2], one, q2.x);
-                if (p.sm_mask != 0x1ffu) {       // a stationary pair the array does not offer never passes
-#pragma unroll
-                    for (int s = 0; s < 9; ++s)
-                        if (!((p.sm_mask >> s) & 1u)) Qc[s] = kRowCap;
-                }
             }
         };
         mid_setup();
@@ -1063,7 +1058,9 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                 for (int s = 0; s < 9; ++s) {
                     const int64_t qd = src[2 * s] - m;
                     const int64_t qs = qd >> p.rel_shift;
-                    tb->Qrel[v][s] = (qs > (int64_t)kTermCap || !((p.sm_mask >> s) & 1u)) ? kTermCap : (int32_t)qs;
+                    // (a pair the array does not offer: kUnfit, which no threshold part, clamped at -kUnfit, can
+                    // bring below zero)
+                    tb->Qrel[v][s] = !((p.sm_mask >> s) & 1u) ? kUnfit : (qs > (int64_t)kTermCap ? kTermCap : (int32_t)qs);
                 }
             }
         }
