@@ -214,11 +214,14 @@ __device__ __forceinline__ void row_test(const int64_t (&k)[9], int64_t thr, int
 // four addends of at most kTermCap follow, 4 * kTermCap < kUnfit, so a sum that was clamped from below
 // stays negative (the group is flagged, which is the safe side), and no 32-bit sum overflows:
 // kRowCap + 2 * kTermCap + kUnfit < 2^31.  Most terms are multiples of the unit, so that a tie with
-// the list's last entry is still told from a better key: groups whose indices lie above that entry
-// use the threshold thr - 1.
+// the list's last entry is still told from a better key: when every index still to be walked in a
+// task lies above that entry's, the threshold is thr - 1 (decided at the start of the task and after
+// each visit of the exact path).
 // Latency: key = P + max(x, Q[s]) (P: the Op1 stage of an unfused task, else 0), and
 // max(a, b) < thr  <=>  a - thr < 0 and b - thr < 0.  a = (x0 + P - thr) + vD + vE with the same
-// clamping; b = (Q[s] - qmin) + (qmin + P - thr), the first part a table entry capped at kTermCap.
+// units, rounding and clamping (the unit is chosen from the largest DRAM term in words);
+// b = (Q[s] - qmin) + (qmin + P - thr), the first part a table entry capped at kTermCap, both parts
+// rounded down.
 // Capacity (Eq. 4): sizes are saturated to kSizeCap, which is above every admissible capacity, so
 // "size <= slack" keeps its truth value in 32 bits.  A row that does not fit has kUnfit added to its
 // keys, which makes them non-negative whatever the threshold.
