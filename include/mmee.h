@@ -170,7 +170,7 @@ int mmee_destroy(mmee_handle_t* handle);
  * library then fails), or a latency-critical loop that cannot afford the device-wide
  * synchronisation of cudaMalloc / cudaFree.  This call makes no cudaMalloc, cudaFree or other
  * allocating call.  Its scratch (work counter, pruning bound, one partial top-k list per CTA) is a
- * fixed 135 200-byte array inside the library image, present on every device that loads the
+ * fixed 139 296-byte array inside the library image, present on every device that loads the
  * library for as long as the process lives.
  *
  *   workload, arch, objective : HOST, as for mmee_create; planned on the host at every call.

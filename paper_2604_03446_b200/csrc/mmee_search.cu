@@ -98,12 +98,17 @@ static_assert(offsetof(RowTab, Ec) % 16 == 0 && offsetof(OrderTab, rt) % 16 == 0
               "Ec rows are read as int4");
 // 21 items per tiling: 9 stationary pairs x 2 recompute flags, 3 unfused Op1 terms
 
+// One warp's k best (key, idx) pairs, best first.  A pair is one 16-byte word, read and written whole.
 struct alignas(16) WarpTop {
-    int64_t key[MMEE_MAX_TOPK];
-    uint64_t idx[MMEE_MAX_TOPK];
+    longlong2 e[MMEE_MAX_TOPK];      // x = key, y = idx
     int32_t count;
-    int32_t pad;
+    int32_t pad[3];
 };
+__device__ __forceinline__ int64_t top_key(const WarpTop* w, int j) { return w->e[j].x; }
+__device__ __forceinline__ uint64_t top_idx(const WarpTop* w, int j) { return (uint64_t)w->e[j].y; }
+__device__ __forceinline__ void top_set(WarpTop* w, int j, int64_t key, uint64_t idx) {
+    w->e[j] = make_longlong2((long long)key, (long long)idx);
+}
 
 struct alignas(16) CtaShared {
     long long G;             // upper bound on the final k-th smallest key (any full list's last key)
@@ -120,14 +125,15 @@ __device__ __forceinline__ bool pair_less(int64_t ka, uint64_t ia, int64_t kb, u
 __device__ __forceinline__ bool warp_insert(WarpTop* wt, int k, int64_t nk, uint64_t ni, int lane) {
     const int count = wt->count;
     const bool have = lane < count;
-    const int64_t ek = have ? wt->key[lane] : kInfKey;
-    const uint64_t ei = have ? wt->idx[lane] : UINT64_MAX;
+    const longlong2 mine = have ? wt->e[lane] : make_longlong2(kInfKey, -1ll);
+    const int64_t ek = mine.x;
+    const uint64_t ei = (uint64_t)mine.y;
     const unsigned smaller = __ballot_sync(kFull, have && pair_less(ek, ei, nk, ni));
     const int pos = __popc(smaller);
     if (pos >= k) return false;
     __syncwarp();
-    if (have && lane >= pos && lane + 1 < k) { wt->key[lane + 1] = ek; wt->idx[lane + 1] = ei; }
-    if (lane == pos) { wt->key[pos] = nk; wt->idx[pos] = ni; }
+    if (have && lane >= pos && lane + 1 < k) top_set(wt, lane + 1, ek, ei);
+    if (lane == pos) top_set(wt, pos, nk, ni);
     if (lane == 0 && count < k) wt->count = count + 1;
     __syncwarp();
     return true;
@@ -139,8 +145,9 @@ __device__ __forceinline__ bool warp_insert(WarpTop* wt, int k, int64_t nk, uint
 __device__ __forceinline__ int64_t lane_threshold(const WarpTop* wt, const CtaShared* cs, int k, uint64_t task_first_idx) {
     int64_t thr = cs->G + 1;                       // G <= INT64_MAX - 1 always
     if (wt->count == k) {
-        const int64_t tk = wt->key[k - 1];
-        const int64_t loc = (task_first_idx > wt->idx[k - 1]) ? tk : tk + 1;
+        const longlong2 last = wt->e[k - 1];
+        const int64_t tk = last.x;
+        const int64_t loc = (task_first_idx > (uint64_t)last.y) ? tk : tk + 1;
         thr = loc < thr ? loc : thr;
     }
     return thr;
@@ -309,7 +316,7 @@ __device__ __noinline__ int64_t slow_row(WarpTop* wt, CtaShared* cs, long long* 
         }
     }
     if (lane == 0 && wt->count == k) {
-        const long long last = wt->key[k - 1];
+        const long long last = top_key(wt, k - 1);
         if (last < cs->G) {
             atomicMin(&cs->G, last);
             atomicMin(global_g, last);       // other CTAs pick it up at their next task
@@ -486,8 +493,9 @@ __device__ __forceinline__ LaneThreshold load_threshold(const WarpTop* wt, const
     const int64_t g1 = cs->G + 1;                 // G <= INT64_MAX - 1 always
     t.T1 = g1; t.ti = UINT64_MAX; t.delta = 0;
     if (wt->count == k) {
-        const int64_t tk1 = wt->key[k - 1] + 1;
-        if (tk1 <= g1) { t.T1 = tk1; t.delta = 1; t.ti = wt->idx[k - 1]; }
+        const longlong2 last = wt->e[k - 1];
+        const int64_t tk1 = last.x + 1;
+        if (tk1 <= g1) { t.T1 = tk1; t.delta = 1; t.ti = (uint64_t)last.y; }
     }
     return t;
 }
@@ -622,9 +630,8 @@ __device__ __noinline__ void exact_group_single(const Plan& p, const TilingTab* 
         const uint64_t oi = __shfl_xor_sync(kFull, best_idx, off);
         if (pair_less(ok, oi, best, best_idx)) { best = ok; best_idx = oi; }
     }
-    if (lane == 0 && best != kInfKey && (wt->count == 0 || pair_less(best, best_idx, wt->key[0], wt->idx[0]))) {
-        wt->key[0] = best;
-        wt->idx[0] = best_idx;
+    if (lane == 0 && best != kInfKey && (wt->count == 0 || pair_less(best, best_idx, top_key(wt, 0), top_idx(wt, 0)))) {
+        top_set(wt, 0, best, best_idx);
         wt->count = 1;
         if (best < cs->G) {
             atomicMin(&cs->G, (long long)best);
@@ -1162,12 +1169,14 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
         for (int w2 = 1; w2 < kSearchThreads / 32; ++w2) {
             const WarpTop* src = &wtops[w2];
             const int n = src->count;
-            for (int j = 0; j < n; ++j)
-                if (!warp_insert(wt, k, src->key[j], src->idx[j], lane)) break;   // sorted: the rest is larger
+            for (int j = 0; j < n; ++j) {
+                const longlong2 sj = src->e[j];
+                if (!warp_insert(wt, k, sj.x, (uint64_t)sj.y, lane)) break;   // sorted: the rest is larger
+            }
         }
         Partial* out = &scratch->partial[blockIdx.x];
         const int n = wt->count;
-        if (lane < n) { out->key[lane] = wt->key[lane]; out->idx[lane] = wt->idx[lane]; }
+        if (lane < n) out->e[lane] = wt->e[lane];
         if (lane == 0) {
             out->count = n;
             if (cs->feasible_rows) atomicAdd(&scratch->feasible_rows, cs->feasible_rows);
@@ -1191,16 +1200,20 @@ finalize_kernel(const __grid_constant__ Plan p, Scratch* __restrict__ scratch, i
     for (int c = warp; c < n_partials; c += 32) {
         const Partial* src = &scratch->partial[c];
         const int n = src->count;
-        for (int j = 0; j < n; ++j)
-            if (!warp_insert(wt, k, src->key[j], src->idx[j], lane)) break;
+        for (int j = 0; j < n; ++j) {
+            const longlong2 sj = src->e[j];
+            if (!warp_insert(wt, k, sj.x, (uint64_t)sj.y, lane)) break;
+        }
     }
     __syncthreads();
     if (warp == 0) {
         for (int w2 = 1; w2 < 32; ++w2) {
             const WarpTop* src = &tops[w2];
             const int n = src->count;
-            for (int j = 0; j < n; ++j)
-                if (!warp_insert(wt, k, src->key[j], src->idx[j], lane)) break;
+            for (int j = 0; j < n; ++j) {
+                const longlong2 sj = src->e[j];
+                if (!warp_insert(wt, k, sj.x, (uint64_t)sj.y, lane)) break;
+            }
         }
         const int found = wt->count;
         const uint64_t n_total = (p.t_end - p.t_begin) * (uint64_t)p.rows_per_tiling * 9u;
@@ -1208,7 +1221,7 @@ finalize_kernel(const __grid_constant__ Plan p, Scratch* __restrict__ scratch, i
         if (lane < k) {
             mmee_result_t r;
             if (lane < found) {
-                evaluate_candidate(p, wt->idx[lane], r);
+                evaluate_candidate(p, top_idx(wt, lane), r);
             } else {
                 // empty slot
                 unsigned char* raw = reinterpret_cast<unsigned char*>(&r);

@@ -13,11 +13,10 @@ constexpr int kWorkerWarps = kSearchThreads / 32 - 1;     // the last warp build
 constexpr int kWorkerThreads = kWorkerWarps * 32;
 
 // One CTA's k best (key, idx) pairs, best first.
-struct Partial {
-    int64_t key[MMEE_MAX_TOPK];
-    uint64_t idx[MMEE_MAX_TOPK];
+struct alignas(16) Partial {
+    longlong2 e[MMEE_MAX_TOPK];     // x = key, y = idx: one 16-byte word per pair, stored and loaded whole
     int32_t count;
-    int32_t pad;
+    int32_t pad[3];
 };
 
 // Global scratch of one handle: a work counter, the feasible-row count, the shared pruning bound
