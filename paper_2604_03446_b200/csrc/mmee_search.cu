@@ -580,6 +580,7 @@ __device__ __noinline__ void exact_group(const Plan& p, const TilingTab* tb, con
         const uint64_t row_first_idx = task_first_idx + (uint64_t)(m * 225 + (d * 5 + e) * 9);
         const int64_t thr_row = lane_threshold(wt, cs, k, row_first_idx);
         bool below = false;
+#pragma unroll
         for (int s = 0; s < 9; ++s)
             below |= ((p.sm_mask >> s) & 1u) &&
                      candidate_key<OBJ>(x, xe, me.wptr[2 * s], me.P[s / 3], me.qptr[2 * s], p.key_cap) < thr_row;
@@ -855,14 +856,14 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
         // the part of the set-up that depends on the threshold: redone after a visit of the exact path
         auto mid_setup = [&]() {
             if constexpr (OBJ == MMEE_OBJ_ENERGY) {
-                u = __viaddmin_s32(base[rc], rc ? bv.w : bv.z, kRowCap);
+                u = __viaddmin_s32(rc ? base[1] : base[0], rc ? bv.w : bv.z, kRowCap);
             } else {
                 int qo[3];
                 const int32_t* qrel;
                 if (fused) {
-                    ua[0] = ua[1] = ua[2] = ua2[rc];
-                    qo[0] = qo[1] = qo[2] = qo2[rc];
-                    qrel = tb->Qrel[rc];
+                    ua[0] = ua[1] = ua[2] = rc ? ua2[1] : ua2[0];
+                    qo[0] = qo[1] = qo[2] = rc ? qo2[1] : qo2[0];
+                    qrel = tb->Qrel[rc];       // (a shared-memory address, not a register array)
                 } else {
                     // unfused latency: max(DA1, C1) + softmax pass + max(DA2, C2); the first two terms are
                     // fixed by (level of A, level of B = m, sm1)
