@@ -67,6 +67,9 @@ extern "C" {
 #define MMEE_ERR_CUDA         5   /* a CUDA runtime call failed (no device, launch error, ...)     */
 #define MMEE_ERR_TIMEOUT      6   /* reserved: the kernels contain no device-side wait             */
 #define MMEE_ERR_RANGE        7   /* request exceeds a documented maximum                          */
+#define MMEE_ERR_CHECK        8   /* out_best->status only: a winner's ranking key is not the key of its full
+                                     evaluation (internal consistency check of the finalize step); the records
+                                     are not to be trusted, search again                              */
 
 /* Attention workload.  Heads are independent instances of one search (Section V, first
  * paragraph); the q_heads/kv_heads query heads that share a K/V head are stacked along I. */
@@ -115,7 +118,7 @@ typedef struct {
     uint32_t row;
     uint32_t bound[8];                       /* i_D,k_D,l_D,j_D,i_G,k_G,l_G,j_G (Section V-E)     */
     uint8_t  phi, pi, beta[5], sm[2], recompute, feasible, reserved[5];
-    int32_t  status;                         /* MMEE_OK or MMEE_ERR_NO_FEASIBLE                   */
+    int32_t  status;                         /* MMEE_OK, MMEE_ERR_NO_FEASIBLE or MMEE_ERR_CHECK   */
     int64_t  bs_x[5];                        /* buffer words of A,B,C,D,E (Section V-B)           */
     int64_t  bs_op1, bs_op2, bs;             /* Eq. (1), (2), (4)                                 */
     int64_t  da_x[5];                        /* DRAM words of A,B,C,D,E (Section V-C); C only unfused */

@@ -17,7 +17,7 @@ ORD_NORECOMP2, ORD_ALL6 = 0, 1
 FUSE_FUSED, FUSE_SOFTMAX_IN_OP1, FUSE_SEPARATE = 1, 2, 4
 MAX_TOPK = 16
 NO_INDEX = 2 ** 64 - 1
-OK, ERR_ARG, ERR_OVERFLOW, ERR_QUANTUM, ERR_NO_FEASIBLE, ERR_CUDA, ERR_TIMEOUT, ERR_RANGE = range(8)
+OK, ERR_ARG, ERR_OVERFLOW, ERR_QUANTUM, ERR_NO_FEASIBLE, ERR_CUDA, ERR_TIMEOUT, ERR_RANGE, ERR_CHECK = range(9)
 
 EXPORTS = ("mmee_create", "mmee_search", "mmee_destroy", "mmee_search_static", "mmee_num_candidates", "mmee_num_tilings",
            "mmee_num_rows", "mmee_strerror", "mmee_last_cuda_error", "mmee_eval", "mmee_dump_keys", "mmee_solve_host", "mmee_pareto_front", "mmee_search_shapes",

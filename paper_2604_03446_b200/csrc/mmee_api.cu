@@ -174,6 +174,7 @@ const char* mmee_strerror(int status) {
         case MMEE_ERR_CUDA: return "CUDA runtime error";
         case MMEE_ERR_TIMEOUT: return "device-side wait timed out";
         case MMEE_ERR_RANGE: return "request exceeds a documented maximum";
+        case MMEE_ERR_CHECK: return "a winner's ranking key differs from its full evaluation";
         default: return "unknown status";
     }
 }
@@ -205,9 +206,12 @@ int mmee_solve_host(const mmee_workload_t* workload, const mmee_arch_t* arch, co
     const size_t bytes = (size_t)(k + 1) * sizeof(mmee_result_t);
     mmee_result_t* dev = nullptr;
     if (cudaMalloc(reinterpret_cast<void**>(&dev), bytes) != cudaSuccess) { mmee_destroy(h); return MMEE_ERR_CUDA; }
-    rc = mmee_search(h, nullptr, dev, dev + 1);
+    for (int attempt = 0; attempt < 3; ++attempt) {       // (search again if the finalize step's check fails)
+        rc = mmee_search(h, nullptr, dev, dev + 1);
+        if (rc == MMEE_OK) rc = cuda_status(cudaMemcpy(out_best, dev, sizeof(mmee_result_t), cudaMemcpyDeviceToHost));
+        if (rc != MMEE_OK || out_best->status != MMEE_ERR_CHECK) break;
+    }
     if (rc == MMEE_OK) {
-        rc = cuda_status(cudaMemcpy(out_best, dev, sizeof(mmee_result_t), cudaMemcpyDeviceToHost));
         if (rc == MMEE_OK && out_topk)
             rc = cuda_status(cudaMemcpy(out_topk, dev + 1, (size_t)k * sizeof(mmee_result_t), cudaMemcpyDeviceToHost));
     }
@@ -280,9 +284,12 @@ int mmee_search_shapes(const mmee_workload_t* workload, const mmee_arch_t* arch,
         a.pe_cols = shapes[2 * i + 1];
         mmee_handle_t* h = nullptr;
         if ((rc = mmee_create(workload, &a, &o, &h))) break;
-        rc = mmee_search(h, nullptr, dev, nullptr);
-        if (rc == MMEE_OK)
-            rc = cuda_status(cudaMemcpy(&out_per_shape[i], dev, sizeof(mmee_result_t), cudaMemcpyDeviceToHost));
+        for (int attempt = 0; attempt < 3; ++attempt) {   // (search again if the finalize step's check fails)
+            rc = mmee_search(h, nullptr, dev, nullptr);
+            if (rc == MMEE_OK)
+                rc = cuda_status(cudaMemcpy(&out_per_shape[i], dev, sizeof(mmee_result_t), cudaMemcpyDeviceToHost));
+            if (rc != MMEE_OK || out_per_shape[i].status != MMEE_ERR_CHECK) break;
+        }
         const int rc2 = mmee_destroy(h);
         if (rc == MMEE_OK) rc = rc2;
         if (rc != MMEE_OK || out_per_shape[i].idx == MMEE_NO_INDEX) continue;

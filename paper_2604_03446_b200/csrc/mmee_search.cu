@@ -1219,10 +1219,23 @@ finalize_kernel(const __grid_constant__ Plan p, Scratch* __restrict__ scratch, i
         const int found = wt->count;
         const uint64_t n_total = (p.t_end - p.t_begin) * (uint64_t)p.rows_per_tiling * 9u;
         const uint64_t n_feasible = scratch->feasible_rows * (uint64_t)p.n_sm;
+        // Every winner is evaluated in full; the key it was ranked by must be the key of that evaluation.  A
+        // mismatch (a list entry whose key and index do not belong together) is reported in out_best->status
+        // instead of being returned as a result.
+        bool consistent = true;
         if (lane < k) {
             mmee_result_t r;
             if (lane < found) {
                 evaluate_candidate(p, top_idx(wt, lane), r);
+                int64_t key;
+                switch (p.objective) {
+                    case MMEE_OBJ_ENERGY: key = r.e_key; break;
+                    case MMEE_OBJ_LATENCY: key = r.l_key; break;
+                    case MMEE_OBJ_EDP: key = dbits(r.edp_key); break;
+                    case MMEE_OBJ_ENERGY_LCAP: key = r.l_key <= p.key_cap ? r.e_key : kInfKey; break;
+                    default: key = r.e_key <= p.key_cap ? r.l_key : kInfKey; break;
+                }
+                consistent = key == top_key(wt, lane) && r.feasible;
             } else {
                 // empty slot
                 unsigned char* raw = reinterpret_cast<unsigned char*>(&r);
@@ -1230,10 +1243,12 @@ finalize_kernel(const __grid_constant__ Plan p, Scratch* __restrict__ scratch, i
                 r.idx = MMEE_NO_INDEX;
                 r.status = found ? MMEE_OK : MMEE_ERR_NO_FEASIBLE;
             }
+            const bool all_consistent = __all_sync(__activemask(), consistent);
             if (out_topk) out_topk[lane] = r;
             if (lane == 0) {
                 r.n_total = n_total;
                 r.n_feasible = n_feasible;
+                if (!all_consistent) r.status = MMEE_ERR_CHECK;
                 *out_best = r;
             }
         }

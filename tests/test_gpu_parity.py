@@ -530,21 +530,24 @@ def test_repeated_searches_after_a_cache_flush_agree():
     separate words about one launch in a hundred returned a pair whose halves came from different mappings;
     with whole 16-byte pairs the rate is below one in a thousand (a known residue, not understood: without the
     preceding writing kernel no launch has ever differed).  The test fails when more than 3 of 1500 launches
-    differ from the oracle's optimum and feasible count, i.e. when the torn-pair rate is back."""
+    differ from the oracle's optimum and feasible count (or are flagged MMEE_ERR_CHECK by the finalize step's own
+    check of its winners), i.e. when the torn-pair rate is back."""
     cfg = mi.config1()
     obj = cfg["searches"][0]
     want = oracle.search(oracle.make_problem(cfg["workload"], cfg["arch"], obj))
     expected = (want.topk[0].idx, want.n_feasible, want.topk[0].e_key)
     flush = torch.empty(64 * 1024 * 1024, dtype=torch.uint8, device="cuda")
     best = mm.result_buffer(1)
-    odd = []
+    odd, caught = [], 0
     with Handle(cfg, obj) as h:
         for it in range(1500):
             flush.fill_(it & 255)
             mm.mmee_search(h, best, None)
             torch.cuda.synchronize()
             r = mm.read_results(best, 1)[0]
-            if (r.idx, r.n_feasible, r.e_key) != expected:
+            if r.status == mm.ERR_CHECK:
+                caught += 1            # the finalize step saw a winner whose ranking key is not its own
+            elif (r.idx, r.n_feasible, r.e_key) != expected:
                 odd.append((it, r.idx, r.n_feasible, r.e_key))
         # without the writing kernel in front, every launch agrees
         for it in range(300):
@@ -552,4 +555,4 @@ def test_repeated_searches_after_a_cache_flush_agree():
             torch.cuda.synchronize()
             r = mm.read_results(best, 1)[0]
             assert (r.idx, r.n_feasible, r.e_key) == expected
-    assert len(odd) <= 3, odd
+    assert len(odd) + caught <= 3, (odd, caught)
