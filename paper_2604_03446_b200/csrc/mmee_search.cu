@@ -974,7 +974,8 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
     OrderTab* otabs_all = reinterpret_cast<OrderTab*>(ttabs_all + 2 * shape.slots);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int k = (int)p.topk;
+    // (from the kernel argument: the shared copy of the plan is not complete before the barrier below)
+    const int k = (int)plan_arg.topk;
     WarpTop* wt = &wtops[warp];
     // The last warp builds the tables of the next range while the other warps walk the tasks of
     // the current one (two table buffers); one barrier per range separates the two.
@@ -1235,7 +1236,7 @@ finalize_kernel(const __grid_constant__ Plan p, Scratch* __restrict__ scratch, i
                     case MMEE_OBJ_ENERGY_LCAP: key = r.l_key <= p.key_cap ? r.e_key : kInfKey; break;
                     default: key = r.e_key <= p.key_cap ? r.l_key : kInfKey; break;
                 }
-                consistent = key == top_key(wt, lane) && r.feasible;
+                consistent = key == top_key(wt, lane) && r.feasible && r.t >= p.t_begin && r.t < p.t_end;
             } else {
                 // empty slot
                 unsigned char* raw = reinterpret_cast<unsigned char*>(&r);

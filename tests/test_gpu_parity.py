@@ -524,35 +524,26 @@ def test_more_random_problems_keys_and_optimum(seed):
     check_search(cfg, obj)
 
 
-def test_repeated_searches_after_a_cache_flush_agree():
+@pytest.mark.parametrize("topk", [1, 16])
+def test_repeated_searches_after_a_cache_flush_agree(topk):
     """The same search launched many times, each time directly after a kernel that fills the L2 with written
-    lines (what the benchmark does between steps).  With (key, idx) pairs of the candidate lists kept as two
-    separate words about one launch in a hundred returned a pair whose halves came from different mappings;
-    with whole 16-byte pairs the rate is below one in a thousand (a known residue, not understood: without the
-    preceding writing kernel no launch has ever differed).  The test fails when more than 3 of 1500 launches
-    differ from the oracle's optimum and feasible count (or are flagged MMEE_ERR_CHECK by the finalize step's own
-    check of its winners), i.e. when the torn-pair rate is back."""
+    lines (what the benchmark does between steps): every launch returns the oracle's list.  (A search kernel
+    that read the list length k from the shared-memory copy of its plan before the barrier that completes the
+    copy passed every single-launch test and failed this one in about one launch in a hundred: after the
+    writing kernel the copy is slower, and a warp that ran ahead took k from what the previous kernel had left
+    in shared memory.)"""
     cfg = mi.config1()
-    obj = cfg["searches"][0]
+    obj = dict(cfg["searches"][0], topk=topk)
     want = oracle.search(oracle.make_problem(cfg["workload"], cfg["arch"], obj))
-    expected = (want.topk[0].idx, want.n_feasible, want.topk[0].e_key)
+    expected = (want.n_feasible, tuple((w.idx, w.e_key) for w in want.topk))
     flush = torch.empty(64 * 1024 * 1024, dtype=torch.uint8, device="cuda")
-    best = mm.result_buffer(1)
-    odd, caught = [], 0
+    best, top = mm.result_buffer(1), mm.result_buffer(topk)
     with Handle(cfg, obj) as h:
-        for it in range(1500):
-            flush.fill_(it & 255)
-            mm.mmee_search(h, best, None)
+        for it in range(1200):
+            if it < 1000:
+                flush.fill_(it & 255)
+            mm.mmee_search(h, best, top)
             torch.cuda.synchronize()
             r = mm.read_results(best, 1)[0]
-            if r.status == mm.ERR_CHECK:
-                caught += 1            # the finalize step saw a winner whose ranking key is not its own
-            elif (r.idx, r.n_feasible, r.e_key) != expected:
-                odd.append((it, r.idx, r.n_feasible, r.e_key))
-        # without the writing kernel in front, every launch agrees
-        for it in range(300):
-            mm.mmee_search(h, best, None)
-            torch.cuda.synchronize()
-            r = mm.read_results(best, 1)[0]
-            assert (r.idx, r.n_feasible, r.e_key) == expected
-    assert len(odd) + caught <= 3, (odd, caught)
+            got = (r.n_feasible, tuple((x.idx, x.e_key) for x in mm.read_results(top, topk)))
+            assert r.status == mm.OK and got == expected, (it, r.status, got[1][:2], expected[1][:2])
