@@ -1199,24 +1199,46 @@ finalize_kernel(const __grid_constant__ Plan p, Scratch* __restrict__ scratch, i
     WarpTop* wt = &tops[warp];
     if (lane == 0) wt->count = 0;
     __syncwarp();
-    for (int c = warp; c < n_partials; c += 32) {
-        const Partial* src = &scratch->partial[c];
-        const int n = src->count;
-        for (int j = 0; j < n; ++j) {
-            const longlong2 sj = src->e[j];
-            if (!warp_insert(wt, k, sj.x, (uint64_t)sj.y, lane)) break;
+    // Each warp merges every 32nd partial list.  The lists of four partials are fetched at once (lane j takes
+    // entry j; the length and the entries are independent loads), so that the merge waits for one round trip
+    // to global memory per four lists instead of one per entry.
+    constexpr int kBatch = 4;
+    for (int c0 = warp; c0 < n_partials; c0 += 32 * kBatch) {
+        int n[kBatch];
+        longlong2 mine[kBatch];
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) {
+            const int c = c0 + 32 * i;
+            n[i] = 0;
+            mine[i] = make_longlong2(kInfKey, -1ll);
+            if (c < n_partials) {
+                const Partial* src = &scratch->partial[c];
+                n[i] = src->count;
+                if (lane < MMEE_MAX_TOPK) mine[i] = src->e[lane];      // (entries past the length are not used)
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) {
+            for (int j = 0; j < n[i]; ++j) {
+                const long long sk = __shfl_sync(kFull, mine[i].x, j);
+                const long long si = __shfl_sync(kFull, mine[i].y, j);
+                if (!warp_insert(wt, k, sk, (uint64_t)si, lane)) break;   // sorted: the rest is larger
+            }
         }
     }
-    __syncthreads();
-    if (warp == 0) {
-        for (int w2 = 1; w2 < 32; ++w2) {
-            const WarpTop* src = &tops[w2];
+    // The 32 warps' lists are merged pairwise, in five rounds, into warp 0's.
+    for (int stride = 16; stride >= 1; stride >>= 1) {
+        __syncthreads();
+        if (warp < stride) {
+            const WarpTop* src = &tops[warp + stride];
             const int n = src->count;
             for (int j = 0; j < n; ++j) {
                 const longlong2 sj = src->e[j];
                 if (!warp_insert(wt, k, sj.x, (uint64_t)sj.y, lane)) break;
             }
         }
+    }
+    if (warp == 0) {
         const int found = wt->count;
         const uint64_t n_total = (p.t_end - p.t_begin) * (uint64_t)p.rows_per_tiling * 9u;
         const uint64_t n_feasible = scratch->feasible_rows * (uint64_t)p.n_sm;
