@@ -1190,15 +1190,28 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
 // finalize: merge the CTAs' partial lists, evaluate the winners in full, reset the scratch header
 // ------------------------------------------------------------------------------------------------
 
+// A sorted list held by a warp in registers: lane j holds entry j, best first; an empty slot, and every lane
+// from k on, holds (kInfKey, UINT64_MAX), which follows every mapping in the (key, idx) order.  All 32 lanes call
+// this converged.
+__device__ __forceinline__ bool reg_insert(int64_t& ek, uint64_t& ei, int k, int64_t nk, uint64_t ni, int lane) {
+    const unsigned smaller = __ballot_sync(kFull, pair_less(ek, ei, nk, ni));
+    const int pos = __popc(smaller);
+    if (pos >= k) return false;
+    const int64_t uk = __shfl_up_sync(kFull, ek, 1);
+    const uint64_t ui = __shfl_up_sync(kFull, ei, 1);
+    if (lane == pos) { ek = nk; ei = ni; }
+    else if (lane > pos && lane < k) { ek = uk; ei = ui; }
+    return true;
+}
+
 __global__ void __launch_bounds__(1024, 1)
 finalize_kernel(const __grid_constant__ Plan p, Scratch* __restrict__ scratch, int n_partials,
                 mmee_result_t* __restrict__ out_best, mmee_result_t* __restrict__ out_topk) {
-    __shared__ WarpTop tops[32];
+    __shared__ longlong2 tops[32][MMEE_MAX_TOPK];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int k = (int)p.topk;
-    WarpTop* wt = &tops[warp];
-    if (lane == 0) wt->count = 0;
-    __syncwarp();
+    int64_t ek = kInfKey;
+    uint64_t ei = UINT64_MAX;
     // Each warp merges every 32nd partial list.  The lists of four partials are fetched at once (lane j takes
     // entry j; the length and the entries are independent loads), so that the merge waits for one round trip
     // to global memory per four lists instead of one per entry.
@@ -1222,24 +1235,26 @@ finalize_kernel(const __grid_constant__ Plan p, Scratch* __restrict__ scratch, i
             for (int j = 0; j < n[i]; ++j) {
                 const long long sk = __shfl_sync(kFull, mine[i].x, j);
                 const long long si = __shfl_sync(kFull, mine[i].y, j);
-                if (!warp_insert(wt, k, sk, (uint64_t)si, lane)) break;   // sorted: the rest is larger
+                if (!reg_insert(ek, ei, k, sk, (uint64_t)si, lane)) break;   // sorted: the rest is larger
             }
         }
     }
     // The 32 warps' lists are merged pairwise, in five rounds, into warp 0's.
+    if (lane < MMEE_MAX_TOPK) tops[warp][lane] = make_longlong2((long long)ek, (long long)ei);
     for (int stride = 16; stride >= 1; stride >>= 1) {
         __syncthreads();
         if (warp < stride) {
-            const WarpTop* src = &tops[warp + stride];
-            const int n = src->count;
-            for (int j = 0; j < n; ++j) {
-                const longlong2 sj = src->e[j];
-                if (!warp_insert(wt, k, sj.x, (uint64_t)sj.y, lane)) break;
+            const longlong2 theirs = lane < MMEE_MAX_TOPK ? tops[warp + stride][lane] : make_longlong2(kInfKey, -1ll);
+            for (int j = 0; j < k; ++j) {
+                const long long sk = __shfl_sync(kFull, theirs.x, j);
+                const long long si = __shfl_sync(kFull, theirs.y, j);
+                if (!reg_insert(ek, ei, k, sk, (uint64_t)si, lane)) break;   // (an empty slot never enters)
             }
+            if (lane < MMEE_MAX_TOPK) tops[warp][lane] = make_longlong2((long long)ek, (long long)ei);
         }
     }
     if (warp == 0) {
-        const int found = wt->count;
+        const int found = __popc(__ballot_sync(kFull, ek != kInfKey || ei != UINT64_MAX));
         const uint64_t n_total = (p.t_end - p.t_begin) * (uint64_t)p.rows_per_tiling * 9u;
         const uint64_t n_feasible = scratch->feasible_rows * (uint64_t)p.n_sm;
         // Every winner is evaluated in full; the key it was ranked by must be the key of that evaluation.  A
@@ -1249,7 +1264,7 @@ finalize_kernel(const __grid_constant__ Plan p, Scratch* __restrict__ scratch, i
         if (lane < k) {
             mmee_result_t r;
             if (lane < found) {
-                evaluate_candidate(p, top_idx(wt, lane), r);
+                evaluate_candidate(p, ei, r);
                 int64_t key;
                 switch (p.objective) {
                     case MMEE_OBJ_ENERGY: key = r.e_key; break;
@@ -1258,7 +1273,7 @@ finalize_kernel(const __grid_constant__ Plan p, Scratch* __restrict__ scratch, i
                     case MMEE_OBJ_ENERGY_LCAP: key = r.l_key <= p.key_cap ? r.e_key : kInfKey; break;
                     default: key = r.e_key <= p.key_cap ? r.l_key : kInfKey; break;
                 }
-                consistent = key == top_key(wt, lane) && r.feasible && r.t >= p.t_begin && r.t < p.t_end;
+                consistent = key == ek && r.feasible && r.t >= p.t_begin && r.t < p.t_end;
             } else {
                 // empty slot
                 unsigned char* raw = reinterpret_cast<unsigned char*>(&r);
