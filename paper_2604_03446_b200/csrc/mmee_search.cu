@@ -139,6 +139,20 @@ __device__ __forceinline__ bool warp_insert(WarpTop* wt, int k, int64_t nk, uint
     return true;
 }
 
+// A sorted list held by a warp in registers: lane j holds entry j, best first; an empty slot, and every lane
+// from k on, holds (kInfKey, UINT64_MAX), which follows every mapping in the (key, idx) order.  All 32 lanes call
+// this converged.
+__device__ __forceinline__ bool reg_insert(int64_t& ek, uint64_t& ei, int k, int64_t nk, uint64_t ni, int lane) {
+    const unsigned smaller = __ballot_sync(kFull, pair_less(ek, ei, nk, ni));
+    const int pos = __popc(smaller);
+    if (pos >= k) return false;
+    const int64_t uk = __shfl_up_sync(kFull, ek, 1);
+    const uint64_t ui = __shfl_up_sync(kFull, ei, 1);
+    if (lane == pos) { ek = nk; ei = ni; }
+    else if (lane > pos && lane < k) { ek = uk; ei = ui; }
+    return true;
+}
+
 // Threshold for candidates whose indices are all >= first_idx: a key passes iff it can still enter
 // the warp's list and is not above the CTA-wide bound G.  Strict against the list's last key
 // when first_idx lies above that entry's index (a tie could then not displace it).
@@ -1168,17 +1182,26 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
 
     // ---- merge the warps' lists into warp 0's, then publish this CTA's partial list
     if (warp == 0) {
+        // (in registers, lane j holding entry j: see reg_insert)
+        int64_t ek = kInfKey;
+        uint64_t ei = UINT64_MAX;
+        if (lane < wt->count) {
+            const longlong2 own = wt->e[lane];
+            ek = own.x; ei = (uint64_t)own.y;
+        }
         for (int w2 = 1; w2 < kSearchThreads / 32; ++w2) {
             const WarpTop* src = &wtops[w2];
             const int n = src->count;
+            const longlong2 theirs = lane < n ? src->e[lane] : make_longlong2(kInfKey, -1ll);
             for (int j = 0; j < n; ++j) {
-                const longlong2 sj = src->e[j];
-                if (!warp_insert(wt, k, sj.x, (uint64_t)sj.y, lane)) break;   // sorted: the rest is larger
+                const long long sk = __shfl_sync(kFull, theirs.x, j);
+                const long long si = __shfl_sync(kFull, theirs.y, j);
+                if (!reg_insert(ek, ei, k, sk, (uint64_t)si, lane)) break;   // sorted: the rest is larger
             }
         }
         Partial* out = &scratch->partial[blockIdx.x];
-        const int n = wt->count;
-        if (lane < n) out->e[lane] = wt->e[lane];
+        const int n = __popc(__ballot_sync(kFull, ek != kInfKey || ei != UINT64_MAX));
+        if (lane < n) out->e[lane] = make_longlong2((long long)ek, (long long)ei);
         if (lane == 0) {
             out->count = n;
             if (cs->feasible_rows) atomicAdd(&scratch->feasible_rows, cs->feasible_rows);
@@ -1189,20 +1212,6 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
 // ------------------------------------------------------------------------------------------------
 // finalize: merge the CTAs' partial lists, evaluate the winners in full, reset the scratch header
 // ------------------------------------------------------------------------------------------------
-
-// A sorted list held by a warp in registers: lane j holds entry j, best first; an empty slot, and every lane
-// from k on, holds (kInfKey, UINT64_MAX), which follows every mapping in the (key, idx) order.  All 32 lanes call
-// this converged.
-__device__ __forceinline__ bool reg_insert(int64_t& ek, uint64_t& ei, int k, int64_t nk, uint64_t ni, int lane) {
-    const unsigned smaller = __ballot_sync(kFull, pair_less(ek, ei, nk, ni));
-    const int pos = __popc(smaller);
-    if (pos >= k) return false;
-    const int64_t uk = __shfl_up_sync(kFull, ek, 1);
-    const uint64_t ui = __shfl_up_sync(kFull, ei, 1);
-    if (lane == pos) { ek = nk; ei = ni; }
-    else if (lane > pos && lane < k) { ek = uk; ei = ui; }
-    return true;
-}
 
 __global__ void __launch_bounds__(1024, 1)
 finalize_kernel(const __grid_constant__ Plan p, Scratch* __restrict__ scratch, int n_partials,
