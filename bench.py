@@ -43,7 +43,7 @@ ALG_OPS_PER_CANDIDATE = {0: 1.0 + 5.0 / 9.0, 1: 2.0, 2: 6.0 + 15.0 / 9.0}
 INT_LANES_PER_SM = 64          # 4 sub-partitions x 16 integer-ALU lanes
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the exhaustive search kernels on the BERT workload,
 # from the ncu capture summarised under profiles/ (energy, latency); None for other workloads.
-NCU_DRAM_BYTES_PER_LAUNCH = {"bert": {0: 108288, 1: 121856}}
+NCU_DRAM_BYTES_PER_LAUNCH = {"bert": {0: 108032, 1: 121600}}
 
 
 WORKLOADS = {"tiny": mi.config1, "bert": mi.config2, "llama": mi.config3, "gqa": mi.config4}
