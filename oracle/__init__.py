@@ -214,5 +214,49 @@ def symbolic_prune():
     return keep, list(kept), list(total)
 
 
+class SimUnfusedOut(C.Structure):
+    _fields_ = [("loads", C.c_int64 * 5), ("c_stores", C.c_int64), ("softmax_words", C.c_int64),
+                ("op1_stages", C.c_int64), ("op2_stages", C.c_int64),
+                ("peak_op1", C.c_int64), ("peak_op2", C.c_int64)]
+
+
+def simulate_unfused(bound, pi: int, beta, phi: int) -> SimUnfusedOut:
+    """Tile-granular execution of the producer nest, the softmax pass and the consumer nest of an unfused mapping."""
+    out = SimUnfusedOut()
+    L = lib()
+    L.mo_simulate_unfused.argtypes = [C.POINTER(C.c_uint32), C.c_uint32, C.POINTER(C.c_uint32), C.c_uint32,
+                                      C.POINTER(SimUnfusedOut)]
+    rc = L.mo_simulate_unfused((C.c_uint32 * 8)(*bound), pi, (C.c_uint32 * 5)(*beta), phi, out)
+    if rc:
+        raise OracleError(rc)
+    return out
+
+
+class ArrayCounts(C.Structure):
+    _fields_ = [("cycles", C.c_int64), ("words", C.c_int64), ("macs", C.c_int64), ("rf", C.c_int64)]
+
+
+def array_tile(sm: int, m: int, r: int, n: int, rows: int, cols: int, resume: bool = False) -> ArrayCounts:
+    """Element-level execution of one (m x r) * (r x n) tile on a rows x cols PE array."""
+    out = ArrayCounts()
+    L = lib()
+    L.mo_array_tile.argtypes = [C.c_uint32] * 6 + [C.c_int, C.POINTER(ArrayCounts)]
+    rc = L.mo_array_tile(sm, m, r, n, rows, cols, int(resume), out)
+    if rc:
+        raise OracleError(rc)
+    return out
+
+
+def array_chain(bound, productions: int, sm1: int, sm2: int, rows: int, cols: int):
+    """Element-level execution of every tile invocation of both operators: (Op1 counts, Op2 counts)."""
+    out = (ArrayCounts * 2)()
+    L = lib()
+    L.mo_array_chain.argtypes = [C.POINTER(C.c_uint32)] + [C.c_uint32] * 5 + [C.POINTER(ArrayCounts)]
+    rc = L.mo_array_chain((C.c_uint32 * 8)(*bound), productions, sm1, sm2, rows, cols, out)
+    if rc:
+        raise OracleError(rc)
+    return out[0], out[1]
+
+
 def threads_used() -> int:
     return lib().mo_threads_used()

@@ -765,3 +765,194 @@ int mo_simulate(const uint32_t bound[8], uint32_t pi, const uint32_t beta[5], mo
 #undef RECORD
 #undef DROP_IF_L3
 }
+
+/* ------------------------------------------------------------------------------------------ */
+/* element-level execution of tiles on the PE array (Section V-D: compute latency from the     */
+/* array size and its utilisation, buffer<->register traffic by stationary mode)               */
+/* ------------------------------------------------------------------------------------------ */
+/*
+ * The array is rows x cols PEs.  A tile multiplies an (m x r) input block by an (r x n) weight
+ * block into an (m x n) output block.  One operand is pinned to the PEs ("stationary"), fold by
+ * fold when it is larger than the array; the other two move:
+ *   weight stationary : PE(p, q) holds weight (reduction index p, output column q); the m input
+ *                       rows stream through, one per cycle; every cycle each active column emits
+ *                       one partial sum;
+ *   input stationary  : PE(p, q) holds input (output row p, reduction index q); the n weight
+ *                       columns stream through; every cycle each active row emits one partial sum;
+ *   output stationary : PE(p, q) accumulates output (row p, column q); the r reduction steps
+ *                       stream through, each bringing one input per active row and one weight per
+ *                       active column; the outputs leave once per fold.
+ * Partial sums that leave the array before the reduction is complete are written to the buffer
+ * and read back by the fold that continues them.  Every word that crosses the buffer<->array
+ * boundary is one register-file access at the PE that takes or gives it; every MAC reads two
+ * operand registers and updates one accumulator register.
+ */
+static uint32_t active(uint32_t total, uint32_t fold, uint32_t width)
+{
+    uint32_t left = total - fold * width;
+    return left < width ? left : width;
+}
+
+int mo_array_tile(uint32_t sm, uint32_t m, uint32_t r, uint32_t n, uint32_t rows, uint32_t cols,
+                  int resume, mo_array_counts* acc)
+{
+    if (!acc || sm > 2 || !m || !r || !n || !rows || !cols) return MO_ERR_ARG;
+    int64_t cycles = 0, words = 0, macs = 0;
+    if (sm == SM_WS) {
+        for (uint32_t fr = 0; fr * rows < r; ++fr)            /* folds of the reduction dim over the rows */
+        for (uint32_t fc = 0; fc * cols < n; ++fc) {          /* folds of the output columns over the cols */
+            uint32_t ar = active(r, fr, rows), ac = active(n, fc, cols);
+            for (uint32_t pe = 0; pe < ar * ac; ++pe) ++words;             /* pin this fold's weights */
+            for (uint32_t v = 0; v < m; ++v) {                             /* stream the input rows   */
+                ++cycles;
+                for (uint32_t p = 0; p < ar; ++p) ++words;                 /* one input per active row */
+                for (uint32_t pe = 0; pe < ar * ac; ++pe) ++macs;
+                for (uint32_t q = 0; q < ac; ++q) {
+                    if (fr > 0 || resume) ++words;                         /* partial sum so far, read */
+                    ++words;                                               /* partial sum, written     */
+                }
+            }
+        }
+    } else if (sm == SM_IS) {
+        for (uint32_t fr = 0; fr * rows < m; ++fr)            /* folds of the output rows over the rows   */
+        for (uint32_t fc = 0; fc * cols < r; ++fc) {          /* folds of the reduction dim over the cols */
+            uint32_t ar = active(m, fr, rows), ac = active(r, fc, cols);
+            for (uint32_t pe = 0; pe < ar * ac; ++pe) ++words;             /* pin this fold's inputs */
+            for (uint32_t v = 0; v < n; ++v) {                             /* stream the weight columns */
+                ++cycles;
+                for (uint32_t q = 0; q < ac; ++q) ++words;                 /* one weight per active col */
+                for (uint32_t pe = 0; pe < ar * ac; ++pe) ++macs;
+                for (uint32_t p = 0; p < ar; ++p) {
+                    if (fc > 0 || resume) ++words;
+                    ++words;
+                }
+            }
+        }
+    } else {
+        for (uint32_t fr = 0; fr * rows < m; ++fr)            /* folds of the output rows over the rows    */
+        for (uint32_t fc = 0; fc * cols < n; ++fc) {          /* folds of the output columns over the cols */
+            uint32_t ar = active(m, fr, rows), ac = active(n, fc, cols);
+            if (resume)
+                for (uint32_t pe = 0; pe < ar * ac; ++pe) ++words;         /* take the partial outputs in */
+            for (uint32_t v = 0; v < r; ++v) {                             /* stream the reduction steps */
+                ++cycles;
+                for (uint32_t p = 0; p < ar; ++p) ++words;
+                for (uint32_t q = 0; q < ac; ++q) ++words;
+                for (uint32_t pe = 0; pe < ar * ac; ++pe) ++macs;
+            }
+            for (uint32_t pe = 0; pe < ar * ac; ++pe) ++words;             /* outputs leave the array */
+        }
+    }
+    acc->cycles += cycles;
+    acc->words += words;
+    acc->macs += macs;
+    acc->rf += words + 3 * macs;
+    return MO_OK;
+}
+
+int mo_array_chain(const uint32_t bound[8], uint32_t productions, uint32_t sm1, uint32_t sm2,
+                   uint32_t rows, uint32_t cols, mo_array_counts out[2])
+{
+    if (!bound || !out || !productions) return MO_ERR_ARG;
+    memset(out, 0, 2 * sizeof(mo_array_counts));
+    const uint32_t iD = bound[0], kD = bound[1], lD = bound[2], jD = bound[3];
+    const uint32_t iG = bound[4], kG = bound[5], lG = bound[6], jG = bound[7];
+    int rc = MO_OK;
+    /* Op1: every C tile is accumulated over the k2 steps; the whole of C `productions` times */
+    for (uint32_t rep = 0; rep < productions; ++rep)
+        for (uint32_t i2 = 0; i2 < iD; ++i2)
+            for (uint32_t l2 = 0; l2 < lD; ++l2)
+                for (uint32_t k2 = 0; k2 < kD; ++k2)
+                    if ((rc = mo_array_tile(sm1, iG, kG, lG, rows, cols, k2 > 0, &out[0]))) return rc;
+    /* Op2: every E tile is accumulated over the l2 steps */
+    for (uint32_t i2 = 0; i2 < iD; ++i2)
+        for (uint32_t j2 = 0; j2 < jD; ++j2)
+            for (uint32_t l2 = 0; l2 < lD; ++l2)
+                if ((rc = mo_array_tile(sm2, iG, lG, jG, rows, cols, l2 > 0, &out[1]))) return rc;
+    return MO_OK;
+}
+
+/* ------------------------------------------------------------------------------------------ */
+/* tile-granular simulator of the two unfused loop nests                                       */
+/* ------------------------------------------------------------------------------------------ */
+/*
+ * Without fusion each operator is mapped on its own (the "no fusion" baseline of Section VII-C):
+ * the producer runs its whole nest and stores every finished C tile, an optional separate pass
+ * applies the softmax to C in DRAM, then the consumer runs its nest and reads C back.  Buffer
+ * blocks behave as in mo_simulate: an operand keeps the tiles of its own loops at levels <= beta
+ * for the current values of its own loops above beta.
+ */
+int mo_simulate_unfused(const uint32_t bound[8], uint32_t pi, const uint32_t beta[5], uint32_t phi,
+                        mo_sim_unfused_out* out)
+{
+    if (!bound || !beta || !out || pi > 5 || phi < 1 || phi > 2) return MO_ERR_ARG;
+    memset(out, 0, sizeof(*out));
+    int64_t dD[4], g[4];
+    for (int d = 0; d < 4; ++d) {
+        dD[d] = bound[d]; g[d] = bound[4 + d];
+        if (dD[d] < 1 || g[d] < 1 || dD[d] > 64) return MO_ERR_ARG;
+    }
+    for (int x = 0; x < 5; ++x) if (beta[x] < 3 || beta[x] > 7) return MO_ERR_ARG;
+    if (beta[OPD_C] != 3) return MO_ERR_ARG;      /* the intermediate is not retained across the two nests */
+
+    int level_of[4];
+    level_of[LP_K] = 4;
+    level_of[ORDERS[pi][2]] = 5; level_of[ORDERS[pi][1]] = 6; level_of[ORDERS[pi][0]] = 7;
+
+    sim_block blk[5]; int64_t tile[5];
+    for (int x = 0; x < 5; ++x) {
+        blk[x].n0 = dD[OWN[x][0]]; blk[x].n1 = dD[OWN[x][1]];
+        blk[x].present = (uint8_t*)calloc((size_t)(blk[x].n0 * blk[x].n1), 1);
+        blk[x].count = 0; blk[x].valid = 0; blk[x].ident[0] = blk[x].ident[1] = -1;
+        tile[x] = g[OWN[x][0]] * g[OWN[x][1]];
+    }
+    int64_t val[4] = {0, 0, 0, 0};
+
+    /* producer nest: i2 and l2 in the order's relative order, k2 innermost */
+    int outer1 = -1, inner1 = -1;
+    for (int q = 0; q < 3; ++q) {
+        int lp = ORDERS[pi][q];
+        if (lp == LP_J) continue;
+        if (outer1 < 0) outer1 = lp; else inner1 = lp;
+    }
+    for (int64_t a = 0; a < dD[outer1]; ++a)
+    for (int64_t b = 0; b < dD[inner1]; ++b) {
+        val[outer1] = a; val[inner1] = b;
+        for (int64_t k2 = 0; k2 < dD[LP_K]; ++k2) {
+            val[LP_K] = k2;
+            out->loads[OPD_A] += block_touch(&blk[OPD_A], OPD_A, (int)beta[OPD_A], level_of, val);
+            out->loads[OPD_B] += block_touch(&blk[OPD_B], OPD_B, (int)beta[OPD_B], level_of, val);
+            (void)block_touch(&blk[OPD_C], OPD_C, 3, level_of, val);
+            int64_t occ = blk[OPD_A].count * tile[OPD_A] + blk[OPD_B].count * tile[OPD_B]
+                        + blk[OPD_C].count * tile[OPD_C];
+            if (occ > out->peak_op1) out->peak_op1 = occ;
+            out->op1_stages++;
+        }
+        out->c_stores += tile[OPD_C];              /* the finished tile goes to DRAM */
+    }
+    block_clear(&blk[OPD_C]);
+
+    /* separate softmax pass: every C tile is read and written once more */
+    if (phi == 2)
+        for (int64_t a = 0; a < dD[LP_I]; ++a)
+            for (int64_t b = 0; b < dD[LP_L]; ++b)
+                out->softmax_words += 2 * tile[OPD_C];
+
+    /* consumer nest: the order's three loops */
+    const int o7 = ORDERS[pi][0], o6 = ORDERS[pi][1], o5 = ORDERS[pi][2];
+    val[LP_K] = 0;
+    for (int64_t a7 = 0; a7 < dD[o7]; ++a7)
+    for (int64_t a6 = 0; a6 < dD[o6]; ++a6)
+    for (int64_t a5 = 0; a5 < dD[o5]; ++a5) {
+        val[o7] = a7; val[o6] = a6; val[o5] = a5;
+        out->loads[OPD_C] += block_touch(&blk[OPD_C], OPD_C, 3, level_of, val);
+        out->loads[OPD_D] += block_touch(&blk[OPD_D], OPD_D, (int)beta[OPD_D], level_of, val);
+        out->loads[OPD_E] += block_touch(&blk[OPD_E], OPD_E, (int)beta[OPD_E], level_of, val);
+        int64_t occ = blk[OPD_C].count * tile[OPD_C] + blk[OPD_D].count * tile[OPD_D]
+                    + blk[OPD_E].count * tile[OPD_E];
+        if (occ > out->peak_op2) out->peak_op2 = occ;
+        out->op2_stages++;
+    }
+    for (int x = 0; x < 5; ++x) { out->loads[x] *= tile[x]; free(blk[x].present); }
+    return MO_OK;
+}

@@ -16,9 +16,15 @@
  *   - MAC/softmax counts of Section V-D, Table I Accel.-1 closed-form latency,
  *   - row-count arithmetic of Sections VI-B / VII-C (18 750 rows, 18 groups),
  *   - brute-force sort for argmin / top-k.
- * PARITY UNPINNED by the paper (builder-defined readings, checked only by hand
- * on one tile): buffer<->PE traffic BR, register-file count N_RF, the unfused
- * rows (phi = 1, 2), absolute energies.
+ *   - an element-level execution of tiles on the PE array (mo_array_tile /
+ *     mo_array_chain) for cycles, buffer<->array words, carried partial sums,
+ *     MACs and register-file accesses,
+ *   - a tile-granular execution of the two unfused loop nests
+ *     (mo_simulate_unfused) for the rows of phi = 1, 2.
+ * PARITY UNPINNED by the paper: absolute energies (its 28 nm energy table is
+ * not printed); the array model itself (which operand each stationary mode
+ * pins to which array dimension) is this build's reading, stated in
+ * mo_array_tile.
  */
 #ifndef MMEE_ORACLE_H
 #define MMEE_ORACLE_H
@@ -118,6 +124,39 @@ int  mo_keys_range(const mo_problem*, uint64_t begin, uint64_t count, int64_t* k
 int  mo_search(const mo_problem*, mo_record* out_topk, uint64_t* n_total, uint64_t* n_feasible,
                uint32_t* n_found, int n_threads);
 int  mo_simulate(const uint32_t bound[8], uint32_t pi, const uint32_t beta[5], mo_sim_out* out);
+
+/* Tile-granular execution of the two separate loop nests of an unfused mapping (phi = 1, 2): the
+ * producer nest (k2 innermost, then i2 / l2 in the order's relative order; every finished C tile is
+ * stored), the optional softmax pass over C, and the consumer nest (the order's three loops; C at L3
+ * is read back).  Counts tile loads / stores per operand and the peak occupancy of each nest; uses
+ * none of the closed forms. */
+typedef struct {
+    int64_t  loads[5];                     /* words loaded per operand; C: read back by the consumer nest */
+    int64_t  c_stores;                     /* words of C stored by the producer nest                      */
+    int64_t  softmax_words;                /* words moved by the separate softmax pass (phi = 2)          */
+    int64_t  op1_stages, op2_stages;
+    int64_t  peak_op1, peak_op2;           /* occupancy in words                                          */
+} mo_sim_unfused_out;
+int  mo_simulate_unfused(const uint32_t bound[8], uint32_t pi, const uint32_t beta[5], uint32_t phi,
+                         mo_sim_unfused_out* out);
+
+/* Element-level execution of tiles on a rows x cols PE array, for the array-level terms of the
+ * model (compute cycles, buffer<->array words, MACs, register-file accesses).  Written as loops
+ * over folds, streamed vectors and PEs that count events; none of the ceiling formulas appear. */
+typedef struct {
+    int64_t cycles;                        /* one per streamed vector per fold                            */
+    int64_t words;                         /* words crossing the buffer<->array boundary, both directions */
+    int64_t macs;                          /* multiply-accumulates performed by the PEs                   */
+    int64_t rf;                            /* register-file accesses                                      */
+} mo_array_counts;
+/* One (m x r) * (r x n) tile; resume != 0: the output tile already holds partial sums of earlier
+ * reduction steps in the buffer, which the array has to take in first.  Adds to *acc. */
+int  mo_array_tile(uint32_t sm, uint32_t m, uint32_t r, uint32_t n, uint32_t rows, uint32_t cols,
+                   int resume, mo_array_counts* acc);
+/* Every tile invocation of both operators of one tiling in loop order: Op1 = C(i2,l2) += A*B over
+ * k2, the whole of it `productions` times (recomputation), Op2 = E(i2,j2) += C*D over l2. */
+int  mo_array_chain(const uint32_t bound[8], uint32_t productions, uint32_t sm1, uint32_t sm2,
+                    uint32_t rows, uint32_t cols, mo_array_counts out[2]);
 int  mo_threads_used(void);
 
 /* Symbolic form of one fused row (Section V-E): every BS_X / DA_X as the set of loop bounds it is the

@@ -80,7 +80,6 @@ static_assert(offsetof(OrderTab, Ac) % 16 == 0 && offsetof(OrderTab, Bc) % 16 ==
 struct alignas(16) TilingTab {
     uint32_t b[8];
     int64_t half[2][16];    // products of every subset of the four x_D bounds / of the four x_G bounds
-    int32_t Wc[2][12];      // W[s][rc] - wmin[rc], saturated to kTermCap (entries 9..11 unused)
     int64_t W[9][2];        // energy of buffer<->PE traffic, MACs and softmax, in quanta
     int64_t CB[9][2];       // fused compute time in words (cycles * words per cycle)
     int64_t QU[9][2];       // unfused Op2 compute time in words, by s (sm2 = s % 3)
@@ -88,12 +87,12 @@ struct alignas(16) TilingTab {
     int64_t cw, smx;        // C write-back words (I*L); separate softmax pass words (2*I*L)
     int64_t wmin[2];        // min over the stationary pairs of W[.][rc]
     int64_t qmin[3];        // min over the stationary pairs of CB[.][0], CB[.][1], QU[.][0]
-    int32_t Qrel[3][12];    // CB[s][0], CB[s][1], QU[s][0] minus that minimum, saturated to kTermCap (kUnfit: pair not offered)
+    int32_t Qrel[3][12];    // CB[s][0], CB[s][1], QU[s][0] minus that minimum, saturated to kTermCap (kUnfit: pair not offered);
+                            // entries 9..11: the least of the three entries of each sm1
     int32_t live;           // smallest possible buffer need of this tiling fits
     int32_t pad[3];
 };
-static_assert(offsetof(TilingTab, Wc) % 16 == 0 && offsetof(TilingTab, Qrel) % 16 == 0 && sizeof(int32_t[12]) % 16 == 0,
-              "Wc and Qrel rows are read as int4");
+static_assert(offsetof(TilingTab, Qrel) % 16 == 0 && sizeof(int32_t[12]) % 16 == 0, "Qrel rows are read as int4");
 static_assert(offsetof(RowTab, Ec) % 16 == 0 && offsetof(OrderTab, rt) % 16 == 0 && sizeof(RowTab) % 16 == 0,
               "Ec rows are read as int4");
 // 21 items per tiling: 9 stationary pairs x 2 recompute flags, 3 unfused Op1 terms
@@ -438,6 +437,12 @@ __device__ __forceinline__ void build_order_item(const Plan& p, const TilingTab*
         }
         fc[3] = 0;
         uc[3] = 0;
+        if constexpr (OBJ == MMEE_OBJ_EDP) {
+            // the energy-delay filter's first level works on single-precision lower bounds: DRAM words and their
+            // energy, each rounded down
+            fc[2] = __float_as_int(__ll2float_rd(fr[2])); fc[3] = __float_as_int(__ll2float_rd(fr[3]));
+            uc[2] = __float_as_int(__ll2float_rd(ur[2])); uc[3] = __float_as_int(__ll2float_rd(ur[3]));
+        }
     } else {
         const int64_t v = monomial(q.da_unfused[order][OP_C][0]);
         ot->gCr = scale * v;
@@ -522,6 +527,7 @@ struct MidExact {
     int64_t P[3];               // unfused latency: Op1 stage and softmax pass, by sm1
     const int64_t* wptr;        // W[s][rc], stride 2
     const int64_t* qptr;        // compute words by s, stride 2
+    uint32_t rc;                // C is regenerated (fused tasks)
 };
 
 template <int OBJ>
@@ -542,6 +548,7 @@ __device__ __forceinline__ MidExact mid_exact(const Plan& p, const TilingTab* tb
     r.slack2 = live ? p.cap_words - (c1 + a2 + b2) : -1;
     const int64_t gab = ot->gA[la][rc] + ot->gB[lb][rc];
     r.wptr = &tb->W[0][rc];
+    r.rc = rc;
     r.xe0 = 0;
     if constexpr (OBJ == MMEE_OBJ_ENERGY) {
         const int64_t extra = p.c_dram_gb * (tb->cw + (phi == 2 ? tb->smx : 0));
@@ -657,6 +664,36 @@ __device__ __noinline__ void exact_group_single(const Plan& p, const TilingTab* 
     __syncwarp();
 }
 
+// Second level of the energy-delay filter, for a group whose single-precision bound passed in some lane: every
+// mapping of the group's five rows in double precision on the FP64 pipe (energy and latency sums converted once per
+// row, then an add, two multiplies and two compares per mapping).  Each approximate product is within a few 2^-53
+// of the exact key, so comparing against the threshold widened by 1e-14 relative can flag a row needlessly but never
+// miss one; the exact path decides.  Returns 1 if some row fits and holds such a product.
+__device__ __noinline__ unsigned edp_group_test(const MidExact& me, const RowTab* rt, int d, int s1c, int s2c,
+                                                uint32_t kept_rows, uint32_t sm_mask, double dthr) {
+    double dW[9], dQP[9];
+#pragma unroll
+    for (int s = 0; s < 9; ++s) {
+        // (a pair the array does not offer: infinite energy, flagged at most while no bound exists yet)
+        dW[s] = ((sm_mask >> s) & 1u) ? (double)me.wptr[2 * s] : __longlong_as_double(0x7ff0000000000000ll);
+        dQP[s] = (double)(me.qptr[2 * s] + me.P[s / 3]);
+    }
+    const int64_t xd = me.x0 + rt->D[d][2];
+    const int64_t xed = me.xe0 + rt->D[d][3];
+    unsigned hit_any = 0;
+#pragma unroll 1
+    for (int e = 0; e < 5; ++e) {
+        const unsigned fit = (unsigned)(rt->Ec[e][0] <= s1c) & (unsigned)(rt->Ec[e][1] <= s2c) & (kept_rows >> e);   // Eq. (4)
+        const int64_t x = xd + rt->E[e][2];
+        const double de = (double)(xed + rt->E[e][3]);
+        double dl[3];
+#pragma unroll
+        for (int j = 0; j < 3; ++j) dl[j] = (double)(x + me.P[j]);
+        hit_any |= edp_row_test(de, dl, dW, dQP, dthr, fit & 1u);
+    }
+    return hit_any;
+}
+
 // The walk in 64-bit keys: the energy-delay product (double-precision filter, see edp_row_test),
 // the capped objectives and the key dump.  Returns the number of rows that fit.
 template <int OBJ, bool DUMP, bool PRUNE>
@@ -669,10 +706,12 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
     LaneThreshold th = load_threshold(wt, cs, k);
     uint32_t rows = 0;
     int E1c[5], E2c[5];
+    float Egf[5], Eef[5];       // EDP: lower bounds of E's DRAM words and of their energy
 #pragma unroll
     for (int e = 0; e < 5; ++e) {
         const int4 v = *reinterpret_cast<const int4*>(rt->Ec[e]);
         E1c[e] = v.x; E2c[e] = v.y;
+        Egf[e] = __int_as_float(v.z); Eef[e] = __int_as_float(v.w);
     }
 #pragma unroll 1
     for (int mi = 0; mi < (PRUNE ? 1 : 5); ++mi) {
@@ -685,25 +724,33 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
             W[s] = me.wptr[2 * s];
             Q[s] = me.qptr[2 * s];
         }
-        double dW[9], dQP[9], dthr = 0.0;
-        if constexpr (OBJ == MMEE_OBJ_EDP) {
-#pragma unroll
-            for (int s = 0; s < 9; ++s) {
-                // (a pair the array does not offer: infinite energy, flagged at most while no bound exists yet)
-                dW[s] = ((p.sm_mask >> s) & 1u) ? (double)W[s] : __longlong_as_double(0x7ff0000000000000ll);
-                dQP[s] = (double)(Q[s] + me.P[s / 3]);
-            }
+        // Energy-delay product: the first filter level is one single-precision lower bound per row,
+        // (row energy + least stationary-pair energy) * max(row DRAM words + least Op1 stage, least compute
+        // words + least Op1 stage), every conversion, sum and product rounded down, against the threshold
+        // rounded up: no mapping of a row is below its row's bound.
+        double dthr = 0.0;
+        float fthr = 0.f, fe0 = 0.f, fx0 = 0.f, fq = 0.f;
+        if constexpr (!DUMP && OBJ == MMEE_OBJ_EDP) {
+            const int64_t pmin = min(me.P[0], min(me.P[1], me.P[2]));
+            fe0 = __ll2float_rd(me.xe0 + tb->wmin[me.rc]);
+            fx0 = __ll2float_rd(me.x0 + pmin);
+            fq = __ll2float_rd(tb->qmin[c.phi == 0 ? me.rc : 2u] + pmin);
         }
         auto refresh = [&]() {
             if constexpr (OBJ == MMEE_OBJ_EDP) {
                 // EDP keys are bit patterns of positive doubles; anything from +inf up means "no bound yet"
                 dthr = th.T1 >= 0x7ff0000000000000ll ? __longlong_as_double(0x7ff0000000000000ll)
                                                     : __longlong_as_double(th.T1) * (1.0 + 1e-14);
+                fthr = __double2float_ru(dthr);
             }
         };
         refresh();
         const int slack1c = me.slack1 < 0 ? -1 : (int)me.slack1;      // slack <= capacity < 2^30
         const int slack2c = me.slack2 < 0 ? -1 : (int)me.slack2;
+        if constexpr (!DUMP && OBJ == MMEE_OBJ_EDP) {
+            // no lane has room left for D and E at this middle level: none of its 25 rows fits
+            if (!__any_sync(kFull, (slack1c | slack2c) >= 0)) continue;
+        }
 
 #pragma unroll 1
         for (int d = 0; d < 5; ++d) {
@@ -712,29 +759,24 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
             }
             unsigned hit_any = 0, fits = 0;
             if constexpr (!DUMP && OBJ == MMEE_OBJ_EDP) {
-                // The energy-delay product is not separable, so the filter is a double-precision
-                // evaluation of every mapping on the FP64 pipe: energy and latency sums converted
-                // once per row, then an add, two multiplies and two compares per mapping.  Each
-                // approximate product is within a few 2^-53 of the exact key, so comparing against
-                // the threshold widened by 1e-14 relative can flag a row needlessly but never miss
-                // one; the exact path decides.
                 const int4 dc = *reinterpret_cast<const int4*>(rt->Dc[d]);
                 const int s1c = slack1c - dc.x;
                 const int s2c = slack2c - dc.y;
-                const int64_t xd = me.x0 + rt->D[d][2];
-                const int64_t xed = me.xe0 + rt->D[d][3];
+                if (!__any_sync(kFull, (s1c | s2c) >= 0)) continue;     // D leaves no room in any lane
+                const float fxd = __fadd_rd(fx0, __int_as_float(dc.z));
+                const float fed = __fadd_rd(fe0, __int_as_float(dc.w));
+                const uint32_t kd = PRUNE ? (kept >> (d * 5)) : 31u;
+                unsigned hit1 = 0;
 #pragma unroll
                 for (int e = 0; e < 5; ++e) {
                     unsigned fit = (unsigned)(E1c[e] <= s1c) & (unsigned)(E2c[e] <= s2c);             // Eq. (4)
-                    if constexpr (PRUNE) fit &= kept >> (d * 5 + e);
+                    if constexpr (PRUNE) fit &= kd >> e;
                     fits += fit;
-                    const int64_t x = xd + rt->E[e][2];
-                    const double de = (double)(xed + rt->E[e][3]);
-                    double dl[3];
-#pragma unroll
-                    for (int j = 0; j < 3; ++j) dl[j] = (double)(x + me.P[j]);
-                    hit_any |= edp_row_test(de, dl, dW, dQP, dthr, fit);
+                    const float fl = fmaxf(__fadd_rd(fxd, Egf[e]), fq);
+                    const float lb = __fmul_rd(__fadd_rd(fed, Eef[e]), fl);
+                    hit1 |= fit & (unsigned)(lb <= fthr);
                 }
+                if (__any_sync(kFull, hit1 != 0u)) hit_any = edp_group_test(me, rt, d, s1c, s2c, kd, p.sm_mask, dthr);
             } else {
                 const int64_t s1 = me.slack1 - rt->D[d][0];
                 const int64_t s2 = me.slack2 - rt->D[d][1];
@@ -859,44 +901,45 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
         const int slack1c = live ? (fused ? max(room1, -1) : (room1 >= 0 ? kSizeCap : -1)) : -1;
         const int slack2c = live ? max(capc - y2, -1) : -1;
 
-        int u = 0, Wc[9], ua[3], Qc[9];
-        if constexpr (OBJ == MMEE_OBJ_ENERGY) {
-            const int4* wc4 = reinterpret_cast<const int4*>(tb->Wc[rc]);
-            const int4 w0 = wc4[0], w1 = wc4[1], w2 = wc4[2];
-            Wc[0] = w0.x; Wc[1] = w0.y; Wc[2] = w0.z; Wc[3] = w0.w;
-            Wc[4] = w1.x; Wc[5] = w1.y; Wc[6] = w1.z; Wc[7] = w1.w;
-            Wc[8] = w2.x;
+        // No lane has room left for D and E at this middle level: none of its 25 rows fits.
+        if (!__any_sync(kFull, (slack1c | slack2c) >= 0)) {
+            if constexpr (!PRUNE) unfit -= 25;
+            continue;
         }
-        // the part of the set-up that depends on the threshold: redone after a visit of the exact path
+
+        // u: the part of key - thr that is fixed by (task, middle level), with the least stationary-pair term
+        // already inside.  The minimum of a row's nine keys is its row sum plus the least stationary-pair
+        // term (energy), or the larger of its DRAM words and the least compute words (latency), so the
+        // nine mappings of a row need one test, not nine.  (Redone after a visit of the exact path.)
+        int u = 0;
         auto mid_setup = [&]() {
             if constexpr (OBJ == MMEE_OBJ_ENERGY) {
                 u = __viaddmin_s32(rc ? base[1] : base[0], rc ? bv.w : bv.z, kRowCap);
             } else {
-                int qo[3];
-                const int32_t* qrel;
+                // max(x, Q) < thr  <=>  x < thr and Q < thr: when even the least compute words reach the
+                // threshold, no row of this middle level passes
                 if (fused) {
-                    ua[0] = ua[1] = ua[2] = rc ? ua2[1] : ua2[0];
-                    qo[0] = qo[1] = qo[2] = rc ? qo2[1] : qo2[0];
-                    qrel = tb->Qrel[rc];       // (a shared-memory address, not a register array)
+                    u = (rc ? qo2[1] : qo2[0]) < 0 ? (rc ? ua2[1] : ua2[0]) : kRowCap;
                 } else {
                     // unfused latency: max(DA1, C1) + softmax pass + max(DA2, C2); the first two terms are
-                    // fixed by (level of A, level of B = m, sm1)
+                    // fixed by (level of A, level of B = m, sm1).  Least Op1 stage over the sm1 the array
+                    // offers, least (Op1 stage + Op2 compute words) over the offered pairs.
                     const int64_t da1 = ot->gA[c.la][0] + ot->gB[m][0] + tb->cw;
                     const int64_t pass = c.phi == 2 ? tb->smx : 0;
+                    const int4 qr = *reinterpret_cast<const int4*>(&tb->Qrel[2][8]);     // [9..11]: least term by sm1
+                    int um = kRowCap, qm = INT_MAX;
 #pragma unroll
                     for (int j = 0; j < 3; ++j) {
                         const int64_t c1w = tb->C1w[j];
                         const int64_t pj = (da1 > c1w ? da1 : c1w) + pass - thr;
-                        ua[j] = rel32((ot->gCr + pj) >> p.rel_shift);
-                        qo[j] = rel32((tb->qmin[2] + pj) >> p.rel_shift);
+                        const int uaj = rel32((ot->gCr + pj) >> p.rel_shift);
+                        const int qoj = rel32((tb->qmin[2] + pj) >> p.rel_shift);
+                        const int qrj = j == 0 ? qr.y : (j == 1 ? qr.z : qr.w);
+                        um = min(um, qrj < kUnfit ? uaj : kRowCap);
+                        qm = min(qm, qoj + qrj);
                     }
-                    qrel = tb->Qrel[2];
+                    u = qm < 0 ? um : kRowCap;
                 }
-                const int4* q4 = reinterpret_cast<const int4*>(qrel);
-                const int4 q0 = q4[0], q1 = q4[1], q2 = q4[2];
-                Qc[0] = imad(qo[0], one, q0.x); Qc[1] = imad(qo[0], one, q0.y); Qc[2] = imad(qo[0], one, q0.z);
-                Qc[3] = imad(qo[1], one, q0.w); Qc[4] = imad(qo[1], one, q1.x); Qc[5] = imad(qo[1], one, q1.y);
-                Qc[6] = imad(qo[2], one, q1.z); Qc[7] = imad(qo[2], one, q1.w); Qc[8] = imad(qo[2], one, q2.x);
             }
         };
         mid_setup();
@@ -908,7 +951,6 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
             }
             // Five rows (levels of E) are evaluated branch-free; one vote decides whether any lane of the
             // warp has to enter the exact path for this group.
-            if constexpr (PRUNE) ++groups;
             const int4 dc = *reinterpret_cast<const int4*>(rt->Dc[d]);
             const int s1c = imad(dc.x, minus_one, slack1c);
             const int s2c = imad(dc.y, minus_one, slack2c);
@@ -916,43 +958,26 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
             // runs (size <= s2c, given s1c >= 0); retained, it must fit beside both operators' operands
             const int lim_l3 = s1c >= 0 ? s2c : -1;
             const int lim_retained = min(s1c, s2c);
-            const uint32_t kd = kept >> (d * 5);
-            int a0 = INT_MAX, a1 = INT_MAX, a2 = INT_MAX;
-            bool hit;
-            if constexpr (OBJ == MMEE_OBJ_ENERGY) {
-                const int uc = __viaddmin_s32(u, dc.z, kRowCap);
-#pragma unroll
-                for (int e = 0; e < 5; ++e) {
-                    // t = -1 if the row does not fit (Eq. 4), else 0; such a row's keys are moved up by kUnfit,
-                    // which makes them non-negative
-                    int t = sign_mask(imad(E2c[e], minus_one, e == 0 ? lim_l3 : lim_retained));
-                    if constexpr (PRUNE) t |= (int)((kd >> e) & 1u) - 1;
-                    unfit = imad(t, one, unfit);
-                    const int xc = imad(t, -kUnfit, imad(uc, one, Gc[e]));
-                    // one fused add-min per mapping: min(key_s - thr)
-                    a0 = __viaddmin_s32(xc, Wc[0], a0); a1 = __viaddmin_s32(xc, Wc[1], a1); a2 = __viaddmin_s32(xc, Wc[2], a2);
-                    a0 = __viaddmin_s32(xc, Wc[3], a0); a1 = __viaddmin_s32(xc, Wc[4], a1); a2 = __viaddmin_s32(xc, Wc[5], a2);
-                    a0 = __viaddmin_s32(xc, Wc[6], a0); a1 = __viaddmin_s32(xc, Wc[7], a1); a2 = __viaddmin_s32(xc, Wc[8], a2);
-                }
-                hit = __vimin3_s32(a0, a1, a2) < 0;
-            } else {
-                int uc[3];
-#pragma unroll
-                for (int j = 0; j < 3; ++j) uc[j] = __viaddmin_s32(ua[j], dc.z, kRowCap);
-#pragma unroll
-                for (int e = 0; e < 5; ++e) {
-                    int t = sign_mask(imad(E2c[e], minus_one, e == 0 ? lim_l3 : lim_retained));      // -1: the row does not fit
-                    if constexpr (PRUNE) t |= (int)((kd >> e) & 1u) - 1;
-                    unfit = imad(t, one, unfit);
-                    const int ge = imad(t, -kUnfit, Gc[e]);
-                    int v[9];                                    // one fused add-max per mapping: key_s - thr
-#pragma unroll
-                    for (int s = 0; s < 9; ++s) v[s] = __viaddmax_s32(uc[s / 3], ge, Qc[s]);
-                    a0 = __vimin3_s32(a0, v[0], v[1]); a1 = __vimin3_s32(a1, v[2], v[3]); a2 = __vimin3_s32(a2, v[4], v[5]);
-                    a0 = __vimin3_s32(a0, v[6], v[7]); a1 = min(a1, v[8]);
-                }
-                hit = __vimin3_s32(a0, a1, a2) < 0;
+            // D leaves no room in any lane: none of the group's five rows fits
+            if (!__any_sync(kFull, lim_l3 >= 0)) {
+                if constexpr (!PRUNE) unfit -= 5;
+                continue;
             }
+            if constexpr (PRUNE) ++groups;
+            const uint32_t kd = kept >> (d * 5);
+            const int uc = __viaddmin_s32(u, dc.z, kRowCap);
+            int g[5];
+#pragma unroll
+            for (int e = 0; e < 5; ++e) {
+                // t = -1 if the row does not fit (Eq. 4), else 0; such a row's term is moved up by kUnfit,
+                // which makes its keys non-negative whatever the threshold
+                int t = sign_mask(imad(E2c[e], minus_one, e == 0 ? lim_l3 : lim_retained));
+                if constexpr (PRUNE) t |= (int)((kd >> e) & 1u) - 1;
+                unfit = imad(t, one, unfit);
+                g[e] = Gc[e] | (t & kUnfit);             // (Gc <= kTermCap < kUnfit, a single bit)
+            }
+            // least key of the group's 45 mappings, relative to the threshold
+            const bool hit = uc + __vimin3_s32(__vimin3_s32(g[0], g[1], g[2]), g[3], g[4]) < 0;
             if (__any_sync(kFull, hit)) {
                 if (k == 1) exact_group_single<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, lane);
                 else exact_group<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, k, lane);
@@ -1070,7 +1095,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
         tiling_pass(0, 18);     // stationary pairs x recompute flag
         tiling_pass(18, 3);     // unfused Op1 compute words
         sync();
-        if (OBJ == MMEE_OBJ_LATENCY) {
+        if (OBJ == MMEE_OBJ_LATENCY || OBJ == MMEE_OBJ_EDP) {
             // compute words relative to their minimum over the stationary pairs: fused without and with
             // recomputation, and Op2 of an unfused task
             for (uint32_t j = first; j < 3 * n_slots; j += step) {
@@ -1088,24 +1113,23 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                     // bring below zero)
                     tb->Qrel[v][s] = !((p.sm_mask >> s) & 1u) ? kUnfit : (qs > (int64_t)kTermCap ? kTermCap : (int32_t)qs);
                 }
+                // entries 9..11: the least term of each Op1 stationary mode (kUnfit: none of its pairs is offered)
+                for (int j2 = 0; j2 < 3; ++j2) {
+                    const int32_t* r = &tb->Qrel[v][3 * j2];
+                    tb->Qrel[v][9 + j2] = min(r[0], min(r[1], r[2]));
+                }
             }
         }
-        if (OBJ == MMEE_OBJ_ENERGY) {
-            // threshold-relative stationary-pair terms (see "32-bit differential keys")
+        if (OBJ == MMEE_OBJ_ENERGY || OBJ == MMEE_OBJ_EDP) {
+            // The least stationary-pair energy term, over the pairs the array offers (never none): a row's least
+            // energy over its nine mappings is its row sum plus this.
             for (uint32_t j = first; j < 2 * n_slots; j += step) {
                 TilingTab* tb = &ttabs[j >> 1];
                 const int rc = (int)(j & 1);
-                // The minimum runs over the stationary pairs the array offers (never none).  A pair it does not
-                // offer gets the largest term: the row's minimum over s is then still that of an offered pair.
                 int64_t m = kInfKey;
                 for (int s = 0; s < 9; ++s)
                     if ((p.sm_mask >> s) & 1u) m = tb->W[s][rc] < m ? tb->W[s][rc] : m;
                 tb->wmin[rc] = m;
-                for (int s = 0; s < 9; ++s) {
-                    const int64_t wd = tb->W[s][rc] - m;
-                    const int64_t ws = wd >> p.rel_shift;
-                    tb->Wc[rc][s] = (ws > (int64_t)kTermCap || !((p.sm_mask >> s) & 1u)) ? kTermCap : (int32_t)ws;
-                }
             }
         }
     };
