@@ -67,9 +67,10 @@ extern "C" {
 #define MMEE_ERR_CUDA         5   /* a CUDA runtime call failed (no device, launch error, ...)     */
 #define MMEE_ERR_TIMEOUT      6   /* reserved: the kernels contain no device-side wait             */
 #define MMEE_ERR_RANGE        7   /* request exceeds a documented maximum                          */
-#define MMEE_ERR_CHECK        8   /* out_best->status only: a winner's ranking key is not the key of its full
-                                     evaluation (internal consistency check of the finalize step); the records
-                                     are not to be trusted, search again                              */
+#define MMEE_ERR_CHECK        8   /* a winner's ranking key is not the key of its full evaluation (internal
+                                     consistency check of the finalize step): the records are not a result.
+                                     In out_best->status after mmee_search; the return value of the
+                                     synchronous entry points (mmee_solve_host, mmee_search_shapes, ...)  */
 
 /* Attention workload.  Heads are independent instances of one search (Section V, first
  * paragraph); the q_heads/kv_heads query heads that share a K/V head are stacked along I. */
@@ -101,7 +102,8 @@ typedef struct {
                                                 topk = 1.  Rows that a lower-index row dominates for every
                                                 tiling are not evaluated: the optimum is unchanged, but
                                                 n_feasible then counts only the evaluated rows.        */
-    uint64_t t_begin, t_end;                 /* tiling sub-range [t_begin,t_end); 0,0 = all       */
+    uint64_t t_begin, t_end;                 /* tiling sub-range [t_begin,t_end); the pair 0,0 stands for
+                                                the whole space, so an empty range cannot start at 0   */
     int64_t  key_cap;                        /* MMEE_OBJ_*CAP: bound on the other key (energy in quanta,
                                                 latency in words); ignored otherwise                   */
     uint32_t stationary_mask;                /* bit 3*sm1+sm2 set: the array offers that stationary pair
@@ -157,7 +159,9 @@ int mmee_create(const mmee_workload_t* workload, const mmee_arch_t* arch,
  *              fits, status = MMEE_ERR_NO_FEASIBLE with idx = MMEE_NO_INDEX.
  *   out_topk : DEVICE, objective.topk entries, best first, unused slots idx = MMEE_NO_INDEX;
  *              may be NULL.
- * Caller owns both buffers.  Calls on one handle must not overlap on the GPU.
+ * Caller owns both buffers.  Calls on one handle must not overlap on the GPU.  The handle's device
+ * must be the current device (MMEE_ERR_ARG otherwise; the same holds for mmee_eval, mmee_decode and
+ * mmee_dump_keys).
  */
 int mmee_search(mmee_handle_t* handle, void* cuda_stream, mmee_result_t* out_best,
                 mmee_result_t* out_topk);
@@ -173,13 +177,15 @@ int mmee_destroy(mmee_handle_t* handle);
  * library then fails), or a latency-critical loop that cannot afford the device-wide
  * synchronisation of cudaMalloc / cudaFree.  This call makes no cudaMalloc, cudaFree or other
  * allocating call.  Its scratch (work counter, pruning bound, one partial top-k list per CTA) is a
- * fixed 139 296-byte array inside the library image, present on every device that loads the
+ * fixed 139 312-byte array inside the library image, present on every device that loads the
  * library for as long as the process lives.
  *
  *   workload, arch, objective : HOST, as for mmee_create; planned on the host at every call.
  *   out_best, out_topk        : DEVICE, caller-owned, as for mmee_search (out_topk may be NULL).
  * Asynchronous on `cuda_stream`.  The first call on a device looks up the array's device address
- * (with that device current); make that first call before any stream capture begins.
+ * (with that device current); make that first call before any stream capture begins.  The address
+ * is kept for the life of the process: after a cudaDeviceReset it is stale, and this entry point
+ * must not be called on that device again.
  * objective.row_pruning must be 0 here (its kept-row list would need a device allocation).
  * Limits: the array holds the partial lists of at most 512 persistent CTAs; a device whose launch
  * shape needs more is refused with MMEE_ERR_RANGE.  Other errors as mmee_create / mmee_search.
@@ -212,8 +218,20 @@ int mmee_eval(mmee_handle_t* handle, void* cuda_stream, uint64_t idx_begin, uint
               mmee_result_t* out);
 
 /*
- * mmee_dump_keys -- run the search kernel's own evaluation path over the handle's tiling range
- * and store every candidate's objective key instead of reducing (Eq. 11: the full result matrix).
+ * mmee_decode -- one candidate index back to its mapping (tiling, order, levels, stationary pair;
+ * index layout at the top of this file) with its full evaluation (Section VI-A: the output of the
+ * search is the optimal tiling, order and buffering levels with their metrics).  The record is
+ * computed on the device by the same code as mmee_eval and copied to the host.  Synchronous.
+ *   host_out : HOST, one record.  MMEE_ERR_ARG for an index outside the handle's space.
+ */
+int mmee_decode(mmee_handle_t* handle, uint64_t idx, mmee_result_t* host_out);
+
+/*
+ * mmee_dump_keys -- run the search kernel in its key-dump mode over the handle's tiling range and
+ * store every candidate's objective key instead of reducing (Eq. 11: the full result matrix).  The
+ * dump mode shares the kernel's tables, decode and task walk, and forms every key exactly in 64 bits
+ * (the path the search takes for the energy-delay and capped objectives and for every group of rows
+ * that its 32-bit filter flags); the filter itself is not part of it.
  *   out_keys : DEVICE, (t_end - t_begin) * R * 9 int64; entry idx - t_begin*R*9.  Energy and
  *              latency keys as integers, EDP keys as the bit pattern of the double; INT64_MAX
  *              for a mapping that does not fit the buffer.
@@ -288,7 +306,7 @@ int mmee_recompute_flag(uint32_t pi, uint32_t beta_c, uint32_t* out_flag);
 
 /*
  * mmee_last_search_stats -- HOST counters of the most recent mmee_search on the handle, valid
- * after the stream has been synchronised: kernels launched by that call, persistent CTAs,
+ * after the stream has been synchronised (the call copies one counter from the device): kernels launched by that call, persistent CTAs,
  * threads per CTA, dynamic shared memory per CTA, tasks (groups of 1125 consecutive mappings) and,
  * when mmee_kernel_timing is on, the device time of the search kernel and of the finalize kernel
  * in milliseconds (CUDA events recorded on the search's stream; -1 when timing is off).
@@ -299,6 +317,10 @@ typedef struct {
     float    search_ms, finalize_ms;
     uint32_t rows_per_tiling;                /* R                                                  */
     uint32_t rows_evaluated_per_tiling;      /* R, or the rows that survive symbolic row pruning   */
+    uint64_t exact_path_visits;              /* groups of rows the 32-bit (or floating-point) filter sent to the
+                                                exact 64-bit path during that search               */
+    float    create_ms;                      /* host wall clock of the mmee_create that made the handle */
+    uint32_t reserved;
 } mmee_launch_stats_t;
 int mmee_last_search_stats(const mmee_handle_t* handle, mmee_launch_stats_t* out);
 

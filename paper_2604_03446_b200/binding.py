@@ -20,7 +20,7 @@ NO_INDEX = 2 ** 64 - 1
 OK, ERR_ARG, ERR_OVERFLOW, ERR_QUANTUM, ERR_NO_FEASIBLE, ERR_CUDA, ERR_TIMEOUT, ERR_RANGE, ERR_CHECK = range(9)
 
 EXPORTS = ("mmee_create", "mmee_search", "mmee_destroy", "mmee_search_static", "mmee_num_candidates", "mmee_num_tilings",
-           "mmee_num_rows", "mmee_strerror", "mmee_last_cuda_error", "mmee_eval", "mmee_dump_keys", "mmee_solve_host", "mmee_pareto_front", "mmee_search_shapes",
+           "mmee_num_rows", "mmee_strerror", "mmee_last_cuda_error", "mmee_eval", "mmee_decode", "mmee_dump_keys", "mmee_solve_host", "mmee_pareto_front", "mmee_search_shapes",
            "mmee_query_vector", "mmee_recompute_flag", "mmee_row_pruning_keep", "mmee_last_search_stats", "mmee_kernel_timing",
            "mmee_alu_peak")
 
@@ -64,7 +64,8 @@ class LaunchStats(C.Structure):
     _fields_ = [("kernels_launched", C.c_uint32), ("grid", C.c_uint32), ("block", C.c_uint32),
                 ("smem_bytes", C.c_uint32), ("tasks", C.c_uint64),
                 ("search_ms", C.c_float), ("finalize_ms", C.c_float),
-                ("rows_per_tiling", C.c_uint32), ("rows_evaluated_per_tiling", C.c_uint32)]
+                ("rows_per_tiling", C.c_uint32), ("rows_evaluated_per_tiling", C.c_uint32),
+                ("exact_path_visits", C.c_uint64), ("create_ms", C.c_float), ("reserved", C.c_uint32)]
 
 
 RESULT_BYTES = C.sizeof(Result)
@@ -109,6 +110,7 @@ def library():
     L.mmee_last_cuda_error.argtypes = []
     L.mmee_last_cuda_error.restype = C.c_char_p
     L.mmee_eval.argtypes = [H, C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p]
+    L.mmee_decode.argtypes = [H, C.c_uint64, C.POINTER(Result)]
     L.mmee_dump_keys.argtypes = [H, C.c_void_p, C.c_void_p]
     L.mmee_solve_host.argtypes = [C.POINTER(Workload), C.POINTER(Arch), C.POINTER(Objective),
                                   C.POINTER(Result), C.POINTER(Result),
@@ -195,6 +197,13 @@ def mmee_search_static(workload: dict, arch: dict, objective: dict, out_best, ou
 def mmee_eval(handle, idx_begin: int, count: int, out, stream=None) -> None:
     _check(library().mmee_eval(handle, _stream_ptr(stream), idx_begin, count, C.c_void_p(out.data_ptr())),
            "mmee_eval")
+
+
+def mmee_decode(handle, idx: int) -> Result:
+    """The mapping behind one candidate index with its full evaluation, as a host record (synchronous)."""
+    r = Result()
+    _check(library().mmee_decode(handle, idx, C.byref(r)), "mmee_decode")
+    return r
 
 
 def mmee_dump_keys(handle, out_keys, stream=None) -> None:

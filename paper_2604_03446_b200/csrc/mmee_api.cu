@@ -1,6 +1,7 @@
 // C ABI of libmmee (declared and documented in include/mmee.h).
 #include <cuda_runtime.h>
 
+#include <chrono>
 #include <cstdlib>
 #include <cstring>
 #include <new>
@@ -15,10 +16,13 @@ struct mmee_handle {
     mmee::Plan plan;
     mmee::LaunchShape shape;
     mmee::Scratch* scratch;      // device
+    mmee_result_t* decode_buf;   // device, one record (mmee_decode); part of the scratch allocation
     mmee::PrunedTask* pruned;    // device, row pruning only
     uint32_t kept_rows;          // rows of a tiling that survive pruning (all rows without it)
     int device;
     mmee_launch_stats_t last;
+    float create_ms;             // host wall clock of mmee_create
+    bool dirty;                  // a launch failed half-way: the scratch header is reset before the next search
     bool timing;
     cudaEvent_t ev[3];           // before search kernel, between, after finalize kernel
 };
@@ -27,12 +31,24 @@ namespace {
 
 using namespace mmee;
 
+thread_local cudaError_t g_last_cuda_error = cudaSuccess;
+
+}  // namespace
+
+namespace mmee {
+
+int cuda_status(cudaError_t e) {
+    if (e == cudaSuccess) return MMEE_OK;
+    g_last_cuda_error = e;
+    return MMEE_ERR_CUDA;
+}
+
 // Tasks a CTA pulls per visit of the global counter, and the tilings such a range can touch.
-int choose_shape(const Plan& p, int device, uint32_t search_tpt, LaunchShape* shape) {
+int choose_launch_shape(const Plan& p, int device, uint32_t search_tpt, uint32_t max_ctas, LaunchShape* shape) {
     int sm_count = 0, smem_optin = 0;      // attribute queries: cudaGetDeviceProperties costs milliseconds
-    if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
-        cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess)
-        return MMEE_ERR_CUDA;
+    cudaError_t e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+    if (e != cudaSuccess) return cuda_status(e);
     // A task is 1125 mappings (225 with row pruning, where the searched units are single middle levels).
     const uint32_t rounds = p.row_pruning ? 9 : 3;
     shape->range_tasks = rounds * kWorkerThreads;
@@ -44,19 +60,22 @@ int choose_shape(const Plan& p, int device, uint32_t search_tpt, LaunchShape* sh
     // Many small tilings per range need many table slots: shrink the range until they fit.
     // (Worker warps take 32 tasks at a time, so a range may be as short as one warp's share.)
     while (smem > 110 * 1024 && shape->range_tasks > 32) {
-        shape->range_tasks -= shape->range_tasks > kWorkerThreads ? kWorkerThreads : 32;
+        shape->range_tasks -= shape->range_tasks > (uint32_t)kWorkerThreads ? kWorkerThreads : 32;
         shape->slots = (shape->range_tasks - 1) / search_tpt + 2;
         smem = search_smem_bytes(p, shape->slots);
     }
     if (smem > (size_t)smem_optin) return MMEE_ERR_RANGE;
     shape->smem_bytes = (uint32_t)smem;
     int per_sm = 0;
-    if (search_occupancy(p, smem, &per_sm) != cudaSuccess || per_sm < 1) return MMEE_ERR_CUDA;
+    if ((e = search_occupancy(p, device, smem, &per_sm)) != cudaSuccess) return cuda_status(e);
+    if (per_sm < 1) return MMEE_ERR_RANGE;
     if (per_sm > 2) per_sm = 2;
     uint64_t grid = (uint64_t)sm_count * (uint32_t)per_sm;
     const uint64_t tasks = (p.t_end - p.t_begin) * search_tpt;
     const uint64_t ranges = (tasks + shape->range_tasks - 1) / shape->range_tasks;
     if (grid > ranges) grid = ranges ? ranges : 1;
+    // (a caller with a fixed scratch: a device that would take more CTAs is refused, not silently under-used)
+    if (max_ctas && grid > max_ctas) return MMEE_ERR_RANGE;
     shape->grid = (uint32_t)grid;
     shape->n_ranges = ranges;
     // golden-ratio stride, moved to the next value coprime to the number of ranges
@@ -69,15 +88,7 @@ int choose_shape(const Plan& p, int device, uint32_t search_tpt, LaunchShape* sh
     return MMEE_OK;
 }
 
-thread_local cudaError_t g_last_cuda_error = cudaSuccess;
-
-int cuda_status(cudaError_t e) {
-    if (e == cudaSuccess) return MMEE_OK;
-    g_last_cuda_error = e;
-    return MMEE_ERR_CUDA;
-}
-
-}  // namespace
+}  // namespace mmee
 
 extern "C" {
 
@@ -85,12 +96,13 @@ int mmee_create(const mmee_workload_t* workload, const mmee_arch_t* arch, const 
                 mmee_handle_t** out) {
     if (!out) return MMEE_ERR_ARG;
     *out = nullptr;
+    const auto t0 = std::chrono::steady_clock::now();
     mmee_handle* h = new (std::nothrow) mmee_handle;
     if (!h) return MMEE_ERR_ARG;
     std::memset(h, 0, sizeof(*h));
     int rc = build_plan(workload, arch, objective, &h->plan);
     if (rc) { delete h; return rc; }
-    if (cudaGetDevice(&h->device) != cudaSuccess) { delete h; return MMEE_ERR_CUDA; }
+    if ((rc = cuda_status(cudaGetDevice(&h->device)))) { delete h; return rc; }
     // Row pruning: the searched task space lists only the tasks that keep at least one row.
     std::vector<PrunedTask> kept_tasks;
     uint32_t search_tpt = h->plan.tasks_per_tiling;
@@ -102,41 +114,62 @@ int mmee_create(const mmee_workload_t* workload, const mmee_arch_t* arch, const 
         kept_tasks.resize(n);
         search_tpt = n;
     }
-    rc = choose_shape(h->plan, h->device, search_tpt, &h->shape);
+    rc = choose_launch_shape(h->plan, h->device, search_tpt, 0, &h->shape);
     if (rc) { delete h; return rc; }
     if (h->plan.row_pruning) {
         const size_t bytes = kept_tasks.size() * sizeof(PrunedTask);
-        if (cudaMalloc(reinterpret_cast<void**>(&h->pruned), bytes) != cudaSuccess ||
-            cudaMemcpy(h->pruned, kept_tasks.data(), bytes, cudaMemcpyHostToDevice) != cudaSuccess) {
+        cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&h->pruned), bytes);
+        if (e == cudaSuccess) e = cudaMemcpy(h->pruned, kept_tasks.data(), bytes, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) {
             if (h->pruned) cudaFree(h->pruned);
             delete h;
-            return MMEE_ERR_CUDA;
+            return cuda_status(e);
         }
         h->shape.pruned = h->pruned;
     }
-    if (cudaMalloc(reinterpret_cast<void**>(&h->scratch), scratch_bytes(h->shape.grid)) != cudaSuccess) {
+    // one allocation: the search scratch, then one result record for mmee_decode
+    const size_t sbytes = (scratch_bytes(h->shape.grid) + 15) / 16 * 16;
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&h->scratch), sbytes + sizeof(mmee_result_t));
+    if (e == cudaSuccess) {
+        h->decode_buf = reinterpret_cast<mmee_result_t*>(reinterpret_cast<unsigned char*>(h->scratch) + sbytes);
+        e = launch_reset(h->scratch, 0);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(0);
+    }
+    if (e != cudaSuccess) {
+        if (h->scratch) cudaFree(h->scratch);
         if (h->pruned) cudaFree(h->pruned);
         delete h;
-        return MMEE_ERR_CUDA;
+        return cuda_status(e);
     }
-    if (launch_reset(h->scratch, 0) != cudaSuccess || cudaStreamSynchronize(0) != cudaSuccess) {
-        cudaFree(h->scratch);
-        if (h->pruned) cudaFree(h->pruned);
-        delete h;
-        return MMEE_ERR_CUDA;
-    }
+    h->create_ms = std::chrono::duration<float, std::milli>(std::chrono::steady_clock::now() - t0).count();
     *out = h;
     return MMEE_OK;
 }
 
+// The handle's device must be the current one: its scratch and tables live there, and a launch from another
+// device's context would fail (or, with peer access enabled, silently run on the wrong device).
+static int check_device(const mmee_handle* h) {
+    int cur = -1;
+    const cudaError_t e = cudaGetDevice(&cur);
+    if (e != cudaSuccess) return cuda_status(e);
+    return cur == h->device ? MMEE_OK : MMEE_ERR_ARG;
+}
+
 int mmee_search(mmee_handle_t* h, void* cuda_stream, mmee_result_t* out_best, mmee_result_t* out_topk) {
     if (!h || !out_best) return MMEE_ERR_ARG;
+    int rc = check_device(h);
+    if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (h->dirty) {        // an earlier call failed between its two launches: the header may hold a used work counter
+        if ((rc = cuda_status(launch_reset(h->scratch, st)))) return rc;
+        h->dirty = false;
+    }
     if (h->timing) cudaEventRecord(h->ev[0], st);
-    cudaError_t e = launch_search(h->plan, h->shape, h->scratch, nullptr, st);
-    if (e != cudaSuccess) return MMEE_ERR_CUDA;
+    cudaError_t e = launch_search(h->plan, h->shape, h->device, h->scratch, nullptr, st);
+    if (e != cudaSuccess) { h->dirty = true; return cuda_status(e); }
     if (h->timing) cudaEventRecord(h->ev[1], st);
     e = launch_finalize(h->plan, h->scratch, (int)h->shape.grid, out_best, out_topk, st);
+    if (e != cudaSuccess) { h->dirty = true; return cuda_status(e); }
     if (h->timing) cudaEventRecord(h->ev[2], st);
     h->last.kernels_launched = 2;
     h->last.grid = h->shape.grid;
@@ -145,7 +178,7 @@ int mmee_search(mmee_handle_t* h, void* cuda_stream, mmee_result_t* out_best, mm
     h->last.tasks = (h->plan.t_end - h->plan.t_begin) * h->shape.search_tpt;
     h->last.rows_per_tiling = h->plan.rows_per_tiling;
     h->last.rows_evaluated_per_tiling = h->kept_rows;
-    return cuda_status(e);
+    return MMEE_OK;
 }
 
 int mmee_destroy(mmee_handle_t* h) {
@@ -183,17 +216,34 @@ int mmee_eval(mmee_handle_t* h, void* cuda_stream, uint64_t idx_begin, uint64_t 
     if (!h || (!out && count)) return MMEE_ERR_ARG;
     const uint64_t n = mmee_num_candidates(h);
     if (idx_begin > n || count > n - idx_begin) return MMEE_ERR_ARG;
+    const int rc = check_device(h);
+    if (rc) return rc;
     return cuda_status(launch_eval(h->plan, idx_begin, count, out, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+int mmee_decode(mmee_handle_t* h, uint64_t idx, mmee_result_t* host_out) {
+    if (!h || !host_out || idx >= mmee_num_candidates(h)) return MMEE_ERR_ARG;
+    int rc = check_device(h);
+    if (rc) return rc;
+    if ((rc = cuda_status(launch_eval(h->plan, idx, 1, h->decode_buf, nullptr)))) return rc;
+    return cuda_status(cudaMemcpy(host_out, h->decode_buf, sizeof(mmee_result_t), cudaMemcpyDeviceToHost));
 }
 
 int mmee_dump_keys(mmee_handle_t* h, void* cuda_stream, int64_t* out_keys) {
     if (!h || !out_keys || h->plan.row_pruning) return MMEE_ERR_ARG;
     const uint64_t n = (h->plan.t_end - h->plan.t_begin) * (uint64_t)h->plan.rows_per_tiling * 9u;
     if (n > (1ull << 31)) return MMEE_ERR_RANGE;
+    int rc = check_device(h);
+    if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    cudaError_t e = launch_search(h->plan, h->shape, h->scratch, out_keys, st);
-    if (e != cudaSuccess) return MMEE_ERR_CUDA;
-    return cuda_status(launch_reset(h->scratch, st));
+    if (h->dirty) {
+        if ((rc = cuda_status(launch_reset(h->scratch, st)))) return rc;
+        h->dirty = false;
+    }
+    cudaError_t e = launch_search(h->plan, h->shape, h->device, h->scratch, out_keys, st);
+    if (e != cudaSuccess) { h->dirty = true; return cuda_status(e); }
+    if ((e = launch_reset(h->scratch, st)) != cudaSuccess) { h->dirty = true; return cuda_status(e); }
+    return MMEE_OK;
 }
 
 int mmee_solve_host(const mmee_workload_t* workload, const mmee_arch_t* arch, const mmee_objective_t* objective,
@@ -205,16 +255,13 @@ int mmee_solve_host(const mmee_workload_t* workload, const mmee_arch_t* arch, co
     const uint32_t k = h->plan.topk;
     const size_t bytes = (size_t)(k + 1) * sizeof(mmee_result_t);
     mmee_result_t* dev = nullptr;
-    if (cudaMalloc(reinterpret_cast<void**>(&dev), bytes) != cudaSuccess) { mmee_destroy(h); return MMEE_ERR_CUDA; }
-    for (int attempt = 0; attempt < 3; ++attempt) {       // (search again if the finalize step's check fails)
-        rc = mmee_search(h, nullptr, dev, dev + 1);
-        if (rc == MMEE_OK) rc = cuda_status(cudaMemcpy(out_best, dev, sizeof(mmee_result_t), cudaMemcpyDeviceToHost));
-        if (rc != MMEE_OK || out_best->status != MMEE_ERR_CHECK) break;
-    }
-    if (rc == MMEE_OK) {
-        if (rc == MMEE_OK && out_topk)
-            rc = cuda_status(cudaMemcpy(out_topk, dev + 1, (size_t)k * sizeof(mmee_result_t), cudaMemcpyDeviceToHost));
-    }
+    if ((rc = cuda_status(cudaMalloc(reinterpret_cast<void**>(&dev), bytes)))) { mmee_destroy(h); return rc; }
+    rc = mmee_search(h, nullptr, dev, dev + 1);
+    if (rc == MMEE_OK) rc = cuda_status(cudaMemcpy(out_best, dev, sizeof(mmee_result_t), cudaMemcpyDeviceToHost));
+    if (rc == MMEE_OK && out_topk)
+        rc = cuda_status(cudaMemcpy(out_topk, dev + 1, (size_t)k * sizeof(mmee_result_t), cudaMemcpyDeviceToHost));
+    // the finalize step's self-check failed: the records are not a result
+    if (rc == MMEE_OK && out_best->status == MMEE_ERR_CHECK) rc = MMEE_ERR_CHECK;
     // The plan (divisor lists, query vectors, coefficients) travels to the device as the kernels'
     // parameter block: once per launch.
     if (h2d_bytes) *h2d_bytes = 2ull * sizeof(mmee::Plan);
@@ -237,7 +284,7 @@ int mmee_pareto_front(const mmee_workload_t* workload, const mmee_arch_t* arch, 
     rc = mmee_create(workload, arch, &ol, &hl);
     if (rc) { mmee_destroy(he); return rc; }
     mmee_result_t* dev = nullptr;
-    if (cudaMalloc(reinterpret_cast<void**>(&dev), sizeof(mmee_result_t)) != cudaSuccess) rc = MMEE_ERR_CUDA;
+    rc = cuda_status(cudaMalloc(reinterpret_cast<void**>(&dev), sizeof(mmee_result_t)));
     mmee_result_t r;
     int64_t latency_cap = INT64_MAX - 1;
     uint32_t n = 0;
@@ -251,7 +298,7 @@ int mmee_pareto_front(const mmee_workload_t* workload, const mmee_arch_t* arch, 
         hl->plan.key_cap = r.e_key;
         if ((rc = mmee_search(hl, nullptr, dev, nullptr))) break;
         if ((rc = cuda_status(cudaMemcpy(&r, dev, sizeof(r), cudaMemcpyDeviceToHost)))) break;
-        if (r.idx == MMEE_NO_INDEX) { rc = MMEE_ERR_CUDA; break; }   // cannot happen: the previous optimum qualifies
+        if (r.idx == MMEE_NO_INDEX) { rc = MMEE_ERR_CHECK; break; }   // cannot happen: the previous optimum qualifies
         if (n < capacity) out_points[n] = r;
         ++n;
         if (r.l_key == 0) break;
@@ -274,8 +321,8 @@ int mmee_search_shapes(const mmee_workload_t* workload, const mmee_arch_t* arch,
     o.topk = 1;
     o.row_pruning = 0;
     mmee_result_t* dev = nullptr;
-    if (cudaMalloc(reinterpret_cast<void**>(&dev), sizeof(mmee_result_t)) != cudaSuccess) return MMEE_ERR_CUDA;
-    int rc = MMEE_OK;
+    int rc = cuda_status(cudaMalloc(reinterpret_cast<void**>(&dev), sizeof(mmee_result_t)));
+    if (rc) return rc;
     bool have = false;
     int64_t best_key = 0;
     for (uint32_t i = 0; i < n_shapes && rc == MMEE_OK; ++i) {
@@ -284,12 +331,10 @@ int mmee_search_shapes(const mmee_workload_t* workload, const mmee_arch_t* arch,
         a.pe_cols = shapes[2 * i + 1];
         mmee_handle_t* h = nullptr;
         if ((rc = mmee_create(workload, &a, &o, &h))) break;
-        for (int attempt = 0; attempt < 3; ++attempt) {   // (search again if the finalize step's check fails)
-            rc = mmee_search(h, nullptr, dev, nullptr);
-            if (rc == MMEE_OK)
-                rc = cuda_status(cudaMemcpy(&out_per_shape[i], dev, sizeof(mmee_result_t), cudaMemcpyDeviceToHost));
-            if (rc != MMEE_OK || out_per_shape[i].status != MMEE_ERR_CHECK) break;
-        }
+        rc = mmee_search(h, nullptr, dev, nullptr);
+        if (rc == MMEE_OK)
+            rc = cuda_status(cudaMemcpy(&out_per_shape[i], dev, sizeof(mmee_result_t), cudaMemcpyDeviceToHost));
+        if (rc == MMEE_OK && out_per_shape[i].status == MMEE_ERR_CHECK) rc = MMEE_ERR_CHECK;
         const int rc2 = mmee_destroy(h);
         if (rc == MMEE_OK) rc = rc2;
         if (rc != MMEE_OK || out_per_shape[i].idx == MMEE_NO_INDEX) continue;
@@ -368,10 +413,18 @@ int mmee_last_search_stats(const mmee_handle_t* h, mmee_launch_stats_t* out) {
     if (!h || !out) return MMEE_ERR_ARG;
     *out = h->last;
     out->search_ms = out->finalize_ms = -1.0f;
+    out->create_ms = h->create_ms;
+    out->exact_path_visits = 0;
+    if (h->last.kernels_launched) {
+        unsigned long long visits = 0;
+        const int rc = cuda_status(cudaMemcpy(&visits, &h->scratch->last_exact_visits, sizeof(visits), cudaMemcpyDeviceToHost));
+        if (rc) return rc;
+        out->exact_path_visits = visits;
+    }
     if (h->timing && h->last.kernels_launched) {
-        if (cudaEventElapsedTime(&out->search_ms, h->ev[0], h->ev[1]) != cudaSuccess ||
-            cudaEventElapsedTime(&out->finalize_ms, h->ev[1], h->ev[2]) != cudaSuccess)
-            return MMEE_ERR_CUDA;
+        cudaError_t e = cudaEventElapsedTime(&out->search_ms, h->ev[0], h->ev[1]);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&out->finalize_ms, h->ev[1], h->ev[2]);
+        if (e != cudaSuccess) return cuda_status(e);
     }
     return MMEE_OK;
 }
@@ -379,8 +432,10 @@ int mmee_last_search_stats(const mmee_handle_t* h, mmee_launch_stats_t* out) {
 int mmee_kernel_timing(mmee_handle_t* h, int enable) {
     if (!h) return MMEE_ERR_ARG;
     if (enable && !h->timing) {
-        for (int i = 0; i < 3; ++i)
-            if (cudaEventCreate(&h->ev[i]) != cudaSuccess) return MMEE_ERR_CUDA;
+        for (int i = 0; i < 3; ++i) {
+            const int rc = cuda_status(cudaEventCreate(&h->ev[i]));
+            if (rc) return rc;
+        }
         h->timing = true;
     } else if (!enable && h->timing) {
         for (int i = 0; i < 3; ++i) cudaEventDestroy(h->ev[i]);

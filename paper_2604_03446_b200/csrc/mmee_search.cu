@@ -22,6 +22,7 @@
 
 #include <climits>
 #include <cstddef>
+#include <mutex>
 #include <type_traits>
 
 #include "mmee_eval.cuh"
@@ -112,6 +113,7 @@ __device__ __forceinline__ void top_set(WarpTop* w, int j, int64_t key, uint64_t
 struct alignas(16) CtaShared {
     long long G;             // upper bound on the final k-th smallest key (any full list's last key)
     unsigned long long feasible_rows;
+    unsigned long long exact_visits;         // groups that some warp of this CTA took to the exact path
     unsigned long long range_begin[2];       // first task of the range whose tables sit in buffer 0 / 1
     unsigned int cursor[2];                  // next unassigned task of that range, relative to its begin
 };
@@ -701,7 +703,7 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
                                                     const TaskChoice& c, bool live, bool valid, uint32_t kept,
                                                     uint32_t kept_mid, uint64_t task_first_idx, WarpTop* wt,
                                                     CtaShared* cs, long long* global_g, int k, int lane,
-                                                    int64_t* __restrict__ dump, uint64_t dump_origin) {
+                                                    int64_t* __restrict__ dump, uint64_t dump_origin, uint32_t& visits) {
     const RowTab* rt = &ot->rt[c.phi == 0 ? 0 : 1];
     LaneThreshold th = load_threshold(wt, cs, k);
     uint32_t rows = 0;
@@ -808,6 +810,7 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
             }
             rows += fits;
             if (__any_sync(kFull, hit_any != 0u)) {
+                ++visits;
                 if (k == 1) exact_group_single<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, lane);
                 else exact_group<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, k, lane);
                 th = load_threshold(wt, cs, k);
@@ -826,7 +829,7 @@ template <int OBJ, bool PRUNE>
 __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const TilingTab* tb, const OrderTab* ot,
                                                        const TaskChoice& c, bool live, uint32_t kept, uint32_t kept_mid,
                                                        uint64_t task_first_idx, WarpTop* wt, CtaShared* cs,
-                                                       long long* global_g, int k, int lane) {
+                                                       long long* global_g, int k, int lane, uint32_t& visits) {
     const bool fused = c.phi == 0;
     const RowTab* rt = &ot->rt[fused ? 0 : 1];
     // Row-side terms of E.  Its buffer need while Op1 runs is its size when retained (level >= L4 of a
@@ -979,6 +982,7 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
             // least key of the group's 45 mappings, relative to the threshold
             const bool hit = uc + __vimin3_s32(__vimin3_s32(g[0], g[1], g[2]), g[3], g[4]) < 0;
             if (__any_sync(kFull, hit)) {
+                ++visits;
                 if (k == 1) exact_group_single<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, lane);
                 else exact_group<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, k, lane);
                 rebase(m * 225 + d * 45 + 45);
@@ -1023,6 +1027,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
     if (tid == 0) {
         cs->G = scratch->G;
         cs->feasible_rows = 0;
+        cs->exact_visits = 0;
     }
     if (lane == 0) wt->count = 0;
     __syncthreads();      // the shared copy of the plan is complete
@@ -1032,6 +1037,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
     const uint64_t dump_origin = task_begin * kCandPerTask;
     const uint32_t n_orders = p.n_orders;
     unsigned long long my_rows = 0;
+    uint32_t my_visits = 0;
 
     // Builder: pull the next range and build its tables into buffer `buf`.  Ranges are visited in a
     // stride-permuted order (stride coprime to their number), so that the first pull of every CTA
@@ -1188,10 +1194,10 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
             const long long g_seen = (lane == 0) ? *reinterpret_cast<volatile long long*>(&scratch->G) : 0;
             if constexpr (!DUMP && OBJ <= MMEE_OBJ_LATENCY) {
                 my_rows += walk_task_relative<OBJ, PRUNE>(p, tb, ot, c, live, kept, kept_mid, task_first_idx, wt, cs,
-                                                          &scratch->G, k, lane);
+                                                          &scratch->G, k, lane, my_visits);
             } else {
                 my_rows += walk_task_exact<OBJ, DUMP, PRUNE>(p, tb, ot, c, live, valid, kept, kept_mid, task_first_idx, wt,
-                                                             cs, &scratch->G, k, lane, dump, dump_origin);
+                                                             cs, &scratch->G, k, lane, dump, dump_origin, my_visits);
             }
             if (lane == 0 && g_seen < cs->G) atomicMin(&cs->G, g_seen);
         }
@@ -1202,6 +1208,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
     // ---- feasible count
     for (int off = 16; off; off >>= 1) my_rows += __shfl_down_sync(kFull, my_rows, off);
     if (lane == 0 && my_rows) atomicAdd(&cs->feasible_rows, my_rows);
+    if (lane == 0 && my_visits) atomicAdd(&cs->exact_visits, (unsigned long long)my_visits);
     __syncthreads();
 
     // ---- merge the warps' lists into warp 0's, then publish this CTA's partial list
@@ -1229,6 +1236,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
         if (lane == 0) {
             out->count = n;
             if (cs->feasible_rows) atomicAdd(&scratch->feasible_rows, cs->feasible_rows);
+            if (cs->exact_visits) atomicAdd(&scratch->exact_visits, cs->exact_visits);
         }
     }
 }
@@ -1328,6 +1336,8 @@ finalize_kernel(const __grid_constant__ Plan p, Scratch* __restrict__ scratch, i
             scratch->next_task = 0;
             scratch->feasible_rows = 0;
             scratch->G = kInfKey - 1;
+            scratch->last_exact_visits = scratch->exact_visits;
+            scratch->exact_visits = 0;
         }
     }
 }
@@ -1336,6 +1346,7 @@ __global__ void reset_kernel(Scratch* scratch) {
     scratch->next_task = 0;
     scratch->feasible_rows = 0;
     scratch->G = kInfKey - 1;
+    scratch->exact_visits = 0;
 }
 
 __global__ void eval_kernel(const __grid_constant__ Plan p, uint64_t idx_begin, uint64_t count,
@@ -1348,18 +1359,35 @@ __global__ void eval_kernel(const __grid_constant__ Plan p, uint64_t idx_begin, 
     }
 }
 
+// The kernels take more dynamic shared memory than the default limit: the limit of each instantiation is
+// raised once per device, to the device's opt-in maximum, so that a launch is one driver call and two host
+// threads with different table sizes cannot undo each other's setting.
 template <int OBJ, int MODE>
-cudaError_t launch_search_t(const Plan& p, const LaunchShape& shape, Scratch* scratch, int64_t* dump, cudaStream_t st) {
-    cudaError_t e = cudaFuncSetAttribute(search_kernel<OBJ, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)shape.smem_bytes);
+cudaError_t allow_large_smem(int device) {
+    static std::mutex mu;
+    static unsigned long long done = 0;       // one bit per device
+    std::lock_guard<std::mutex> lock(mu);
+    if (device >= 0 && device < 64 && (done >> device & 1ull)) return cudaSuccess;
+    int optin = 0;
+    cudaError_t e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(search_kernel<OBJ, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, optin);
+    if (e == cudaSuccess && device >= 0 && device < 64) done |= 1ull << device;
+    return e;
+}
+
+template <int OBJ, int MODE>
+cudaError_t launch_search_t(const Plan& p, const LaunchShape& shape, int device, Scratch* scratch, int64_t* dump,
+                            cudaStream_t st) {
+    cudaError_t e = allow_large_smem<OBJ, MODE>(device);
     if (e != cudaSuccess) return e;
     search_kernel<OBJ, MODE><<<shape.grid, kSearchThreads, shape.smem_bytes, st>>>(p, shape, scratch, dump);
     return cudaGetLastError();
 }
 
 template <int OBJ, int MODE>
-cudaError_t occupancy_t(int* blocks_per_sm, size_t smem) {
-    cudaError_t e = cudaFuncSetAttribute(search_kernel<OBJ, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+cudaError_t occupancy_t(int device, int* blocks_per_sm, size_t smem) {
+    cudaError_t e = allow_large_smem<OBJ, MODE>(device);
     if (e != cudaSuccess) return e;
     return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, search_kernel<OBJ, MODE>, kSearchThreads, smem);
 }
@@ -1371,41 +1399,42 @@ size_t search_smem_bytes(const Plan& p, uint32_t slots) {
            2 * (size_t)slots * p.n_orders * sizeof(OrderTab);
 }
 
-cudaError_t search_occupancy(const Plan& p, size_t smem, int* blocks_per_sm) {
+cudaError_t search_occupancy(const Plan& p, int device, size_t smem, int* blocks_per_sm) {
     switch (p.objective) {
-        case MMEE_OBJ_ENERGY: return occupancy_t<MMEE_OBJ_ENERGY, kModeSearch>(blocks_per_sm, smem);
-        case MMEE_OBJ_LATENCY: return occupancy_t<MMEE_OBJ_LATENCY, kModeSearch>(blocks_per_sm, smem);
-        case MMEE_OBJ_EDP: return occupancy_t<MMEE_OBJ_EDP, kModeSearch>(blocks_per_sm, smem);
-        case MMEE_OBJ_ENERGY_LCAP: return occupancy_t<MMEE_OBJ_ENERGY_LCAP, kModeSearch>(blocks_per_sm, smem);
-        default: return occupancy_t<MMEE_OBJ_LATENCY_ECAP, kModeSearch>(blocks_per_sm, smem);
+        case MMEE_OBJ_ENERGY: return occupancy_t<MMEE_OBJ_ENERGY, kModeSearch>(device, blocks_per_sm, smem);
+        case MMEE_OBJ_LATENCY: return occupancy_t<MMEE_OBJ_LATENCY, kModeSearch>(device, blocks_per_sm, smem);
+        case MMEE_OBJ_EDP: return occupancy_t<MMEE_OBJ_EDP, kModeSearch>(device, blocks_per_sm, smem);
+        case MMEE_OBJ_ENERGY_LCAP: return occupancy_t<MMEE_OBJ_ENERGY_LCAP, kModeSearch>(device, blocks_per_sm, smem);
+        default: return occupancy_t<MMEE_OBJ_LATENCY_ECAP, kModeSearch>(device, blocks_per_sm, smem);
     }
 }
 
-cudaError_t launch_search(const Plan& p, const LaunchShape& shape, Scratch* scratch, int64_t* dump, cudaStream_t st) {
+cudaError_t launch_search(const Plan& p, const LaunchShape& shape, int device, Scratch* scratch, int64_t* dump,
+                          cudaStream_t st) {
     if (dump) {
         switch (p.objective) {
-            case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, kModeDump>(p, shape, scratch, dump, st);
-            case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, kModeDump>(p, shape, scratch, dump, st);
-            case MMEE_OBJ_EDP: return launch_search_t<MMEE_OBJ_EDP, kModeDump>(p, shape, scratch, dump, st);
-            case MMEE_OBJ_ENERGY_LCAP: return launch_search_t<MMEE_OBJ_ENERGY_LCAP, kModeDump>(p, shape, scratch, dump, st);
-            default: return launch_search_t<MMEE_OBJ_LATENCY_ECAP, kModeDump>(p, shape, scratch, dump, st);
+            case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, kModeDump>(p, shape, device, scratch, dump, st);
+            case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, kModeDump>(p, shape, device, scratch, dump, st);
+            case MMEE_OBJ_EDP: return launch_search_t<MMEE_OBJ_EDP, kModeDump>(p, shape, device, scratch, dump, st);
+            case MMEE_OBJ_ENERGY_LCAP: return launch_search_t<MMEE_OBJ_ENERGY_LCAP, kModeDump>(p, shape, device, scratch, dump, st);
+            default: return launch_search_t<MMEE_OBJ_LATENCY_ECAP, kModeDump>(p, shape, device, scratch, dump, st);
         }
     }
     if (shape.pruned) {
         switch (p.objective) {
-            case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, kModePrune>(p, shape, scratch, nullptr, st);
-            case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, kModePrune>(p, shape, scratch, nullptr, st);
-            case MMEE_OBJ_EDP: return launch_search_t<MMEE_OBJ_EDP, kModePrune>(p, shape, scratch, nullptr, st);
-            case MMEE_OBJ_ENERGY_LCAP: return launch_search_t<MMEE_OBJ_ENERGY_LCAP, kModePrune>(p, shape, scratch, nullptr, st);
-            default: return launch_search_t<MMEE_OBJ_LATENCY_ECAP, kModePrune>(p, shape, scratch, nullptr, st);
+            case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, kModePrune>(p, shape, device, scratch, nullptr, st);
+            case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, kModePrune>(p, shape, device, scratch, nullptr, st);
+            case MMEE_OBJ_EDP: return launch_search_t<MMEE_OBJ_EDP, kModePrune>(p, shape, device, scratch, nullptr, st);
+            case MMEE_OBJ_ENERGY_LCAP: return launch_search_t<MMEE_OBJ_ENERGY_LCAP, kModePrune>(p, shape, device, scratch, nullptr, st);
+            default: return launch_search_t<MMEE_OBJ_LATENCY_ECAP, kModePrune>(p, shape, device, scratch, nullptr, st);
         }
     }
     switch (p.objective) {
-        case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, kModeSearch>(p, shape, scratch, nullptr, st);
-        case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, kModeSearch>(p, shape, scratch, nullptr, st);
-        case MMEE_OBJ_EDP: return launch_search_t<MMEE_OBJ_EDP, kModeSearch>(p, shape, scratch, nullptr, st);
-        case MMEE_OBJ_ENERGY_LCAP: return launch_search_t<MMEE_OBJ_ENERGY_LCAP, kModeSearch>(p, shape, scratch, nullptr, st);
-        default: return launch_search_t<MMEE_OBJ_LATENCY_ECAP, kModeSearch>(p, shape, scratch, nullptr, st);
+        case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, kModeSearch>(p, shape, device, scratch, nullptr, st);
+        case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, kModeSearch>(p, shape, device, scratch, nullptr, st);
+        case MMEE_OBJ_EDP: return launch_search_t<MMEE_OBJ_EDP, kModeSearch>(p, shape, device, scratch, nullptr, st);
+        case MMEE_OBJ_ENERGY_LCAP: return launch_search_t<MMEE_OBJ_ENERGY_LCAP, kModeSearch>(p, shape, device, scratch, nullptr, st);
+        default: return launch_search_t<MMEE_OBJ_LATENCY_ECAP, kModeSearch>(p, shape, device, scratch, nullptr, st);
     }
 }
 

@@ -19,13 +19,16 @@ struct alignas(16) Partial {
     int32_t pad[3];
 };
 
-// Global scratch of one handle: a work counter, the feasible-row count, the shared pruning bound
-// and one partial list per CTA.  The header is reset by the finalize kernel.
+// Global scratch of one handle: a work counter, the feasible-row count, the shared pruning bound,
+// the count of exact-path visits and one partial list per CTA.  The header is reset by the finalize
+// kernel, which also keeps the finished search's visit count in `last_exact_visits`.
 struct Scratch {
     unsigned long long next_task;
     unsigned long long feasible_rows;
     long long G;
-    long long pad;
+    unsigned long long exact_visits;
+    unsigned long long last_exact_visits;
+    unsigned long long pad;
     Partial partial[1];     // grid entries follow
 };
 
@@ -44,12 +47,20 @@ struct LaunchShape {
 inline size_t scratch_bytes(uint32_t grid) { return sizeof(Scratch) + (size_t)(grid ? grid - 1 : 0) * sizeof(Partial); }
 
 size_t search_smem_bytes(const Plan& p, uint32_t slots);
-cudaError_t search_occupancy(const Plan& p, size_t smem, int* blocks_per_sm);
-cudaError_t launch_search(const Plan& p, const LaunchShape& shape, Scratch* scratch, int64_t* dump, cudaStream_t st);
+cudaError_t search_occupancy(const Plan& p, int device, size_t smem, int* blocks_per_sm);
+cudaError_t launch_search(const Plan& p, const LaunchShape& shape, int device, Scratch* scratch, int64_t* dump,
+                          cudaStream_t st);
 cudaError_t launch_finalize(const Plan& p, Scratch* scratch, int n_partials, mmee_result_t* out_best,
                             mmee_result_t* out_topk, cudaStream_t st);
 cudaError_t launch_reset(Scratch* scratch, cudaStream_t st);
 cudaError_t launch_eval(const Plan& p, uint64_t idx_begin, uint64_t count, mmee_result_t* out, cudaStream_t st);
 cudaError_t measure_alu_peak(double* giops);
+
+// Launch shape of a search on `device`: tasks per range, table slots, shared memory, persistent CTAs
+// (at most max_ctas when that is not 0: MMEE_ERR_RANGE if the device would take more), range order.
+int choose_launch_shape(const Plan& p, int device, uint32_t search_tpt, uint32_t max_ctas, LaunchShape* shape);
+
+// MMEE_OK, or MMEE_ERR_CUDA with the error kept for mmee_last_cuda_error (per host thread).
+int cuda_status(cudaError_t e);
 
 }  // namespace mmee

@@ -45,6 +45,19 @@ def test_static_scratch_search_matches_the_handle_search_twice_in_a_row():
     got = mm.read_results(bufs[0][0], 1)[0]
     assert got.status == mm.OK and got.n_total == 162067500 and got.idx != mm.NO_INDEX
 
+    # What the entry point is for: once the first call on the device has looked the array up, further calls
+    # take no device memory at all (the free-memory figure of the device does not move).
+    free_before, _ = torch.cuda.mem_get_info()
+    for _ in range(3):
+        for (cfg, obj), (best, topk) in zip(cases, bufs):
+            mm.mmee_search_static(cfg["workload"], cfg["arch"], obj, best, topk)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    for (best, topk), (want_best, want_topk) in zip(bufs, want):
+        assert bytes(best.cpu().numpy().tobytes()) == want_best
+        assert bytes(topk.cpu().numpy().tobytes()) == want_topk
+
 
 def test_static_scratch_search_rejects_bad_arguments():
     cfg = mi.config1()
