@@ -1,10 +1,12 @@
 """Benchmark of the MMEE search path: candidate mappings evaluated per second on B200.
 
-A step is one pass of the whole hot path over one workload: for each search of the workload
-(BERT-base-shaped attention on the edge accelerator: energy-driven, then latency-driven) the plan
-is decoded, every mapping evaluated, capacity-pruned and reduced to the optimum on the device.
+A step is one pass of the whole hot path over one workload: for each search of the workload the plan
+is decoded, every mapping's cost bounded or evaluated, capacity-pruned and reduced to the optimum on
+the device, in one kernel launch per search.  The default workload is the largest single-GPU
+configuration: grouped-query attention (batch 4, 32 query heads on 8 KV heads, S = 8192, d = 128) on
+the cloud accelerator, latency-driven then energy-delay-product-driven, 3.39e9 mappings per search.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
 
 Prints one JSON line.  With N > 1 (under torchrun) every rank runs an independent replica on its
 own GPU: the search is launched per workload and does not shard in this build.
@@ -30,20 +32,19 @@ METRIC = "candidate mappings evaluated/sec"
 UNIT = "candidates/s"
 OBJ_NAMES = {0: "energy", 1: "latency", 2: "edp", 3: "energy_lcap", 4: "latency_ecap"}
 
-# Algorithmic integer work per mapping in the hoisted separable form of the model, counted in
-# thread-level 32-bit integer instructions.  Energy: one fused add-min per mapping (its key relative
-# to the threshold) plus, per row of 9 mappings, the row add, the capacity difference, its sign mask,
-# the masking multiply-add and the feasible count (5).  Latency: one fused add-max per mapping and
-# five 3-/2-input mins per row (14), plus the capacity difference, its sign mask, the masking
-# multiply-add and the feasible count (4).  EDP (not separable) is evaluated in double precision on
-# the FP64 pipe, which has the same 64 lanes per SM: add, two multiplies, two compares and a
-# predicate OR per mapping (6) plus, per row, four conversions, four 64-bit adds and the capacity
-# test (15).
-ALG_OPS_PER_CANDIDATE = {0: 1.0 + 5.0 / 9.0, 1: 2.0, 2: 6.0 + 15.0 / 9.0}
-INT_LANES_PER_SM = 64          # 4 sub-partitions x 16 integer-ALU lanes
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the exhaustive search kernels on the BERT workload,
-# from the ncu capture summarised under profiles/ (energy, latency); None for other workloads.
-NCU_DRAM_BYTES_PER_LAUNCH = {"bert": {0: 108032, 1: 121600}}
+# Algorithmic work of the search kernels, per TESTED ROW (a row is the nine mappings that share tiling, order
+# and buffering levels; the kernel reports how many rows it tested, the others lay in tilings, middle levels
+# or groups that a coarser capacity test showed not to fit).  The least key of a row's nine mappings is its
+# row sum plus the least stationary-pair term, which is taken once per tiling, so a row needs one test.
+# Energy / latency, in thread-level 32-bit integer instructions: capacity difference of Eq. (4), its sign mask,
+# the feasible count, the masked row term, and 2/5 of a three-input minimum (five rows share two).
+# Energy-delay product: two capacity compares, their AND, the feasible count, and the single-precision row
+# bound (two adds, a max, a multiply, a compare, the predicate merge).
+ALG_OPS_PER_ROW = {0: 4.4, 1: 4.4, 2: 10.0}
+LANES_PER_SM = 64          # 4 sub-partitions x 16 lanes: width of the integer-ALU pipe, the busiest pipe of these kernels
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, recorded from the ncu captures summarised under
+# profiles/ (not measured in this run); workload -> objective -> bytes.  None where no capture backs it.
+NCU_DRAM_BYTES_PER_LAUNCH = {}
 
 
 WORKLOADS = {"tiny": mi.config1, "bert": mi.config2, "llama": mi.config3, "gqa": mi.config4}
@@ -51,8 +52,8 @@ WORKLOADS = {"tiny": mi.config1, "bert": mi.config2, "llama": mi.config3, "gqa":
 
 def workload_jobs(name):
     """(workload name, [(problem, search), ...]): one step runs every listed search once.
-    The default, "bert", is the configuration the headline metric is quoted on; "sweep" is the
-    28-point sequence-length sweep (one energy search per point)."""
+    The default, "gqa", is the largest single-GPU configuration; "sweep" is the 28-point
+    sequence-length sweep (one energy search per point)."""
     if name == "sweep":
         pts = mi.config5()
         return "sweep_s1k_to_64k", [(c, c["searches"][0]) for c in pts]
@@ -113,7 +114,8 @@ class ClockSampler:
 
 
 def cpu_baseline(cfg, obj, budget_s: float = 12.0):
-    """The oracle as it stands on the host cores, on a bounded tiling sub-range of the workload."""
+    """The oracle as it stands on the host cores, on a bounded tiling sub-range of the workload; then the same
+    on one core, on a quarter-size budget."""
     import oracle
     p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
     probe = max(1, min(p.T, 40))
@@ -126,9 +128,17 @@ def cpu_baseline(cfg, obj, budget_s: float = 12.0):
     t0 = time.perf_counter()
     res = oracle.search(q)
     dt = time.perf_counter() - t0
-    return dict(value=res.n_total / dt, unit=UNIT, cores=oracle.threads_used(), kind="oracle",
+    cores = oracle.threads_used()
+    n_1 = max(1, int(n_t / max(cores, 1) / 4))
+    q1 = oracle.make_problem(cfg["workload"], cfg["arch"], dict(obj, t_begin=lo, t_end=lo + n_1))
+    t0 = time.perf_counter()
+    res1 = oracle.search(q1, threads=1)
+    dt1 = time.perf_counter() - t0
+    return dict(value=res.n_total / dt, unit=UNIT, cores=cores, kind="oracle",
                 sample="%s objective, tilings [%d,%d) of %d (%d mappings, %.1f s)" %
-                       (OBJ_NAMES[obj["objective"]], lo, lo + n_t, p.T, res.n_total, dt))
+                       (OBJ_NAMES[obj["objective"]], lo, lo + n_t, p.T, res.n_total, dt),
+                one_core=dict(value=res1.n_total / dt1, unit=UNIT, cores=1,
+                              sample="tilings [%d,%d) (%d mappings, %.1f s)" % (lo, lo + n_1, res1.n_total, dt1)))
 
 
 def run_reference(args, rank):
@@ -192,11 +202,11 @@ def run_reconfig(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="bert", choices=sorted(WORKLOADS) + ["sweep", "ffn", "beyond", "reconfig"])
+    ap.add_argument("--workload", default="gqa", choices=sorted(WORKLOADS) + ["sweep", "ffn", "beyond", "reconfig"])
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -242,8 +252,7 @@ def main():
         torch.cuda.synchronize()
         if not timed:
             return None
-        ks = [mm.mmee_last_search_stats(h) for h in handles]
-        return ev0.elapsed_time(ev1), [(k.search_ms, k.finalize_ms) for k in ks]
+        return ev0.elapsed_time(ev1), [mm.mmee_last_search_stats(h).search_ms for h in handles]
 
     for _ in range(args.warmup):
         one_step(False)
@@ -273,24 +282,24 @@ def main():
     # parity of what was timed is the tests' job; here only the counters of the last step
     bests = [mm.read_results(b, 1)[0] for b, _ in outs]
     stats = [mm.mmee_last_search_stats(h) for h in handles]
+    check_failures = sum(1 for b in bests if b.status == mm.ERR_CHECK)
 
-    # time to optimum per search: host wall clock from the mmee_search call until the optimum is
-    # readable on the host (warm handle)
+    # time to optimum per search: host wall clock of mmee_search_host on the warm handle (launch, device
+    # search, copy of the optimum record to host memory)
     tto_ms = []
-    for h, (b, t) in zip(handles, outs):
+    for h in handles:
         samples = []
         for _ in range(21):
             torch.cuda.synchronize()
             t0 = time.perf_counter()
-            mm.mmee_search(h, b, t)
-            mm.read_results(b, 1)
+            mm.mmee_search_host(h)
             samples.append(1e3 * (time.perf_counter() - t0))
         tto_ms.append(statistics.median(samples))
 
     # offline symbolic row pruning (single-optimum searches only): same optimum, fewer rows evaluated
     pruning = []
     for i, (c, s) in enumerate(jobs):
-        if s["topk"] != 1:
+        if s["topk"] != 1 or len(jobs) > 4:
             continue
         hp = mm.mmee_create(c["workload"], c["arch"], dict(s, row_pruning=1))
         mm.mmee_kernel_timing(hp, True)
@@ -309,7 +318,7 @@ def main():
                                          energy_pj=got.energy_pj, latency_cycles=got.latency_cycles)))
         mm.mmee_destroy(hp)
 
-    # end to end through the host-buffer entry point: plan, launch, copy back, every step
+    # end to end through the host-buffer entry point: plan, allocate, launch, copy back, release, every step
     e2e_steps = max(3, min(args.steps, 30))
     h2d = d2h = 0
     for _ in range(2):
@@ -332,29 +341,34 @@ def main():
         mm.mmee_destroy(h)
 
     if rank == 0:
-        per_kernel = []
-        for i, (s, n) in enumerate(n_cand):
-            sm = statistics.mean(k[i][0] for k in kernel_ms)
-            fm = statistics.mean(k[i][1] for k in kernel_ms)
-            ops = bests[i].n_feasible * ALG_OPS_PER_CANDIDATE[s["objective"]]
-            per_kernel.append(dict(kernel="search_kernel<%s>" % OBJ_NAMES[s["objective"]], objective=s["objective"],
-                                   problem=jobs[i][0]["name"],
-                                   avg_ms=sm, median_ms=statistics.median(k[i][0] for k in kernel_ms),
-                                   max_ms=max(k[i][0] for k in kernel_ms), finalize_avg_ms=fm, candidates=n, feasible=bests[i].n_feasible,
-                                   pruned_fraction=1.0 - bests[i].n_feasible / n, time_to_optimum_ms=tto_ms[i],
-                                   candidates_per_s=n / (sm * 1e-3), achieved_gops=ops / (sm * 1e-3) / 1e9))
-        dom = max(per_kernel, key=lambda k: k["avg_ms"])
         sm_mhz = clocks.get("sm_mhz") or peaks[3]
         n_sm = torch.cuda.get_device_properties(local_rank).multi_processor_count
-        peak = n_sm * INT_LANES_PER_SM * sm_mhz * 1e6 / 1e9
+        peak = n_sm * LANES_PER_SM * sm_mhz * 1e6 / 1e9
+        per_kernel = []
+        for i, (s, n) in enumerate(n_cand):
+            ks = [k[i] for k in kernel_ms]
+            sm = statistics.mean(ks)
+            ops = stats[i].rows_tested * ALG_OPS_PER_ROW.get(s["objective"], 10.0)
+            per_kernel.append(dict(
+                kernel="search_kernel<%s>" % OBJ_NAMES[s["objective"]], objective=s["objective"], problem=jobs[i][0]["name"],
+                avg_ms=sm, median_ms=statistics.median(ks), max_ms=max(ks), create_ms=stats[i].create_ms,
+                candidates=n, feasible=bests[i].n_feasible, pruned_fraction=1.0 - bests[i].n_feasible / n,
+                rows_tested=stats[i].rows_tested, rows_total=n // 9, exact_path_visits=stats[i].exact_path_visits,
+                time_to_optimum_ms=tto_ms[i], candidates_per_s=n / (sm * 1e-3),
+                evaluated_per_s=9 * stats[i].rows_tested / (sm * 1e-3),
+                achieved_gops=ops / (sm * 1e-3) / 1e9, frac=ops / (sm * 1e-3) / 1e9 / peak))
+        dom = max(per_kernel, key=lambda k: k["avg_ms"])
+        traffic = NCU_DRAM_BYTES_PER_LAUNCH.get(args.workload, {}).get(dom["objective"])
         roofline = dict(bound="alu", kernel=dom["kernel"], achieved=dom["achieved_gops"], peak=peak,
-                        unit="Gop/s (32-bit integer instructions)", frac=dom["achieved_gops"] / peak,
-                        traffic=NCU_DRAM_BYTES_PER_LAUNCH.get(args.workload, {}).get(dom["objective"]),
-                        peak_source="%d SMs x %d integer-ALU lanes x %.0f MHz (clock sampled during the run)" %
-                                    (n_sm, INT_LANES_PER_SM, sm_mhz),
+                        unit="Gop/s (thread-level 32-bit instructions of the row tests)", frac=dom["achieved_gops"] / peak,
+                        traffic=traffic,
+                        traffic_note=("recorded from the ncu capture under profiles/, not measured in this run"
+                                      if traffic is not None else "no capture of this kernel on this workload"),
+                        peak_source="%d SMs x %d lanes of the integer-ALU pipe x %.0f MHz (clock sampled during the run)" %
+                                    (n_sm, LANES_PER_SM, sm_mhz),
+                        ops_per_tested_row=ALG_OPS_PER_ROW.get(dom["objective"], 10.0),
                         measured_rates_gops=dict(logic=peaks[0], add_logic=peaks[1], key_mix=peaks[2],
-                                                 sm_mhz=peaks[3]),
-                        frac_of_measured_key_mix=dom["achieved_gops"] / peaks[2] if peaks[2] else None)
+                                                 sm_mhz=peaks[3]))
         line = dict(
             metric=METRIC, value=world * cand_per_step * args.steps / (total_ms * 1e-3), unit=UNIT,
             n_gpus=world, steps=args.steps, warmup=args.warmup, ms_per_step=total_ms / args.steps,
@@ -363,11 +377,11 @@ def main():
                         candidates_per_step=cand_per_step, parallelism="replicas only",
                         l2="flushed between steps (256 MB write); the path reads no HBM-resident input",
                         grid=stats[0].grid, block=stats[0].block, smem_bytes=stats[0].smem_bytes),
-            clocks=clocks, gpu_launches=2 * len(searches) * args.steps,
+            clocks=clocks, gpu_launches=len(searches) * args.steps, check_failures=check_failures,
             e2e=dict(value=world * cand_per_step * e2e_steps / e2e_s, unit=UNIT, h2d_bytes_per_step=h2d,
                      d2h_bytes_per_step=d2h, ms_per_step=1e3 * e2e_s / e2e_steps,
-                     note="mmee_solve_host: plan + launch + result copy to host buffers, host wall clock"),
-            time_to_optimum_ms=tto_ms, device_time_to_optimum_ms=[k["avg_ms"] + k["finalize_avg_ms"] for k in per_kernel],
+                     note="mmee_solve_host: plan + allocate + launch + result copy to host buffers + release, host wall clock"),
+            time_to_optimum_ms=tto_ms, create_ms=[k["create_ms"] for k in per_kernel],
             kernels=per_kernel, roofline=roofline, row_pruning=pruning)
         if not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(*jobs[0])

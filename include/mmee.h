@@ -166,6 +166,15 @@ int mmee_create(const mmee_workload_t* workload, const mmee_arch_t* arch,
 int mmee_search(mmee_handle_t* handle, void* cuda_stream, mmee_result_t* out_best,
                 mmee_result_t* out_topk);
 
+/*
+ * mmee_search_host -- mmee_search on the default stream of the handle's device followed by the copy of
+ * the records to HOST memory: the time to the optimal mapping of a planned search (the handle is warm;
+ * nothing is allocated).  Synchronous.
+ *   out_best : HOST, one record.   out_topk : HOST, objective.topk records, or NULL.
+ * Returns MMEE_ERR_CHECK if the finalize step's self-check failed (the records are then not a result).
+ */
+int mmee_search_host(mmee_handle_t* handle, mmee_result_t* out_best, mmee_result_t* out_topk);
+
 int mmee_destroy(mmee_handle_t* handle);
 
 /*
@@ -177,7 +186,7 @@ int mmee_destroy(mmee_handle_t* handle);
  * library then fails), or a latency-critical loop that cannot afford the device-wide
  * synchronisation of cudaMalloc / cudaFree.  This call makes no cudaMalloc, cudaFree or other
  * allocating call.  Its scratch (work counter, pruning bound, one partial top-k list per CTA) is a
- * fixed 139 312-byte array inside the library image, present on every device that loads the
+ * fixed 139 328-byte array inside the library image, present on every device that loads the
  * library for as long as the process lives.
  *
  *   workload, arch, objective : HOST, as for mmee_create; planned on the host at every call.
@@ -306,10 +315,12 @@ int mmee_recompute_flag(uint32_t pi, uint32_t beta_c, uint32_t* out_flag);
 
 /*
  * mmee_last_search_stats -- HOST counters of the most recent mmee_search on the handle, valid
- * after the stream has been synchronised (the call copies one counter from the device): kernels launched by that call, persistent CTAs,
- * threads per CTA, dynamic shared memory per CTA, tasks (groups of 1125 consecutive mappings) and,
- * when mmee_kernel_timing is on, the device time of the search kernel and of the finalize kernel
- * in milliseconds (CUDA events recorded on the search's stream; -1 when timing is off).
+ * after the stream has been synchronised (the call copies one counter from the device): kernels
+ * launched by that call (one: the CTA that finishes last merges the partial results and writes the
+ * records), persistent CTAs, threads per CTA, dynamic shared memory per CTA, tasks (groups of 1125
+ * consecutive mappings) and, when mmee_kernel_timing is on, the device time of the search kernel in
+ * milliseconds (CUDA events recorded on the search's stream; -1 when timing is off).  finalize_ms
+ * is 0: the finalize step is part of the search kernel.
  */
 typedef struct {
     uint32_t kernels_launched, grid, block, smem_bytes;
@@ -321,6 +332,9 @@ typedef struct {
                                                 exact 64-bit path during that search               */
     float    create_ms;                      /* host wall clock of the mmee_create that made the handle */
     uint32_t reserved;
+    uint64_t rows_tested;                    /* rows (of nine mappings each) whose capacity test (Eq. 4) and
+                                                bound the search evaluated; the rest lay in tilings, middle
+                                                levels or groups that a coarser test showed not to fit   */
 } mmee_launch_stats_t;
 int mmee_last_search_stats(const mmee_handle_t* handle, mmee_launch_stats_t* out);
 

@@ -19,7 +19,7 @@ MAX_TOPK = 16
 NO_INDEX = 2 ** 64 - 1
 OK, ERR_ARG, ERR_OVERFLOW, ERR_QUANTUM, ERR_NO_FEASIBLE, ERR_CUDA, ERR_TIMEOUT, ERR_RANGE, ERR_CHECK = range(9)
 
-EXPORTS = ("mmee_create", "mmee_search", "mmee_destroy", "mmee_search_static", "mmee_num_candidates", "mmee_num_tilings",
+EXPORTS = ("mmee_create", "mmee_search", "mmee_search_host", "mmee_destroy", "mmee_search_static", "mmee_num_candidates", "mmee_num_tilings",
            "mmee_num_rows", "mmee_strerror", "mmee_last_cuda_error", "mmee_eval", "mmee_decode", "mmee_dump_keys", "mmee_solve_host", "mmee_pareto_front", "mmee_search_shapes",
            "mmee_query_vector", "mmee_recompute_flag", "mmee_row_pruning_keep", "mmee_last_search_stats", "mmee_kernel_timing",
            "mmee_alu_peak")
@@ -65,7 +65,8 @@ class LaunchStats(C.Structure):
                 ("smem_bytes", C.c_uint32), ("tasks", C.c_uint64),
                 ("search_ms", C.c_float), ("finalize_ms", C.c_float),
                 ("rows_per_tiling", C.c_uint32), ("rows_evaluated_per_tiling", C.c_uint32),
-                ("exact_path_visits", C.c_uint64), ("create_ms", C.c_float), ("reserved", C.c_uint32)]
+                ("exact_path_visits", C.c_uint64), ("create_ms", C.c_float), ("reserved", C.c_uint32),
+                ("rows_tested", C.c_uint64)]
 
 
 RESULT_BYTES = C.sizeof(Result)
@@ -99,6 +100,7 @@ def library():
     H = C.c_void_p
     L.mmee_create.argtypes = [C.POINTER(Workload), C.POINTER(Arch), C.POINTER(Objective), C.POINTER(H)]
     L.mmee_search.argtypes = [H, C.c_void_p, C.c_void_p, C.c_void_p]
+    L.mmee_search_host.argtypes = [H, C.POINTER(Result), C.POINTER(Result)]
     L.mmee_destroy.argtypes = [H]
     L.mmee_search_static.argtypes = [C.POINTER(Workload), C.POINTER(Arch), C.POINTER(Objective),
                                      C.c_void_p, C.c_void_p, C.c_void_p]
@@ -182,6 +184,14 @@ def mmee_search(handle, out_best, out_topk=None, stream=None) -> None:
     _check(library().mmee_search(handle, _stream_ptr(stream), C.c_void_p(out_best.data_ptr()),
                                  C.c_void_p(out_topk.data_ptr()) if out_topk is not None else None),
            "mmee_search")
+
+
+def mmee_search_host(handle, want_topk: bool = False, topk: int = 0):
+    """Search through a planned handle with the records copied to host structs: (best, list of top-k or None)."""
+    best = Result()
+    arr = (Result * topk)() if want_topk else None
+    _check(library().mmee_search_host(handle, C.byref(best), arr), "mmee_search_host")
+    return best, (list(arr) if want_topk else None)
 
 
 def mmee_search_static(workload: dict, arch: dict, objective: dict, out_best, out_topk=None, stream=None) -> None:

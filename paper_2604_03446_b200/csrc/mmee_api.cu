@@ -17,6 +17,7 @@ struct mmee_handle {
     mmee::LaunchShape shape;
     mmee::Scratch* scratch;      // device
     mmee_result_t* decode_buf;   // device, one record (mmee_decode); part of the scratch allocation
+    mmee_result_t* host_out;     // device, 1 + topk records (mmee_search_host); part of the scratch allocation
     mmee::PrunedTask* pruned;    // device, row pruning only
     uint32_t kept_rows;          // rows of a tiling that survive pruning (all rows without it)
     int device;
@@ -24,7 +25,7 @@ struct mmee_handle {
     float create_ms;             // host wall clock of mmee_create
     bool dirty;                  // a launch failed half-way: the scratch header is reset before the next search
     bool timing;
-    cudaEvent_t ev[3];           // before search kernel, between, after finalize kernel
+    cudaEvent_t ev[2];           // before and after the search kernel
 };
 
 namespace {
@@ -127,11 +128,12 @@ int mmee_create(const mmee_workload_t* workload, const mmee_arch_t* arch, const 
         }
         h->shape.pruned = h->pruned;
     }
-    // one allocation: the search scratch, then one result record for mmee_decode
+    // one allocation: the search scratch, one result record for mmee_decode, 1 + topk records for mmee_search_host
     const size_t sbytes = (scratch_bytes(h->shape.grid) + 15) / 16 * 16;
-    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&h->scratch), sbytes + sizeof(mmee_result_t));
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&h->scratch), sbytes + (2 + h->plan.topk) * sizeof(mmee_result_t));
     if (e == cudaSuccess) {
         h->decode_buf = reinterpret_cast<mmee_result_t*>(reinterpret_cast<unsigned char*>(h->scratch) + sbytes);
+        h->host_out = h->decode_buf + 1;
         e = launch_reset(h->scratch, 0);
         if (e == cudaSuccess) e = cudaStreamSynchronize(0);
     }
@@ -165,13 +167,10 @@ int mmee_search(mmee_handle_t* h, void* cuda_stream, mmee_result_t* out_best, mm
         h->dirty = false;
     }
     if (h->timing) cudaEventRecord(h->ev[0], st);
-    cudaError_t e = launch_search(h->plan, h->shape, h->device, h->scratch, nullptr, st);
+    const cudaError_t e = launch_search(h->plan, h->shape, h->device, h->scratch, nullptr, out_best, out_topk, st);
     if (e != cudaSuccess) { h->dirty = true; return cuda_status(e); }
     if (h->timing) cudaEventRecord(h->ev[1], st);
-    e = launch_finalize(h->plan, h->scratch, (int)h->shape.grid, out_best, out_topk, st);
-    if (e != cudaSuccess) { h->dirty = true; return cuda_status(e); }
-    if (h->timing) cudaEventRecord(h->ev[2], st);
-    h->last.kernels_launched = 2;
+    h->last.kernels_launched = 1;
     h->last.grid = h->shape.grid;
     h->last.block = kSearchThreads;
     h->last.smem_bytes = h->shape.smem_bytes;
@@ -181,10 +180,23 @@ int mmee_search(mmee_handle_t* h, void* cuda_stream, mmee_result_t* out_best, mm
     return MMEE_OK;
 }
 
+int mmee_search_host(mmee_handle_t* h, mmee_result_t* out_best, mmee_result_t* out_topk) {
+    if (!h || !out_best) return MMEE_ERR_ARG;
+    const uint32_t k = h->plan.topk;
+    int rc = mmee_search(h, nullptr, h->host_out, h->host_out + 1);
+    if (rc) return rc;
+    // (a copy to pageable host memory returns when the data is there: no further synchronisation needed)
+    if ((rc = cuda_status(cudaMemcpy(out_best, h->host_out, sizeof(mmee_result_t), cudaMemcpyDeviceToHost)))) return rc;
+    if (out_topk &&
+        (rc = cuda_status(cudaMemcpy(out_topk, h->host_out + 1, (size_t)k * sizeof(mmee_result_t), cudaMemcpyDeviceToHost))))
+        return rc;
+    return out_best->status == MMEE_ERR_CHECK ? MMEE_ERR_CHECK : MMEE_OK;
+}
+
 int mmee_destroy(mmee_handle_t* h) {
     if (!h) return MMEE_ERR_ARG;
     cudaError_t e = cudaSuccess;
-    if (h->timing) for (int i = 0; i < 3; ++i) cudaEventDestroy(h->ev[i]);
+    if (h->timing) for (int i = 0; i < 2; ++i) cudaEventDestroy(h->ev[i]);
     if (h->scratch) e = cudaFree(h->scratch);
     if (h->pruned) cudaFree(h->pruned);
     delete h;
@@ -240,7 +252,7 @@ int mmee_dump_keys(mmee_handle_t* h, void* cuda_stream, int64_t* out_keys) {
         if ((rc = cuda_status(launch_reset(h->scratch, st)))) return rc;
         h->dirty = false;
     }
-    cudaError_t e = launch_search(h->plan, h->shape, h->device, h->scratch, out_keys, st);
+    cudaError_t e = launch_search(h->plan, h->shape, h->device, h->scratch, out_keys, nullptr, nullptr, st);
     if (e != cudaSuccess) { h->dirty = true; return cuda_status(e); }
     if ((e = launch_reset(h->scratch, st)) != cudaSuccess) { h->dirty = true; return cuda_status(e); }
     return MMEE_OK;
@@ -415,16 +427,18 @@ int mmee_last_search_stats(const mmee_handle_t* h, mmee_launch_stats_t* out) {
     out->search_ms = out->finalize_ms = -1.0f;
     out->create_ms = h->create_ms;
     out->exact_path_visits = 0;
+    out->rows_tested = 0;
     if (h->last.kernels_launched) {
-        unsigned long long visits = 0;
-        const int rc = cuda_status(cudaMemcpy(&visits, &h->scratch->last_exact_visits, sizeof(visits), cudaMemcpyDeviceToHost));
+        unsigned long long counters[3] = {0, 0, 0};      // last_exact_visits, tested_rows, last_tested_rows
+        const int rc = cuda_status(cudaMemcpy(counters, &h->scratch->last_exact_visits, sizeof(counters), cudaMemcpyDeviceToHost));
         if (rc) return rc;
-        out->exact_path_visits = visits;
+        out->exact_path_visits = counters[0];
+        out->rows_tested = counters[2];
     }
     if (h->timing && h->last.kernels_launched) {
-        cudaError_t e = cudaEventElapsedTime(&out->search_ms, h->ev[0], h->ev[1]);
-        if (e == cudaSuccess) e = cudaEventElapsedTime(&out->finalize_ms, h->ev[1], h->ev[2]);
+        const cudaError_t e = cudaEventElapsedTime(&out->search_ms, h->ev[0], h->ev[1]);
         if (e != cudaSuccess) return cuda_status(e);
+        out->finalize_ms = 0.0f;        // the finalize step runs inside the search kernel (its last CTA)
     }
     return MMEE_OK;
 }
@@ -432,13 +446,13 @@ int mmee_last_search_stats(const mmee_handle_t* h, mmee_launch_stats_t* out) {
 int mmee_kernel_timing(mmee_handle_t* h, int enable) {
     if (!h) return MMEE_ERR_ARG;
     if (enable && !h->timing) {
-        for (int i = 0; i < 3; ++i) {
+        for (int i = 0; i < 2; ++i) {
             const int rc = cuda_status(cudaEventCreate(&h->ev[i]));
             if (rc) return rc;
         }
         h->timing = true;
     } else if (!enable && h->timing) {
-        for (int i = 0; i < 3; ++i) cudaEventDestroy(h->ev[i]);
+        for (int i = 0; i < 2; ++i) cudaEventDestroy(h->ev[i]);
         h->timing = false;
     }
     return MMEE_OK;

@@ -119,43 +119,83 @@ __device__ __forceinline__ TaskChoice decode_task(const Plan& p, uint32_t w) {
     return c;
 }
 
-// Full evaluation of one mapping: all five metric groups of Section VI-A (buffer sizes of
+// One candidate index taken apart (index layout: include/mmee.h).
+struct CandidateChoice {
+    uint64_t t;
+    uint32_t row, s;
+    TaskChoice c;
+    uint32_t lv[5];             // beta - 3 of A, B, C, D, E
+    int sm1, sm2;
+    bool fused;
+    uint32_t rc;                // C is regenerated (Section III-C)
+};
+
+__device__ __forceinline__ CandidateChoice decode_candidate(const Plan& p, uint64_t idx) {
+    CandidateChoice d;
+    const uint64_t per_t = (uint64_t)p.rows_per_tiling * 9u;
+    d.t = idx / per_t;
+    const uint32_t rem = (uint32_t)(idx - d.t * per_t);
+    d.row = rem / 9u;
+    d.s = rem % 9u;
+    const uint32_t w = d.row / 125u, mid = (d.row % 125u) / 25u, de = d.row % 25u;
+    d.c = decode_task(p, w);
+    d.fused = d.c.phi == 0;
+    d.lv[OP_A] = d.c.la;
+    d.lv[OP_B] = d.fused ? d.c.lb : mid;
+    d.lv[OP_C] = d.fused ? mid : 0u;
+    d.lv[OP_D] = de / 5u;
+    d.lv[OP_E] = de % 5u;
+    d.sm1 = (int)(d.s / 3u);
+    d.sm2 = (int)(d.s % 3u);
+    d.rc = d.fused ? p.q.recompute[d.c.order][d.lv[OP_C]] : 0u;
+    return d;
+}
+
+// Buffer words and DRAM words of one operand (Section V-B, V-C) from its two query vectors.  For the
+// intermediate C of an unfused mapping `da` is the read-back by the consumer nest only.
+__device__ __forceinline__ void operand_terms(const Plan& p, const CandidateChoice& d, const uint32_t b[8], int x,
+                                              int64_t& bs, int64_t& da) {
+    const QueryTables& q = p.q;
+    bs = monomial(q.bs[d.c.order][x][d.lv[x]], b);
+    if (d.fused) da = (x == OP_C) ? 0 : monomial(q.da[d.c.order][x][d.lv[x]][d.rc], b);
+    else da = monomial(q.da_unfused[d.c.order][x][d.lv[x]], b);
+}
+
+// Array-level terms of one operator (0: C = A*B, 1: E = C*D) under one stationary mode: buffer<->PE words
+// including the carried partial sums, and compute cycles.
+__device__ __forceinline__ void operator_array_terms(const Plan& p, const uint32_t b[8], const TilingCounts& c, int op,
+                                                     int sm, bool recompute, int64_t& words, int64_t& cycles) {
+    if (op == 0) {
+        const int64_t rho = recompute ? (int64_t)b[3] : 1;
+        const int64_t t1 = rho * c.t1;
+        words = t1 * tile_traffic(sm, b[4], b[5], b[6], p.pe_rows, p.pe_cols) + rho * c.carry1;
+        cycles = t1 * tile_cycles(sm, b[4], b[5], b[6], p.pe_rows, p.pe_cols);
+    } else {
+        words = c.t2 * tile_traffic(sm, b[4], b[6], b[7], p.pe_rows, p.pe_cols) + c.carry2;
+        cycles = c.t2 * tile_cycles(sm, b[4], b[6], b[7], p.pe_rows, p.pe_cols);
+    }
+}
+
+// The record of one mapping from its parts: all five metric groups of Section VI-A (buffer sizes of
 // producer and consumer, DRAM access, compute latency of both operators, buffer<->register
 // traffic), then energy and latency (Section V-D).
-__device__ inline void evaluate_candidate(const Plan& p, uint64_t idx, mmee_result_t& o) {
-    const uint64_t per_t = (uint64_t)p.rows_per_tiling * 9u;
-    const uint64_t t = idx / per_t;
-    const uint32_t rem = (uint32_t)(idx - t * per_t);
-    const uint32_t row = rem / 9u, s = rem % 9u;
-    const uint32_t w = row / 125u, mid = (row % 125u) / 25u, de = row % 25u;
-    const TaskChoice c = decode_task(p, w);
-    const uint32_t lv[5] = {c.la, c.phi == 0 ? c.lb : mid, c.phi == 0 ? mid : 0u, de / 5u, de % 5u};
-    const int sm1 = (int)(s / 3u), sm2 = (int)(s % 3u);
-
-    uint32_t b[8];
-    tiling_bounds(p, t, b);
-    const TilingCounts tt = tiling_counts(p, b);
-
-    o.idx = idx; o.t = t; o.row = row;
-    for (int d = 0; d < 8; ++d) o.bound[d] = b[d];
-    o.phi = (uint8_t)c.phi; o.pi = (uint8_t)c.order;
+__device__ __forceinline__ void assemble_record(const Plan& p, uint64_t idx, const CandidateChoice& d, const uint32_t b[8],
+                                                const TilingCounts& tt, const int64_t bs[5], const int64_t da_in[5],
+                                                int64_t words1, int64_t cyc1, int64_t words2, int64_t cyc2,
+                                                mmee_result_t& o) {
+    const uint32_t* lv = d.lv;
+    o.idx = idx; o.t = d.t; o.row = d.row;
+    for (int i = 0; i < 8; ++i) o.bound[i] = b[i];
+    o.phi = (uint8_t)d.c.phi; o.pi = (uint8_t)d.c.order;
     for (int x = 0; x < 5; ++x) o.beta[x] = (uint8_t)(lv[x] + 3);
-    o.sm[0] = (uint8_t)sm1; o.sm[1] = (uint8_t)sm2;
+    o.sm[0] = (uint8_t)d.sm1; o.sm[1] = (uint8_t)d.sm2;
     for (int i = 0; i < 5; ++i) o.reserved[i] = 0;
     o.status = MMEE_OK;
 
-    const QueryTables& q = p.q;
-    const bool fused = c.phi == 0;
-    const uint32_t rc = fused ? q.recompute[c.order][lv[OP_C]] : 0u;
-
-    int64_t bs[5], da[5];
-    for (int x = 0; x < 5; ++x) {
-        bs[x] = monomial(q.bs[c.order][x][lv[x]], b);
-        if (fused) da[x] = (x == OP_C) ? 0 : monomial(q.da[c.order][x][lv[x]][rc], b);
-        else da[x] = monomial(q.da_unfused[c.order][x][lv[x]], b);
-    }
+    int64_t da[5];
+    for (int x = 0; x < 5; ++x) da[x] = da_in[x];
     int64_t bs1, bs2, da_sm = 0, da1 = 0, da2 = 0;
-    if (fused) {
+    if (d.fused) {
         // Eq. (1)/(2): operands of the other operator count only when retained (tau = 1).
         bs1 = bs[OP_A] + bs[OP_B] + bs[OP_C] + (lv[OP_D] ? bs[OP_D] : 0) + (lv[OP_E] ? bs[OP_E] : 0);
         bs2 = bs[OP_C] + bs[OP_D] + bs[OP_E] + (lv[OP_A] ? bs[OP_A] : 0) + (lv[OP_B] ? bs[OP_B] : 0);
@@ -166,17 +206,17 @@ __device__ inline void evaluate_candidate(const Plan& p, uint64_t idx, mmee_resu
         da1 = da[OP_A] + da[OP_B] + c_write;
         da2 = da[OP_C] + da[OP_D] + da[OP_E];
         da[OP_C] += c_write;
-        if (c.phi == 2) da_sm = 2 * tt.il;             // separate softmax pass: read S, write P
+        if (d.c.phi == 2) da_sm = 2 * tt.il;           // separate softmax pass: read S, write P
     }
     const int64_t n_dram = da[0] + da[1] + da[2] + da[3] + da[4] + da_sm;
-    const ArrayTerms at = array_terms(p, b, tt, sm1, sm2, rc != 0);
-    const int64_t n_mac = at.n_mac, n_sfu = at.n_sfu, br = at.br, cyc1 = at.cyc1, cyc2 = at.cyc2;
+    const int64_t rho = d.rc ? (int64_t)b[3] : 1;
+    const int64_t n_mac = rho * tt.ikl + tt.ilj, n_sfu = rho * tt.il, br = words1 + words2;
     const int64_t n_gb = n_dram + br;
     const int64_t n_rf = p.has_rf ? br + 3 * n_mac : 0;
 
     const int64_t e_key = p.cq[0] * n_dram + p.cq[1] * n_gb + p.cq[2] * n_rf + p.cq[3] * n_mac + p.cq[4] * n_sfu;
     int64_t l_key;
-    if (fused) {
+    if (d.fused) {
         const int64_t comp = (cyc1 + cyc2) * (int64_t)p.bw;
         l_key = n_dram > comp ? n_dram : comp;
     } else {
@@ -190,13 +230,46 @@ __device__ inline void evaluate_candidate(const Plan& p, uint64_t idx, mmee_resu
     o.br = br; o.cyc1 = cyc1; o.cyc2 = cyc2;
     o.n[0] = n_dram; o.n[1] = n_gb; o.n[2] = n_rf; o.n[3] = n_mac; o.n[4] = n_sfu;
     o.e_key = e_key; o.l_key = l_key;
-    o.recompute = (uint8_t)rc;
-    o.feasible = (uint8_t)(o.bs <= p.cap_words && ((p.sm_mask >> s) & 1u));
+    o.recompute = (uint8_t)d.rc;
+    o.feasible = (uint8_t)(o.bs <= p.cap_words && ((p.sm_mask >> d.s) & 1u));
     o.edp_key = __dmul_rn((double)e_key, (double)l_key);
     o.energy_pj = __dmul_rn(__dmul_rn((double)e_key, p.quantum_pj), (double)p.instances);
     const uint32_t waves = (p.instances + p.n_arrays - 1) / p.n_arrays;
     o.latency_cycles = __dmul_rn(__ddiv_rn((double)l_key, (double)p.bw), (double)waves);
     o.n_total = 0; o.n_feasible = 0;
+}
+
+// Full evaluation of one mapping by one thread.
+__device__ inline void evaluate_candidate(const Plan& p, uint64_t idx, mmee_result_t& o) {
+    const CandidateChoice d = decode_candidate(p, idx);
+    uint32_t b[8];
+    tiling_bounds(p, d.t, b);
+    const TilingCounts tt = tiling_counts(p, b);
+    int64_t bs[5], da[5];
+    for (int x = 0; x < 5; ++x) operand_terms(p, d, b, x, bs[x], da[x]);
+    int64_t w1, c1, w2, c2;
+    operator_array_terms(p, b, tt, 0, d.sm1, d.rc != 0, w1, c1);
+    operator_array_terms(p, b, tt, 1, d.sm2, d.rc != 0, w2, c2);
+    assemble_record(p, idx, d, b, tt, bs, da, w1, c1, w2, c2, o);
+}
+
+// The same by one warp (all 32 lanes call it converged): lanes 0..4 take one operand each, lanes 5 and 6 one
+// operator's array-level terms each; lane 0 gathers the parts and holds the record on return.
+__device__ inline void evaluate_candidate_warp(const Plan& p, uint64_t idx, int lane, mmee_result_t& o) {
+    const CandidateChoice d = decode_candidate(p, idx);
+    uint32_t b[8];
+    tiling_bounds(p, d.t, b);
+    const TilingCounts tt = tiling_counts(p, b);
+    int64_t v0 = 0, v1 = 0;
+    if (lane < 5) operand_terms(p, d, b, lane, v0, v1);
+    else if (lane < 7) operator_array_terms(p, b, tt, lane - 5, lane == 5 ? d.sm1 : d.sm2, d.rc != 0, v0, v1);
+    int64_t part0[7], part1[7];
+#pragma unroll
+    for (int i = 0; i < 7; ++i) {
+        part0[i] = __shfl_sync(0xffffffffu, v0, i);
+        part1[i] = __shfl_sync(0xffffffffu, v1, i);
+    }
+    if (lane == 0) assemble_record(p, idx, d, b, tt, part0, part1, part0[5], part1[5], part0[6], part1[6], o);
 }
 
 }  // namespace mmee

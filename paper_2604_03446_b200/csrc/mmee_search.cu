@@ -114,8 +114,11 @@ struct alignas(16) CtaShared {
     long long G;             // upper bound on the final k-th smallest key (any full list's last key)
     unsigned long long feasible_rows;
     unsigned long long exact_visits;         // groups that some warp of this CTA took to the exact path
+    unsigned long long tested_rows;          // rows whose capacity test and bound were evaluated
     unsigned long long range_begin[2];       // first task of the range whose tables sit in buffer 0 / 1
     unsigned int cursor[2];                  // next unassigned task of that range, relative to its begin
+    unsigned int last_cta;                   // this CTA drew the last ticket: it runs the finalize step
+    unsigned int check_failed;               // finalize step: a winner's key is not the key of its evaluation
 };
 
 __device__ __forceinline__ bool pair_less(int64_t ka, uint64_t ia, int64_t kb, uint64_t ib) {
@@ -152,6 +155,39 @@ __device__ __forceinline__ bool reg_insert(int64_t& ek, uint64_t& ei, int k, int
     if (lane == pos) { ek = nk; ei = ni; }
     else if (lane > pos && lane < k) { ek = uk; ei = ui; }
     return true;
+}
+
+// Merge of two such lists (both sorted, (kInfKey, UINT64_MAX) in every unused lane): the k smallest pairs of
+// both, sorted, stay in (ek, ei).  The other list reversed and the lane-wise minimum of the two give the 16
+// smallest of the 32 pairs as a bitonic sequence, which four compare-exchange stages sort.  All 32 lanes call
+// this converged.  Cheaper than insertion one by one when the other list is long.
+__device__ __forceinline__ void reg_merge(int64_t& ek, uint64_t& ei, int k, int64_t ok, uint64_t oi, int lane) {
+    const int rev = (MMEE_MAX_TOPK - 1 - lane) & 31;
+    const int64_t rk = __shfl_sync(kFull, ok, rev);
+    const uint64_t ri = __shfl_sync(kFull, oi, rev);
+    if (lane < (int)MMEE_MAX_TOPK && pair_less(rk, ri, ek, ei)) { ek = rk; ei = ri; }
+#pragma unroll
+    for (int stride = MMEE_MAX_TOPK / 2; stride >= 1; stride >>= 1) {
+        const int64_t pk = __shfl_xor_sync(kFull, ek, stride);
+        const uint64_t pi = __shfl_xor_sync(kFull, ei, stride);
+        const bool keep_smaller = (lane & stride) == 0;
+        if (pair_less(pk, pi, ek, ei) == keep_smaller) { ek = pk; ei = pi; }
+    }
+    if (lane >= k) { ek = kInfKey; ei = UINT64_MAX; }
+}
+
+// The other list has n entries, lane j holding entry j: by insertion when it is short, else by the merge above.
+__device__ __forceinline__ void reg_absorb(int64_t& ek, uint64_t& ei, int k, int n, int64_t ok, uint64_t oi, int lane) {
+    if (n > 3) {
+        if (lane >= n) { ok = kInfKey; oi = UINT64_MAX; }
+        reg_merge(ek, ei, k, ok, oi, lane);
+        return;
+    }
+    for (int j = 0; j < n; ++j) {
+        const long long sk = __shfl_sync(kFull, ok, j);
+        const uint64_t si = __shfl_sync(kFull, oi, j);
+        if (!reg_insert(ek, ei, k, sk, si, lane)) break;   // sorted: the rest is larger
+    }
 }
 
 // Threshold for candidates whose indices are all >= first_idx: a key passes iff it can still enter
@@ -703,7 +739,8 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
                                                     const TaskChoice& c, bool live, bool valid, uint32_t kept,
                                                     uint32_t kept_mid, uint64_t task_first_idx, WarpTop* wt,
                                                     CtaShared* cs, long long* global_g, int k, int lane,
-                                                    int64_t* __restrict__ dump, uint64_t dump_origin, uint32_t& visits) {
+                                                    int64_t* __restrict__ dump, uint64_t dump_origin, uint32_t& visits,
+                                                    uint32_t& tested) {
     const RowTab* rt = &ot->rt[c.phi == 0 ? 0 : 1];
     LaneThreshold th = load_threshold(wt, cs, k);
     uint32_t rows = 0;
@@ -753,6 +790,7 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
             // no lane has room left for D and E at this middle level: none of its 25 rows fits
             if (!__any_sync(kFull, (slack1c | slack2c) >= 0)) continue;
         }
+        uint32_t groups_walked = 0;
 
 #pragma unroll 1
         for (int d = 0; d < 5; ++d) {
@@ -765,6 +803,7 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
                 const int s1c = slack1c - dc.x;
                 const int s2c = slack2c - dc.y;
                 if (!__any_sync(kFull, (s1c | s2c) >= 0)) continue;     // D leaves no room in any lane
+                ++groups_walked;
                 const float fxd = __fadd_rd(fx0, __int_as_float(dc.z));
                 const float fed = __fadd_rd(fe0, __int_as_float(dc.w));
                 const uint32_t kd = PRUNE ? (kept >> (d * 5)) : 31u;
@@ -780,6 +819,7 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
                 }
                 if (__any_sync(kFull, hit1 != 0u)) hit_any = edp_group_test(me, rt, d, s1c, s2c, kd, p.sm_mask, dthr);
             } else {
+                ++groups_walked;
                 const int64_t s1 = me.slack1 - rt->D[d][0];
                 const int64_t s2 = me.slack2 - rt->D[d][1];
                 const int64_t xd = me.x0 + rt->D[d][2];
@@ -817,6 +857,7 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
                 refresh();
             }
         }
+        if (live) tested += groups_walked * 5u;
     }
     return rows;
 }
@@ -829,7 +870,8 @@ template <int OBJ, bool PRUNE>
 __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const TilingTab* tb, const OrderTab* ot,
                                                        const TaskChoice& c, bool live, uint32_t kept, uint32_t kept_mid,
                                                        uint64_t task_first_idx, WarpTop* wt, CtaShared* cs,
-                                                       long long* global_g, int k, int lane, uint32_t& visits) {
+                                                       long long* global_g, int k, int lane, uint32_t& visits,
+                                                       uint32_t& tested) {
     const bool fused = c.phi == 0;
     const RowTab* rt = &ot->rt[fused ? 0 : 1];
     // Row-side terms of E.  Its buffer need while Op1 runs is its size when retained (level >= L4 of a
@@ -845,7 +887,7 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
     const int capc = (int)p.cap_words;
     // Additions that need no saturation are written x * one + y: an integer multiply-add runs on the FMA
     // pipe, which is otherwise idle, instead of the integer ALU pipe that bounds this kernel.
-    const int one = p.unit, minus_one = -p.unit;
+    const int minus_one = -p.unit;
     const int gxc = (OBJ == MMEE_OBJ_ENERGY && !fused) ? ot->gXc[c.phi == 2 ? 1 : 0] : 0;
     // task-level part of key - thr, clamped to [-kUnfit, kRowCap]: clamping from below keeps the sign of every
     // sum that follows (at most 4 * kTermCap < kUnfit is added), clamping from above only lowers
@@ -884,7 +926,9 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
     };
     rebase(0);
 
-    int unfit = 0;          // minus the number of visited rows that do not fit
+    // low half: the number of rows that do not fit; high half: how many of them lay in middle levels and groups
+    // that no lane of the warp had room for (their rows were not tested one by one)
+    int unfit = 0;
     uint32_t groups = 0;
 #pragma unroll 1
     for (int mi = 0; mi < (PRUNE ? 1 : 5); ++mi) {
@@ -906,7 +950,7 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
 
         // No lane has room left for D and E at this middle level: none of its 25 rows fits.
         if (!__any_sync(kFull, (slack1c | slack2c) >= 0)) {
-            if constexpr (!PRUNE) unfit -= 25;
+            if constexpr (!PRUNE) unfit += 25 + (25 << 16);
             continue;
         }
 
@@ -963,7 +1007,7 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
             const int lim_retained = min(s1c, s2c);
             // D leaves no room in any lane: none of the group's five rows fits
             if (!__any_sync(kFull, lim_l3 >= 0)) {
-                if constexpr (!PRUNE) unfit -= 5;
+                if constexpr (!PRUNE) unfit += 5 + (5 << 16);
                 continue;
             }
             if constexpr (PRUNE) ++groups;
@@ -976,7 +1020,7 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
                 // which makes its keys non-negative whatever the threshold
                 int t = sign_mask(imad(E2c[e], minus_one, e == 0 ? lim_l3 : lim_retained));
                 if constexpr (PRUNE) t |= (int)((kd >> e) & 1u) - 1;
-                unfit = imad(t, one, unfit);
+                unfit = imad(t, minus_one, unfit);
                 g[e] = Gc[e] | (t & kUnfit);             // (Gc <= kTermCap < kUnfit, a single bit)
             }
             // least key of the group's 45 mappings, relative to the threshold
@@ -991,7 +1035,114 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
         }
     }
     if constexpr (!PRUNE) groups = 25;
-    return (uint32_t)((int)(groups * 5u) + unfit);
+    if (live) tested += groups * 5u - ((uint32_t)unfit >> 16);
+    return groups * 5u - ((uint32_t)unfit & 0xffffu);
+}
+
+// ------------------------------------------------------------------------------------------------
+// finalize: merge the CTAs' partial lists, evaluate the winners in full, reset the scratch header
+// ------------------------------------------------------------------------------------------------
+// Run by every thread of ONE CTA (the last one to finish its search) after all CTAs have published their
+// partial lists.  `tops` is shared memory for one list per warp, `check_failed` a shared flag (zero on entry).
+__device__ __noinline__ void finalize_step(const Plan& p, Scratch* __restrict__ scratch, int n_partials,
+                                              mmee_result_t* __restrict__ out_best, mmee_result_t* __restrict__ out_topk,
+                                              longlong2 (*tops)[MMEE_MAX_TOPK], unsigned int* check_failed) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int kWarps = kSearchThreads / 32;
+    const int k = (int)p.topk;
+    int64_t ek = kInfKey;
+    uint64_t ei = UINT64_MAX;
+    // Thread i looks at the length of partial list i (+ a multiple of the CTA size): one round trip to the L2
+    // for all lengths.  Most lists are empty, because a CTA publishes only the entries that are not above the
+    // bound G it knew at its end.  Each warp then merges the non-empty lists among its 32, eight at a time
+    // (lane j takes entry j of each; the loads bypass the L1 cache).
+    constexpr int kBatch = 8;
+    for (int c0 = 0; c0 < n_partials; c0 += kSearchThreads) {
+        const int c = c0 + tid;
+        const int len = c < n_partials ? __ldcg(&scratch->partial[c].count) : 0;
+        unsigned todo = __ballot_sync(kFull, len > 0);
+        while (todo) {
+            int n[kBatch];
+            longlong2 mine[kBatch];
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) {
+                n[i] = 0;
+                mine[i] = make_longlong2(kInfKey, -1ll);
+                if (todo) {
+                    const int src_lane = __ffs(todo) - 1;
+                    todo &= todo - 1;
+                    n[i] = __shfl_sync(kFull, len, src_lane);
+                    if (lane < n[i]) mine[i] = __ldcg(&scratch->partial[c0 + warp * 32 + src_lane].e[lane]);
+                }
+            }
+            // (unrolled: with a run-time index the batch would live in local memory, and the store of each
+            // loaded entry there would wait for its load before the next load could issue)
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) reg_absorb(ek, ei, k, n[i], mine[i].x, (uint64_t)mine[i].y, lane);
+        }
+    }
+    // The warps' lists are merged pairwise into warp 0's.
+    if (lane < MMEE_MAX_TOPK) tops[warp][lane] = make_longlong2((long long)ek, (long long)ei);
+    for (int stride = kWarps / 2; stride >= 1; stride >>= 1) {
+        __syncthreads();
+        if (warp < stride) {
+            const longlong2 theirs = lane < MMEE_MAX_TOPK ? tops[warp + stride][lane] : make_longlong2(kInfKey, -1ll);
+            const int n_theirs = __popc(__ballot_sync(kFull, theirs.x != kInfKey || theirs.y != -1ll));
+            reg_absorb(ek, ei, k, n_theirs, theirs.x, (uint64_t)theirs.y, lane);
+            if (lane < MMEE_MAX_TOPK) tops[warp][lane] = make_longlong2((long long)ek, (long long)ei);
+        }
+    }
+    __syncthreads();
+    // Every winner is evaluated in full, one warp per record (the parts of a record on different lanes); the key
+    // it was ranked by must be the key of that evaluation.  A mismatch (a list entry whose key and index do not
+    // belong together) is reported in out_best->status instead of being returned as a result.
+    const longlong2 final_entry = lane < MMEE_MAX_TOPK ? tops[0][lane] : make_longlong2(kInfKey, -1ll);
+    const int found = __popc(__ballot_sync(kFull, lane < k && (final_entry.x != kInfKey || final_entry.y != -1ll)));
+    mmee_result_t r, first;
+    for (int rec = warp; rec < k; rec += kWarps) {
+        const long long rk = __shfl_sync(kFull, final_entry.x, rec);
+        const uint64_t ri = (uint64_t)__shfl_sync(kFull, final_entry.y, rec);
+        if (rec < found) {
+            evaluate_candidate_warp(p, ri, lane, r);
+            if (lane == 0) {
+                int64_t key;
+                switch (p.objective) {
+                    case MMEE_OBJ_ENERGY: key = r.e_key; break;
+                    case MMEE_OBJ_LATENCY: key = r.l_key; break;
+                    case MMEE_OBJ_EDP: key = dbits(r.edp_key); break;
+                    case MMEE_OBJ_ENERGY_LCAP: key = r.l_key <= p.key_cap ? r.e_key : kInfKey; break;
+                    default: key = r.e_key <= p.key_cap ? r.l_key : kInfKey; break;
+                }
+                if (!(key == rk && r.feasible && r.t >= p.t_begin && r.t < p.t_end)) atomicOr(check_failed, 1u);
+            }
+        } else if (lane == 0) {
+            // empty slot
+            unsigned long long* raw = reinterpret_cast<unsigned long long*>(&r);
+            for (unsigned i = 0; i < sizeof(r) / 8; ++i) raw[i] = 0;
+            r.idx = MMEE_NO_INDEX;
+            r.status = found ? MMEE_OK : MMEE_ERR_NO_FEASIBLE;
+        }
+        if (lane == 0) {
+            if (out_topk) out_topk[rec] = r;
+            if (rec == 0) first = r;
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        first.n_total = (p.t_end - p.t_begin) * (uint64_t)p.rows_per_tiling * 9u;
+        first.n_feasible = __ldcg(&scratch->feasible_rows) * (uint64_t)p.n_sm;
+        if (*check_failed) first.status = MMEE_ERR_CHECK;
+        *out_best = first;
+        // ready for the next search on this scratch
+        scratch->next_task = 0;
+        scratch->feasible_rows = 0;
+        scratch->G = kInfKey - 1;
+        scratch->last_exact_visits = __ldcg(&scratch->exact_visits);
+        scratch->exact_visits = 0;
+        scratch->last_tested_rows = __ldcg(&scratch->tested_rows);
+        scratch->tested_rows = 0;
+        scratch->done_ctas = 0;
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1001,7 +1152,7 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
 template <int OBJ, int MODE>
 __global__ void __launch_bounds__(kSearchThreads, 2)
 search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Scratch* __restrict__ scratch,
-              int64_t* __restrict__ dump) {
+              int64_t* __restrict__ dump, mmee_result_t* __restrict__ out_best, mmee_result_t* __restrict__ out_topk) {
     constexpr bool DUMP = MODE == kModeDump;        // store every key instead of reducing
     constexpr bool PRUNE = MODE == kModePrune;      // visit only the rows kept by symbolic pruning
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -1028,6 +1179,8 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
         cs->G = scratch->G;
         cs->feasible_rows = 0;
         cs->exact_visits = 0;
+        cs->tested_rows = 0;
+        cs->check_failed = 0;
     }
     if (lane == 0) wt->count = 0;
     __syncthreads();      // the shared copy of the plan is complete
@@ -1038,6 +1191,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
     const uint32_t n_orders = p.n_orders;
     unsigned long long my_rows = 0;
     uint32_t my_visits = 0;
+    uint32_t my_tested = 0;       // rows whose capacity test and bound this lane evaluated (fewer than 2^32 per lane)
 
     // Builder: pull the next range and build its tables into buffer `buf`.  Ranges are visited in a
     // stride-permuted order (stride coprime to their number), so that the first pull of every CTA
@@ -1194,10 +1348,10 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
             const long long g_seen = (lane == 0) ? *reinterpret_cast<volatile long long*>(&scratch->G) : 0;
             if constexpr (!DUMP && OBJ <= MMEE_OBJ_LATENCY) {
                 my_rows += walk_task_relative<OBJ, PRUNE>(p, tb, ot, c, live, kept, kept_mid, task_first_idx, wt, cs,
-                                                          &scratch->G, k, lane, my_visits);
+                                                          &scratch->G, k, lane, my_visits, my_tested);
             } else {
                 my_rows += walk_task_exact<OBJ, DUMP, PRUNE>(p, tb, ot, c, live, valid, kept, kept_mid, task_first_idx, wt,
-                                                             cs, &scratch->G, k, lane, dump, dump_origin, my_visits);
+                                                             cs, &scratch->G, k, lane, dump, dump_origin, my_visits, my_tested);
             }
             if (lane == 0 && g_seen < cs->G) atomicMin(&cs->G, g_seen);
         }
@@ -1206,8 +1360,13 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
     }
 
     // ---- feasible count
-    for (int off = 16; off; off >>= 1) my_rows += __shfl_down_sync(kFull, my_rows, off);
+    unsigned long long tested_rows = my_tested;
+    for (int off = 16; off; off >>= 1) {
+        my_rows += __shfl_down_sync(kFull, my_rows, off);
+        tested_rows += __shfl_down_sync(kFull, tested_rows, off);
+    }
     if (lane == 0 && my_rows) atomicAdd(&cs->feasible_rows, my_rows);
+    if (lane == 0 && tested_rows) atomicAdd(&cs->tested_rows, tested_rows);
     if (lane == 0 && my_visits) atomicAdd(&cs->exact_visits, (unsigned long long)my_visits);
     __syncthreads();
 
@@ -1224,120 +1383,37 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
             const WarpTop* src = &wtops[w2];
             const int n = src->count;
             const longlong2 theirs = lane < n ? src->e[lane] : make_longlong2(kInfKey, -1ll);
-            for (int j = 0; j < n; ++j) {
-                const long long sk = __shfl_sync(kFull, theirs.x, j);
-                const long long si = __shfl_sync(kFull, theirs.y, j);
-                if (!reg_insert(ek, ei, k, sk, (uint64_t)si, lane)) break;   // sorted: the rest is larger
-            }
+            reg_absorb(ek, ei, k, n, theirs.x, (uint64_t)theirs.y, lane);
         }
+        // An entry above the bound G (some full list's last key, here or in another CTA) cannot be among the
+        // k best of the whole search: it is not published.
         Partial* out = &scratch->partial[blockIdx.x];
-        const int n = __popc(__ballot_sync(kFull, ek != kInfKey || ei != UINT64_MAX));
+        long long g_end = (lane == 0) ? *reinterpret_cast<volatile long long*>(&scratch->G) : 0;
+        g_end = __shfl_sync(kFull, g_end, 0);
+        if (cs->G < g_end) g_end = cs->G;
+        const int n = __popc(__ballot_sync(kFull, (ek != kInfKey || ei != UINT64_MAX) && ek <= g_end));
         if (lane < n) out->e[lane] = make_longlong2((long long)ek, (long long)ei);
         if (lane == 0) {
             out->count = n;
             if (cs->feasible_rows) atomicAdd(&scratch->feasible_rows, cs->feasible_rows);
             if (cs->exact_visits) atomicAdd(&scratch->exact_visits, cs->exact_visits);
+            if (cs->tested_rows) atomicAdd(&scratch->tested_rows, cs->tested_rows);
+        }
+        if constexpr (!DUMP) {
+            // Grid reduction without a wait: every CTA makes its partial list visible, then draws a ticket; the
+            // CTA that draws the last one knows that all lists are there and runs the finalize step.
+            __threadfence();
+            __syncwarp();
+            if (lane == 0) cs->last_cta = atomicAdd(&scratch->done_ctas, 1u) == gridDim.x - 1 ? 1u : 0u;
         }
     }
-}
-
-// ------------------------------------------------------------------------------------------------
-// finalize: merge the CTAs' partial lists, evaluate the winners in full, reset the scratch header
-// ------------------------------------------------------------------------------------------------
-
-__global__ void __launch_bounds__(1024, 1)
-finalize_kernel(const __grid_constant__ Plan p, Scratch* __restrict__ scratch, int n_partials,
-                mmee_result_t* __restrict__ out_best, mmee_result_t* __restrict__ out_topk) {
-    __shared__ longlong2 tops[32][MMEE_MAX_TOPK];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int k = (int)p.topk;
-    int64_t ek = kInfKey;
-    uint64_t ei = UINT64_MAX;
-    // Each warp merges every 32nd partial list.  The lists of four partials are fetched at once (lane j takes
-    // entry j; the length and the entries are independent loads), so that the merge waits for one round trip
-    // to global memory per four lists instead of one per entry.
-    constexpr int kBatch = 4;
-    for (int c0 = warp; c0 < n_partials; c0 += 32 * kBatch) {
-        int n[kBatch];
-        longlong2 mine[kBatch];
-#pragma unroll
-        for (int i = 0; i < kBatch; ++i) {
-            const int c = c0 + 32 * i;
-            n[i] = 0;
-            mine[i] = make_longlong2(kInfKey, -1ll);
-            if (c < n_partials) {
-                const Partial* src = &scratch->partial[c];
-                n[i] = src->count;
-                if (lane < MMEE_MAX_TOPK) mine[i] = src->e[lane];      // (entries past the length are not used)
-            }
-        }
-#pragma unroll
-        for (int i = 0; i < kBatch; ++i) {
-            for (int j = 0; j < n[i]; ++j) {
-                const long long sk = __shfl_sync(kFull, mine[i].x, j);
-                const long long si = __shfl_sync(kFull, mine[i].y, j);
-                if (!reg_insert(ek, ei, k, sk, (uint64_t)si, lane)) break;   // sorted: the rest is larger
-            }
-        }
-    }
-    // The 32 warps' lists are merged pairwise, in five rounds, into warp 0's.
-    if (lane < MMEE_MAX_TOPK) tops[warp][lane] = make_longlong2((long long)ek, (long long)ei);
-    for (int stride = 16; stride >= 1; stride >>= 1) {
+    if constexpr (!DUMP) {
         __syncthreads();
-        if (warp < stride) {
-            const longlong2 theirs = lane < MMEE_MAX_TOPK ? tops[warp + stride][lane] : make_longlong2(kInfKey, -1ll);
-            for (int j = 0; j < k; ++j) {
-                const long long sk = __shfl_sync(kFull, theirs.x, j);
-                const long long si = __shfl_sync(kFull, theirs.y, j);
-                if (!reg_insert(ek, ei, k, sk, (uint64_t)si, lane)) break;   // (an empty slot never enters)
-            }
-            if (lane < MMEE_MAX_TOPK) tops[warp][lane] = make_longlong2((long long)ek, (long long)ei);
-        }
-    }
-    if (warp == 0) {
-        const int found = __popc(__ballot_sync(kFull, ek != kInfKey || ei != UINT64_MAX));
-        const uint64_t n_total = (p.t_end - p.t_begin) * (uint64_t)p.rows_per_tiling * 9u;
-        const uint64_t n_feasible = scratch->feasible_rows * (uint64_t)p.n_sm;
-        // Every winner is evaluated in full; the key it was ranked by must be the key of that evaluation.  A
-        // mismatch (a list entry whose key and index do not belong together) is reported in out_best->status
-        // instead of being returned as a result.
-        bool consistent = true;
-        if (lane < k) {
-            mmee_result_t r;
-            if (lane < found) {
-                evaluate_candidate(p, ei, r);
-                int64_t key;
-                switch (p.objective) {
-                    case MMEE_OBJ_ENERGY: key = r.e_key; break;
-                    case MMEE_OBJ_LATENCY: key = r.l_key; break;
-                    case MMEE_OBJ_EDP: key = dbits(r.edp_key); break;
-                    case MMEE_OBJ_ENERGY_LCAP: key = r.l_key <= p.key_cap ? r.e_key : kInfKey; break;
-                    default: key = r.e_key <= p.key_cap ? r.l_key : kInfKey; break;
-                }
-                consistent = key == ek && r.feasible && r.t >= p.t_begin && r.t < p.t_end;
-            } else {
-                // empty slot
-                unsigned char* raw = reinterpret_cast<unsigned char*>(&r);
-                for (unsigned i = 0; i < sizeof(r); ++i) raw[i] = 0;
-                r.idx = MMEE_NO_INDEX;
-                r.status = found ? MMEE_OK : MMEE_ERR_NO_FEASIBLE;
-            }
-            const bool all_consistent = __all_sync(__activemask(), consistent);
-            if (out_topk) out_topk[lane] = r;
-            if (lane == 0) {
-                r.n_total = n_total;
-                r.n_feasible = n_feasible;
-                if (!all_consistent) r.status = MMEE_ERR_CHECK;
-                *out_best = r;
-            }
-        }
-        __syncwarp();
-        if (lane == 0) {         // ready for the next search on this handle
-            scratch->next_task = 0;
-            scratch->feasible_rows = 0;
-            scratch->G = kInfKey - 1;
-            scratch->last_exact_visits = scratch->exact_visits;
-            scratch->exact_visits = 0;
+        if (cs->last_cta) {
+            __threadfence();
+            // (the table buffers are no longer in use: their first bytes hold the warps' lists of the merge)
+            finalize_step(p, scratch, (int)gridDim.x, out_best, out_topk,
+                          reinterpret_cast<longlong2 (*)[MMEE_MAX_TOPK]>(ttabs_all), &cs->check_failed);
         }
     }
 }
@@ -1347,6 +1423,8 @@ __global__ void reset_kernel(Scratch* scratch) {
     scratch->feasible_rows = 0;
     scratch->G = kInfKey - 1;
     scratch->exact_visits = 0;
+    scratch->tested_rows = 0;
+    scratch->done_ctas = 0;
 }
 
 __global__ void eval_kernel(const __grid_constant__ Plan p, uint64_t idx_begin, uint64_t count,
@@ -1378,10 +1456,10 @@ cudaError_t allow_large_smem(int device) {
 
 template <int OBJ, int MODE>
 cudaError_t launch_search_t(const Plan& p, const LaunchShape& shape, int device, Scratch* scratch, int64_t* dump,
-                            cudaStream_t st) {
+                            mmee_result_t* out_best, mmee_result_t* out_topk, cudaStream_t st) {
     cudaError_t e = allow_large_smem<OBJ, MODE>(device);
     if (e != cudaSuccess) return e;
-    search_kernel<OBJ, MODE><<<shape.grid, kSearchThreads, shape.smem_bytes, st>>>(p, shape, scratch, dump);
+    search_kernel<OBJ, MODE><<<shape.grid, kSearchThreads, shape.smem_bytes, st>>>(p, shape, scratch, dump, out_best, out_topk);
     return cudaGetLastError();
 }
 
@@ -1410,38 +1488,32 @@ cudaError_t search_occupancy(const Plan& p, int device, size_t smem, int* blocks
 }
 
 cudaError_t launch_search(const Plan& p, const LaunchShape& shape, int device, Scratch* scratch, int64_t* dump,
-                          cudaStream_t st) {
+                          mmee_result_t* out_best, mmee_result_t* out_topk, cudaStream_t st) {
     if (dump) {
         switch (p.objective) {
-            case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, kModeDump>(p, shape, device, scratch, dump, st);
-            case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, kModeDump>(p, shape, device, scratch, dump, st);
-            case MMEE_OBJ_EDP: return launch_search_t<MMEE_OBJ_EDP, kModeDump>(p, shape, device, scratch, dump, st);
-            case MMEE_OBJ_ENERGY_LCAP: return launch_search_t<MMEE_OBJ_ENERGY_LCAP, kModeDump>(p, shape, device, scratch, dump, st);
-            default: return launch_search_t<MMEE_OBJ_LATENCY_ECAP, kModeDump>(p, shape, device, scratch, dump, st);
+            case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, kModeDump>(p, shape, device, scratch, dump, out_best, out_topk, st);
+            case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, kModeDump>(p, shape, device, scratch, dump, out_best, out_topk, st);
+            case MMEE_OBJ_EDP: return launch_search_t<MMEE_OBJ_EDP, kModeDump>(p, shape, device, scratch, dump, out_best, out_topk, st);
+            case MMEE_OBJ_ENERGY_LCAP: return launch_search_t<MMEE_OBJ_ENERGY_LCAP, kModeDump>(p, shape, device, scratch, dump, out_best, out_topk, st);
+            default: return launch_search_t<MMEE_OBJ_LATENCY_ECAP, kModeDump>(p, shape, device, scratch, dump, out_best, out_topk, st);
         }
     }
     if (shape.pruned) {
         switch (p.objective) {
-            case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, kModePrune>(p, shape, device, scratch, nullptr, st);
-            case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, kModePrune>(p, shape, device, scratch, nullptr, st);
-            case MMEE_OBJ_EDP: return launch_search_t<MMEE_OBJ_EDP, kModePrune>(p, shape, device, scratch, nullptr, st);
-            case MMEE_OBJ_ENERGY_LCAP: return launch_search_t<MMEE_OBJ_ENERGY_LCAP, kModePrune>(p, shape, device, scratch, nullptr, st);
-            default: return launch_search_t<MMEE_OBJ_LATENCY_ECAP, kModePrune>(p, shape, device, scratch, nullptr, st);
+            case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, kModePrune>(p, shape, device, scratch, nullptr, out_best, out_topk, st);
+            case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, kModePrune>(p, shape, device, scratch, nullptr, out_best, out_topk, st);
+            case MMEE_OBJ_EDP: return launch_search_t<MMEE_OBJ_EDP, kModePrune>(p, shape, device, scratch, nullptr, out_best, out_topk, st);
+            case MMEE_OBJ_ENERGY_LCAP: return launch_search_t<MMEE_OBJ_ENERGY_LCAP, kModePrune>(p, shape, device, scratch, nullptr, out_best, out_topk, st);
+            default: return launch_search_t<MMEE_OBJ_LATENCY_ECAP, kModePrune>(p, shape, device, scratch, nullptr, out_best, out_topk, st);
         }
     }
     switch (p.objective) {
-        case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, kModeSearch>(p, shape, device, scratch, nullptr, st);
-        case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, kModeSearch>(p, shape, device, scratch, nullptr, st);
-        case MMEE_OBJ_EDP: return launch_search_t<MMEE_OBJ_EDP, kModeSearch>(p, shape, device, scratch, nullptr, st);
-        case MMEE_OBJ_ENERGY_LCAP: return launch_search_t<MMEE_OBJ_ENERGY_LCAP, kModeSearch>(p, shape, device, scratch, nullptr, st);
-        default: return launch_search_t<MMEE_OBJ_LATENCY_ECAP, kModeSearch>(p, shape, device, scratch, nullptr, st);
+        case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, kModeSearch>(p, shape, device, scratch, nullptr, out_best, out_topk, st);
+        case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, kModeSearch>(p, shape, device, scratch, nullptr, out_best, out_topk, st);
+        case MMEE_OBJ_EDP: return launch_search_t<MMEE_OBJ_EDP, kModeSearch>(p, shape, device, scratch, nullptr, out_best, out_topk, st);
+        case MMEE_OBJ_ENERGY_LCAP: return launch_search_t<MMEE_OBJ_ENERGY_LCAP, kModeSearch>(p, shape, device, scratch, nullptr, out_best, out_topk, st);
+        default: return launch_search_t<MMEE_OBJ_LATENCY_ECAP, kModeSearch>(p, shape, device, scratch, nullptr, out_best, out_topk, st);
     }
-}
-
-cudaError_t launch_finalize(const Plan& p, Scratch* scratch, int n_partials, mmee_result_t* out_best,
-                            mmee_result_t* out_topk, cudaStream_t st) {
-    finalize_kernel<<<1, 1024, 0, st>>>(p, scratch, n_partials, out_best, out_topk);
-    return cudaGetLastError();
 }
 
 cudaError_t launch_reset(Scratch* scratch, cudaStream_t st) {

@@ -21,14 +21,17 @@ struct alignas(16) Partial {
 
 // Global scratch of one handle: a work counter, the feasible-row count, the shared pruning bound,
 // the count of exact-path visits and one partial list per CTA.  The header is reset by the finalize
-// kernel, which also keeps the finished search's visit count in `last_exact_visits`.
+// step, which also keeps the finished search's visit count in `last_exact_visits`.
 struct Scratch {
     unsigned long long next_task;
     unsigned long long feasible_rows;
     long long G;
     unsigned long long exact_visits;
     unsigned long long last_exact_visits;
-    unsigned long long pad;
+    unsigned long long tested_rows;         // rows whose capacity test and bound were evaluated
+    unsigned long long last_tested_rows;
+    unsigned int done_ctas;         // ticket counter: the CTA that draws the last ticket runs the finalize step
+    unsigned int pad;
     Partial partial[1];     // grid entries follow
 };
 
@@ -48,10 +51,11 @@ inline size_t scratch_bytes(uint32_t grid) { return sizeof(Scratch) + (size_t)(g
 
 size_t search_smem_bytes(const Plan& p, uint32_t slots);
 cudaError_t search_occupancy(const Plan& p, int device, size_t smem, int* blocks_per_sm);
+// One launch per search: the last CTA to finish merges the partial lists, evaluates the winners into
+// out_best / out_topk (device) and resets the scratch header.  With `dump` set the kernel stores every
+// key instead and writes no result (the caller resets the header).
 cudaError_t launch_search(const Plan& p, const LaunchShape& shape, int device, Scratch* scratch, int64_t* dump,
-                          cudaStream_t st);
-cudaError_t launch_finalize(const Plan& p, Scratch* scratch, int n_partials, mmee_result_t* out_best,
-                            mmee_result_t* out_topk, cudaStream_t st);
+                          mmee_result_t* out_best, mmee_result_t* out_topk, cudaStream_t st);
 cudaError_t launch_reset(Scratch* scratch, cudaStream_t st);
 cudaError_t launch_eval(const Plan& p, uint64_t idx_begin, uint64_t count, mmee_result_t* out, cudaStream_t st);
 cudaError_t measure_alu_peak(double* giops);

@@ -21,8 +21,8 @@ constexpr uint32_t kStaticMaxCtas = 512;       // persistent CTAs the fixed scra
 constexpr int kMaxDevices = 64;
 constexpr size_t kStaticScratchBytes = sizeof(Scratch) + (size_t)(kStaticMaxCtas - 1) * sizeof(Partial);
 
-// 139 312 bytes on every device that loads the library.
-static_assert(kStaticScratchBytes == 139312, "documented size of the fixed scratch");
+// 139 328 bytes on every device that loads the library.
+static_assert(kStaticScratchBytes == 139328, "documented size of the fixed scratch");
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 std::mutex g_setup_mutex;
@@ -65,8 +65,7 @@ extern "C" int mmee_search_static(const mmee_workload_t* workload, const mmee_ar
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     // The array keeps whatever the previous call left in it.  The header (work counter, feasible
     // count, pruning bound) must start clean; the partial lists need no clearing, every CTA of
-    // this launch overwrites its own before the finalize kernel reads them.
+    // this launch overwrites its own before the finalize step reads them.
     if ((rc = cuda_status(launch_reset(scratch, st)))) return rc;
-    if ((rc = cuda_status(launch_search(plan, shape, device, scratch, nullptr, st)))) return rc;
-    return cuda_status(launch_finalize(plan, scratch, (int)shape.grid, out_best, out_topk, st));
+    return cuda_status(launch_search(plan, shape, device, scratch, nullptr, out_best, out_topk, st));
 }
