@@ -168,8 +168,9 @@ int mmee_search(mmee_handle_t* handle, void* cuda_stream, mmee_result_t* out_bes
 
 /*
  * mmee_search_host -- mmee_search on the default stream of the handle's device followed by the copy of
- * the records to HOST memory: the time to the optimal mapping of a planned search (the handle is warm;
- * nothing is allocated).  Synchronous.
+ * the records to HOST memory: the time to the optimal mapping of a planned search.  The first call on
+ * a handle allocates 1 + topk records of pinned host memory that the kernel writes its records into;
+ * later calls allocate nothing.  Synchronous.
  *   out_best : HOST, one record.   out_topk : HOST, objective.topk records, or NULL.
  * Returns MMEE_ERR_CHECK if the finalize step's self-check failed (the records are then not a result).
  */
@@ -249,6 +250,21 @@ int mmee_decode(mmee_handle_t* handle, uint64_t idx, mmee_result_t* host_out);
 int mmee_dump_keys(mmee_handle_t* handle, void* cuda_stream, int64_t* out_keys);
 
 /*
+ * mmee_filter_flags -- test view of the search kernel's filter.  The search decides with a cheap bound per group of
+ * five rows (45 mappings: one level of D, the five levels of E, nine stationary pairs) whether the group can hold a
+ * key below the current threshold, and forms exact keys only for flagged groups (32-bit threshold-relative sums for
+ * energy and latency, a single-precision product bound followed by double-precision products for the energy-delay
+ * product).  This call runs that filter over the handle's tiling range against the FIXED threshold `threshold_key`
+ * (a key as the search orders it; for the energy-delay product the bit pattern of the double), inserts nothing, and
+ * stores one byte per group: 1 = flagged.  A group that holds a mapping that fits, with an offered stationary pair and
+ * a key < threshold_key, must be flagged; the converse need not hold.
+ *   out_flags : DEVICE, (t_end - t_begin) * (R / 125) * 25 bytes; group g of middle level m of task w (a task is 125
+ *               consecutive rows of a tiling) at ((t - t_begin) * (R / 125) + w) * 25 + m * 5 + g.
+ * Energy, latency and energy-delay objectives without row pruning; MMEE_ERR_ARG otherwise.  Asynchronous.
+ */
+int mmee_filter_flags(mmee_handle_t* handle, void* cuda_stream, int64_t threshold_key, uint8_t* out_flags);
+
+/*
  * mmee_solve_host -- whole path with HOST buffers: plan, upload, search, copy the results back,
  * release.  Synchronous.  out_best: HOST, one record; out_topk: HOST, objective.topk records or
  * NULL.  h2d_bytes / d2h_bytes (HOST, may be NULL) receive the bytes copied in each direction.
@@ -271,6 +287,21 @@ int mmee_solve_host(const mmee_workload_t* workload, const mmee_arch_t* arch,
 int mmee_pareto_front(const mmee_workload_t* workload, const mmee_arch_t* arch,
                       const mmee_objective_t* objective, mmee_result_t* out_points, uint32_t capacity,
                       uint32_t* n_points);
+
+/*
+ * mmee_pareto_front_bs_da -- the buffer-size / DRAM-traffic trade-off of the whole mapping space (Section VI-A,
+ * Section VII-C): every pair (BS, DA) of a mapping with BS <= arch.gb_bytes / word_bytes that no other mapping
+ * improves in one of the two without losing in the other, by decreasing buffer size / increasing traffic, each
+ * with the lowest-index mapping of least traffic among those that need no more buffer.  Computed by device
+ * searches for the least DRAM traffic under a shrinking buffer (one search per distinct buffer need met on the
+ * way down).  The energies of arch and objective.objective, .topk, .row_pruning, .key_cap are ignored: the key
+ * of the returned records (e_key) is the DRAM word count n[0].  Synchronous.
+ *   out_points : HOST, `capacity` records; *n_points receives the number of points of the front, also when it
+ *                exceeds capacity (then MMEE_ERR_RANGE is returned and the first `capacity` points are valid).
+ */
+int mmee_pareto_front_bs_da(const mmee_workload_t* workload, const mmee_arch_t* arch,
+                            const mmee_objective_t* objective, mmee_result_t* out_points, uint32_t capacity,
+                            uint32_t* n_points);
 
 /*
  * mmee_search_shapes -- reconfigurable PE arrays (Section VII-K): the same search on each of several logical

@@ -20,7 +20,7 @@ NO_INDEX = 2 ** 64 - 1
 OK, ERR_ARG, ERR_OVERFLOW, ERR_QUANTUM, ERR_NO_FEASIBLE, ERR_CUDA, ERR_TIMEOUT, ERR_RANGE, ERR_CHECK = range(9)
 
 EXPORTS = ("mmee_create", "mmee_search", "mmee_search_host", "mmee_destroy", "mmee_search_static", "mmee_num_candidates", "mmee_num_tilings",
-           "mmee_num_rows", "mmee_strerror", "mmee_last_cuda_error", "mmee_eval", "mmee_decode", "mmee_dump_keys", "mmee_solve_host", "mmee_pareto_front", "mmee_search_shapes",
+           "mmee_num_rows", "mmee_strerror", "mmee_last_cuda_error", "mmee_eval", "mmee_decode", "mmee_dump_keys", "mmee_filter_flags", "mmee_solve_host", "mmee_pareto_front", "mmee_pareto_front_bs_da", "mmee_search_shapes",
            "mmee_query_vector", "mmee_recompute_flag", "mmee_row_pruning_keep", "mmee_last_search_stats", "mmee_kernel_timing",
            "mmee_alu_peak")
 
@@ -114,11 +114,13 @@ def library():
     L.mmee_eval.argtypes = [H, C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p]
     L.mmee_decode.argtypes = [H, C.c_uint64, C.POINTER(Result)]
     L.mmee_dump_keys.argtypes = [H, C.c_void_p, C.c_void_p]
+    L.mmee_filter_flags.argtypes = [H, C.c_void_p, C.c_int64, C.c_void_p]
     L.mmee_solve_host.argtypes = [C.POINTER(Workload), C.POINTER(Arch), C.POINTER(Objective),
                                   C.POINTER(Result), C.POINTER(Result),
                                   C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
     L.mmee_pareto_front.argtypes = [C.POINTER(Workload), C.POINTER(Arch), C.POINTER(Objective),
                                     C.POINTER(Result), C.c_uint32, C.POINTER(C.c_uint32)]
+    L.mmee_pareto_front_bs_da.argtypes = L.mmee_pareto_front.argtypes
     L.mmee_search_shapes.argtypes = [C.POINTER(Workload), C.POINTER(Arch), C.POINTER(Objective),
                                      C.POINTER(C.c_uint32), C.c_uint32, C.POINTER(Result), C.POINTER(C.c_uint32)]
     L.mmee_query_vector.argtypes = [C.c_uint32] * 6 + [C.POINTER(C.c_uint8)]
@@ -222,6 +224,12 @@ def mmee_dump_keys(handle, out_keys, stream=None) -> None:
            "mmee_dump_keys")
 
 
+def mmee_filter_flags(handle, threshold_key: int, out_flags, stream=None) -> None:
+    """out_flags: uint8 CUDA tensor with 25 entries per task of the handle's tiling range (1 = group flagged)."""
+    _check(library().mmee_filter_flags(handle, _stream_ptr(stream), threshold_key, C.c_void_p(out_flags.data_ptr())),
+           "mmee_filter_flags")
+
+
 def mmee_solve_host(workload: dict, arch: dict, objective: dict):
     """(best, topk list, h2d bytes, d2h bytes) with host buffers."""
     k = objective["topk"]
@@ -240,6 +248,16 @@ def mmee_pareto_front(workload: dict, arch: dict, objective: dict, capacity: int
     _check(library().mmee_pareto_front(_fill(Workload(), workload), _fill(Arch(), arch),
                                        _fill(Objective(), objective), pts, capacity, C.byref(n)),
            "mmee_pareto_front")
+    return list(pts[:n.value])
+
+
+def mmee_pareto_front_bs_da(workload: dict, arch: dict, objective: dict, capacity: int = 1024):
+    """Buffer-size / DRAM-traffic Pareto front of the whole mapping space: list of Result, by decreasing buffer size."""
+    pts = (Result * capacity)()
+    n = C.c_uint32()
+    _check(library().mmee_pareto_front_bs_da(_fill(Workload(), workload), _fill(Arch(), arch),
+                                             _fill(Objective(), objective), pts, capacity, C.byref(n)),
+           "mmee_pareto_front_bs_da")
     return list(pts[:n.value])
 
 

@@ -17,7 +17,8 @@ struct mmee_handle {
     mmee::LaunchShape shape;
     mmee::Scratch* scratch;      // device
     mmee_result_t* decode_buf;   // device, one record (mmee_decode); part of the scratch allocation
-    mmee_result_t* host_out;     // device, 1 + topk records (mmee_search_host); part of the scratch allocation
+    mmee_result_t* host_out;     // pinned host memory mapped into the device's address space, 1 + topk records:
+                                 // mmee_search_host lets the kernel write its records there (made at its first call)
     mmee::PrunedTask* pruned;    // device, row pruning only
     uint32_t kept_rows;          // rows of a tiling that survive pruning (all rows without it)
     int device;
@@ -128,12 +129,11 @@ int mmee_create(const mmee_workload_t* workload, const mmee_arch_t* arch, const 
         }
         h->shape.pruned = h->pruned;
     }
-    // one allocation: the search scratch, one result record for mmee_decode, 1 + topk records for mmee_search_host
+    // one allocation: the search scratch, then one result record for mmee_decode
     const size_t sbytes = (scratch_bytes(h->shape.grid) + 15) / 16 * 16;
-    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&h->scratch), sbytes + (2 + h->plan.topk) * sizeof(mmee_result_t));
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&h->scratch), sbytes + sizeof(mmee_result_t));
     if (e == cudaSuccess) {
         h->decode_buf = reinterpret_cast<mmee_result_t*>(reinterpret_cast<unsigned char*>(h->scratch) + sbytes);
-        h->host_out = h->decode_buf + 1;
         e = launch_reset(h->scratch, 0);
         if (e == cudaSuccess) e = cudaStreamSynchronize(0);
     }
@@ -183,13 +183,20 @@ int mmee_search(mmee_handle_t* h, void* cuda_stream, mmee_result_t* out_best, mm
 int mmee_search_host(mmee_handle_t* h, mmee_result_t* out_best, mmee_result_t* out_topk) {
     if (!h || !out_best) return MMEE_ERR_ARG;
     const uint32_t k = h->plan.topk;
-    int rc = mmee_search(h, nullptr, h->host_out, h->host_out + 1);
-    if (rc) return rc;
-    // (a copy to pageable host memory returns when the data is there: no further synchronisation needed)
-    if ((rc = cuda_status(cudaMemcpy(out_best, h->host_out, sizeof(mmee_result_t), cudaMemcpyDeviceToHost)))) return rc;
-    if (out_topk &&
-        (rc = cuda_status(cudaMemcpy(out_topk, h->host_out + 1, (size_t)k * sizeof(mmee_result_t), cudaMemcpyDeviceToHost))))
-        return rc;
+    int rc;
+    if (!h->host_out) {
+        // Pinned, mapped host memory: the kernel's last CTA writes the records straight into it, so that the
+        // host needs no copy call after the search, only the synchronisation.
+        rc = cuda_status(cudaHostAlloc(reinterpret_cast<void**>(&h->host_out), (size_t)(1 + k) * sizeof(mmee_result_t),
+                                       cudaHostAllocMapped));
+        if (rc) { h->host_out = nullptr; return rc; }
+    }
+    mmee_result_t* dev = nullptr;
+    if ((rc = cuda_status(cudaHostGetDevicePointer(reinterpret_cast<void**>(&dev), h->host_out, 0)))) return rc;
+    if ((rc = mmee_search(h, nullptr, dev, dev + 1))) return rc;
+    if ((rc = cuda_status(cudaStreamSynchronize(nullptr)))) return rc;
+    std::memcpy(out_best, h->host_out, sizeof(mmee_result_t));
+    if (out_topk) std::memcpy(out_topk, h->host_out + 1, (size_t)k * sizeof(mmee_result_t));
     return out_best->status == MMEE_ERR_CHECK ? MMEE_ERR_CHECK : MMEE_OK;
 }
 
@@ -199,6 +206,7 @@ int mmee_destroy(mmee_handle_t* h) {
     if (h->timing) for (int i = 0; i < 2; ++i) cudaEventDestroy(h->ev[i]);
     if (h->scratch) e = cudaFree(h->scratch);
     if (h->pruned) cudaFree(h->pruned);
+    if (h->host_out) cudaFreeHost(h->host_out);
     delete h;
     return cuda_status(e);
 }
@@ -253,6 +261,25 @@ int mmee_dump_keys(mmee_handle_t* h, void* cuda_stream, int64_t* out_keys) {
         h->dirty = false;
     }
     cudaError_t e = launch_search(h->plan, h->shape, h->device, h->scratch, out_keys, nullptr, nullptr, st);
+    if (e != cudaSuccess) { h->dirty = true; return cuda_status(e); }
+    if ((e = launch_reset(h->scratch, st)) != cudaSuccess) { h->dirty = true; return cuda_status(e); }
+    return MMEE_OK;
+}
+
+int mmee_filter_flags(mmee_handle_t* h, void* cuda_stream, int64_t threshold_key, uint8_t* out_flags) {
+    if (!h || !out_flags || h->plan.row_pruning || h->plan.objective > MMEE_OBJ_EDP) return MMEE_ERR_ARG;
+    int rc = check_device(h);
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (h->dirty) {
+        if ((rc = cuda_status(launch_reset(h->scratch, st)))) return rc;
+        h->dirty = false;
+    }
+    const uint64_t bytes = (h->plan.t_end - h->plan.t_begin) * (uint64_t)h->plan.tasks_per_tiling * 25u;
+    if ((rc = cuda_status(cudaMemsetAsync(out_flags, 0, bytes, st)))) return rc;
+    Plan p = h->plan;
+    p.key_cap = threshold_key;
+    cudaError_t e = launch_filter_flags(p, h->shape, h->device, h->scratch, out_flags, st);
     if (e != cudaSuccess) { h->dirty = true; return cuda_status(e); }
     if ((e = launch_reset(h->scratch, st)) != cudaSuccess) { h->dirty = true; return cuda_status(e); }
     return MMEE_OK;
@@ -319,6 +346,48 @@ int mmee_pareto_front(const mmee_workload_t* workload, const mmee_arch_t* arch, 
     if (dev) cudaFree(dev);
     mmee_destroy(he);
     mmee_destroy(hl);
+    *n_points = n;
+    if (rc == MMEE_OK && n > capacity) rc = MMEE_ERR_RANGE;
+    return rc;
+}
+
+int mmee_pareto_front_bs_da(const mmee_workload_t* workload, const mmee_arch_t* arch, const mmee_objective_t* objective,
+                            mmee_result_t* out_points, uint32_t capacity, uint32_t* n_points) {
+    if (!arch || !objective || !n_points || (!out_points && capacity)) return MMEE_ERR_ARG;
+    *n_points = 0;
+    // DRAM words as the key: one quantum per DRAM word, nothing else costs anything
+    mmee_arch_t a = *arch;
+    a.e_dram_pj = 1.0; a.e_gb_pj = a.e_rf_pj = a.e_mac_pj = 0.0; a.c_softmax = 0.0; a.energy_quantum_pj = 1.0;
+    mmee_objective_t o = *objective;
+    o.objective = MMEE_OBJ_ENERGY; o.topk = 1; o.row_pruning = 0; o.key_cap = 0;
+    mmee_handle_t* h = nullptr;
+    int rc = mmee_create(workload, &a, &o, &h);
+    if (rc) return rc;
+    mmee_result_t* dev = nullptr;
+    rc = cuda_status(cudaMalloc(reinterpret_cast<void**>(&dev), sizeof(mmee_result_t)));
+    mmee_result_t r, held;
+    bool have = false;
+    uint32_t n = 0;
+    // Searches with a shrinking buffer: each returns the least DRAM traffic that fits, with the buffer words its
+    // mapping needs; the next one allows one word less than that.  While the traffic stays the same the mapping
+    // found needs less buffer for the same traffic; when it rises, the mapping held is a point of the front.
+    while (rc == MMEE_OK) {
+        if ((rc = mmee_search(h, nullptr, dev, nullptr))) break;
+        if ((rc = cuda_status(cudaMemcpy(&r, dev, sizeof(r), cudaMemcpyDeviceToHost)))) break;
+        if (r.status == MMEE_ERR_CHECK) { rc = MMEE_ERR_CHECK; break; }
+        const bool found = r.idx != MMEE_NO_INDEX;
+        if (have && (!found || r.e_key != held.e_key)) {
+            if (n < capacity) out_points[n] = held;
+            ++n;
+        }
+        if (!found) break;
+        held = r;
+        have = true;
+        if (r.bs <= 0) { if (n < capacity) out_points[n] = held; ++n; break; }      // (cannot happen: tiles take words)
+        h->plan.cap_words = r.bs - 1;
+    }
+    if (dev) cudaFree(dev);
+    mmee_destroy(h);
     *n_points = n;
     if (rc == MMEE_OK && n > capacity) rc = MMEE_ERR_RANGE;
     return rc;

@@ -33,7 +33,7 @@ namespace mmee {
 namespace {
 
 constexpr unsigned kFull = 0xffffffffu;
-constexpr int kModeSearch = 0, kModeDump = 1, kModePrune = 2;
+constexpr int kModeSearch = 0, kModeDump = 1, kModePrune = 2, kModeFlags = 3;
 constexpr size_t kPlanBytes = (sizeof(Plan) + 15) / 16 * 16;
 static_assert(sizeof(Plan) % 4 == 0, "the plan is copied word by word");
 constexpr int kTermCap = (1 << 28) - 1;    // cap of each non-negative addend of such a sum (at most six of them)
@@ -734,15 +734,16 @@ __device__ __noinline__ unsigned edp_group_test(const MidExact& me, const RowTab
 
 // The walk in 64-bit keys: the energy-delay product (double-precision filter, see edp_row_test),
 // the capped objectives and the key dump.  Returns the number of rows that fit.
-template <int OBJ, bool DUMP, bool PRUNE>
+template <int OBJ, bool DUMP, bool PRUNE, bool FLAGS>
 __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingTab* tb, const OrderTab* ot,
                                                     const TaskChoice& c, bool live, bool valid, uint32_t kept,
                                                     uint32_t kept_mid, uint64_t task_first_idx, WarpTop* wt,
                                                     CtaShared* cs, long long* global_g, int k, int lane,
                                                     int64_t* __restrict__ dump, uint64_t dump_origin, uint32_t& visits,
-                                                    uint32_t& tested) {
+                                                    uint32_t& tested, unsigned char* flags) {
     const RowTab* rt = &ot->rt[c.phi == 0 ? 0 : 1];
     LaneThreshold th = load_threshold(wt, cs, k);
+    if constexpr (FLAGS) { th.T1 = p.key_cap; th.ti = UINT64_MAX; th.delta = 0; }
     uint32_t rows = 0;
     int E1c[5], E2c[5];
     float Egf[5], Eef[5];       // EDP: lower bounds of E's DRAM words and of their energy
@@ -849,7 +850,9 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
                 }
             }
             rows += fits;
-            if (__any_sync(kFull, hit_any != 0u)) {
+            if constexpr (FLAGS) {
+                if (hit_any && flags) flags[m * 5 + d] = 1;
+            } else if (__any_sync(kFull, hit_any != 0u)) {
                 ++visits;
                 if (k == 1) exact_group_single<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, lane);
                 else exact_group<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, k, lane);
@@ -866,12 +869,14 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
 // objectives.  Everything a middle level, a group or a row needs is a 32-bit table entry or a
 // register; 64-bit arithmetic is left to the places where the threshold enters (once per task and
 // after each visit of the exact path).  Returns the number of rows that fit.
-template <int OBJ, bool PRUNE>
+// FLAGS (a test mode): the threshold is the fixed key p.key_cap, nothing is inserted, and flags[mid * 5 + group]
+// is set for every group the filter would send to the exact path.
+template <int OBJ, bool PRUNE, bool FLAGS>
 __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const TilingTab* tb, const OrderTab* ot,
                                                        const TaskChoice& c, bool live, uint32_t kept, uint32_t kept_mid,
                                                        uint64_t task_first_idx, WarpTop* wt, CtaShared* cs,
                                                        long long* global_g, int k, int lane, uint32_t& visits,
-                                                       uint32_t& tested) {
+                                                       uint32_t& tested, unsigned char* flags) {
     const bool fused = c.phi == 0;
     const RowTab* rt = &ot->rt[fused ? 0 : 1];
     // Row-side terms of E.  Its buffer need while Op1 runs is its size when retained (level >= L4 of a
@@ -903,8 +908,12 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
     int base[2] = {0, 0}, ua2[2] = {0, 0}, qo2[2] = {0, 0};
     int64_t thr = 0;
     auto rebase = [&](int next_pos) {
-        const LaneThreshold th = load_threshold(wt, cs, k);
-        thr = th.T1 - ((task_first_idx + (uint64_t)next_pos > th.ti) ? th.delta : 0);
+        if constexpr (FLAGS) {
+            thr = p.key_cap;
+        } else {
+            const LaneThreshold th = load_threshold(wt, cs, k);
+            thr = th.T1 - ((task_first_idx + (uint64_t)next_pos > th.ti) ? th.delta : 0);
+        }
         if constexpr (OBJ == MMEE_OBJ_ENERGY) {
 #pragma unroll
             for (int rc = 0; rc < 2; ++rc) {
@@ -1025,7 +1034,9 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
             }
             // least key of the group's 45 mappings, relative to the threshold
             const bool hit = uc + __vimin3_s32(__vimin3_s32(g[0], g[1], g[2]), g[3], g[4]) < 0;
-            if (__any_sync(kFull, hit)) {
+            if constexpr (FLAGS) {
+                if (hit && flags) flags[m * 5 + d] = 1;
+            } else if (__any_sync(kFull, hit)) {
                 ++visits;
                 if (k == 1) exact_group_single<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, lane);
                 else exact_group<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, k, lane);
@@ -1155,6 +1166,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
               int64_t* __restrict__ dump, mmee_result_t* __restrict__ out_best, mmee_result_t* __restrict__ out_topk) {
     constexpr bool DUMP = MODE == kModeDump;        // store every key instead of reducing
     constexpr bool PRUNE = MODE == kModePrune;      // visit only the rows kept by symbolic pruning
+    constexpr bool FLAGS = MODE == kModeFlags;      // test mode: record which groups the filter flags (in `dump`)
     extern __shared__ __align__(16) unsigned char smem_raw[];
     // The plan is copied to shared memory: lanes index its tables (query vectors, divisor lists,
     // block lists) with different indices, which the constant bank would serialise.
@@ -1346,12 +1358,15 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
             // The other CTAs' pruning bound: the load is issued here and consumed at the end of the
             // task, so that its latency is covered by the task's own work.
             const long long g_seen = (lane == 0) ? *reinterpret_cast<volatile long long*>(&scratch->G) : 0;
+            // (flags mode: 25 bytes per task, relative to the first task of the searched range)
+            unsigned char* flags = (FLAGS && live) ? reinterpret_cast<unsigned char*>(dump) + (tq - task_begin) * 25u : nullptr;
             if constexpr (!DUMP && OBJ <= MMEE_OBJ_LATENCY) {
-                my_rows += walk_task_relative<OBJ, PRUNE>(p, tb, ot, c, live, kept, kept_mid, task_first_idx, wt, cs,
-                                                          &scratch->G, k, lane, my_visits, my_tested);
+                my_rows += walk_task_relative<OBJ, PRUNE, FLAGS>(p, tb, ot, c, live, kept, kept_mid, task_first_idx, wt, cs,
+                                                                 &scratch->G, k, lane, my_visits, my_tested, flags);
             } else {
-                my_rows += walk_task_exact<OBJ, DUMP, PRUNE>(p, tb, ot, c, live, valid, kept, kept_mid, task_first_idx, wt,
-                                                             cs, &scratch->G, k, lane, dump, dump_origin, my_visits, my_tested);
+                my_rows += walk_task_exact<OBJ, DUMP, PRUNE, FLAGS>(p, tb, ot, c, live, valid, kept, kept_mid, task_first_idx,
+                                                                    wt, cs, &scratch->G, k, lane, dump, dump_origin, my_visits,
+                                                                    my_tested, flags);
             }
             if (lane == 0 && g_seen < cs->G) atomicMin(&cs->G, g_seen);
         }
@@ -1399,7 +1414,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
             if (cs->exact_visits) atomicAdd(&scratch->exact_visits, cs->exact_visits);
             if (cs->tested_rows) atomicAdd(&scratch->tested_rows, cs->tested_rows);
         }
-        if constexpr (!DUMP) {
+        if constexpr (!DUMP && !FLAGS) {
             // Grid reduction without a wait: every CTA makes its partial list visible, then draws a ticket; the
             // CTA that draws the last one knows that all lists are there and runs the finalize step.
             __threadfence();
@@ -1407,7 +1422,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
             if (lane == 0) cs->last_cta = atomicAdd(&scratch->done_ctas, 1u) == gridDim.x - 1 ? 1u : 0u;
         }
     }
-    if constexpr (!DUMP) {
+    if constexpr (!DUMP && !FLAGS) {
         __syncthreads();
         if (cs->last_cta) {
             __threadfence();
@@ -1484,6 +1499,17 @@ cudaError_t search_occupancy(const Plan& p, int device, size_t smem, int* blocks
         case MMEE_OBJ_EDP: return occupancy_t<MMEE_OBJ_EDP, kModeSearch>(device, blocks_per_sm, smem);
         case MMEE_OBJ_ENERGY_LCAP: return occupancy_t<MMEE_OBJ_ENERGY_LCAP, kModeSearch>(device, blocks_per_sm, smem);
         default: return occupancy_t<MMEE_OBJ_LATENCY_ECAP, kModeSearch>(device, blocks_per_sm, smem);
+    }
+}
+
+cudaError_t launch_filter_flags(const Plan& p, const LaunchShape& shape, int device, Scratch* scratch, unsigned char* flags,
+                                cudaStream_t st) {
+    int64_t* out = reinterpret_cast<int64_t*>(flags);
+    switch (p.objective) {
+        case MMEE_OBJ_ENERGY: return launch_search_t<MMEE_OBJ_ENERGY, kModeFlags>(p, shape, device, scratch, out, nullptr, nullptr, st);
+        case MMEE_OBJ_LATENCY: return launch_search_t<MMEE_OBJ_LATENCY, kModeFlags>(p, shape, device, scratch, out, nullptr, nullptr, st);
+        case MMEE_OBJ_EDP: return launch_search_t<MMEE_OBJ_EDP, kModeFlags>(p, shape, device, scratch, out, nullptr, nullptr, st);
+        default: return cudaErrorInvalidValue;
     }
 }
 

@@ -56,6 +56,11 @@ cudaError_t search_occupancy(const Plan& p, int device, size_t smem, int* blocks
 // key instead and writes no result (the caller resets the header).
 cudaError_t launch_search(const Plan& p, const LaunchShape& shape, int device, Scratch* scratch, int64_t* dump,
                           mmee_result_t* out_best, mmee_result_t* out_topk, cudaStream_t st);
+// Test mode: the search kernel's filter alone against the fixed threshold p.key_cap; flags[(task - first task) * 25
+// + middle level * 5 + group] is set to 1 for every flagged group (the caller clears the buffer first and resets
+// the scratch header afterwards).  Energy, latency and energy-delay objectives.
+cudaError_t launch_filter_flags(const Plan& p, const LaunchShape& shape, int device, Scratch* scratch, unsigned char* flags,
+                                cudaStream_t st);
 cudaError_t launch_reset(Scratch* scratch, cudaStream_t st);
 cudaError_t launch_eval(const Plan& p, uint64_t idx_begin, uint64_t count, mmee_result_t* out, cudaStream_t st);
 cudaError_t measure_alu_peak(double* giops);

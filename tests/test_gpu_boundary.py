@@ -98,3 +98,135 @@ def test_a_handle_is_refused_on_another_device():
     finally:
         with torch.cuda.device(0):
             mm.mmee_destroy(h)
+
+
+def _bs_da_of_every_candidate(cfg, obj, limit):
+    """(buffer words, DRAM words, idx) of every candidate of the range-limited problem, from the oracle's records."""
+    p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
+    if p.N > limit:
+        obj = dict(obj, t_begin=0, t_end=max(1, limit // (p.R * 9)))
+        p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
+    begin, count = p.t_begin * p.R * 9, (p.t_end - p.t_begin) * p.R * 9
+    recs = oracle.evaluate_range(p, begin, count)
+    raw = np.frombuffer(recs, dtype=np.uint8).reshape(count, C.sizeof(oracle.Record))
+    field = lambda off: raw[:, off:off + 8].copy().view(np.int64).ravel()
+    bs = field(oracle.Record.bs.offset)
+    da = field(oracle.Record.n.offset)
+    return obj, p, bs, da, np.arange(begin, begin + count, dtype=np.int64)
+
+
+@pytest.mark.parametrize("seed", [2, 3, 6, 8, 11])
+def test_buffer_size_dram_traffic_pareto_front(seed):
+    """The buffer-size / DRAM-traffic front (Section VI-A, Section VII-C) by device searches under a shrinking buffer,
+    against a brute-force front over the oracle's (BS, N_DRAM) pair of every candidate: by increasing traffic,
+    each point the least buffer that reaches that traffic, with the lowest index that attains the pair."""
+    cfg = mi.random_tiny_problem(seed)
+    obj, p, bs, da, idx = _bs_da_of_every_candidate(cfg, dict(cfg["searches"][0], objective=mi.OBJ_ENERGY, topk=1), 250_000)
+    fits = bs <= p.cap_words
+    want, best_bs = [], None
+    for d in np.unique(da[fits]):
+        sel = fits & (da == d)
+        b = int(bs[sel].min())
+        if best_bs is None or b < best_bs:
+            want.append((b, int(d), int(idx[sel & (bs == b)].min())))
+            best_bs = b
+    got = mm.mmee_pareto_front_bs_da(cfg["workload"], cfg["arch"], obj)
+    assert [(r.bs, r.n[0], r.idx) for r in got] == want
+    assert len(want) >= 2
+    for r in got:
+        assert r.e_key == r.n[0]                # the search's key was the DRAM word count
+
+
+def test_buffer_size_dram_traffic_front_of_the_ffn_task():
+    """On the fused feed-forward GEMMs of the paper's buffer-size study the front is a staircase: strictly less
+    buffer and strictly more traffic from point to point, no point above the buffer, the last one at the
+    smallest buffer any mapping needs; a plain search at a point's buffer size finds that point's traffic."""
+    cfg = [c for c in mi.ffn_dram_sweep_configs() if c["name"] == "ffn_gpt3_dram_1024KB"][0]
+    obj = dict(cfg["searches"][0], t_begin=0, t_end=4000)
+    got = mm.mmee_pareto_front_bs_da(cfg["workload"], cfg["arch"], obj)
+    cap = cfg["arch"]["gb_bytes"] // cfg["workload"]["word_bytes"]
+    assert len(got) >= 3 and got[0].bs <= cap
+    for a, b in zip(got, got[1:]):
+        assert b.bs < a.bs and b.n[0] > a.n[0]
+    mid = got[len(got) // 2]
+    arch = dict(cfg["arch"], gb_bytes=mid.bs * cfg["workload"]["word_bytes"])
+    best = mm.mmee_solve_host(cfg["workload"], arch, obj)[0]
+    assert (best.n[0], best.bs, best.idx) == (mid.n[0], mid.bs, mid.idx)
+    below = dict(cfg["arch"], gb_bytes=(got[-1].bs - 1) * cfg["workload"]["word_bytes"])
+    assert mm.mmee_solve_host(cfg["workload"], below, obj)[0].idx == mm.NO_INDEX
+
+
+def _group_minima(cfg, obj):
+    """Least key of the feasible mappings of every group of 45 consecutive candidates (INT64_MAX: none), from the
+    oracle's keys."""
+    p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
+    begin, count = p.t_begin * p.R * 9, (p.t_end - p.t_begin) * p.R * 9
+    keys, feas = oracle.keys_range(p, begin, count)
+    masked = np.where(feas.astype(bool), keys, np.iinfo(np.int64).max)
+    return masked.reshape(-1, 45).min(axis=1), keys[feas.astype(bool)]
+
+
+def _filter_flags(cfg, obj, thr, n_groups):
+    flags = torch.empty(n_groups, dtype=torch.uint8, device="cuda")
+    with Handle(cfg, obj) as h:
+        mm.mmee_filter_flags(h, int(thr), flags)
+        torch.cuda.synchronize()
+    return flags.cpu().numpy().astype(bool)
+
+
+@pytest.mark.parametrize("objective", [mi.OBJ_ENERGY, mi.OBJ_LATENCY, mi.OBJ_EDP])
+@pytest.mark.parametrize("seed", [1, 2, 5, 7, 10, 12])
+def test_the_filter_flags_every_group_that_holds_a_passing_mapping(seed, objective):
+    """The search kernel's filter against fixed thresholds (the 1st, 50th and 99th percentile of the oracle's feasible
+    keys, just above the optimum, the optimum itself and the largest key): every group of five rows that holds a
+    feasible mapping with a key below the threshold is flagged.  In these small problems the energy and latency
+    filters work in units of one quantum / one word, where they are exact: nothing else is flagged either; the
+    energy-delay filter also flags groups whose least key equals the threshold or lies within its rounding margin."""
+    cfg = mi.random_tiny_problem(seed)
+    obj = shrink_to(cfg, dict(cfg["searches"][0], objective=objective, topk=1), 1_200_000)
+    gmin, fkeys = _group_minima(cfg, obj)
+    if fkeys.size == 0:
+        pytest.skip("nothing fits")
+    ranked = np.sort(fkeys)
+    thresholds = [ranked[(ranked.size - 1) * q // 100] for q in (1, 50, 99)] + [ranked[0] + 1, ranked[0], ranked[-1] + 1]
+    for thr in thresholds:
+        flags = _filter_flags(cfg, obj, thr, gmin.size)
+        must = gmin < int(thr)
+        assert not (must & ~flags).any(), "a group with a passing mapping was not flagged (threshold %d)" % thr
+        extra = flags & ~must
+        if objective == mi.OBJ_EDP:
+            # (keys are bit patterns of positive doubles; the filter compares products rounded in floating point
+            # with "<=" against the threshold widened by 1e-14: a group is flagged beyond need only if its least key
+            # is within that margin of the threshold)
+            as_double = lambda a: np.asarray(a, dtype=np.int64).view(np.float64)
+            assert (as_double(gmin[extra]) <= as_double([int(thr)])[0] * (1.0 + 1e-13)).all()
+        else:
+            assert not extra.any()
+
+
+@pytest.mark.parametrize("log2_quantum", [-12, -24])
+@pytest.mark.parametrize("seed", [3, 4, 8])
+def test_the_filter_in_coarse_units_never_misses(seed, log2_quantum):
+    """The same with a tiny energy quantum: keys are then large, the 32-bit filter works in units of many quanta with
+    every term rounded down (and the largest ones capped), so it may flag more groups than pass, never fewer."""
+    cfg = mi.random_tiny_problem(seed)
+    arch = dict(cfg["arch"], energy_quantum_pj=cfg["arch"]["energy_quantum_pj"] * 2.0 ** log2_quantum)
+    cfg = dict(cfg, arch=arch)
+    obj = shrink_to(cfg, dict(cfg["searches"][0], objective=mi.OBJ_ENERGY, topk=1), 1_200_000)
+    gmin, fkeys = _group_minima(cfg, obj)
+    if fkeys.size == 0:
+        pytest.skip("nothing fits")
+    ranked = np.sort(fkeys)
+    for q in (1, 50, 99):
+        thr = ranked[(ranked.size - 1) * q // 100]
+        flags = _filter_flags(cfg, obj, thr, gmin.size)
+        must = gmin < int(thr)
+        assert not (must & ~flags).any()
+        assert (flags & ~must).sum() <= max(16, gmin.size // 4)
+
+
+def shrink_to(cfg, obj, limit):
+    p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
+    if p.N <= limit:
+        return dict(obj)
+    return dict(obj, t_begin=0, t_end=max(1, limit // (p.R * 9)))
