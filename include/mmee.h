@@ -110,7 +110,21 @@ typedef struct {
                                                 (Section VII-K: a fixed array offers one, a reconfigurable
                                                 one several); 0 = all nine.  A mapping with another pair
                                                 is outside the space: never selected, not in n_feasible */
-    uint32_t reserved;                       /* 0 */
+    uint32_t rf_tiling;                      /* 1: a third tiling level below the buffer tile, in the PEs' register files
+                                                (the register-file level of the accelerator template, Section II-B).
+                                                The stationary operand of each operator's tile is processed in blocks
+                                                of a x b elements (divisors of its two extents; weight stationary:
+                                                reduction x output columns, input stationary: output rows x reduction,
+                                                output stationary: output rows x columns).  A block lives in the register
+                                                files, element (x, y) in PE (x mod pe_rows, y mod pe_cols), beside one
+                                                register each for the streamed operand and the partial sum: it is
+                                                admissible iff ceil(a/pe_rows)*ceil(b/pe_cols) + 2 <= rf_bytes/word_bytes.
+                                                The streamed vectors pass once per block, one cycle per element a PE
+                                                holds.  Each mapping takes, per operator, the admissible block with the
+                                                fewest buffer<->array words (energy objective; then the fewest cycles) or
+                                                the fewest cycles (latency objective; then the fewest words), the first
+                                                such block in ascending (a, b) order.  Energy and latency objectives on
+                                                an architecture with a register file only; 0: one array fold per pass. */
 } mmee_objective_t;
 
 /* One fully evaluated mapping.  Counts are per instance. */
@@ -134,6 +148,9 @@ typedef struct {
     double   latency_cycles;                 /* l_key / words_per_cycle * ceil(instances/n_arrays) */
     uint64_t n_total;                        /* candidates of the searched range (in out_best)    */
     uint64_t n_feasible;                     /* of which fit the buffer, with an offered stationary pair (in out_best) */
+    uint32_t rf_block[6];                    /* objective.rf_tiling: register-file block (m, r, n) of the first operator's
+                                                tile, then of the second's (1 for the streamed extent); else 0        */
+    uint32_t reserved2[2];
 } mmee_result_t;
 
 typedef struct mmee_handle mmee_handle_t;

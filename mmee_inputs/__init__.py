@@ -34,10 +34,10 @@ def arch(pe_rows, pe_cols, n_arrays, gb_bytes, rf_bytes, dram_words_per_cycle,
 
 
 def objective(objective=OBJ_ENERGY, topk=1, tiling_set=TILE_ALL_DIVISORS, order_set=ORD_ALL6,
-              fuse_mask=FUSE_ALL, t_begin=0, t_end=0, row_pruning=0, key_cap=0, stationary_mask=0):
+              fuse_mask=FUSE_ALL, t_begin=0, t_end=0, row_pruning=0, key_cap=0, stationary_mask=0, rf_tiling=0):
     return dict(objective=objective, topk=topk, tiling_set=tiling_set, order_set=order_set,
                 fuse_mask=fuse_mask, row_pruning=row_pruning, t_begin=t_begin, t_end=t_end, key_cap=key_cap,
-                stationary_mask=stationary_mask)
+                stationary_mask=stationary_mask, rf_tiling=rf_tiling)
 
 
 # --- accelerators -----------------------------------------------------------------------------

@@ -41,7 +41,7 @@ class Arch(C.Structure):
 class Objective(C.Structure):
     _fields_ = [("objective", C.c_uint32), ("topk", C.c_uint32), ("tiling_set", C.c_uint32),
                 ("order_set", C.c_uint32), ("fuse_mask", C.c_uint32), ("stationary_mask", C.c_uint32),
-                ("t_begin", C.c_uint64), ("t_end", C.c_uint64)]
+                ("t_begin", C.c_uint64), ("t_end", C.c_uint64), ("rf_tiling", C.c_uint32), ("pad", C.c_uint32)]
 
 
 class Problem(C.Structure):
@@ -55,7 +55,7 @@ class Problem(C.Structure):
                 ("has_rf", C.c_int), ("cap_words", C.c_uint64),
                 ("pe_rows", C.c_uint32), ("pe_cols", C.c_uint32), ("n_arrays", C.c_uint32),
                 ("bw", C.c_uint32), ("objective", C.c_uint32), ("topk", C.c_uint32),
-                ("stationary_mask", C.c_uint32)]
+                ("stationary_mask", C.c_uint32), ("rf_tiling", C.c_uint32), ("rf_words", C.c_uint64)]
 
 
 class Record(C.Structure):
@@ -68,7 +68,8 @@ class Record(C.Structure):
                 ("da1", C.c_int64), ("da2", C.c_int64),
                 ("br", C.c_int64), ("cyc1", C.c_int64), ("cyc2", C.c_int64),
                 ("n", C.c_int64 * 5), ("e_key", C.c_int64), ("l_key", C.c_int64),
-                ("edp_key", C.c_double), ("energy_pj", C.c_double), ("latency_cycles", C.c_double)]
+                ("edp_key", C.c_double), ("energy_pj", C.c_double), ("latency_cycles", C.c_double),
+                ("rf_block", C.c_uint32 * 6)]
 
 
 class SimOut(C.Structure):
@@ -119,8 +120,10 @@ class OracleError(RuntimeError):
 
 
 def _fill(struct, values: dict):
+    names = {f[0] for f in struct._fields_}
     for k, v in values.items():
-        setattr(struct, k, v)
+        if k in names:            # (the three input dicts also serve the CUDA binding, whose structs have more fields)
+            setattr(struct, k, v)
     return struct
 
 
@@ -256,6 +259,31 @@ def array_chain(bound, productions: int, sm1: int, sm2: int, rows: int, cols: in
     if rc:
         raise OracleError(rc)
     return out[0], out[1]
+
+
+def array_tile_blocked(sm: int, m: int, r: int, n: int, rows: int, cols: int, a: int, b: int,
+                       resume: bool = False) -> ArrayCounts:
+    """Element-level execution of one tile whose stationary operand is processed in register-file blocks of a x b."""
+    out = ArrayCounts()
+    L = lib()
+    L.mo_array_tile_blocked.argtypes = [C.c_uint32] * 8 + [C.c_int, C.POINTER(ArrayCounts)]
+    rc = L.mo_array_tile_blocked(sm, m, r, n, rows, cols, a, b, int(resume), out)
+    if rc:
+        raise OracleError(rc)
+    return out
+
+
+def rf_block(objective: int, sm: int, m: int, r: int, n: int, rows: int, cols: int, rf_words: int):
+    """The register-file block the model picks for one tile: ((m, r, n) block, words, cycles)."""
+    blk = (C.c_uint32 * 3)()
+    w, c = C.c_int64(), C.c_int64()
+    L = lib()
+    L.mo_rf_block.argtypes = [C.c_uint32] * 7 + [C.c_uint64, C.POINTER(C.c_uint32), C.POINTER(C.c_int64),
+                                                 C.POINTER(C.c_int64)]
+    rc = L.mo_rf_block(objective, sm, m, r, n, rows, cols, rf_words, blk, C.byref(w), C.byref(c))
+    if rc:
+        raise OracleError(rc)
+    return tuple(blk), w.value, c.value
 
 
 def threads_used() -> int:

@@ -70,6 +70,8 @@ int mo_problem_init(const mo_workload* w, const mo_arch* a, const mo_objective* 
     if (o->tiling_set > MO_TILE_ALL_DIVISORS || o->order_set > MO_ORD_ALL6) return MO_ERR_ARG;
     if ((o->fuse_mask & 7u) == 0 || (o->fuse_mask & ~7u)) return MO_ERR_ARG;
     if (o->stationary_mask & ~0x1ffu) return MO_ERR_ARG;
+    if (o->rf_tiling > 1 || o->pad) return MO_ERR_ARG;
+    if (o->rf_tiling && (o->objective > MO_OBJ_LATENCY || !a->rf_bytes)) return MO_ERR_ARG;
 
     /* Heads are independent instances (Section V, "we omit the head dimension"); the g query
      * heads that share one K/V head are stacked along I, so K and V are loaded once per group. */
@@ -126,6 +128,8 @@ int mo_problem_init(const mo_workload* w, const mo_arch* a, const mo_objective* 
     p->bw = a->dram_words_per_cycle;
     p->objective = o->objective; p->topk = o->topk;
     p->stationary_mask = o->stationary_mask ? o->stationary_mask : 0x1ffu;
+    p->rf_tiling = o->rf_tiling;
+    p->rf_words = a->rf_bytes / w->word_bytes;
 
     /* Worst-case key bound.  With M = I*L*J*(K+1) >= the largest MAC count (recomputation factor
      * at most J): every DRAM term is at most I*K*L*J <= M and there are at most 7 of them; array
@@ -194,6 +198,61 @@ static i128 tile_buffer_traffic(int sm, uint64_t m, uint64_t r, uint64_t n, uint
     default:      /* outputs stay in the array; both inputs re-streamed per fold */
         return (i128)m * r * ceil_div(n, cols) + (i128)r * n * ceil_div(m, rows) + (i128)m * n;
     }
+}
+
+/* Register-file-level tiling: a tile whose stationary operand is processed in blocks of a x b elements.
+ * The block is pinned once (a*b words); every streamed vector passes once per block; partial sums leave the
+ * array after every block of the reduction dimension and are read back by the next one. */
+static void blocked_tile_terms(int sm, uint64_t m, uint64_t r, uint64_t n, uint64_t rows, uint64_t cols,
+                               uint64_t a, uint64_t b, i128* words, i128* cycles)
+{
+    i128 held = (i128)ceil_div(a, rows) * ceil_div(b, cols);      /* stationary elements per PE */
+    switch (sm) {
+    case SM_WS:   /* block = a reduction indices x b output columns; the m input rows stream */
+        *words = (i128)r * n + (i128)m * r * (n / b) + (i128)m * n * (2 * (r / a) - 1);
+        *cycles = (i128)(r / a) * (n / b) * m * held;
+        break;
+    case SM_IS:   /* block = a output rows x b reduction indices; the n weight columns stream */
+        *words = (i128)m * r + (i128)r * n * (m / a) + (i128)m * n * (2 * (r / b) - 1);
+        *cycles = (i128)(m / a) * (r / b) * n * held;
+        break;
+    default:      /* block = a output rows x b output columns; the r reduction steps stream */
+        *words = (i128)m * r * (n / b) + (i128)r * n * (m / a) + (i128)m * n;
+        *cycles = (i128)(m / a) * (n / b) * r * held;
+        break;
+    }
+}
+
+int mo_rf_block(uint32_t objective, uint32_t sm, uint32_t m, uint32_t r, uint32_t n, uint32_t rows, uint32_t cols,
+                uint64_t rf_words, uint32_t block_mrn[3], int64_t* words, int64_t* cycles)
+{
+    if (sm > 2 || !m || !r || !n || !rows || !cols || !block_mrn || !words || !cycles) return MO_ERR_ARG;
+    uint64_t ea = sm == SM_WS ? r : m;                   /* extents of the stationary operand */
+    uint64_t eb = sm == SM_WS ? n : (sm == SM_IS ? r : n);
+    int have = 0;
+    i128 best_w = 0, best_c = 0;
+    uint64_t best_a = 0, best_b = 0;
+    for (uint64_t a = 1; a <= ea; ++a) {
+        if (ea % a) continue;
+        for (uint64_t b = 1; b <= eb; ++b) {
+            if (eb % b) continue;
+            if ((i128)ceil_div(a, rows) * ceil_div(b, cols) + 2 > (i128)rf_words) continue;
+            i128 w, c;
+            blocked_tile_terms((int)sm, m, r, n, rows, cols, a, b, &w, &c);
+            int better;
+            if (!have) better = 1;
+            else if (objective == MO_OBJ_LATENCY) better = c < best_c || (c == best_c && w < best_w);
+            else better = w < best_w || (w == best_w && c < best_c);
+            if (better) { have = 1; best_w = w; best_c = c; best_a = a; best_b = b; }
+        }
+    }
+    if (!have || !fits64(best_w) || !fits64(best_c)) return MO_ERR_ARG;
+    block_mrn[0] = sm == SM_WS ? 1u : (uint32_t)best_a;
+    block_mrn[1] = sm == SM_WS ? (uint32_t)best_a : (sm == SM_IS ? (uint32_t)best_b : 1u);
+    block_mrn[2] = sm == SM_IS ? 1u : (uint32_t)best_b;
+    *words = (int64_t)best_w;
+    *cycles = (int64_t)best_c;
+    return MO_OK;
 }
 
 static int decode(const mo_problem* p, uint64_t idx, mo_record* o)
@@ -344,12 +403,25 @@ int mo_eval(const mo_problem* p, uint64_t idx, mo_record* o)
     i128 t2 = (i128)dD[LP_I] * dD[LP_L] * dD[LP_J];
     i128 carry1 = (t1 - t1 / dD[LP_K]) * g[LP_I] * g[LP_L];
     i128 carry2 = (t2 - t2 / dD[LP_L]) * g[LP_I] * g[LP_J];
-    i128 br = t1 * tile_buffer_traffic((int)o->sm[0], g[LP_I], g[LP_K], g[LP_L], p->pe_rows, p->pe_cols)
-            + carry1
-            + t2 * tile_buffer_traffic((int)o->sm[1], g[LP_I], g[LP_L], g[LP_J], p->pe_rows, p->pe_cols)
-            + carry2;
-    i128 cyc1 = t1 * tile_cycles((int)o->sm[0], g[LP_I], g[LP_K], g[LP_L], p->pe_rows, p->pe_cols);
-    i128 cyc2 = t2 * tile_cycles((int)o->sm[1], g[LP_I], g[LP_L], g[LP_J], p->pe_rows, p->pe_cols);
+    i128 w1, w2, c1t, c2t;                  /* buffer<->array words and cycles of one tile of each operator */
+    if (p->rf_tiling) {
+        /* third tiling level: the register-file block of each operator's tile, picked by the objective */
+        int64_t bw_, bc_;
+        if (mo_rf_block(p->objective, o->sm[0], (uint32_t)g[LP_I], (uint32_t)g[LP_K], (uint32_t)g[LP_L],
+                        p->pe_rows, p->pe_cols, p->rf_words, &o->rf_block[0], &bw_, &bc_)) return MO_ERR_ARG;
+        w1 = bw_; c1t = bc_;
+        if (mo_rf_block(p->objective, o->sm[1], (uint32_t)g[LP_I], (uint32_t)g[LP_L], (uint32_t)g[LP_J],
+                        p->pe_rows, p->pe_cols, p->rf_words, &o->rf_block[3], &bw_, &bc_)) return MO_ERR_ARG;
+        w2 = bw_; c2t = bc_;
+    } else {
+        w1 = tile_buffer_traffic((int)o->sm[0], g[LP_I], g[LP_K], g[LP_L], p->pe_rows, p->pe_cols);
+        w2 = tile_buffer_traffic((int)o->sm[1], g[LP_I], g[LP_L], g[LP_J], p->pe_rows, p->pe_cols);
+        c1t = tile_cycles((int)o->sm[0], g[LP_I], g[LP_K], g[LP_L], p->pe_rows, p->pe_cols);
+        c2t = tile_cycles((int)o->sm[1], g[LP_I], g[LP_L], g[LP_J], p->pe_rows, p->pe_cols);
+    }
+    i128 br = t1 * w1 + carry1 + t2 * w2 + carry2;
+    i128 cyc1 = t1 * c1t;
+    i128 cyc2 = t2 * c2t;
 
     i128 n_gb = n_dram + br;
     i128 n_rf = p->has_rf ? br + 3 * n_mac : 0;
@@ -954,5 +1026,58 @@ int mo_simulate_unfused(const uint32_t bound[8], uint32_t pi, const uint32_t bet
         out->op2_stages++;
     }
     for (int x = 0; x < 5; ++x) { out->loads[x] *= tile[x]; free(blk[x].present); }
+    return MO_OK;
+}
+
+/* One tile with register-file-level blocks (see mmee_oracle.h), executed block by block, element by element. */
+int mo_array_tile_blocked(uint32_t sm, uint32_t m, uint32_t r, uint32_t n, uint32_t rows, uint32_t cols,
+                          uint32_t a, uint32_t b, int resume, mo_array_counts* acc)
+{
+    if (!acc || sm > 2 || !m || !r || !n || !rows || !cols || !a || !b) return MO_ERR_ARG;
+    const uint32_t ea = sm == SM_WS ? r : m;                   /* extents of the stationary operand */
+    const uint32_t eb = sm == SM_WS ? n : (sm == SM_IS ? r : n);
+    const uint32_t stream = sm == SM_WS ? m : (sm == SM_IS ? n : r);
+    if (ea % a || eb % b) return MO_ERR_ARG;
+    /* how many elements of a block each PE holds: element (x, y) lives in PE (x mod rows, y mod cols) */
+    uint32_t* held = (uint32_t*)calloc((size_t)rows * cols, sizeof(uint32_t));
+    if (!held) return MO_ERR_ARG;
+    uint32_t busiest = 0;
+    for (uint32_t x = 0; x < a; ++x)
+        for (uint32_t y = 0; y < b; ++y) {
+            uint32_t c = ++held[(size_t)(x % rows) * cols + (y % cols)];
+            if (c > busiest) busiest = c;
+        }
+    free(held);
+    int64_t cycles = 0, words = 0, macs = 0;
+    for (uint32_t ba = 0; ba * a < ea; ++ba)
+    for (uint32_t bb = 0; bb * b < eb; ++bb) {
+        /* the reduction dimension is the first block index under weight stationary, the second under input
+         * stationary; output stationary keeps the whole reduction inside one block */
+        const int continues = sm == SM_WS ? (ba > 0) : (sm == SM_IS ? (bb > 0) : 0);
+        if (sm != SM_OS)
+            for (uint32_t e = 0; e < a * b; ++e) ++words;                      /* pin the block */
+        else if (resume)
+            for (uint32_t e = 0; e < a * b; ++e) ++words;                      /* take the partial outputs in */
+        for (uint32_t v = 0; v < stream; ++v) {
+            for (uint32_t c = 0; c < busiest; ++c) ++cycles;                   /* one cycle per element of the busiest PE */
+            for (uint32_t e = 0; e < a * b; ++e) ++macs;
+            if (sm == SM_WS) {
+                for (uint32_t x = 0; x < a; ++x) ++words;                      /* the input row's a elements */
+                for (uint32_t y = 0; y < b; ++y) { if (continues || resume) ++words; ++words; }
+            } else if (sm == SM_IS) {
+                for (uint32_t y = 0; y < b; ++y) ++words;                      /* the weight column's b elements */
+                for (uint32_t x = 0; x < a; ++x) { if (continues || resume) ++words; ++words; }
+            } else {
+                for (uint32_t x = 0; x < a; ++x) ++words;
+                for (uint32_t y = 0; y < b; ++y) ++words;
+            }
+        }
+        if (sm == SM_OS)
+            for (uint32_t e = 0; e < a * b; ++e) ++words;                      /* outputs leave the array */
+    }
+    acc->cycles += cycles;
+    acc->words += words;
+    acc->macs += macs;
+    acc->rf += words + 3 * macs;
     return MO_OK;
 }

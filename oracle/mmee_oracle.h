@@ -60,6 +60,8 @@ typedef struct {
     uint32_t stationary_mask;              /* bit 3*sm1+sm2 set: that stationary pair is in the space; 0 = all nine
                                               (a reconfigurable array offers several, a fixed one a single pair) */
     uint64_t t_begin, t_end;
+    uint32_t rf_tiling;                    /* 1: register-file-level tiling (see mo_rf_block); energy / latency only */
+    uint32_t pad;
 } mo_objective;
 
 /* Everything derived once from the three input structs. */
@@ -81,6 +83,8 @@ typedef struct {
     uint32_t pe_rows, pe_cols, n_arrays, bw;
     uint32_t objective, topk;
     uint32_t stationary_mask;              /* never 0 */
+    uint32_t rf_tiling;
+    uint64_t rf_words;                     /* floor(rf_bytes / word_bytes)          */
 } mo_problem;
 
 typedef struct {
@@ -101,6 +105,7 @@ typedef struct {
     int64_t  e_key, l_key;
     double   edp_key;
     double   energy_pj, latency_cycles;
+    uint32_t rf_block[6];                  /* register-file-level tiling: block (m, r, n) of Op1, then of Op2; 0 when off */
 } mo_record;
 
 typedef struct {
@@ -153,6 +158,22 @@ typedef struct {
  * reduction steps in the buffer, which the array has to take in first.  Adds to *acc. */
 int  mo_array_tile(uint32_t sm, uint32_t m, uint32_t r, uint32_t n, uint32_t rows, uint32_t cols,
                    int resume, mo_array_counts* acc);
+/* Register-file-level tiling (third tiling level, below the buffer tile).  The stationary operand of a tile is
+ * cut into blocks of a x b elements (a, b divisors of its two extents); one block at a time lives in the PEs'
+ * register files, element (x, y) in PE (x mod rows, y mod cols), so that a PE holds ceil(a/rows) * ceil(b/cols)
+ * of them, beside one register for the streamed operand and one for the partial sum: a block is admissible iff
+ * that count + 2 <= rf_words.  The streamed vectors pass once per block; a vector takes one cycle per element a
+ * PE holds.  mo_array_tile_blocked executes one tile that way, element by element (block (a, b) as the two
+ * stationary extents: weight stationary (r, n), input stationary (m, r), output stationary (m, n)). */
+int  mo_array_tile_blocked(uint32_t sm, uint32_t m, uint32_t r, uint32_t n, uint32_t rows, uint32_t cols,
+                           uint32_t a, uint32_t b, int resume, mo_array_counts* acc);
+/* The block the model picks for one tile: every admissible (a, b) is tried in ascending (a, b) order; the energy
+ * objective keeps the block with the fewest buffer<->array words (then the fewest cycles, then the first), the
+ * latency objective the one with the fewest cycles (then the fewest words, then the first).  Returns MO_ERR_ARG
+ * if no block is admissible (cannot happen for rf_words >= 3). */
+int  mo_rf_block(uint32_t objective, uint32_t sm, uint32_t m, uint32_t r, uint32_t n, uint32_t rows, uint32_t cols,
+                 uint64_t rf_words, uint32_t block_mrn[3], int64_t* words, int64_t* cycles);
+
 /* Every tile invocation of both operators of one tiling in loop order: Op1 = C(i2,l2) += A*B over
  * k2, the whole of it `productions` times (recomputation), Op2 = E(i2,j2) += C*D over l2. */
 int  mo_array_chain(const uint32_t bound[8], uint32_t productions, uint32_t sm1, uint32_t sm2,

@@ -43,7 +43,7 @@ class Objective(C.Structure):
     _fields_ = [("objective", C.c_uint32), ("topk", C.c_uint32), ("tiling_set", C.c_uint32),
                 ("order_set", C.c_uint32), ("fuse_mask", C.c_uint32), ("row_pruning", C.c_uint32),
                 ("t_begin", C.c_uint64), ("t_end", C.c_uint64), ("key_cap", C.c_int64),
-                ("stationary_mask", C.c_uint32), ("reserved", C.c_uint32)]
+                ("stationary_mask", C.c_uint32), ("rf_tiling", C.c_uint32)]
 
 
 class Result(C.Structure):
@@ -57,7 +57,8 @@ class Result(C.Structure):
                 ("br", C.c_int64), ("cyc1", C.c_int64), ("cyc2", C.c_int64),
                 ("n", C.c_int64 * 5), ("e_key", C.c_int64), ("l_key", C.c_int64),
                 ("edp_key", C.c_double), ("energy_pj", C.c_double), ("latency_cycles", C.c_double),
-                ("n_total", C.c_uint64), ("n_feasible", C.c_uint64)]
+                ("n_total", C.c_uint64), ("n_feasible", C.c_uint64),
+                ("rf_block", C.c_uint32 * 6), ("reserved2", C.c_uint32 * 2)]
 
 
 class LaunchStats(C.Structure):

@@ -9,7 +9,7 @@
 
 #include "mmee_search.h"
 
-static_assert(sizeof(mmee_result_t) == 304, "mmee_result_t is part of the ABI");
+static_assert(sizeof(mmee_result_t) == 336, "mmee_result_t is part of the ABI");
 static_assert(sizeof(mmee::Plan) <= 4096, "the plan travels as a kernel parameter");
 
 struct mmee_handle {

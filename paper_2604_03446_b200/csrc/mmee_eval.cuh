@@ -38,6 +38,70 @@ __device__ __forceinline__ int64_t tile_traffic(int sm, uint32_t m, uint32_t r, 
     return M * R * ceil_div(n, cols) + R * N * ceil_div(m, rows) + M * N;
 }
 
+// Register-file-level tiling (objective.rf_tiling): buffer<->array words and compute cycles of one tile when
+// its stationary operand is processed in blocks of a x b elements; the block is searched over the divisors of the
+// operand's two extents (dimension ids da, db: the extents are tile extents of those dimensions, so their
+// divisors are among the plan's divisor lists), in ascending (a, b) order, keeping the admissible block with
+// the least (words, cycles) for the energy objective and the least (cycles, words) for the latency objective.
+// blk receives the block as (m, r, n) extents, 1 for the streamed extent.
+__device__ __forceinline__ void rf_block_terms(const Plan& p, int sm, uint32_t m, uint32_t r, uint32_t n, int da, int db,
+                                               int64_t& words, int64_t& cycles, uint32_t blk[3]) {
+    const uint32_t ea = sm == 0 ? r : m, eb = sm == 0 ? n : (sm == 1 ? r : n);
+    const int64_t M = m, R = r, N = n;
+    bool have = false;
+    int64_t bw = 0, bc = 0;
+    uint32_t ba = 0, bb = 0;
+    for (uint32_t ia = 0; ia < p.ndiv[da]; ++ia) {
+        const uint32_t a = p.divs[da][ia];
+        if (a > ea) break;
+        if (ea % a) continue;
+        const int64_t ha = ceil_div(a, p.pe_rows);
+        for (uint32_t ib = 0; ib < p.ndiv[db]; ++ib) {
+            const uint32_t b = p.divs[db][ib];
+            if (b > eb) break;
+            if (eb % b) continue;
+            const int64_t held = ha * ceil_div(b, p.pe_cols);       // stationary elements per PE
+            if (held + 2 > (int64_t)p.rf_words) continue;
+            int64_t w, c;
+            if (sm == 0) {
+                w = R * N + M * R * (int64_t)(n / b) + M * N * (2 * (int64_t)(r / a) - 1);
+                c = (int64_t)(r / a) * (int64_t)(n / b) * M * held;
+            } else if (sm == 1) {
+                w = M * R + R * N * (int64_t)(m / a) + M * N * (2 * (int64_t)(r / b) - 1);
+                c = (int64_t)(m / a) * (int64_t)(r / b) * N * held;
+            } else {
+                w = M * R * (int64_t)(n / b) + R * N * (int64_t)(m / a) + M * N;
+                c = (int64_t)(m / a) * (int64_t)(n / b) * R * held;
+            }
+            const bool better = !have || (p.objective == MMEE_OBJ_LATENCY ? (c < bc || (c == bc && w < bw))
+                                                                          : (w < bw || (w == bw && c < bc)));
+            if (better) { have = true; bw = w; bc = c; ba = a; bb = b; }
+        }
+    }
+    // (a block of one element needs three registers, which the planner requires: some block is always admissible)
+    words = bw;
+    cycles = bc;
+    blk[0] = sm == 0 ? 1u : ba;
+    blk[1] = sm == 0 ? ba : (sm == 1 ? bb : 1u);
+    blk[2] = sm == 1 ? 1u : bb;
+}
+
+// Words and cycles of one tile of operator `op` (0: (i_G x k_G)(k_G x l_G), 1: (i_G x l_G)(l_G x j_G)) under
+// stationary mode sm: one array fold per pass, or the register-file block search.
+__device__ __forceinline__ void tile_array_terms(const Plan& p, const uint32_t b[8], int op, int sm, int64_t& words,
+                                                 int64_t& cycles, uint32_t blk[3]) {
+    const uint32_t m = b[4], r = op == 0 ? b[5] : b[6], n = op == 0 ? b[6] : b[7];
+    if (p.rf_tiling) {
+        // dimensions of the stationary operand's two extents
+        const int dm = LOOP_I, dr = op == 0 ? LOOP_K : LOOP_L, dn = op == 0 ? LOOP_L : LOOP_J;
+        rf_block_terms(p, sm, m, r, n, sm == 0 ? dr : dm, sm == 0 ? dn : (sm == 1 ? dr : dn), words, cycles, blk);
+    } else {
+        words = tile_traffic(sm, m, r, n, p.pe_rows, p.pe_cols);
+        cycles = tile_cycles(sm, m, r, n, p.pe_rows, p.pe_cols);
+        blk[0] = blk[1] = blk[2] = 0;
+    }
+}
+
 // Tile invocations and carried partial sums of one tiling (no recomputation).
 struct TilingCounts {
     int64_t t1, t2;             // tile invocations of Op1 and Op2
@@ -56,26 +120,6 @@ __device__ __forceinline__ TilingCounts tiling_counts(const Plan& p, const uint3
     c.ilj = (int64_t)p.dim[0] * p.dim[2] * p.dim[3];
     c.il = (int64_t)p.dim[0] * p.dim[2];
     return c;
-}
-
-// Array-level terms of one (stationary pair, recompute flag) of one tiling: buffer<->PE words,
-// compute cycles of each operator, MAC and softmax counts.
-struct ArrayTerms {
-    int64_t br, cyc1, cyc2, n_mac, n_sfu;
-};
-
-__device__ __forceinline__ ArrayTerms array_terms(const Plan& p, const uint32_t b[8], const TilingCounts& c,
-                                                  int sm1, int sm2, bool recompute) {
-    const int64_t rho = recompute ? (int64_t)b[3] : 1;
-    const int64_t t1 = rho * c.t1;
-    ArrayTerms a;
-    a.br = t1 * tile_traffic(sm1, b[4], b[5], b[6], p.pe_rows, p.pe_cols) + rho * c.carry1 +
-           c.t2 * tile_traffic(sm2, b[4], b[6], b[7], p.pe_rows, p.pe_cols) + c.carry2;
-    a.cyc1 = t1 * tile_cycles(sm1, b[4], b[5], b[6], p.pe_rows, p.pe_cols);
-    a.cyc2 = c.t2 * tile_cycles(sm2, b[4], b[6], b[7], p.pe_rows, p.pe_cols);
-    a.n_mac = rho * c.ikl + c.ilj;
-    a.n_sfu = rho * c.il;
-    return a;
 }
 
 // Tiling index -> boundary vector b (one column of the boundary matrix, Section VI-A).
@@ -164,15 +208,18 @@ __device__ __forceinline__ void operand_terms(const Plan& p, const CandidateChoi
 // Array-level terms of one operator (0: C = A*B, 1: E = C*D) under one stationary mode: buffer<->PE words
 // including the carried partial sums, and compute cycles.
 __device__ __forceinline__ void operator_array_terms(const Plan& p, const uint32_t b[8], const TilingCounts& c, int op,
-                                                     int sm, bool recompute, int64_t& words, int64_t& cycles) {
+                                                     int sm, bool recompute, int64_t& words, int64_t& cycles,
+                                                     uint32_t blk[3]) {
+    int64_t w, cy;
+    tile_array_terms(p, b, op, sm, w, cy, blk);
     if (op == 0) {
         const int64_t rho = recompute ? (int64_t)b[3] : 1;
         const int64_t t1 = rho * c.t1;
-        words = t1 * tile_traffic(sm, b[4], b[5], b[6], p.pe_rows, p.pe_cols) + rho * c.carry1;
-        cycles = t1 * tile_cycles(sm, b[4], b[5], b[6], p.pe_rows, p.pe_cols);
+        words = t1 * w + rho * c.carry1;
+        cycles = t1 * cy;
     } else {
-        words = c.t2 * tile_traffic(sm, b[4], b[6], b[7], p.pe_rows, p.pe_cols) + c.carry2;
-        cycles = c.t2 * tile_cycles(sm, b[4], b[6], b[7], p.pe_rows, p.pe_cols);
+        words = c.t2 * w + c.carry2;
+        cycles = c.t2 * cy;
     }
 }
 
@@ -182,7 +229,7 @@ __device__ __forceinline__ void operator_array_terms(const Plan& p, const uint32
 __device__ __forceinline__ void assemble_record(const Plan& p, uint64_t idx, const CandidateChoice& d, const uint32_t b[8],
                                                 const TilingCounts& tt, const int64_t bs[5], const int64_t da_in[5],
                                                 int64_t words1, int64_t cyc1, int64_t words2, int64_t cyc2,
-                                                mmee_result_t& o) {
+                                                const uint32_t blk1[3], const uint32_t blk2[3], mmee_result_t& o) {
     const uint32_t* lv = d.lv;
     o.idx = idx; o.t = d.t; o.row = d.row;
     for (int i = 0; i < 8; ++i) o.bound[i] = b[i];
@@ -237,6 +284,8 @@ __device__ __forceinline__ void assemble_record(const Plan& p, uint64_t idx, con
     const uint32_t waves = (p.instances + p.n_arrays - 1) / p.n_arrays;
     o.latency_cycles = __dmul_rn(__ddiv_rn((double)l_key, (double)p.bw), (double)waves);
     o.n_total = 0; o.n_feasible = 0;
+    for (int i = 0; i < 3; ++i) { o.rf_block[i] = blk1[i]; o.rf_block[3 + i] = blk2[i]; }
+    o.reserved2[0] = o.reserved2[1] = 0;
 }
 
 // Full evaluation of one mapping by one thread.
@@ -248,9 +297,10 @@ __device__ inline void evaluate_candidate(const Plan& p, uint64_t idx, mmee_resu
     int64_t bs[5], da[5];
     for (int x = 0; x < 5; ++x) operand_terms(p, d, b, x, bs[x], da[x]);
     int64_t w1, c1, w2, c2;
-    operator_array_terms(p, b, tt, 0, d.sm1, d.rc != 0, w1, c1);
-    operator_array_terms(p, b, tt, 1, d.sm2, d.rc != 0, w2, c2);
-    assemble_record(p, idx, d, b, tt, bs, da, w1, c1, w2, c2, o);
+    uint32_t blk1[3], blk2[3];
+    operator_array_terms(p, b, tt, 0, d.sm1, d.rc != 0, w1, c1, blk1);
+    operator_array_terms(p, b, tt, 1, d.sm2, d.rc != 0, w2, c2, blk2);
+    assemble_record(p, idx, d, b, tt, bs, da, w1, c1, w2, c2, blk1, blk2, o);
 }
 
 // The same by one warp (all 32 lanes call it converged): lanes 0..4 take one operand each, lanes 5 and 6 one
@@ -261,15 +311,22 @@ __device__ inline void evaluate_candidate_warp(const Plan& p, uint64_t idx, int 
     tiling_bounds(p, d.t, b);
     const TilingCounts tt = tiling_counts(p, b);
     int64_t v0 = 0, v1 = 0;
+    uint32_t blk[3] = {0, 0, 0};
     if (lane < 5) operand_terms(p, d, b, lane, v0, v1);
-    else if (lane < 7) operator_array_terms(p, b, tt, lane - 5, lane == 5 ? d.sm1 : d.sm2, d.rc != 0, v0, v1);
+    else if (lane < 7) operator_array_terms(p, b, tt, lane - 5, lane == 5 ? d.sm1 : d.sm2, d.rc != 0, v0, v1, blk);
     int64_t part0[7], part1[7];
 #pragma unroll
     for (int i = 0; i < 7; ++i) {
         part0[i] = __shfl_sync(0xffffffffu, v0, i);
         part1[i] = __shfl_sync(0xffffffffu, v1, i);
     }
-    if (lane == 0) assemble_record(p, idx, d, b, tt, part0, part1, part0[5], part1[5], part0[6], part1[6], o);
+    uint32_t blk1[3], blk2[3];
+#pragma unroll
+    for (int i = 0; i < 3; ++i) {
+        blk1[i] = __shfl_sync(0xffffffffu, blk[i], 5);
+        blk2[i] = __shfl_sync(0xffffffffu, blk[i], 6);
+    }
+    if (lane == 0) assemble_record(p, idx, d, b, tt, part0, part1, part0[5], part1[5], part0[6], part1[6], blk1, blk2, o);
 }
 
 }  // namespace mmee

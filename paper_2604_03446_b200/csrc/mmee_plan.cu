@@ -145,7 +145,8 @@ int build_plan(const mmee_workload_t* w, const mmee_arch_t* a, const mmee_object
     if (o->row_pruning > 1 || (o->row_pruning && o->topk != 1)) return MMEE_ERR_ARG;
     if (o->tiling_set > MMEE_TILE_ALL_DIVISORS || o->order_set > MMEE_ORD_ALL6) return MMEE_ERR_ARG;
     if (!(o->fuse_mask & 7u) || (o->fuse_mask & ~7u)) return MMEE_ERR_ARG;
-    if ((o->stationary_mask & ~0x1ffu) || o->reserved) return MMEE_ERR_ARG;
+    if ((o->stationary_mask & ~0x1ffu) || o->rf_tiling > 1) return MMEE_ERR_ARG;
+    if (o->rf_tiling && (o->objective > MMEE_OBJ_LATENCY || !a->rf_bytes)) return MMEE_ERR_ARG;
 
     // The g = q_heads/kv_heads query heads of one K/V head are stacked along I, so that K and V
     // are fetched once per group; each (batch, kv head) pair is one independent instance.
@@ -230,6 +231,11 @@ int build_plan(const mmee_workload_t* w, const mmee_arch_t* a, const mmee_object
     p->sm_mask = o->stationary_mask ? o->stationary_mask : 0x1ffu;
     for (uint32_t b = 0; b < 9; ++b) p->n_sm += (p->sm_mask >> b) & 1u;
     p->key_cap = o->key_cap;
+    p->rf_tiling = o->rf_tiling;
+    {
+        const uint64_t rfw = a->rf_bytes / w->word_bytes;
+        p->rf_words = rfw > 0xffffffffull ? 0xffffffffu : (uint32_t)rfw;
+    }
 
     // Largest key any mapping of this problem can have.  M bounds the MAC count with the largest
     // recomputation factor (j_D <= J); each of at most seven DRAM terms is <= I*K*L*J <= M, the

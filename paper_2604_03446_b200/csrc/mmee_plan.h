@@ -55,6 +55,8 @@ struct Plan {
     uint32_t rel_shift;           // energy: threshold-relative keys are kept in units of 2^rel_shift quanta
     int32_t  unit;                // the constant 1, as a run-time value: x * unit + y is issued as an integer
                                   // multiply-add, which the FMA pipe executes beside the integer ALU pipe
+    uint32_t rf_tiling;           // register-file-level tiling: the block of each operator's tile is searched
+    uint32_t rf_words;            // register-file capacity of one PE in words
     double   quantum_pj;
     QueryTables q;
     uint32_t divs[4][MMEE_MAX_DIVISORS];

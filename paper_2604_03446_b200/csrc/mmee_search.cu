@@ -84,6 +84,8 @@ struct alignas(16) TilingTab {
     int64_t W[9][2];        // energy of buffer<->PE traffic, MACs and softmax, in quanta
     int64_t CB[9][2];       // fused compute time in words (cycles * words per cycle)
     int64_t QU[9][2];       // unfused Op2 compute time in words, by s (sm2 = s % 3)
+    int64_t opw[2][3];      // buffer<->array words of one tile of each operator, by stationary mode
+    int64_t opc[2][3];      // compute cycles of one tile of each operator, by stationary mode
     int64_t C1w[3];         // unfused Op1 compute time in words, by sm1
     int64_t cw, smx;        // C write-back words (I*L); separate softmax pass words (2*I*L)
     int64_t wmin[2];        // min over the stationary pairs of W[.][rc]
@@ -508,19 +510,31 @@ __device__ __forceinline__ void build_tiling_head(const Plan& p, uint64_t t, Til
     tb->pad[0] = tb->pad[1] = tb->pad[2] = 0;
 }
 
+// One thread per (tiling slot, operator, stationary mode): words and cycles of one tile (the only part of the
+// array-level terms that needs divisions, or the register-file block search).
+__device__ __forceinline__ void build_tile_terms(const Plan& p, TilingTab* tb, int item) {
+    const int op = item / 3, sm = item % 3;
+    uint32_t blk[3];
+    tile_array_terms(p, tb->b, op, sm, tb->opw[op][sm], tb->opc[op][sm], blk);
+}
+
 // One thread per (tiling slot, item): stationary-pair terms with the cost coefficients applied.
 __device__ __forceinline__ void build_tiling_item(const Plan& p, TilingTab* tb, int item) {
     const TilingCounts c = tiling_counts(p, tb->b);
     const int64_t bw = p.bw;
     if (item < 18) {
         const int s = item >> 1, rc = item & 1;
-        const ArrayTerms a = array_terms(p, tb->b, c, s / 3, s % 3, rc != 0);
-        tb->W[s][rc] = p.c_br * a.br + p.c_mac * a.n_mac + p.c_sfu * a.n_sfu;
-        tb->CB[s][rc] = (a.cyc1 + a.cyc2) * bw;
-        tb->QU[s][rc] = a.cyc2 * bw;
+        const int sm1 = s / 3, sm2 = s % 3;
+        const int64_t rho = rc ? (int64_t)tb->b[3] : 1;
+        const int64_t t1 = rho * c.t1;
+        const int64_t br = t1 * tb->opw[0][sm1] + rho * c.carry1 + c.t2 * tb->opw[1][sm2] + c.carry2;
+        const int64_t cyc1 = t1 * tb->opc[0][sm1], cyc2 = c.t2 * tb->opc[1][sm2];
+        tb->W[s][rc] = p.c_br * br + p.c_mac * (rho * c.ikl + c.ilj) + p.c_sfu * (rho * c.il);
+        tb->CB[s][rc] = (cyc1 + cyc2) * bw;
+        tb->QU[s][rc] = cyc2 * bw;
     } else {
         const int sm1 = item - 18;
-        tb->C1w[sm1] = c.t1 * tile_cycles(sm1, tb->b[4], tb->b[5], tb->b[6], p.pe_rows, p.pe_cols) * bw;
+        tb->C1w[sm1] = c.t1 * tb->opc[0][sm1] * bw;
     }
 }
 
@@ -1264,6 +1278,9 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                 build_tiling_item(p, &ttabs[slot], (int)e);
             }
         };
+        for (uint32_t it = first; it < n_slots * 6u; it += step)      // one tile of each operator under each mode
+            if (ttabs[it / 6u].live) build_tile_terms(p, &ttabs[it / 6u], (int)(it % 6u));
+        sync();
         tiling_pass(0, 18);     // stationary pairs x recompute flag
         tiling_pass(18, 3);     // unfused Op1 compute words
         sync();

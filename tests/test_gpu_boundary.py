@@ -230,3 +230,66 @@ def shrink_to(cfg, obj, limit):
     if p.N <= limit:
         return dict(obj)
     return dict(obj, t_begin=0, t_end=max(1, limit // (p.R * 9)))
+
+
+# ---- register-file-level tiling ------------------------------------------------------------------------------------
+
+def _with_register_file_tiling(cfg, objective, rf_words, topk=1):
+    arch = dict(cfg["arch"], rf_bytes=rf_words * cfg["workload"]["word_bytes"])
+    if arch["e_rf_pj"] == 0:
+        arch["e_rf_pj"] = arch["energy_quantum_pj"]
+    obj = dict(cfg["searches"][0], objective=objective, topk=topk, rf_tiling=1, row_pruning=0)
+    return dict(cfg, arch=arch), obj
+
+
+@pytest.mark.parametrize("objective", [mi.OBJ_ENERGY, mi.OBJ_LATENCY])
+@pytest.mark.parametrize("seed,rf_words", [(1, 6), (2, 7), (4, 8), (6, 16), (9, 64)])
+def test_register_file_tiling_keys_records_and_search(seed, rf_words, objective):
+    """The third tiling level on small problems: every candidate's key, sampled full records (with the register-file
+    block of each operator) and the top-5 of the search equal the oracle's, from a register file that holds a single
+    stationary element per PE to one that holds whole tiles."""
+    cfg, obj = _with_register_file_tiling(mi.random_tiny_problem(seed), objective, rf_words, topk=5)
+    obj = shrink_to(cfg, obj, 600_000)
+    p = oracle.make_problem(cfg["workload"], cfg["arch"], obj)
+    begin, count = p.t_begin * p.R * 9, (p.t_end - p.t_begin) * p.R * 9
+    want_keys, want_feas = oracle.keys_range(p, begin, count)
+    want_keys = np.where(want_feas.astype(bool), want_keys, np.iinfo(np.int64).max)
+    keys = torch.empty(count, dtype=torch.int64, device="cuda")
+    with Handle(cfg, obj) as h:
+        mm.mmee_dump_keys(h, keys)
+        torch.cuda.synchronize()
+        rng = np.random.default_rng(seed)
+        for idx in [begin, begin + count - 1] + [int(i) for i in rng.integers(begin, begin + count, size=60)]:
+            assert_same_record(mm.mmee_decode(h, idx), oracle.evaluate(p, idx), "idx %d" % idx)
+        best, topk = mm.mmee_search_host(h, True, 5)
+    assert np.array_equal(keys.cpu().numpy(), want_keys)
+    want = oracle.search(p)
+    assert [r.idx for r in topk if r.idx != mm.NO_INDEX] == [r.idx for r in want.topk]
+    assert best.n_feasible == want.n_feasible
+    for g, o in zip(topk, want.topk):
+        assert_same_record(g, o)
+        assert any(g.rf_block)
+
+
+def test_register_file_tiling_at_full_size_sampled():
+    """BERT-base on the edge accelerator with the third tiling level: sampled candidates against the oracle, and the
+    search's optimum is a mapping whose record the oracle reproduces and whose key no sampled candidate beats; a
+    larger register file never makes the optimum worse."""
+    cfg = mi.config2()
+    rng = np.random.default_rng(17)
+    best_keys = []
+    for rf_words in (8, 512):
+        cfgr, obj = _with_register_file_tiling(cfg, mi.OBJ_ENERGY, rf_words)
+        p = oracle.make_problem(cfgr["workload"], cfgr["arch"], obj)
+        with Handle(cfgr, obj) as h:
+            best, _ = mm.mmee_search_host(h)
+            assert best.status == mm.OK
+            assert_same_record(best, oracle.evaluate(p, best.idx), "optimum")
+            for idx in rng.integers(0, p.N, size=300):
+                o = oracle.evaluate(p, int(idx))
+                assert_same_record(mm.mmee_decode(h, int(idx)), o, "idx %d" % idx)
+                assert not o.feasible or (o.e_key, o.idx) >= (best.e_key, best.idx)
+        best_keys.append(best.e_key)
+    assert best_keys[1] <= best_keys[0]
+    plain, _, _ = __import__("test_gpu_parity").gpu_search(cfg, cfg["searches"][0])
+    assert plain.rf_block[0] == 0

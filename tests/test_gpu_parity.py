@@ -21,7 +21,7 @@ GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 REL_TOL = 1e-12
 INT_FIELDS = ("idx", "t", "row", "phi", "pi", "recompute", "feasible", "bs_op1", "bs_op2", "bs",
               "da_sm", "br", "cyc1", "cyc2", "e_key", "l_key")
-ARRAY_FIELDS = ("bound", "beta", "sm", "bs_x", "da_x", "n")
+ARRAY_FIELDS = ("bound", "beta", "sm", "bs_x", "da_x", "n", "rf_block")
 FLOAT_FIELDS = ("edp_key", "energy_pj", "latency_cycles")
 
 

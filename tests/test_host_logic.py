@@ -27,7 +27,7 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_result_record_layout():
-    assert C.sizeof(mm.Result) == 72 + 8 * 24 + 8 * 3 + 16 == 304
+    assert C.sizeof(mm.Result) == 72 + 8 * 24 + 8 * 3 + 16 + 32 == 336
     assert mm.Result.status.offset == 68 and mm.Result.bs_x.offset == 72
 
 
@@ -84,7 +84,7 @@ def test_argument_errors_come_before_any_device_call():
     for bad_o, code in ((dict(o, fuse_mask=0), mm.ERR_ARG), (dict(o, topk=0), mm.ERR_ARG),
                         (dict(o, topk=17), mm.ERR_RANGE), (dict(o, objective=5), mm.ERR_ARG), (dict(o, objective=3, key_cap=-1), mm.ERR_ARG),
                         (dict(o, t_begin=5, t_end=2), mm.ERR_ARG), (dict(o, stationary_mask=0x200), mm.ERR_ARG),
-                        (dict(o, reserved=1), mm.ERR_ARG)):
+                        (dict(o, rf_tiling=2), mm.ERR_ARG), (dict(o, rf_tiling=1, objective=2), mm.ERR_ARG)):
         with pytest.raises(mm.MmeeError) as e:
             mm.mmee_create(w, a, bad_o)
         assert e.value.code == code

@@ -181,3 +181,100 @@ def test_fused_keys_from_counted_events():
         assert rec.l_key == max(n_dram, (op1.cycles + op2.cycles) * bw)
         assert rec.e_key == 7 * n_dram + 5 * (n_dram + op1.words + op2.words) + 3 * (op1.rf + op2.rf) \
             + 2 * (op1.macs + op2.macs) + 4 * 2 * I * L
+
+
+# ---- register-file-level tiling -----------------------------------------------------------------------------------
+
+def _divisors(x):
+    return [d for d in range(1, x + 1) if x % d == 0]
+
+
+def _stationary_extents(sm, m, r, n):
+    return {WS: (r, n), IS: (m, r), OS: (m, n)}[sm]
+
+
+def _best_block_by_execution(objective, sm, m, r, n, rows, cols, rf_words):
+    """Every admissible block executed element by element; the choice rule applied to the counted figures."""
+    ea, eb = _stationary_extents(sm, m, r, n)
+    best = None
+    for a in _divisors(ea):
+        for b in _divisors(eb):
+            per_pe = max(sum(1 for x in range(a) for y in range(b) if (x % rows, y % cols) == pe)
+                         for pe in {(x % rows, y % cols) for x in range(a) for y in range(b)})
+            if per_pe + 2 > rf_words:
+                continue
+            c = oracle.array_tile_blocked(sm, m, r, n, rows, cols, a, b)
+            key = (c.cycles, c.words) if objective == mi.OBJ_LATENCY else (c.words, c.cycles)
+            if best is None or key < best[0]:
+                best = (key, (a, b), c.words, c.cycles)
+    return best
+
+
+@pytest.mark.parametrize("rows,cols,rf_words", [(2, 3, 3), (2, 3, 6), (3, 2, 12), (4, 4, 4), (1, 5, 40)])
+def test_register_file_block_choice_against_element_level_execution(rows, cols, rf_words):
+    """Register-file-level tiling: for every stationary mode and several tile shapes, the block the oracle picks and
+    the words and cycles it reports equal what an element-by-element execution of every admissible block gives
+    under the same choice rule (fewest words, then cycles, for energy; fewest cycles, then words, for latency;
+    the first such block in ascending order)."""
+    for m, r, n in [(4, 6, 6), (6, 4, 9), (8, 12, 6), (5, 7, 3), (12, 2, 8)]:
+        for sm in (WS, IS, OS):
+            for objective in (mi.OBJ_ENERGY, mi.OBJ_LATENCY):
+                blk, words, cycles = oracle.rf_block(objective, sm, m, r, n, rows, cols, rf_words)
+                _, (a, b), w_sim, c_sim = _best_block_by_execution(objective, sm, m, r, n, rows, cols, rf_words)
+                want_blk = {WS: (1, a, b), IS: (a, b, 1), OS: (a, 1, b)}[sm]
+                assert (blk, words, cycles) == (want_blk, w_sim, c_sim), (sm, objective, m, r, n)
+                # a resumed tile takes its partial outputs in first: m * n words more, same cycles
+                res = oracle.array_tile_blocked(sm, m, r, n, rows, cols, a, b, resume=True)
+                assert res.words == w_sim + m * n and res.cycles == c_sim and res.macs == m * r * n
+
+
+def test_mappings_under_register_file_tiling_from_counted_events():
+    """Whole mappings with the third tiling level: BR, cycles, N_RF and both keys of sampled fused and unfused rows
+    equal the sums over all tile invocations of the element-level execution with the picked blocks (a reduction
+    step after the first of an output tile resumes it); the level changes nothing above the array: buffer need,
+    DRAM words and MACs are those of the same mapping without it."""
+    I, K, L, J = 8, 6, 6, 4
+    rows, cols, bw = 2, 3, 3
+    w = mi.workload(1, 1, 1, I, L, K, J, 1)
+    a = mi.arch(rows, cols, 1, 10 ** 9, 6, bw, 7.0, 5.0, 3.0, 2.0, c_softmax=4.0)
+    rng = np.random.default_rng(3)
+    for objective in (mi.OBJ_ENERGY, mi.OBJ_LATENCY):
+        p = oracle.make_problem(w, a, dict(mi.objective(objective), rf_tiling=1))
+        plain = oracle.make_problem(w, a, mi.objective(objective))
+        t = tiling_index(p, (4, 3, 2, 2))
+        for r in list(rng.integers(0, 6250, size=20)) + list(rng.integers(18750, 26250, size=10)):
+            s = int(r) % 9
+            idx = (t * p.R + int(r)) * 9 + s
+            rec, ref = oracle.evaluate(p, idx), oracle.evaluate(plain, idx)
+            assert list(rec.bs_x) == list(ref.bs_x) and list(rec.da_x) == list(ref.da_x) and rec.n[3] == ref.n[3]
+            iD, kD, lD, jD, iG, kG, lG, jG = rec.bound
+            rho = jD if rec.recompute else 1
+            blocks = (tuple(rec.rf_block[:3]), tuple(rec.rf_block[3:]))
+            tiles = ((s // 3, iG, kG, lG, rho * iD * lD, kD), (s % 3, iG, lG, jG, iD * jD, lD))
+            words, cyc = [], []
+            for (sm, m, rr, n, outputs, steps), blk in zip(tiles, blocks):
+                ab = {WS: (blk[1], blk[2]), IS: (blk[0], blk[1]), OS: (blk[0], blk[2])}[sm]
+                first = oracle.array_tile_blocked(sm, m, rr, n, rows, cols, *ab)
+                again = oracle.array_tile_blocked(sm, m, rr, n, rows, cols, *ab, resume=True)
+                words.append(outputs * (first.words + (steps - 1) * again.words))
+                cyc.append(outputs * steps * first.cycles)
+            assert (rec.cyc1, rec.cyc2) == tuple(cyc) and rec.br == sum(words)
+            assert rec.n[2] == rec.br + 3 * rec.n[3] and rec.n[1] == rec.n[0] + rec.br
+            assert rec.e_key == 7 * rec.n[0] + 5 * rec.n[1] + 3 * rec.n[2] + 2 * rec.n[3] + 8 * rec.n[4]
+            if rec.phi == 0:
+                assert rec.l_key == max(rec.n[0], (rec.cyc1 + rec.cyc2) * bw)
+            # the level is a refinement: the energy objective never moves more words between buffer and array than
+            # the best single block shape of the plain model's kind could, and every block respects the capacity
+            for sm, blk in zip((s // 3, s % 3), blocks):
+                held = {WS: (blk[1], blk[2]), IS: (blk[0], blk[1]), OS: (blk[0], blk[2])}[sm]
+                assert -(-held[0] // rows) * -(-held[1] // cols) + 2 <= 6
+
+
+def test_register_file_tiling_is_refused_where_it_is_not_defined():
+    w, a = mi.workload(1, 1, 1, 8, 8, 4, 4), mi.arch(2, 2, 1, 4096, 0, 1, 1, 1, 0, 1)
+    for obj in (dict(mi.objective(mi.OBJ_ENERGY), rf_tiling=1),                      # no register-file level
+                ):
+        with pytest.raises(oracle.OracleError):
+            oracle.make_problem(w, a, obj)
+    with pytest.raises(oracle.OracleError):                                           # product objective
+        oracle.make_problem(w, dict(a, rf_bytes=64, e_rf_pj=1), dict(mi.objective(mi.OBJ_EDP), rf_tiling=1))
