@@ -73,7 +73,7 @@ int mo_problem_init(const mo_workload* w, const mo_arch* a, const mo_objective* 
     if (o->rf_tiling > 1 || o->pad) return MO_ERR_ARG;
     if (o->rf_tiling && (o->objective > MO_OBJ_LATENCY || !a->rf_bytes)) return MO_ERR_ARG;
 
-    /* Heads are independent instances (Section V, "we omit the head dimension"); the g query
+    /* Heads are independent instances (Section V, opening paragraph: the model is stated per head); the g query
      * heads that share one K/V head are stacked along I, so K and V are loaded once per group. */
     uint64_t g = w->q_heads / w->kv_heads;
     p->dim[LP_I] = g * (uint64_t)w->seq_q;
@@ -152,7 +152,7 @@ typedef struct {
 } nest_t;
 
 /* Operand buffer words: tile footprint times the bounds of the operand's own loops at and
- * below its buffering level (Section V-B, "Operand's buffer size requirement"). */
+ * below its buffering level (Section V-B, first definition). */
 static i128 buffer_words(int x, int beta, const nest_t* n, const uint64_t* dD, i128 tile)
 {
     i128 bs = tile;
@@ -644,7 +644,7 @@ typedef struct { int n; uint8_t term[6]; } sym_sum;
 
 /* P >= Q for every assignment of the bounds if the terms of Q can be matched one-to-one into
  * terms of P with term_Q a subset of term_P (a product over a superset of bounds >= 1 is not
- * smaller).  This is the comparison "without specific tiling solutions" of Section VI-B. */
+ * smaller).  This is the tiling-independent comparison of Section VI-B. */
 static int match_terms(const sym_sum* p, const sym_sum* q, int qi, unsigned used)
 {
     if (qi == q->n) return 1;

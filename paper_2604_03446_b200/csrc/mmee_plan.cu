@@ -40,8 +40,8 @@ Nest nest_of(int order, uint8_t absent) {
     return n;
 }
 
-// BS_X: tile footprint times the bounds of the operand's own loops at levels 4..beta
-// (Section V-B, "Operand's buffer size requirement").
+// Query row of BS_X (Section V-B): the two x_G bits of the operand's tile plus the x_D bit of every own loop
+// that sits at or below the buffering level.
 uint8_t buffer_query(const Nest& n, int x, int beta) {
     uint8_t q = (uint8_t)(bit_g(kOwn[x][0]) | bit_g(kOwn[x][1]));
     for (int s = 0; s < 2; ++s) {
