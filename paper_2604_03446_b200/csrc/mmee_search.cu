@@ -9,15 +9,17 @@
 // per-operand monomials; Section V-D: energy is linear in the access counts), so the query-matrix
 // product exp(Q . ln B) (Eq. 11) is evaluated once per (tiling, order, operand, level) into small
 // shared-memory tables -- each entry an exact integer monomial already multiplied by its energy
-// coefficient -- and a candidate's key is a short sum of table entries.  The row loop evaluates
-// every candidate's key relative to the current top-k threshold in saturated 32-bit arithmetic
-// (one fused add-min per candidate for energy, one fused add-max for latency); exact 64-bit keys
-// are formed only for groups of rows that can enter the list.  Nothing per candidate ever touches
-// global memory.
+// coefficient -- and a candidate's key is a short sum of table entries.  The least key of the nine
+// mappings of a row (one per stationary pair) is the row's sum plus the least stationary-pair term,
+// which is taken once per tiling: the row loop tests one key per row, relative to the current top-k
+// threshold in saturated 32-bit arithmetic (a single-precision product bound for the energy-delay
+// objective); exact 64-bit keys of single mappings are formed only for groups of rows that can enter
+// the list.  Nothing per candidate ever touches global memory.
 //
 // CTAs are persistent and pull ranges of tasks from a global counter.  All warps build the tables
 // of a CTA's first range together; after that seven warps walk tasks while the eighth builds the
-// tables of the next range into a second buffer and then joins them.
+// tables of the next range into a second buffer and then joins them.  The CTA that finishes last
+// (a ticket counter, no wait) merges the CTAs' partial lists and evaluates the winners in full.
 #include <cuda_runtime.h>
 
 #include <climits>
@@ -260,31 +262,33 @@ __device__ __forceinline__ void row_test(const int64_t (&k)[9], int64_t thr, int
 // 32-bit differential keys
 // ------------------------------------------------------------------------------------------------
 // Whether a candidate enters the top-k depends only on the sign of key - thr.  The row loops
-// therefore evaluate every candidate's key RELATIVE to the lane's current threshold, in saturated
-// 32-bit arithmetic, and keep the minimum over a group of five rows; a negative minimum sends the
-// warp to the exact 64-bit path, which re-evaluates the group in full.  The filter may flag a group
-// needlessly; it must never miss a candidate that passes.
+// therefore evaluate the least key of every row (nine mappings) RELATIVE to the lane's current
+// threshold, in saturated 32-bit arithmetic, and keep the minimum over a group of five rows; a
+// negative minimum sends the warp to the exact 64-bit path, which re-evaluates the group's 45
+// mappings in full.  The filter may flag a group needlessly; it must never miss a candidate that
+// passes.
 //
-// Energy: key = x + W[s].  With wmin = min_s W[s], B = thr - wmin and W' = W - wmin >= 0:
-// key < thr  <=>  (gA + gX - B) + gB + vD + vE + W' < 0, the g / v terms being the DRAM energies of the
-// operands at their levels (gX: the C round trip of an unfused task).  All terms are kept in units of
-// 2^rel_shift quanta (the plan picks the shift from the largest possible DRAM term): every addend is
-// rounded down and capped at kTermCap, B is rounded up, so that the 32-bit sum is never above the
-// true one.  The task-level part (gA + gX - ceil(B / unit)) is clamped to [-kUnfit, kRowCap]; at most
-// four addends of at most kTermCap follow, 4 * kTermCap < kUnfit, so a sum that was clamped from below
-// stays negative (the group is flagged, which is the safe side), and no 32-bit sum overflows:
-// kRowCap + 2 * kTermCap + kUnfit < 2^31.  Most terms are multiples of the unit, so that a tie with
-// the list's last entry is still told from a better key: when every index still to be walked in a
-// task lies above that entry's, the threshold is thr - 1 (decided at the start of the task and after
-// each visit of the exact path).
+// Energy: key = x + W[s], so the row's least key is x + wmin with wmin = min_s W[s] over the offered
+// pairs.  With B = thr - wmin:  x + wmin < thr  <=>  (gA + gX - B) + gB + vD + vE < 0, the g / v terms
+// being the DRAM energies of the operands at their levels (gX: the C round trip of an unfused task).
+// All terms are kept in units of 2^rel_shift quanta (the plan picks the shift from the largest possible
+// DRAM term): every addend is rounded down and capped at kTermCap, B is rounded up, so that the 32-bit
+// sum is never above the true one.  The task-level part (gA + gX - ceil(B / unit)) is clamped to
+// [-kUnfit, kRowCap]; at most three addends of at most kTermCap follow, 3 * kTermCap < kUnfit, so a sum
+// that was clamped from below stays negative (the group is flagged, which is the safe side), and no
+// 32-bit sum overflows: kRowCap + kTermCap + kUnfit < 2^31.  Most terms are multiples of the unit, so
+// that a tie with the list's last entry is still told from a better key: when every index still to be
+// walked in a task lies above that entry's, the threshold is thr - 1 (decided at the start of the task
+// and after each visit of the exact path).
 // Latency: key = P + max(x, Q[s]) (P: the Op1 stage of an unfused task, else 0), and
-// max(a, b) < thr  <=>  a - thr < 0 and b - thr < 0.  a = (x0 + P - thr) + vD + vE with the same
-// units, rounding and clamping (the unit is chosen from the largest DRAM term in words);
-// b = (Q[s] - qmin) + (qmin + P - thr), the first part a table entry capped at kTermCap, both parts
-// rounded down.
+// max(a, b) < thr  <=>  a - thr < 0 and b - thr < 0.  The row's least key over s has b = qmin (the
+// least compute words over the offered pairs; with the least Op1 stage for an unfused task): when
+// qmin + P - thr >= 0 no row of the middle level can pass, otherwise only a = (x0 + P - thr) + vD + vE
+// decides, with the same units, rounding and clamping (the unit is chosen from the largest DRAM term
+// in words).
 // Capacity (Eq. 4): sizes are saturated to kSizeCap, which is above every admissible capacity, so
-// "size <= slack" keeps its truth value in 32 bits.  A row that does not fit has kUnfit added to its
-// keys, which makes them non-negative whatever the threshold.
+// "size <= slack" keeps its truth value in 32 bits.  A row that does not fit has kUnfit OR-ed into
+// its term, which makes its key non-negative whatever the threshold.
 // Integer multiply-add and arithmetic shift as single PTX instructions, opaque to the optimiser: the row
 // loops use them to keep additions on the FMA pipe and sign masks out of compare-and-select form.
 __device__ __forceinline__ int imad(int a, int b, int c) {
