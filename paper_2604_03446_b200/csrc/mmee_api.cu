@@ -162,7 +162,7 @@ int mmee_search(mmee_handle_t* h, void* cuda_stream, mmee_result_t* out_best, mm
     int rc = check_device(h);
     if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    if (h->dirty) {        // an earlier call failed between its two launches: the header may hold a used work counter
+    if (h->dirty) {        // an earlier launch on this handle failed: the header may hold a used work counter
         if ((rc = cuda_status(launch_reset(h->scratch, st)))) return rc;
         h->dirty = false;
     }

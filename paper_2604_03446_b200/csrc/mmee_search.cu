@@ -908,8 +908,8 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
     const int4 av = *reinterpret_cast<const int4*>(ot->Ac[c.la]);
     const int a1c = av.x, a2c = fused ? av.y : 0;
     const int capc = (int)p.cap_words;
-    // Additions that need no saturation are written x * one + y: an integer multiply-add runs on the FMA
-    // pipe, which is otherwise idle, instead of the integer ALU pipe that bounds this kernel.
+    // Differences and counts that need no saturation are written x * (-1) + y with a run-time -1: an integer
+    // multiply-add runs on the FMA pipe, which is otherwise idle, instead of the integer ALU pipe.
     const int minus_one = -p.unit;
     const int gxc = (OBJ == MMEE_OBJ_ENERGY && !fused) ? ot->gXc[c.phi == 2 ? 1 : 0] : 0;
     // task-level part of key - thr, clamped to [-kUnfit, kRowCap]: clamping from below keeps the sign of every
