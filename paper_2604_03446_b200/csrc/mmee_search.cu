@@ -725,8 +725,14 @@ __device__ __noinline__ void exact_group_single(const Plan& p, const TilingTab* 
 // row, then an add, two multiplies and two compares per mapping).  Each approximate product is within a few 2^-53
 // of the exact key, so comparing against the threshold widened by 1e-14 relative can flag a row needlessly but never
 // miss one; the exact path decides.  Returns 1 if some row fits and holds such a product.
-__device__ __noinline__ unsigned edp_group_test(const MidExact& me, const RowTab* rt, int d, int s1c, int s2c,
-                                                uint32_t kept_rows, uint32_t sm_mask, double dthr) {
+__device__ __noinline__ unsigned edp_group_test(const Plan& p, const TilingTab* tb, const OrderTab* ot, uint32_t phi,
+                                                uint32_t la, uint32_t lb_task, int m, bool live, int d, int s1c, int s2c,
+                                                uint32_t kept_rows, double dthr) {
+    // (the 64-bit terms of the middle level are formed again here, so that the caller's row loop need not keep
+    // them, in registers or in local memory, for this rare path)
+    const MidExact me = mid_exact<MMEE_OBJ_EDP>(p, tb, ot, phi, la, lb_task, m, live);
+    const RowTab* rt = &ot->rt[phi == 0 ? 0 : 1];
+    const uint32_t sm_mask = p.sm_mask;
     double dW[9], dQP[9];
 #pragma unroll
     for (int s = 0; s < 9; ++s) {
@@ -836,7 +842,8 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
                     const float lb = __fmul_rd(__fadd_rd(fed, Eef[e]), fl);
                     hit1 |= fit & (unsigned)(lb <= fthr);
                 }
-                if (__any_sync(kFull, hit1 != 0u)) hit_any = edp_group_test(me, rt, d, s1c, s2c, kd, p.sm_mask, dthr);
+                if (__any_sync(kFull, hit1 != 0u))
+                    hit_any = edp_group_test(p, tb, ot, c.phi, c.la, c.lb, m, live, d, s1c, s2c, kd, dthr);
             } else {
                 ++groups_walked;
                 const int64_t s1 = me.slack1 - rt->D[d][0];
