@@ -293,3 +293,21 @@ def test_register_file_tiling_at_full_size_sampled():
     assert best_keys[1] <= best_keys[0]
     plain, _, _ = __import__("test_gpu_parity").gpu_search(cfg, cfg["searches"][0])
     assert plain.rf_block[0] == 0
+
+
+def test_fronts_and_flags_on_a_problem_in_which_nothing_fits():
+    """A buffer smaller than any tile set: both Pareto fronts are empty, no group is flagged, and the plain search
+    reports that nothing fits."""
+    cfg = mi.random_tiny_problem(3)
+    arch = dict(cfg["arch"], gb_bytes=2 * cfg["workload"]["word_bytes"])
+    obj = dict(cfg["searches"][0], objective=mi.OBJ_ENERGY, topk=1)
+    assert mm.mmee_pareto_front_bs_da(cfg["workload"], arch, obj) == []
+    assert mm.mmee_pareto_front(cfg["workload"], arch, obj) == []
+    small = dict(cfg, arch=arch)
+    obj = shrink_to(small, obj, 400_000)
+    p = oracle.make_problem(small["workload"], small["arch"], obj)
+    n_groups = (p.t_end - p.t_begin) * p.R // 5
+    assert not _filter_flags(small, obj, 2 ** 62, n_groups).any()
+    with Handle(small, obj) as h:
+        best, _ = mm.mmee_search_host(h)
+    assert best.idx == mm.NO_INDEX and best.status == mm.ERR_NO_FEASIBLE and best.n_feasible == 0

@@ -102,6 +102,12 @@ def test_argument_errors_come_before_any_device_call():
     lib = mm.library()
     assert lib.mmee_destroy(None) == mm.ERR_ARG
     assert lib.mmee_search(None, None, None, None) == mm.ERR_ARG
+    assert lib.mmee_search_host(None, None, None) == mm.ERR_ARG
+    assert lib.mmee_decode(None, 0, None) == mm.ERR_ARG
+    assert lib.mmee_filter_flags(None, None, 0, None) == mm.ERR_ARG
+    n = C.c_uint32(7)
+    assert lib.mmee_pareto_front_bs_da(None, None, None, None, 0, C.byref(n)) == mm.ERR_ARG
+    assert lib.mmee_pareto_front_bs_da(None, None, None, None, 0, None) == mm.ERR_ARG
     assert lib.mmee_query_vector(0, 0, 9, 0, 3, 0, (C.c_uint8 * 8)()) == mm.ERR_ARG
     assert lib.mmee_query_vector(1, 0, 0, 2, 3, 0, (C.c_uint8 * 8)()) == mm.ERR_ARG
 
