@@ -817,7 +817,9 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
         }
         uint32_t groups_walked = 0;
 
-#pragma unroll 1
+        // (the energy-delay search's group loop is unrolled: its body is short; the 64-bit walks' is not)
+        constexpr int kUnrollGroups = (!DUMP && !PRUNE && OBJ == MMEE_OBJ_EDP) ? 5 : 1;
+#pragma unroll kUnrollGroups
         for (int d = 0; d < 5; ++d) {
             if constexpr (PRUNE) {
                 if (!__any_sync(kFull, live && ((kept >> (d * 5)) & 31u))) continue;
