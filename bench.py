@@ -44,7 +44,7 @@ ALG_OPS_PER_ROW = {0: 4.4, 1: 4.4, 2: 10.0}
 LANES_PER_SM = 64          # 4 sub-partitions x 16 lanes: width of the integer-ALU pipe, the busiest pipe of these kernels
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, recorded from the ncu captures summarised under
 # profiles/ (not measured in this run); workload -> objective -> bytes.  None where no capture backs it.
-NCU_DRAM_BYTES_PER_LAUNCH = {"gqa": {1: 212736, 2: 194048}, "llama": {0: 193024, 1: 185856},
+NCU_DRAM_BYTES_PER_LAUNCH = {"gqa": {1: 212736, 2: 205312}, "llama": {0: 193024, 1: 185856},
                              "bert": {0: 192512, 1: 212224}}
 
 
