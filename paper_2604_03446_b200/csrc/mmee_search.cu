@@ -96,8 +96,12 @@ struct alignas(16) TilingTab {
                             // entries 9..11: the least of the three entries of each sm1
     int32_t live;           // smallest possible buffer need of this tiling fits
     int32_t pad[3];
+    // energy-delay search: single-precision lower bounds (rounded down) of wmin[0], wmin[1], qmin[0], qmin[1],
+    // qmin[2], the least of C1w[0..2], cw and smx
+    float fl[8];
 };
 static_assert(offsetof(TilingTab, Qrel) % 16 == 0 && sizeof(int32_t[12]) % 16 == 0, "Qrel rows are read as int4");
+static_assert(offsetof(TilingTab, fl) % 16 == 0, "fl is read as two float4");
 static_assert(offsetof(RowTab, Ec) % 16 == 0 && offsetof(OrderTab, rt) % 16 == 0 && sizeof(RowTab) % 16 == 0,
               "Ec rows are read as int4");
 // 21 items per tiling: 9 stationary pairs x 2 recompute flags, 3 unfused Op1 terms
@@ -451,6 +455,12 @@ __device__ __forceinline__ void build_order_item(const Plan& p, const TilingTab*
         c[1] = l ? size32(bs) : 0;
         c[2] = term32(scale * v0);
         c[3] = term32(scale * v1);
+        if constexpr (OBJ == MMEE_OBJ_EDP) {
+            // the energy-delay filter's first level: DRAM words as single-precision lower bounds (their energy is
+            // the same words times the cost of a DRAM word)
+            c[2] = __float_as_int(__ll2float_rd(v0));
+            c[3] = __float_as_int(__ll2float_rd(v1));
+        }
     } else if (item < 15) {                            // C
         const int64_t bs = monomial(q.bs[order][OP_C][l]);
         ot->C1[l] = bs;
@@ -494,6 +504,7 @@ __device__ __forceinline__ void build_order_item(const Plan& p, const TilingTab*
         // energy of an unfused task's C round trip: read-back, write, and the separate softmax pass of phi = 2
         ot->gXc[0] = term32(p.c_dram_gb * (v + tb->cw));
         ot->gXc[1] = term32(p.c_dram_gb * (v + tb->cw + tb->smx));
+        if constexpr (OBJ == MMEE_OBJ_EDP) ot->gXc[0] = __float_as_int(__ll2float_rd(v));
     }
 }
 
@@ -765,10 +776,18 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
                                                     CtaShared* cs, long long* global_g, int k, int lane,
                                                     int64_t* __restrict__ dump, uint64_t dump_origin, uint32_t& visits,
                                                     uint32_t& tested, unsigned char* flags) {
-    const RowTab* rt = &ot->rt[c.phi == 0 ? 0 : 1];
+    // The energy-delay search sets a middle level up from the 32-bit tables alone (saturated sizes as in the
+    // threshold-relative walk, single-precision lower bounds of the DRAM words); the other walks need the exact terms.
+    constexpr bool FAST = !DUMP && OBJ == MMEE_OBJ_EDP;
+    const bool fused = c.phi == 0;
+    const RowTab* rt = &ot->rt[fused ? 0 : 1];
     LaneThreshold th = load_threshold(wt, cs, k);
     if constexpr (FLAGS) { th.T1 = p.key_cap; th.ti = UINT64_MAX; th.delta = 0; }
     uint32_t rows = 0;
+    const int4 av = FAST ? *reinterpret_cast<const int4*>(ot->Ac[c.la]) : make_int4(0, 0, 0, 0);
+    const int a1c = av.x, a2c = fused ? av.y : 0;
+    const int capc = (int)p.cap_words;
+    const float cdf = FAST ? __ll2float_rd(p.c_dram_gb) : 0.f;        // cost of a DRAM word, rounded down
     int E1c[5], E2c[5];
     float Egf[5], Eef[5];       // EDP: lower bounds of E's DRAM words and of their energy
 #pragma unroll
@@ -781,24 +800,57 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
     for (int mi = 0; mi < (PRUNE ? 1 : 5); ++mi) {
         const int m = PRUNE ? (int)kept_mid : mi;
         const uint64_t mid_first_idx = task_first_idx + (uint64_t)(m * 225);
-        const MidExact me = mid_exact<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, live);
-        int64_t W[9], Q[9];
+        MidExact me{};
+        int64_t W[9] = {}, Q[9] = {};
+        if constexpr (!FAST) {
+            me = mid_exact<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, live);
 #pragma unroll
-        for (int s = 0; s < 9; ++s) {
-            W[s] = me.wptr[2 * s];
-            Q[s] = me.qptr[2 * s];
+            for (int s = 0; s < 9; ++s) {
+                W[s] = me.wptr[2 * s];
+                Q[s] = me.qptr[2 * s];
+            }
         }
         // Energy-delay product: the first filter level is one single-precision lower bound per row,
         // (row energy + least stationary-pair energy) * max(row DRAM words + least Op1 stage, least compute
         // words + least Op1 stage), every conversion, sum and product rounded down, against the threshold
         // rounded up: no mapping of a row is below its row's bound.
+        // All terms are non-negative, so a sum or product of rounded-down terms, itself rounded down, stays a
+        // lower bound.  The energy of the task's DRAM words is their number times the cost of a word.
         double dthr = 0.0;
         float fthr = 0.f, fe0 = 0.f, fx0 = 0.f, fq = 0.f;
-        if constexpr (!DUMP && OBJ == MMEE_OBJ_EDP) {
-            const int64_t pmin = min(me.P[0], min(me.P[1], me.P[2]));
-            fe0 = __ll2float_rd(me.xe0 + tb->wmin[me.rc]);
-            fx0 = __ll2float_rd(me.x0 + pmin);
-            fq = __ll2float_rd(tb->qmin[c.phi == 0 ? me.rc : 2u] + pmin);
+        int slack1c, slack2c;
+        if constexpr (FAST) {
+            const int4 bv = *reinterpret_cast<const int4*>(ot->Bc[fused ? c.lb : (uint32_t)m]);
+            const int2 cv = *reinterpret_cast<const int2*>(ot->Cc[fused ? m : 0]);
+            // (a lane without a live task may read the constant tables of a tiling that cannot fit)
+            const uint32_t rc = (fused && live) ? ((uint32_t)cv.y & 1u) : 0u;
+            // Eq. (1)/(2) in saturated 32-bit sizes: a retained operand of the other operator keeps its space
+            int y1 = __viaddmin_s32(a1c, bv.x, kSizeCap);
+            y1 = __viaddmin_s32(y1, cv.x, kSizeCap);
+            int y2 = __viaddmin_s32(a2c, fused ? bv.y : 0, kSizeCap);
+            y2 = __viaddmin_s32(y2, cv.x, kSizeCap);
+            slack1c = live ? max(capc - y1, -1) : -1;       // (a lane without a live task: none of its rows fits)
+            slack2c = live ? max(capc - y2, -1) : -1;
+            const float4 t0 = *reinterpret_cast<const float4*>(&tb->fl[0]);
+            const float4 t1 = *reinterpret_cast<const float4*>(&tb->fl[4]);
+            const float fgab = __fadd_rd(__int_as_float(rc ? av.w : av.z), __int_as_float(rc ? bv.w : bv.z));
+            if (fused) {
+                fx0 = fgab;
+                fe0 = __fadd_rd(__fmul_rd(cdf, fgab), rc ? t0.y : t0.x);
+                fq = rc ? t0.w : t0.z;
+            } else {
+                // unfused: least Op1 stage max(DRAM words of A and B + C write-back, least Op1 compute words) plus the
+                // softmax pass; the row's DRAM words start from the C read-back
+                const float fgcr = __int_as_float(ot->gXc[0]);
+                const float fpass = c.phi == 2 ? t1.w : 0.f;
+                const float fp = __fadd_rd(fmaxf(__fadd_rd(fgab, t1.z), t1.y), fpass);
+                fx0 = __fadd_rd(fgcr, fp);
+                fq = __fadd_rd(t1.x, fp);
+                fe0 = __fadd_rd(__fmul_rd(cdf, __fadd_rd(__fadd_rd(fgab, fgcr), __fadd_rd(t1.z, fpass))), t0.x);
+            }
+        } else {
+            slack1c = me.slack1 < 0 ? -1 : (int)me.slack1;      // slack <= capacity < 2^30
+            slack2c = me.slack2 < 0 ? -1 : (int)me.slack2;
         }
         auto refresh = [&]() {
             if constexpr (OBJ == MMEE_OBJ_EDP) {
@@ -809,9 +861,7 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
             }
         };
         refresh();
-        const int slack1c = me.slack1 < 0 ? -1 : (int)me.slack1;      // slack <= capacity < 2^30
-        const int slack2c = me.slack2 < 0 ? -1 : (int)me.slack2;
-        if constexpr (!DUMP && OBJ == MMEE_OBJ_EDP) {
+        if constexpr (FAST) {
             // no lane has room left for D and E at this middle level: none of its 25 rows fits
             if (!__any_sync(kFull, (slack1c | slack2c) >= 0)) continue;
         }
@@ -1308,6 +1358,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                 for (int s = 0; s < 9; ++s)
                     if ((p.sm_mask >> s) & 1u) m = src[2 * s] < m ? src[2 * s] : m;
                 tb->qmin[v] = m;
+                if constexpr (OBJ == MMEE_OBJ_EDP) tb->fl[2 + v] = __ll2float_rd(m);
                 for (int s = 0; s < 9; ++s) {
                     const int64_t qd = src[2 * s] - m;
                     const int64_t qs = qd >> p.rel_shift;
@@ -1332,6 +1383,15 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                 for (int s = 0; s < 9; ++s)
                     if ((p.sm_mask >> s) & 1u) m = tb->W[s][rc] < m ? tb->W[s][rc] : m;
                 tb->wmin[rc] = m;
+                if constexpr (OBJ == MMEE_OBJ_EDP) {
+                    tb->fl[rc] = __ll2float_rd(m);
+                    if (rc == 0) {
+                        const int64_t c1 = min(tb->C1w[0], min(tb->C1w[1], tb->C1w[2]));
+                        tb->fl[5] = __ll2float_rd(c1);
+                        tb->fl[6] = __ll2float_rd(tb->cw);
+                        tb->fl[7] = __ll2float_rd(tb->smx);
+                    }
+                }
             }
         }
     };
