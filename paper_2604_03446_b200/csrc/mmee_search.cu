@@ -94,8 +94,9 @@ struct alignas(16) TilingTab {
     int64_t qmin[3];        // min over the stationary pairs of CB[.][0], CB[.][1], QU[.][0]
     int32_t Qrel[3][12];    // CB[s][0], CB[s][1], QU[s][0] minus that minimum, saturated to kTermCap (kUnfit: pair not offered);
                             // entries 9..11: the least of the three entries of each sm1
+    int64_t c1min;          // least C1w over the sm1 that have an offered pair
     int32_t live;           // smallest possible buffer need of this tiling fits
-    int32_t pad[3];
+    int32_t pad[1];
     // energy-delay search: single-precision lower bounds (rounded down) of wmin[0], wmin[1], qmin[0], qmin[1],
     // qmin[2], the least of C1w[0..2], cw and smx
     float fl[8];
@@ -522,7 +523,7 @@ __device__ __forceinline__ void build_tiling_head(const Plan& p, uint64_t t, Til
     const int64_t td = (int64_t)b[6] * b[7], te = (int64_t)b[4] * b[7];
     const int64_t need1 = ta + tbb + tc, need2 = tc + td + te;
     tb->live = ((need1 > need2 ? need1 : need2) <= p.cap_words) ? 1 : 0;
-    tb->pad[0] = tb->pad[1] = tb->pad[2] = 0;
+    tb->pad[0] = 0;
 }
 
 // One thread per (tiling slot, operator, stationary mode): words and cycles of one tile (the only part of the
@@ -1059,19 +1060,26 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
                     // offers, least (Op1 stage + Op2 compute words) over the offered pairs.
                     const int64_t da1 = ot->gA[c.la][0] + ot->gB[m][0] + tb->cw;
                     const int64_t pass = c.phi == 2 ? tb->smx : 0;
-                    const int4 qr = *reinterpret_cast<const int4*>(&tb->Qrel[2][8]);     // [9..11]: least term by sm1
-                    int um = kRowCap, qm = INT_MAX;
+                    // With the least stage over the offered sm1 (all 32-bit forms are monotone in the stage): the
+                    // DRAM-side bound is the least over the sm1, and the compute-side gate a lower bound of every
+                    // sm1's.  Only when that gate lets the middle level through are the three sm1 looked at.
+                    const int64_t c1m = tb->c1min;
+                    const int64_t pm = (da1 > c1m ? da1 : c1m) + pass - thr;
+                    u = kRowCap;
+                    if (rel32((tb->qmin[2] + pm) >> p.rel_shift) < 0) {
+                        const int um = rel32((ot->gCr + pm) >> p.rel_shift);
+                        const int4 qr = *reinterpret_cast<const int4*>(&tb->Qrel[2][8]);     // [9..11]: least term by sm1
+                        int qm = INT_MAX;
 #pragma unroll
-                    for (int j = 0; j < 3; ++j) {
-                        const int64_t c1w = tb->C1w[j];
-                        const int64_t pj = (da1 > c1w ? da1 : c1w) + pass - thr;
-                        const int uaj = rel32((ot->gCr + pj) >> p.rel_shift);
-                        const int qoj = rel32((tb->qmin[2] + pj) >> p.rel_shift);
-                        const int qrj = j == 0 ? qr.y : (j == 1 ? qr.z : qr.w);
-                        um = min(um, qrj < kUnfit ? uaj : kRowCap);
-                        qm = min(qm, qoj + qrj);
+                        for (int j = 0; j < 3; ++j) {
+                            const int64_t c1w = tb->C1w[j];
+                            const int64_t pj = (da1 > c1w ? da1 : c1w) + pass - thr;
+                            const int qoj = rel32((tb->qmin[2] + pj) >> p.rel_shift);
+                            const int qrj = j == 0 ? qr.y : (j == 1 ? qr.z : qr.w);
+                            qm = min(qm, qoj + qrj);
+                        }
+                        u = qm < 0 ? um : kRowCap;
                     }
-                    u = qm < 0 ? um : kRowCap;
                 }
             }
         };
@@ -1370,6 +1378,12 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                 for (int j2 = 0; j2 < 3; ++j2) {
                     const int32_t* r = &tb->Qrel[v][3 * j2];
                     tb->Qrel[v][9 + j2] = min(r[0], min(r[1], r[2]));
+                }
+                if (v == 2) {
+                    int64_t c1 = kInfKey;
+                    for (int j2 = 0; j2 < 3; ++j2)
+                        if ((p.sm_mask >> (3 * j2)) & 7u) c1 = tb->C1w[j2] < c1 ? tb->C1w[j2] : c1;
+                    tb->c1min = c1;
                 }
             }
         }
