@@ -80,13 +80,8 @@ int choose_launch_shape(const Plan& p, int device, uint32_t search_tpt, uint32_t
     if (max_ctas && grid > max_ctas) return MMEE_ERR_RANGE;
     shape->grid = (uint32_t)grid;
     shape->n_ranges = ranges;
-    // golden-ratio stride, moved to the next value coprime to the number of ranges
-    uint64_t stride = ranges > 2 ? (uint64_t)((double)ranges * 0.6180339887498949) : 1;
-    if (stride < 1) stride = 1;
-    auto gcd = [](uint64_t a, uint64_t b) { while (b) { const uint64_t t = a % b; a = b; b = t; } return a; };
-    while (ranges > 1 && gcd(stride, ranges) != 1) ++stride;
-    shape->range_stride = ranges > 1 ? stride % ranges : 0;
-    if (ranges > 1 && shape->range_stride == 0) shape->range_stride = 1;
+    // one spread range per CTA while at least as many ranges remain for the ascending part
+    shape->n_spread = grid < ranges / 2 ? grid : ranges / 2;
     return MMEE_OK;
 }
 

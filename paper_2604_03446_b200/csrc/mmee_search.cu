@@ -185,6 +185,21 @@ __device__ __forceinline__ void reg_merge(int64_t& ek, uint64_t& ei, int k, int6
     if (lane >= k) { ek = kInfKey; ei = UINT64_MAX; }
 }
 
+// Ascending sort of 32 (key, idx) pairs, one per lane (a bitonic network of 15 compare-exchange stages).  All 32
+// lanes call this converged.
+__device__ __forceinline__ void warp_sort_pairs(int64_t& ck, uint64_t& ci, int lane) {
+#pragma unroll
+    for (int size = 2; size <= 32; size <<= 1) {
+#pragma unroll
+        for (int stride = size >> 1; stride >= 1; stride >>= 1) {
+            const int64_t pk = __shfl_xor_sync(kFull, ck, stride);
+            const uint64_t pi = __shfl_xor_sync(kFull, ci, stride);
+            const bool keep_smaller = ((lane & size) == 0) == ((lane & stride) == 0);
+            if (pair_less(pk, pi, ck, ci) == keep_smaller) { ck = pk; ci = pi; }
+        }
+    }
+}
+
 // The other list has n entries, lane j holding entry j: by insertion when it is short, else by the merge above.
 __device__ __forceinline__ void reg_absorb(int64_t& ek, uint64_t& ei, int k, int n, int64_t ok, uint64_t oi, int lane) {
     if (n > 3) {
@@ -353,6 +368,11 @@ __device__ __forceinline__ unsigned edp_row_test(double de, const double (&dl)[3
     return hit;
 }
 
+#ifndef MMEE_BULK_MIN
+#define MMEE_BULK_MIN 3
+#endif
+constexpr int kBulkMin = MMEE_BULK_MIN;     // more pending candidates than this are merged in one step
+
 // Rare path: some lane of the warp has a key below its threshold in this row.  Every lane
 // re-evaluates its nine candidates of the row from the shared tables and the warp inserts the
 // passing ones, one at a time, into its sorted list.
@@ -369,6 +389,28 @@ __device__ __noinline__ int64_t slow_row(WarpTop* wt, CtaShared* cs, long long* 
         while (true) {
             const unsigned m = __ballot_sync(kFull, pend);
             if (!m) break;
+            if (__popc(m) > kBulkMin) {
+                // Many lanes at once (an empty list at the start of a search, or mappings tied at the threshold):
+                // the pending candidates are sorted across the lanes and merged into the list in one step.
+                int64_t ck = pend ? key : kInfKey;
+                uint64_t ci = pend ? row_first_idx + (uint64_t)s : UINT64_MAX;
+                warp_sort_pairs(ck, ci, lane);
+                const int count = wt->count;
+                int64_t ek = kInfKey;
+                uint64_t ei = UINT64_MAX;
+                if (lane < count) {
+                    const longlong2 own = wt->e[lane];
+                    ek = own.x; ei = (uint64_t)own.y;
+                }
+                reg_merge(ek, ei, k, ck, ci, lane);
+                const int n_new = min(k, count + __popc(m));
+                __syncwarp();
+                if (lane < n_new) wt->e[lane] = make_longlong2((long long)ek, (long long)ei);
+                if (lane == 0) wt->count = n_new;
+                __syncwarp();
+                thr = lane_threshold(wt, cs, k, row_first_idx);
+                break;          // every pending candidate has been considered
+            }
             const int leader = __ffs(m) - 1;
             const int64_t lk = __shfl_sync(kFull, key, leader);
             const uint64_t li = __shfl_sync(kFull, row_first_idx + (uint64_t)s, leader);
@@ -649,7 +691,7 @@ __device__ __forceinline__ MidExact mid_exact(const Plan& p, const TilingTab* tb
 // Every lane finds its rows that hold a passing candidate, exactly, and the warp inserts them.
 template <int OBJ>
 __device__ __noinline__ void exact_group(const Plan& p, const TilingTab* tb, const OrderTab* ot, uint32_t phi, uint32_t la,
-                                         uint32_t lb_task, int m, int d, bool live, uint32_t kept,
+                                         uint32_t lb_task, int m, int d, uint32_t rows, bool live, uint32_t kept,
                                          uint64_t task_first_idx, WarpTop* wt, CtaShared* cs, long long* global_g, int k,
                                          int lane) {
     // The other CTAs' bound, read afresh: a lane that visits this path with a stale threshold would come back for
@@ -663,6 +705,7 @@ __device__ __noinline__ void exact_group(const Plan& p, const TilingTab* tb, con
     const int64_t xed = (OBJ >= MMEE_OBJ_EDP) ? me.xe0 + rt->D[d][3] : 0;
 #pragma unroll 1
     for (int e = 0; e < 5; ++e) {
+        if (!((rows >> e) & 1u)) continue;      // the filter flagged this row in no lane
         const bool fit = (rt->E[e][0] <= s1) && (rt->E[e][1] <= s2) && ((kept >> (d * 5 + e)) & 1u);
         const int64_t x = xd + rt->E[e][2];
         const int64_t xe = (OBJ >= MMEE_OBJ_EDP) ? xed + rt->E[e][3] : 0;
@@ -686,9 +729,9 @@ __device__ __noinline__ void exact_group(const Plan& p, const TilingTab* tb, con
 // (key, idx) pair, and one lane replaces the list's entry if that pair precedes it.
 template <int OBJ>
 __device__ __noinline__ void exact_group_single(const Plan& p, const TilingTab* tb, const OrderTab* ot, uint32_t phi,
-                                                uint32_t la, uint32_t lb_task, int m, int d, bool live, uint32_t kept,
-                                                uint64_t task_first_idx, WarpTop* wt, CtaShared* cs, long long* global_g,
-                                                int lane) {
+                                                uint32_t la, uint32_t lb_task, int m, int d, uint32_t rows, bool live,
+                                                uint32_t kept, uint64_t task_first_idx, WarpTop* wt, CtaShared* cs,
+                                                long long* global_g, int lane) {
     // The other CTAs' bound, read afresh: a lane that visits this path with a stale threshold would come back for
     // every group.  The load is consumed at the end of the visit, before the caller renews its threshold.
     const long long g_now = (lane == 0) ? *reinterpret_cast<volatile long long*>(global_g) : 0;
@@ -702,6 +745,7 @@ __device__ __noinline__ void exact_group_single(const Plan& p, const TilingTab* 
     uint32_t best_pos = 0;
 #pragma unroll 1
     for (int e = 0; e < 5; ++e) {
+        if (!((rows >> e) & 1u)) continue;      // the filter flagged this row in no lane
         const bool fit = (rt->E[e][0] <= s1) && (rt->E[e][1] <= s2) && ((kept >> (d * 5 + e)) & 1u);
         const int64_t x = xd + rt->E[e][2];
         const int64_t xe = (OBJ >= MMEE_OBJ_EDP) ? xed + rt->E[e][3] : 0;
@@ -714,11 +758,18 @@ __device__ __noinline__ void exact_group_single(const Plan& p, const TilingTab* 
     uint64_t best_idx = task_first_idx + (uint64_t)(m * 225 + d * 45) + best_pos;
     // a key above the CTA-wide bound cannot be the optimum; an infeasible or capped-out lane holds kInfKey > G
     if (best > cs->G) { best = kInfKey; best_idx = UINT64_MAX; }
-#pragma unroll
-    for (int off = 16; off; off >>= 1) {
-        const int64_t ok = __shfl_xor_sync(kFull, best, off);
-        const uint64_t oi = __shfl_xor_sync(kFull, best_idx, off);
-        if (pair_less(ok, oi, best, best_idx)) { best = ok; best_idx = oi; }
+    // The smallest (key, idx) pair of the warp by four 32-bit warp minima: the key's high and low words (keys are
+    // non-negative), then the index's among the lanes that hold that key.  Every lane ends up with the pair.
+    {
+        const uint32_t kh = __reduce_min_sync(kFull, (uint32_t)((uint64_t)best >> 32));
+        const bool m1 = (uint32_t)((uint64_t)best >> 32) == kh;
+        const uint32_t kl = __reduce_min_sync(kFull, m1 ? (uint32_t)best : 0xffffffffu);
+        const bool m2 = m1 && (uint32_t)best == kl;
+        const uint32_t ih = __reduce_min_sync(kFull, m2 ? (uint32_t)(best_idx >> 32) : 0xffffffffu);
+        const bool m3 = m2 && (uint32_t)(best_idx >> 32) == ih;
+        const uint32_t il = __reduce_min_sync(kFull, m3 ? (uint32_t)best_idx : 0xffffffffu);
+        best = (int64_t)(((uint64_t)kh << 32) | kl);
+        best_idx = ((uint64_t)ih << 32) | il;
     }
     if (lane == 0 && best != kInfKey && (wt->count == 0 || pair_less(best, best_idx, top_key(wt, 0), top_idx(wt, 0)))) {
         top_set(wt, 0, best, best_idx);
@@ -736,7 +787,7 @@ __device__ __noinline__ void exact_group_single(const Plan& p, const TilingTab* 
 // mapping of the group's five rows in double precision on the FP64 pipe (energy and latency sums converted once per
 // row, then an add, two multiplies and two compares per mapping).  Each approximate product is within a few 2^-53
 // of the exact key, so comparing against the threshold widened by 1e-14 relative can flag a row needlessly but never
-// miss one; the exact path decides.  Returns 1 if some row fits and holds such a product.
+// miss one; the exact path decides.  Returns the mask of the rows that fit and hold such a product.
 __device__ __noinline__ unsigned edp_group_test(const Plan& p, const TilingTab* tb, const OrderTab* ot, uint32_t phi,
                                                 uint32_t la, uint32_t lb_task, int m, bool live, int d, int s1c, int s2c,
                                                 uint32_t kept_rows, double dthr) {
@@ -763,7 +814,7 @@ __device__ __noinline__ unsigned edp_group_test(const Plan& p, const TilingTab* 
         double dl[3];
 #pragma unroll
         for (int j = 0; j < 3; ++j) dl[j] = (double)(x + me.P[j]);
-        hit_any |= edp_row_test(de, dl, dW, dQP, dthr, fit & 1u);
+        hit_any |= edp_row_test(de, dl, dW, dQP, dthr, fit & 1u) << e;
     }
     return hit_any;
 }
@@ -917,7 +968,7 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
                     row_test(key, thr, rt->E[e][0], s1, rt->E[e][1], s2, fit, hit);
                     if constexpr (PRUNE) { fit &= kept >> (d * 5 + e); hit &= fit; }
                     fits += fit;
-                    hit_any |= hit;
+                    hit_any |= hit << e;
                     if (DUMP) {
                         if (valid) {
 #pragma unroll
@@ -932,8 +983,9 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
                 if (hit_any && flags) flags[m * 5 + d] = 1;
             } else if (__any_sync(kFull, hit_any != 0u)) {
                 ++visits;
-                if (k == 1) exact_group_single<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, lane);
-                else exact_group<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, k, lane);
+                const uint32_t rows = __reduce_or_sync(kFull, hit_any);     // the rows that some lane's filter flags
+                if (k == 1) exact_group_single<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, rows, live, kept, task_first_idx, wt, cs, global_g, lane);
+                else exact_group<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, rows, live, kept, task_first_idx, wt, cs, global_g, k, lane);
                 th = load_threshold(wt, cs, k);
                 refresh();
             }
@@ -1084,6 +1136,8 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
             }
         };
         mid_setup();
+        // (u is a value from here on: the compiler must not form it again from its inputs in every group)
+        asm volatile("" : "+r"(u));
 
 #pragma unroll
         for (int d = 0; d < 5; ++d) {
@@ -1123,10 +1177,23 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
                 if (hit && flags) flags[m * 5 + d] = 1;
             } else if (__any_sync(kFull, hit)) {
                 ++visits;
-                if (k == 1) exact_group_single<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, lane);
-                else exact_group<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, live, kept, task_first_idx, wt, cs, global_g, k, lane);
+                // the rows that some lane's bound flags: the exact path looks at no other
+                // (the row terms are formed again, through an opaque instruction, so that the five of the common
+                // path need not stay in registers for this rare one)
+                uint32_t rows = 0;
+#pragma unroll
+                for (int e = 0; e < 5; ++e) {
+                    int t;
+                    asm volatile("shr.s32 %0, %1, 31;" : "=r"(t) : "r"(imad(E2c[e], minus_one, e == 0 ? lim_l3 : lim_retained)));
+                    if constexpr (PRUNE) t |= (int)((kd >> e) & 1u) - 1;
+                    rows |= (uc + (Gc[e] | (t & kUnfit)) < 0) ? (1u << e) : 0u;
+                }
+                rows = __reduce_or_sync(kFull, rows);
+                if (k == 1) exact_group_single<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, rows, live, kept, task_first_idx, wt, cs, global_g, lane);
+                else exact_group<OBJ>(p, tb, ot, c.phi, c.la, c.lb, m, d, rows, live, kept, task_first_idx, wt, cs, global_g, k, lane);
                 rebase(m * 225 + d * 45 + 45);
                 mid_setup();
+                asm volatile("" : "+r"(u));
             }
         }
     }
@@ -1290,9 +1357,11 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
     uint32_t my_visits = 0;
     uint32_t my_tested = 0;       // rows whose capacity test and bound this lane evaluated (fewer than 2^32 per lane)
 
-    // Builder: pull the next range and build its tables into buffer `buf`.  Ranges are visited in a
-    // stride-permuted order (stride coprime to their number), so that the first pull of every CTA
-    // samples the whole index space and the pruning bound G is near its final value from the start.
+    // Builder: pull the next range and build its tables into buffer `buf`.  The first n_spread pulls (one per
+    // CTA) take ranges spread evenly over the index space, so that the pruning bound G is near its final value
+    // from the start; the other ranges follow in ascending order.  Ascending matters where many mappings tie at
+    // the best key (latency at the compute bound): a tie enters a list only with a lower index than the list's last
+    // entry, and in ascending order the later candidates never have one.
     // `coop` (a std::bool_constant): the whole CTA builds together (the first range, when there is nothing to walk
     // yet) instead of the builder warp alone.
     auto build_next = [&](int buf, auto coop) {
@@ -1302,9 +1371,20 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
         auto sync = [] { if constexpr (COOP) __syncthreads(); else __syncwarp(); };
         if (first == 0) {
             const unsigned long long got = atomicAdd(&scratch->next_task, 1ull);
-            cs->range_begin[buf] = got < shape.n_ranges
-                                       ? task_begin + ((got * shape.range_stride) % shape.n_ranges) * shape.range_tasks
-                                       : task_end;
+            // pull number -> range: multiples of `step` first, then the ranges between them, then the tail
+            uint64_t range = got;
+            if (shape.n_spread && got < shape.n_ranges) {
+                const uint64_t step = shape.n_ranges / shape.n_spread;       // >= 2
+                if (got < shape.n_spread) {
+                    range = got * step;
+                } else {
+                    const uint64_t r = got - shape.n_spread;
+                    const uint64_t block = r / (step - 1), offset = r % (step - 1);
+                    range = block < shape.n_spread ? block * step + 1 + offset
+                                                   : shape.n_spread * step + (r - shape.n_spread * (step - 1));
+                }
+            }
+            cs->range_begin[buf] = got < shape.n_ranges ? task_begin + range * shape.range_tasks : task_end;
             cs->cursor[buf] = 0;
         }
         sync();

@@ -44,7 +44,8 @@ struct LaunchShape {
     uint32_t pad;
     const PrunedTask* pruned;   // device: the kept tasks of a tiling (row pruning), else null
     uint64_t n_ranges;      // ranges of the searched task interval
-    uint64_t range_stride;  // ranges are visited as (i * range_stride) mod n_ranges; coprime to n_ranges
+    uint64_t n_spread;      // the first n_spread pulls take ranges spread evenly over the interval (multiples of
+                            // n_ranges / n_spread >= 2), the others follow in ascending order; 0: ascending only
 };
 
 inline size_t scratch_bytes(uint32_t grid) { return sizeof(Scratch) + (size_t)(grid ? grid - 1 : 0) * sizeof(Partial); }
