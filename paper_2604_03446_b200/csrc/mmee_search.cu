@@ -1220,6 +1220,26 @@ __device__ __noinline__ void finalize_step(const Plan& p, Scratch* __restrict__ 
     // bound G it knew at its end.  Each warp then merges the non-empty lists among its 32, eight at a time
     // (lane j takes entry j of each; the loads bypass the L1 cache).
     constexpr int kBatch = 8;
+    if (k == 1) {
+        // A single optimum: every thread reads the only entry of its lists (all loads in flight at once), and the
+        // warp's smallest pair is found by four 32-bit warp minima (key high / low word, index high / low word).
+        for (int c = tid; c < n_partials; c += kSearchThreads) {
+            if (__ldcg(&scratch->partial[c].count) > 0) {
+                const longlong2 head = __ldcg(&scratch->partial[c].e[0]);
+                if (pair_less(head.x, (uint64_t)head.y, ek, ei)) { ek = head.x; ei = (uint64_t)head.y; }
+            }
+        }
+        const uint32_t kh = __reduce_min_sync(kFull, (uint32_t)((uint64_t)ek >> 32));
+        const bool m1 = (uint32_t)((uint64_t)ek >> 32) == kh;
+        const uint32_t kl = __reduce_min_sync(kFull, m1 ? (uint32_t)ek : 0xffffffffu);
+        const bool m2 = m1 && (uint32_t)ek == kl;
+        const uint32_t ih = __reduce_min_sync(kFull, m2 ? (uint32_t)(ei >> 32) : 0xffffffffu);
+        const bool m3 = m2 && (uint32_t)(ei >> 32) == ih;
+        const uint32_t il = __reduce_min_sync(kFull, m3 ? (uint32_t)ei : 0xffffffffu);
+        // (lane 0 holds the warp's entry, the other lanes the empty pair)
+        ek = lane == 0 ? (int64_t)(((uint64_t)kh << 32) | kl) : kInfKey;
+        ei = lane == 0 ? (((uint64_t)ih << 32) | il) : UINT64_MAX;
+    } else
     for (int c0 = 0; c0 < n_partials; c0 += kSearchThreads) {
         const int c = c0 + tid;
         const int len = c < n_partials ? __ldcg(&scratch->partial[c].count) : 0;
@@ -1241,7 +1261,14 @@ __device__ __noinline__ void finalize_step(const Plan& p, Scratch* __restrict__ 
             // (unrolled: with a run-time index the batch would live in local memory, and the store of each
             // loaded entry there would wait for its load before the next load could issue)
 #pragma unroll
-            for (int i = 0; i < kBatch; ++i) reg_absorb(ek, ei, k, n[i], mine[i].x, (uint64_t)mine[i].y, lane);
+            for (int i = 0; i < kBatch; ++i) {
+                // a list whose first entry does not precede this warp's k-th entry adds nothing
+                const int64_t kth_key = __shfl_sync(kFull, ek, k - 1), head_key = __shfl_sync(kFull, mine[i].x, 0);
+                const uint64_t kth_idx = __shfl_sync(kFull, ei, k - 1);
+                const uint64_t head_idx = (uint64_t)__shfl_sync(kFull, mine[i].y, 0);
+                if (n[i] > 0 && pair_less(head_key, head_idx, kth_key, kth_idx))
+                    reg_absorb(ek, ei, k, n[i], mine[i].x, (uint64_t)mine[i].y, lane);
+            }
         }
     }
     // The warps' lists are merged pairwise into warp 0's.
