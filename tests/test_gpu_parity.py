@@ -292,6 +292,22 @@ def test_sub_ranges_partition_the_search():
     assert sorted(bests)[:len(found)] == [(r.e_key, r.idx) for r in found]
 
 
+@pytest.mark.parametrize("n_tilings", [1, 2, 3, 5, 7, 9, 12, 23, 64])
+def test_interval_lengths_around_the_range_order_cases(n_tilings):
+    """The kernel's CTAs pull ranges of the task interval in a two-part order (some spread evenly, the others
+    ascending, a tail).  Intervals of 1 to 64 tilings give 1 to about 30 ranges (odd and even counts, with and
+    without a tail): every range must be walked exactly once, which the feasible count and the top-k show."""
+    cfg = mi.config2()
+    obj = dict(cfg["searches"][1], topk=3, t_begin=1000, t_end=1000 + n_tilings)
+    check_search(cfg, obj)
+
+
+def test_interval_with_more_ranges_than_ctas_but_fewer_than_twice_as_many():
+    """About 420 ranges on a grid of at most 296 CTAs: the spread part is half the ranges, not one per CTA."""
+    cfg = mi.config2()
+    check_search(cfg, dict(cfg["searches"][0], topk=2, t_begin=300, t_end=1200))
+
+
 def test_nothing_fits():
     cfg = mi.random_tiny_problem(3)
     arch = dict(cfg["arch"], gb_bytes=cfg["workload"]["word_bytes"] * 2)
