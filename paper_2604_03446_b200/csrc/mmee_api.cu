@@ -52,20 +52,39 @@ int choose_launch_shape(const Plan& p, int device, uint32_t search_tpt, uint32_t
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
     if (e != cudaSuccess) return cuda_status(e);
     // A task is 1125 mappings (225 with row pruning, where the searched units are single middle levels).
-    const uint32_t rounds = p.row_pruning ? 9 : 3;
-    shape->range_tasks = rounds * kWorkerThreads;
     shape->search_tpt = search_tpt;
-    shape->pad = 0;
     shape->pruned = nullptr;
-    shape->slots = (shape->range_tasks - 1) / search_tpt + 2;
-    size_t smem = search_smem_bytes(p, shape->slots);
-    // Many small tilings per range need many table slots: shrink the range until they fit.
-    // (Worker warps take 32 tasks at a time, so a range may be as short as one warp's share.)
-    while (smem > 110 * 1024 && shape->range_tasks > 32) {
-        shape->range_tasks -= shape->range_tasks > (uint32_t)kWorkerThreads ? kWorkerThreads : 32;
-        shape->slots = (shape->range_tasks - 1) / search_tpt + 2;
-        smem = search_smem_bytes(p, shape->slots);
+    // Two CTAs per SM under the 196 KB shared-memory carve-out, which leaves the row loops 60 KB of L1 (the next
+    // carve-out, 228 KB, leaves 28 KB and costs the energy-delay search a tenth of its speed).
+    constexpr size_t kSmemTarget = 97 * 1024;
+    // Ranges of whole tilings, as many as the table slots hold: a tiling's tables are then built once, not once
+    // by each of the two ranges it would straddle, and a range needs no slot for a tiling it only touches.
+    constexpr uint32_t kAlignedMaxTasks = 1024;
+    const uint64_t tilings = p.t_end - p.t_begin;
+    bool aligned = search_tpt <= kAlignedMaxTasks && search_smem_bytes(p, 1) <= kSmemTarget;
+    uint32_t per_range = 1;                          // aligned: tilings of a range
+    if (aligned) {
+        while ((per_range + 1) * search_tpt <= kAlignedMaxTasks && search_smem_bytes(p, per_range + 1) <= kSmemTarget)
+            ++per_range;
+        // (a small problem, with fewer than four such ranges per CTA of a full grid, keeps ranges of a fixed number
+        // of tasks: whole tilings would leave most warps of a CTA without work)
+        if (tilings / per_range < 4ull * 2u * (uint64_t)sm_count) aligned = false;
     }
+    if (aligned) {
+        shape->range_tasks = per_range * search_tpt;
+        shape->slots = per_range;
+    } else {
+        const uint32_t rounds = p.row_pruning ? 9 : 3;
+        shape->range_tasks = rounds * kWorkerThreads;
+        shape->slots = (shape->range_tasks - 1) / search_tpt + 2;
+        // Many small tilings per range need many table slots: shrink the range until they fit.
+        // (Worker warps take 32 tasks at a time, so a range may be as short as one warp's share.)
+        while (search_smem_bytes(p, shape->slots) > kSmemTarget && shape->range_tasks > 32) {
+            shape->range_tasks -= shape->range_tasks > (uint32_t)kWorkerThreads ? kWorkerThreads : 32;
+            shape->slots = (shape->range_tasks - 1) / search_tpt + 2;
+        }
+    }
+    const size_t smem = search_smem_bytes(p, shape->slots);
     if (smem > (size_t)smem_optin) return MMEE_ERR_RANGE;
     shape->smem_bytes = (uint32_t)smem;
     int per_sm = 0;
@@ -73,13 +92,26 @@ int choose_launch_shape(const Plan& p, int device, uint32_t search_tpt, uint32_t
     if (per_sm < 1) return MMEE_ERR_RANGE;
     if (per_sm > 2) per_sm = 2;
     uint64_t grid = (uint64_t)sm_count * (uint32_t)per_sm;
-    const uint64_t tasks = (p.t_end - p.t_begin) * search_tpt;
-    const uint64_t ranges = (tasks + shape->range_tasks - 1) / shape->range_tasks;
+    const uint64_t tasks = tilings * search_tpt;
+    if (aligned) {
+        // The last tilings go out one per range, about half a full range's worth per CTA: the CTAs then finish
+        // within one tiling of each other instead of within one full range.  (Measured with a whole, a half and a
+        // quarter of a range per CTA: the searches differ in which they prefer, by 1 to 3 %.)
+        uint64_t tail = grid * per_range / 2;
+        shape->n_big = (tilings - tail) / per_range;
+        tail = tilings - shape->n_big * per_range;
+        shape->tail_tasks = search_tpt;
+        shape->n_ranges = shape->n_big + tail;
+    } else {
+        shape->n_ranges = (tasks + shape->range_tasks - 1) / shape->range_tasks;
+        shape->n_big = shape->n_ranges;
+        shape->tail_tasks = shape->range_tasks;
+    }
+    const uint64_t ranges = shape->n_ranges;
     if (grid > ranges) grid = ranges ? ranges : 1;
     // (a caller with a fixed scratch: a device that would take more CTAs is refused, not silently under-used)
     if (max_ctas && grid > max_ctas) return MMEE_ERR_RANGE;
     shape->grid = (uint32_t)grid;
-    shape->n_ranges = ranges;
     // one spread range per CTA while at least as many ranges remain for the ascending part
     shape->n_spread = grid < ranges / 2 ? grid : ranges / 2;
     return MMEE_OK;

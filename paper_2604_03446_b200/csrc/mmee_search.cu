@@ -125,6 +125,7 @@ struct alignas(16) CtaShared {
     unsigned long long exact_visits;         // groups that some warp of this CTA took to the exact path
     unsigned long long tested_rows;          // rows whose capacity test and bound were evaluated
     unsigned long long range_begin[2];       // first task of the range whose tables sit in buffer 0 / 1
+    unsigned long long range_end[2];         // one past its last task
     unsigned int cursor[2];                  // next unassigned task of that range, relative to its begin
     unsigned int last_cta;                   // this CTA drew the last ticket: it runs the finalize step
     unsigned int check_failed;               // finalize step: a winner's key is not the key of its evaluation
@@ -1411,13 +1412,20 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
                                                    : shape.n_spread * step + (r - shape.n_spread * (step - 1));
                 }
             }
-            cs->range_begin[buf] = got < shape.n_ranges ? task_begin + range * shape.range_tasks : task_end;
+            // range -> tasks: n_big ranges of range_tasks, then short ones of tail_tasks
+            auto first_task = [&](uint64_t r) {
+                return r <= shape.n_big ? r * shape.range_tasks
+                                        : shape.n_big * shape.range_tasks + (r - shape.n_big) * shape.tail_tasks;
+            };
+            const uint64_t b0 = task_begin + first_task(range), b1 = task_begin + first_task(range + 1);
+            cs->range_begin[buf] = got < shape.n_ranges ? b0 : task_end;
+            cs->range_end[buf] = b1 < task_end ? b1 : task_end;
             cs->cursor[buf] = 0;
         }
         sync();
         const uint64_t r0 = cs->range_begin[buf];
         if (r0 >= task_end) return;
-        const uint64_t r1 = (r0 + shape.range_tasks < task_end) ? r0 + shape.range_tasks : task_end;
+        const uint64_t r1 = cs->range_end[buf];
         const uint64_t t_first = r0 / tpt, t_last = (r1 - 1) / tpt;
         const uint32_t n_slots = (uint32_t)(t_last - t_first + 1);
         TilingTab* ttabs = ttabs_all + buf * shape.slots;
@@ -1526,7 +1534,7 @@ search_kernel(const __grid_constant__ Plan plan_arg, const LaunchShape shape, Sc
         if (r0 >= task_end) break;
         if (builder) build_next(buf ^ 1, std::false_type{});
         {       // every warp walks tasks; the builder warp joins once the next range's tables are done
-        const uint64_t r1 = (r0 + shape.range_tasks < task_end) ? r0 + shape.range_tasks : task_end;
+        const uint64_t r1 = cs->range_end[buf];
         const uint64_t t_first = r0 / tpt;
         const TilingTab* ttabs = ttabs_all + buf * shape.slots;
         const OrderTab* otabs = otabs_all + (size_t)buf * shape.slots * n_orders;

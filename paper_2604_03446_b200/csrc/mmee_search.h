@@ -37,13 +37,14 @@ struct Scratch {
 
 struct LaunchShape {
     uint32_t grid;          // persistent CTAs
-    uint32_t range_tasks;   // tasks a CTA takes per pull (multiple of kWorkerThreads)
+    uint32_t range_tasks;   // tasks a CTA takes per pull: those of `slots` whole tilings where that many fit
     uint32_t slots;         // tilings one range can touch
     uint32_t smem_bytes;
     uint32_t search_tpt;    // tasks per tiling in the searched task space (fewer with row pruning)
-    uint32_t pad;
+    uint32_t tail_tasks;    // tasks of each range from number n_big on (one tiling's; the last ranges are short)
     const PrunedTask* pruned;   // device: the kept tasks of a tiling (row pruning), else null
-    uint64_t n_ranges;      // ranges of the searched task interval
+    uint64_t n_ranges;      // ranges of the searched task interval: n_big of range_tasks, the others of tail_tasks
+    uint64_t n_big;
     uint64_t n_spread;      // the first n_spread pulls take ranges spread evenly over the interval (multiples of
                             // n_ranges / n_spread >= 2), the others follow in ascending order; 0: ascending only
 };
