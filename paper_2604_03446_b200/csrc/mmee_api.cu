@@ -59,7 +59,7 @@ int choose_launch_shape(const Plan& p, int device, uint32_t search_tpt, uint32_t
     constexpr size_t kSmemTarget = 97 * 1024;
     // Ranges of whole tilings, as many as the table slots hold: a tiling's tables are then built once, not once
     // by each of the two ranges it would straddle, and a range needs no slot for a tiling it only touches.
-    constexpr uint32_t kAlignedMaxTasks = 1024;
+    constexpr uint32_t kAlignedMaxTasks = 2048;
     const uint64_t tilings = p.t_end - p.t_begin;
     bool aligned = search_tpt <= kAlignedMaxTasks && search_smem_bytes(p, 1) <= kSmemTarget;
     uint32_t per_range = 1;                          // aligned: tilings of a range

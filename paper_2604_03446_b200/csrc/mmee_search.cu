@@ -47,32 +47,32 @@ constexpr int kRowCap = (1 << 29) - 1;     // upper cap of a row sum: kRowCap + 
 // shared-memory tables
 // ------------------------------------------------------------------------------------------------
 
-// Row-side terms (levels of D and E) of one (tiling, order), in the form the row loop consumes:
-// x1 = buffer words counted while Op1 runs (the operand's size if it is retained, else 0),
-// x2 = buffer words while Op2 runs, g = DRAM words times the objective's scale (energy: quanta
-// per DRAM word; latency / EDP: 1), e = energy-scaled copy (EDP only).  One instance for fused
-// rows, one for unfused rows, so that the loops need no selects.
+// Row-side terms (levels of D and E) of one (tiling, order).  One instance for fused rows, one for unfused rows,
+// so that the loops need no selects.  Per level: g = DRAM words times the objective's scale (energy: quanta per
+// DRAM word; latency / EDP: 1), exact; and the 32-bit forms x1 = buffer words counted while Op1 runs (the
+// operand's size if it is retained, else 0), x2 = buffer words while Op2 runs, both saturated to kSizeCap (which
+// is above every admissible capacity, so "fits" has the same truth value as with the exact size), then g in
+// relative units saturated to kTermCap and an unused word (EDP: single-precision lower bounds of the DRAM words
+// and of their energy).  The energy of the DRAM words, where an objective needs both sides, is g times the cost
+// of a DRAM word: it is formed where it is needed, not stored.
 struct alignas(16) RowTab {
-    int64_t D[5][4];        // per level of D: x1, x2, g, e
-    int64_t E[5][4];        // per level of E: x1, x2, g, e
-    int32_t Dc[5][4];       // x1, x2 saturated to kSizeCap, g saturated to kTermCap, unused
+    int64_t Dg[5], Eg[5];
+    int32_t Dc[5][4];
     int32_t Ec[5][4];
 };
 
 // Per (tiling, order): task-side terms (levels of A, B, C) and the two row tables.
 struct alignas(16) OrderTab {
-    int64_t A1[5], A2[5], gA[5][2], eA[5][2];     // [level][recompute]; A2 = size if retained
-    int64_t B1[5], B2[5], gB[5][2], eB[5][2];
-    int64_t C1[5];
-    int64_t gCr, eCr;                             // unfused: C read back by Op2
-    uint32_t rc[5];
-    uint32_t pad;
-    // 32-bit forms for the threshold-relative walk: per level x1 = size, x2 = size if retained,
-    // g[recompute] = DRAM term in relative units; sizes saturated to kSizeCap, terms to kTermCap
+    int64_t gA[5][2], gB[5][2];                   // [level][recompute]: DRAM term, exact
+    int64_t gCr;                                  // unfused: C read back by Op2
+    int32_t gXc[2];                               // energy: C round trip (+ softmax pass) of an unfused task, phi = 1, 2
+                                                  // (EDP: [0] = single-precision lower bound of gCr)
+    // 32-bit forms: per level x1 = size, x2 = size if retained (from L4 upwards), both saturated to kSizeCap;
+    // g[recompute] = DRAM term in relative units saturated to kTermCap (EDP: single-precision lower bounds)
     int32_t Ac[5][4];
     int32_t Bc[5][4];
     int32_t Cc[5][2];                             // size, recompute flag
-    int32_t gXc[2];                               // energy: C round trip (+ softmax pass) of an unfused task, phi = 1, 2
+    int32_t pad[2];
     RowTab rt[2];                                 // 0 fused, 1 unfused
 };
 static_assert(offsetof(OrderTab, Ac) % 16 == 0 && offsetof(OrderTab, Bc) % 16 == 0 && offsetof(OrderTab, Cc) % 8 == 0,
@@ -440,28 +440,22 @@ __device__ __noinline__ int64_t slow_row(WarpTop* wt, CtaShared* cs, long long* 
 __device__ __forceinline__ void fill_dead_order_item(OrderTab* ot, int item) {
     const int l = item % 5;
     if (item < 10) {
-        int64_t* s1 = item < 5 ? ot->A1 : ot->B1;
-        int64_t* s2 = item < 5 ? ot->A2 : ot->B2;
         int64_t (*g)[2] = item < 5 ? ot->gA : ot->gB;
-        int64_t (*e)[2] = item < 5 ? ot->eA : ot->eB;
-        s1[l] = s2[l] = 0;
-        g[l][0] = g[l][1] = e[l][0] = e[l][1] = 0;
+        g[l][0] = g[l][1] = 0;
         int32_t* c = item < 5 ? ot->Ac[l] : ot->Bc[l];
         c[0] = c[1] = kSizeCap; c[2] = c[3] = 0;
     } else if (item < 15) {
-        ot->C1[l] = 0;
-        ot->rc[l] = 0;
         ot->Cc[l][0] = kSizeCap; ot->Cc[l][1] = 0;
     } else if (item < 25) {
         for (int v = 0; v < 2; ++v) {
-            int64_t* r = item < 20 ? ot->rt[v].D[l] : ot->rt[v].E[l];
+            (item < 20 ? ot->rt[v].Dg : ot->rt[v].Eg)[l] = 0;
             int32_t* c = item < 20 ? ot->rt[v].Dc[l] : ot->rt[v].Ec[l];
-            r[0] = r[1] = (int64_t)kSizeCap; r[2] = r[3] = 0;
             c[0] = c[1] = kSizeCap; c[2] = c[3] = 0;
         }
     } else {
-        ot->gCr = ot->eCr = 0;
+        ot->gCr = 0;
         ot->gXc[0] = ot->gXc[1] = 0;
+        ot->pad[0] = ot->pad[1] = 0;
     }
 }
 
@@ -485,18 +479,12 @@ __device__ __forceinline__ void build_order_item(const Plan& p, const TilingTab*
         const int x = item < 5 ? OP_A : OP_B;
         const int64_t bs = monomial(q.bs[order][x][l]);
         const int64_t v0 = monomial(q.da[order][x][l][0]), v1 = monomial(q.da[order][x][l][1]);
-        int64_t* s1 = x == OP_A ? ot->A1 : ot->B1;
-        int64_t* s2 = x == OP_A ? ot->A2 : ot->B2;
         int64_t (*g)[2] = x == OP_A ? ot->gA : ot->gB;
-        int64_t (*e)[2] = x == OP_A ? ot->eA : ot->eB;
-        s1[l] = bs;
-        s2[l] = l ? bs : 0;                            // retained (tau = 1) from L4 upwards
         g[l][0] = scale * v0;
         g[l][1] = scale * v1;
-        if (OBJ >= MMEE_OBJ_EDP) { e[l][0] = escale * v0; e[l][1] = escale * v1; }
         int32_t* c = x == OP_A ? ot->Ac[l] : ot->Bc[l];
         c[0] = size32(bs);
-        c[1] = l ? size32(bs) : 0;
+        c[1] = l ? size32(bs) : 0;                     // retained (tau = 1) from L4 upwards
         c[2] = term32(scale * v0);
         c[3] = term32(scale * v1);
         if constexpr (OBJ == MMEE_OBJ_EDP) {
@@ -506,10 +494,7 @@ __device__ __forceinline__ void build_order_item(const Plan& p, const TilingTab*
             c[3] = __float_as_int(__ll2float_rd(v1));
         }
     } else if (item < 15) {                            // C
-        const int64_t bs = monomial(q.bs[order][OP_C][l]);
-        ot->C1[l] = bs;
-        ot->rc[l] = q.recompute[order][l];
-        ot->Cc[l][0] = size32(bs);
+        ot->Cc[l][0] = size32(monomial(q.bs[order][OP_C][l]));
         ot->Cc[l][1] = (int32_t)q.recompute[order][l];
     } else if (item < 25) {                            // D, E
         const int x = item < 20 ? OP_D : OP_E;
@@ -518,33 +503,23 @@ __device__ __forceinline__ void build_order_item(const Plan& p, const TilingTab*
         const int64_t vu = monomial(q.da_unfused[order][x][l]);
         RowTab* f = &ot->rt[0];
         RowTab* u = &ot->rt[1];
-        int64_t* fr = x == OP_D ? f->D[l] : f->E[l];
-        int64_t* ur = x == OP_D ? u->D[l] : u->E[l];
-        fr[0] = l ? bs : 0; fr[1] = bs; fr[2] = scale * vf; fr[3] = escale * vf;
-        ur[0] = 0;          ur[1] = bs; ur[2] = scale * vu; ur[3] = escale * vu;
+        (x == OP_D ? f->Dg : f->Eg)[l] = scale * vf;
+        (x == OP_D ? u->Dg : u->Eg)[l] = scale * vu;
         int32_t* fc = x == OP_D ? f->Dc[l] : f->Ec[l];
         int32_t* uc = x == OP_D ? u->Dc[l] : u->Ec[l];
-#pragma unroll
-        for (int i = 0; i < 3; ++i) {
-            // sizes saturate; the DRAM term is kept in units of 2^rel_shift (rounded down), then saturated
-            const int64_t lim = i < 2 ? (int64_t)kSizeCap : (int64_t)kTermCap;
-            const int64_t fv = i < 2 ? fr[i] : (fr[i] >> p.rel_shift);
-            const int64_t uv = i < 2 ? ur[i] : (ur[i] >> p.rel_shift);
-            fc[i] = (int32_t)(fv < lim ? fv : lim);
-            uc[i] = (int32_t)(uv < lim ? uv : lim);
-        }
-        fc[3] = 0;
-        uc[3] = 0;
+        // fused rows: retained from L4 upwards while Op1 runs; unfused rows take no space while Op1 runs
+        fc[0] = l ? size32(bs) : 0; fc[1] = size32(bs); fc[2] = term32(scale * vf); fc[3] = 0;
+        uc[0] = 0;                  uc[1] = size32(bs); uc[2] = term32(scale * vu); uc[3] = 0;
         if constexpr (OBJ == MMEE_OBJ_EDP) {
             // the energy-delay filter's first level works on single-precision lower bounds: DRAM words and their
             // energy, each rounded down
-            fc[2] = __float_as_int(__ll2float_rd(fr[2])); fc[3] = __float_as_int(__ll2float_rd(fr[3]));
-            uc[2] = __float_as_int(__ll2float_rd(ur[2])); uc[3] = __float_as_int(__ll2float_rd(ur[3]));
+            fc[2] = __float_as_int(__ll2float_rd(vf)); fc[3] = __float_as_int(__ll2float_rd(escale * vf));
+            uc[2] = __float_as_int(__ll2float_rd(vu)); uc[3] = __float_as_int(__ll2float_rd(escale * vu));
         }
     } else {
         const int64_t v = monomial(q.da_unfused[order][OP_C][0]);
         ot->gCr = scale * v;
-        ot->eCr = escale * v;
+        ot->pad[0] = ot->pad[1] = 0;
         // energy of an unfused task's C round trip: read-back, write, and the separate softmax pass of phi = 2
         ot->gXc[0] = term32(p.c_dram_gb * (v + tb->cw));
         ot->gXc[1] = term32(p.c_dram_gb * (v + tb->cw + tb->smx));
@@ -650,9 +625,10 @@ __device__ __forceinline__ MidExact mid_exact(const Plan& p, const TilingTab* tb
     const uint32_t lc = fused ? (uint32_t)m : 0u;
     // Tables of a tiling that cannot fit are filled with constants: a lane whose task lies in such
     // a tiling must not index with what it reads from them.
-    const uint32_t rc = (fused && live) ? (ot->rc[lc] & 1u) : 0u;
-    const int64_t a1 = ot->A1[la], b1 = ot->B1[lb], c1 = ot->C1[lc];
-    const int64_t a2 = fused ? ot->A2[la] : 0, b2 = fused ? ot->B2[lb] : 0;
+    const uint32_t rc = (fused && live) ? ((uint32_t)ot->Cc[lc][1] & 1u) : 0u;
+    // (sizes saturated to kSizeCap, which is above the capacity: every comparison with a slack keeps its result)
+    const int64_t a1 = ot->Ac[la][0], b1 = ot->Bc[lb][0], c1 = ot->Cc[lc][0];
+    const int64_t a2 = fused ? ot->Ac[la][1] : 0, b2 = fused ? ot->Bc[lb][1] : 0;
     // Eq. (1)/(2): a retained operand (level >= L4) of the other operator keeps its space.
     // A lane without a live task gets a negative slack, so that none of its rows fits.
     r.slack1 = live ? p.cap_words - (a1 + b1 + c1) : -1;
@@ -681,8 +657,8 @@ __device__ __forceinline__ MidExact mid_exact(const Plan& p, const TilingTab* tb
             r.qptr = &tb->QU[0][0];
         }
         if constexpr (OBJ >= MMEE_OBJ_EDP) {
-            const int64_t eab = ot->eA[la][rc] + ot->eB[lb][rc];
-            r.xe0 = fused ? eab : eab + ot->eCr + p.c_dram_gb * (tb->cw + pass);
+            // (for these objectives the g terms are DRAM words; their energy is the words times the cost of one)
+            r.xe0 = p.c_dram_gb * (fused ? gab : gab + ot->gCr + tb->cw + pass);
         }
     }
     return r;
@@ -700,16 +676,16 @@ __device__ __noinline__ void exact_group(const Plan& p, const TilingTab* tb, con
     const long long g_now = (lane == 0) ? *reinterpret_cast<volatile long long*>(global_g) : 0;
     const MidExact me = mid_exact<OBJ>(p, tb, ot, phi, la, lb_task, m, live);
     const RowTab* rt = &ot->rt[phi == 0 ? 0 : 1];
-    const int64_t s1 = me.slack1 - rt->D[d][0];
-    const int64_t s2 = me.slack2 - rt->D[d][1];
-    const int64_t xd = me.x0 + rt->D[d][2];
-    const int64_t xed = (OBJ >= MMEE_OBJ_EDP) ? me.xe0 + rt->D[d][3] : 0;
+    const int64_t s1 = me.slack1 - rt->Dc[d][0];
+    const int64_t s2 = me.slack2 - rt->Dc[d][1];
+    const int64_t xd = me.x0 + rt->Dg[d];
+    const int64_t xed = (OBJ >= MMEE_OBJ_EDP) ? me.xe0 + p.c_dram_gb * rt->Dg[d] : 0;
 #pragma unroll 1
     for (int e = 0; e < 5; ++e) {
         if (!((rows >> e) & 1u)) continue;      // the filter flagged this row in no lane
-        const bool fit = (rt->E[e][0] <= s1) && (rt->E[e][1] <= s2) && ((kept >> (d * 5 + e)) & 1u);
-        const int64_t x = xd + rt->E[e][2];
-        const int64_t xe = (OBJ >= MMEE_OBJ_EDP) ? xed + rt->E[e][3] : 0;
+        const bool fit = (rt->Ec[e][0] <= s1) && (rt->Ec[e][1] <= s2) && ((kept >> (d * 5 + e)) & 1u);
+        const int64_t x = xd + rt->Eg[e];
+        const int64_t xe = (OBJ >= MMEE_OBJ_EDP) ? xed + p.c_dram_gb * rt->Eg[e] : 0;
         const uint64_t row_first_idx = task_first_idx + (uint64_t)(m * 225 + (d * 5 + e) * 9);
         const int64_t thr_row = lane_threshold(wt, cs, k, row_first_idx);
         bool below = false;
@@ -738,18 +714,18 @@ __device__ __noinline__ void exact_group_single(const Plan& p, const TilingTab* 
     const long long g_now = (lane == 0) ? *reinterpret_cast<volatile long long*>(global_g) : 0;
     const MidExact me = mid_exact<OBJ>(p, tb, ot, phi, la, lb_task, m, live);
     const RowTab* rt = &ot->rt[phi == 0 ? 0 : 1];
-    const int64_t s1 = me.slack1 - rt->D[d][0];
-    const int64_t s2 = me.slack2 - rt->D[d][1];
-    const int64_t xd = me.x0 + rt->D[d][2];
-    const int64_t xed = (OBJ >= MMEE_OBJ_EDP) ? me.xe0 + rt->D[d][3] : 0;
+    const int64_t s1 = me.slack1 - rt->Dc[d][0];
+    const int64_t s2 = me.slack2 - rt->Dc[d][1];
+    const int64_t xd = me.x0 + rt->Dg[d];
+    const int64_t xed = (OBJ >= MMEE_OBJ_EDP) ? me.xe0 + p.c_dram_gb * rt->Dg[d] : 0;
     int64_t best = kInfKey;
     uint32_t best_pos = 0;
 #pragma unroll 1
     for (int e = 0; e < 5; ++e) {
         if (!((rows >> e) & 1u)) continue;      // the filter flagged this row in no lane
-        const bool fit = (rt->E[e][0] <= s1) && (rt->E[e][1] <= s2) && ((kept >> (d * 5 + e)) & 1u);
-        const int64_t x = xd + rt->E[e][2];
-        const int64_t xe = (OBJ >= MMEE_OBJ_EDP) ? xed + rt->E[e][3] : 0;
+        const bool fit = (rt->Ec[e][0] <= s1) && (rt->Ec[e][1] <= s2) && ((kept >> (d * 5 + e)) & 1u);
+        const int64_t x = xd + rt->Eg[e];
+        const int64_t xe = (OBJ >= MMEE_OBJ_EDP) ? xed + p.c_dram_gb * rt->Eg[e] : 0;
 #pragma unroll
         for (int s = 0; s < 9; ++s) {
             const int64_t key = candidate_key<OBJ>(x, xe, me.wptr[2 * s], me.P[s / 3], me.qptr[2 * s], p.key_cap);
@@ -804,14 +780,14 @@ __device__ __noinline__ unsigned edp_group_test(const Plan& p, const TilingTab* 
         dW[s] = ((sm_mask >> s) & 1u) ? (double)me.wptr[2 * s] : __longlong_as_double(0x7ff0000000000000ll);
         dQP[s] = (double)(me.qptr[2 * s] + me.P[s / 3]);
     }
-    const int64_t xd = me.x0 + rt->D[d][2];
-    const int64_t xed = me.xe0 + rt->D[d][3];
+    const int64_t xd = me.x0 + rt->Dg[d];
+    const int64_t xed = me.xe0 + p.c_dram_gb * rt->Dg[d];
     unsigned hit_any = 0;
 #pragma unroll 1
     for (int e = 0; e < 5; ++e) {
         const unsigned fit = (unsigned)(rt->Ec[e][0] <= s1c) & (unsigned)(rt->Ec[e][1] <= s2c) & (kept_rows >> e);   // Eq. (4)
-        const int64_t x = xd + rt->E[e][2];
-        const double de = (double)(xed + rt->E[e][3]);
+        const int64_t x = xd + rt->Eg[e];
+        const double de = (double)(xed + p.c_dram_gb * rt->Eg[e]);
         double dl[3];
 #pragma unroll
         for (int j = 0; j < 3; ++j) dl[j] = (double)(x + me.P[j]);
@@ -951,22 +927,22 @@ __device__ __forceinline__ uint32_t walk_task_exact(const Plan& p, const TilingT
                     hit_any = edp_group_test(p, tb, ot, c.phi, c.la, c.lb, m, live, d, s1c, s2c, kd, dthr);
             } else {
                 ++groups_walked;
-                const int64_t s1 = me.slack1 - rt->D[d][0];
-                const int64_t s2 = me.slack2 - rt->D[d][1];
-                const int64_t xd = me.x0 + rt->D[d][2];
-                const int64_t xed = (OBJ >= MMEE_OBJ_EDP) ? me.xe0 + rt->D[d][3] : 0;
+                const int64_t s1 = me.slack1 - rt->Dc[d][0];
+                const int64_t s2 = me.slack2 - rt->Dc[d][1];
+                const int64_t xd = me.x0 + rt->Dg[d];
+                const int64_t xed = (OBJ >= MMEE_OBJ_EDP) ? me.xe0 + p.c_dram_gb * rt->Dg[d] : 0;
                 const uint64_t group_first_idx = mid_first_idx + (uint64_t)(d * 45);
                 const int64_t thr = th.T1 - (group_first_idx > th.ti ? th.delta : 0);
 #pragma unroll
                 for (int e = 0; e < 5; ++e) {
-                    const int64_t x = xd + rt->E[e][2];
-                    const int64_t xe = (OBJ >= MMEE_OBJ_EDP) ? xed + rt->E[e][3] : 0;
+                    const int64_t x = xd + rt->Eg[e];
+                    const int64_t xe = (OBJ >= MMEE_OBJ_EDP) ? xed + p.c_dram_gb * rt->Eg[e] : 0;
                     int64_t key[9];
 #pragma unroll
                     for (int s = 0; s < 9; ++s)
                         key[s] = ((p.sm_mask >> s) & 1u) ? candidate_key<OBJ>(x, xe, W[s], me.P[s / 3], Q[s], p.key_cap) : kInfKey;
                     unsigned fit, hit;
-                    row_test(key, thr, rt->E[e][0], s1, rt->E[e][1], s2, fit, hit);
+                    row_test(key, thr, (int64_t)rt->Ec[e][0], s1, (int64_t)rt->Ec[e][1], s2, fit, hit);
                     if constexpr (PRUNE) { fit &= kept >> (d * 5 + e); hit &= fit; }
                     fits += fit;
                     hit_any |= hit << e;
