@@ -1116,6 +1116,11 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
         // (u is a value from here on: the compiler must not form it again from its inputs in every group)
         asm volatile("" : "+r"(u));
 
+        // The D terms of the five groups are loaded ahead of the group loop: inside it a load could not move above
+        // the (rare) calls of the exact path, and each group would wait for its own.
+        int4 dcs[5];
+#pragma unroll
+        for (int d = 0; d < 5; ++d) dcs[d] = *reinterpret_cast<const int4*>(rt->Dc[d]);
 #pragma unroll
         for (int d = 0; d < 5; ++d) {
             if constexpr (PRUNE) {
@@ -1123,7 +1128,7 @@ __device__ __forceinline__ uint32_t walk_task_relative(const Plan& p, const Tili
             }
             // Five rows (levels of E) are evaluated branch-free; one vote decides whether any lane of the
             // warp has to enter the exact path for this group.
-            const int4 dc = *reinterpret_cast<const int4*>(rt->Dc[d]);
+            const int4 dc = dcs[d];
             const int s1c = imad(dc.x, minus_one, slack1c);
             const int s2c = imad(dc.y, minus_one, slack2c);
             // Eq. (4) for the five levels of E: at L3, and in an unfused task, E takes no space while Op1
