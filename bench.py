@@ -44,8 +44,8 @@ ALG_OPS_PER_ROW = {0: 4.4, 1: 4.4, 2: 10.0}
 LANES_PER_SM = 64          # 4 sub-partitions x 16 lanes: width of the integer-ALU pipe, the busiest pipe of these kernels
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, recorded from the ncu captures summarised under
 # profiles/ (not measured in this run); workload -> objective -> bytes.  None where no capture backs it.
-NCU_DRAM_BYTES_PER_LAUNCH = {"gqa": {1: 198656, 2: 193792}, "llama": {0: 205824, 1: 195328},
-                             "bert": {0: 183040, 1: 199936}}
+NCU_DRAM_BYTES_PER_LAUNCH = {"gqa": {1: 199680, 2: 193024}, "llama": {0: 207360, 1: 198400},
+                             "bert": {0: 182272, 1: 201216}}
 
 
 WORKLOADS = {"tiny": mi.config1, "bert": mi.config2, "llama": mi.config3, "gqa": mi.config4}
