@@ -308,6 +308,28 @@ def test_interval_with_more_ranges_than_ctas_but_fewer_than_twice_as_many():
     check_search(cfg, dict(cfg["searches"][0], topk=2, t_begin=300, t_end=1200))
 
 
+def test_whole_tiling_ranges_with_odd_interval_ends():
+    """An interval long enough for ranges of whole tilings with a tail of short ranges, with ends that are not
+    multiples of the range length: the two small end pieces are checked against the oracle directly, and the three
+    pieces together must give the stored whole-problem answer (feasible count; the best of the pieces)."""
+    with open(os.path.join(GOLDEN, "search_gqa_b4_s8192.json")) as f:
+        gold = json.load(f)
+    cfg = dict(name=gold["name"], workload=gold["workload"], arch=gold["arch"])
+    s = gold["searches"][0]
+    obj = dict(s["objective"], topk=1)
+    T = oracle.make_problem(cfg["workload"], cfg["arch"], obj).T
+    lo, hi = 3, T - 5
+    pieces = [check_search(cfg, dict(obj, t_begin=0, t_end=lo))[0], check_search(cfg, dict(obj, t_begin=hi, t_end=T))[0]]
+    big, _, stats = gpu_search(cfg, dict(obj, t_begin=lo, t_end=hi))
+    assert stats.tasks == (hi - lo) * 210
+    pieces.append(big)
+    assert sum(p.n_feasible for p in pieces) == s["n_feasible"]
+    key = {mi.OBJ_ENERGY: "e_key", mi.OBJ_LATENCY: "l_key"}.get(obj["objective"])
+    best = min((p for p in pieces if p.idx != mm.NO_INDEX),
+               key=lambda p: ((getattr(p, key) if key else p.edp_key), p.idx))
+    assert best.idx == s["topk"][0]["idx"]
+
+
 def test_nothing_fits():
     cfg = mi.random_tiny_problem(3)
     arch = dict(cfg["arch"], gb_bytes=cfg["workload"]["word_bytes"] * 2)
