@@ -369,10 +369,9 @@ __device__ __forceinline__ unsigned edp_row_test(double de, const double (&dl)[3
     return hit;
 }
 
-#ifndef MMEE_BULK_MIN
-#define MMEE_BULK_MIN 3
-#endif
-constexpr int kBulkMin = MMEE_BULK_MIN;     // more pending candidates than this are merged in one step
+// More pending candidates of one position than this are merged into the list in one sorted step (measured with 3, 7,
+// 15 and never: 3 is fastest on the top-16 searches).
+constexpr int kBulkMin = 3;
 
 // Rare path: some lane of the warp has a key below its threshold in this row.  Every lane
 // re-evaluates its nine candidates of the row from the shared tables and the warp inserts the
@@ -1221,35 +1220,36 @@ __device__ __noinline__ void finalize_step(const Plan& p, Scratch* __restrict__ 
         // (lane 0 holds the warp's entry, the other lanes the empty pair)
         ek = lane == 0 ? (int64_t)(((uint64_t)kh << 32) | kl) : kInfKey;
         ei = lane == 0 ? (((uint64_t)ih << 32) | il) : UINT64_MAX;
-    } else
-    for (int c0 = 0; c0 < n_partials; c0 += kSearchThreads) {
-        const int c = c0 + tid;
-        const int len = c < n_partials ? __ldcg(&scratch->partial[c].count) : 0;
-        unsigned todo = __ballot_sync(kFull, len > 0);
-        while (todo) {
-            int n[kBatch];
-            longlong2 mine[kBatch];
+    } else {
+        for (int c0 = 0; c0 < n_partials; c0 += kSearchThreads) {
+            const int c = c0 + tid;
+            const int len = c < n_partials ? __ldcg(&scratch->partial[c].count) : 0;
+            unsigned todo = __ballot_sync(kFull, len > 0);
+            while (todo) {
+                int n[kBatch];
+                longlong2 mine[kBatch];
 #pragma unroll
-            for (int i = 0; i < kBatch; ++i) {
-                n[i] = 0;
-                mine[i] = make_longlong2(kInfKey, -1ll);
-                if (todo) {
-                    const int src_lane = __ffs(todo) - 1;
-                    todo &= todo - 1;
-                    n[i] = __shfl_sync(kFull, len, src_lane);
-                    if (lane < n[i]) mine[i] = __ldcg(&scratch->partial[c0 + warp * 32 + src_lane].e[lane]);
+                for (int i = 0; i < kBatch; ++i) {
+                    n[i] = 0;
+                    mine[i] = make_longlong2(kInfKey, -1ll);
+                    if (todo) {
+                        const int src_lane = __ffs(todo) - 1;
+                        todo &= todo - 1;
+                        n[i] = __shfl_sync(kFull, len, src_lane);
+                        if (lane < n[i]) mine[i] = __ldcg(&scratch->partial[c0 + warp * 32 + src_lane].e[lane]);
+                    }
                 }
-            }
-            // (unrolled: with a run-time index the batch would live in local memory, and the store of each
-            // loaded entry there would wait for its load before the next load could issue)
+                // (unrolled: with a run-time index the batch would live in local memory, and the store of each
+                // loaded entry there would wait for its load before the next load could issue)
 #pragma unroll
-            for (int i = 0; i < kBatch; ++i) {
-                // a list whose first entry does not precede this warp's k-th entry adds nothing
-                const int64_t kth_key = __shfl_sync(kFull, ek, k - 1), head_key = __shfl_sync(kFull, mine[i].x, 0);
-                const uint64_t kth_idx = __shfl_sync(kFull, ei, k - 1);
-                const uint64_t head_idx = (uint64_t)__shfl_sync(kFull, mine[i].y, 0);
-                if (n[i] > 0 && pair_less(head_key, head_idx, kth_key, kth_idx))
-                    reg_absorb(ek, ei, k, n[i], mine[i].x, (uint64_t)mine[i].y, lane);
+                for (int i = 0; i < kBatch; ++i) {
+                    // a list whose first entry does not precede this warp's k-th entry adds nothing
+                    const int64_t kth_key = __shfl_sync(kFull, ek, k - 1), head_key = __shfl_sync(kFull, mine[i].x, 0);
+                    const uint64_t kth_idx = __shfl_sync(kFull, ei, k - 1);
+                    const uint64_t head_idx = (uint64_t)__shfl_sync(kFull, mine[i].y, 0);
+                    if (n[i] > 0 && pair_less(head_key, head_idx, kth_key, kth_idx))
+                        reg_absorb(ek, ei, k, n[i], mine[i].x, (uint64_t)mine[i].y, lane);
+                }
             }
         }
     }
